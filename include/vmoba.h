@@ -1,0 +1,167 @@
+/*
+ * vmoba.h -- C ABI of the VMoBA block-sparse attention layer for NVIDIA B200 (sm_100a).
+ *
+ * VMoBA (Mixture-of-Block Attention for video diffusion models, arXiv 2506.23858)
+ * replaces the dense self-attention of a video DiT layer by three steps (Section 3.1):
+ *   Step 1  partition the keys of the T x H x W latent grid into 1D / 2D / 3D blocks and
+ *           mean-pool each block into a centroid                     (Eq. 1, Eq. 2)
+ *   Step 2  score every query token against every centroid and keep, per head, the
+ *           globally best (query, key-block) pairs until their normalised similarity
+ *           mass reaches a threshold tau                             (Eq. 3, Eq. 4)
+ *   Step 3  softmax attention of each query over the keys of its selected blocks only.
+ *
+ * Conventions shared by every entry point
+ *   - All data pointers are DEVICE pointers, 16-byte aligned, owned by the caller.  The
+ *     library allocates no device memory and keeps no state between calls; scratch memory
+ *     is passed in as `ws` and must hold vmoba_workspace_bytes() bytes.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it and
+ *     return; they never synchronise.
+ *   - The return value reports errors the host can see (bad arguments, shapes, workspace
+ *     size, a failed launch).  Errors that depend on device data (work-list capacity
+ *     exceeded, a bounded device-side wait that expired) are written to the int32 word
+ *     `dev_status` (first error wins; the caller zeroes it and reads it after
+ *     synchronising).  After any error the outputs are unspecified but every access stayed
+ *     inside the buffers described here.
+ *   - Token order at the boundary is raster (t, h, w), w fastest, S = T*H*W.  "Block-major"
+ *     means position p = block * s_b + slot, blocks ordered (nT, nH, nW) with nW fastest and
+ *     slots (sT, sH, sW) with sW fastest (Eq. 1).  Block-major tensors are [B, heads, S, head_dim],
+ *     contiguous.  G = (b * heads + head) * S + p is the flat query index used by the lists.
+ *   - The partition type is implied by the block shape: (bT, H, W) is the 1D temporal
+ *     partition, (T, bH, bW) the 2D spatial one, anything else 3D; one index formula covers
+ *     all three.  A layer l of the recurrent schedule uses l mod 3 -> 1D, 2D, 3D.
+ *   - dtype VMOBA_BF16 runs QK^T and PV on the tensor cores (head_dim 128); VMOBA_F32 is the
+ *     fp32 CUDA-core path (head_dim 64 or 128).  Scores, LSE and all selection arithmetic are
+ *     fp32 (fp64 for the cumulative mass) for both.
+ */
+#ifndef VMOBA_H_
+#define VMOBA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  VMOBA_OK = 0,
+  VMOBA_ERR_ARG = 1,            /* null or misaligned pointer, tau not in (0, 1], bad enum          */
+  VMOBA_ERR_SHAPE = 2,          /* non-positive size, grid not divisible by the block, head_dim     */
+  VMOBA_ERR_WORKSPACE = 3,      /* ws_bytes smaller than vmoba_workspace_bytes()                    */
+  VMOBA_ERR_CAPACITY = 4,       /* (dev_status) more selected pairs than the lists can hold         */
+  VMOBA_ERR_TIMEOUT = 5,        /* (dev_status) a bounded device-side wait expired                  */
+  VMOBA_ERR_CUDA = 6,           /* a CUDA runtime / driver call failed                              */
+  VMOBA_ERR_NOT_IMPLEMENTED = 7 /* combination of dtype / head_dim without a kernel                 */
+} vmoba_status;
+
+typedef enum { VMOBA_F32 = 0, VMOBA_BF16 = 1 } vmoba_dtype;
+
+typedef enum {
+  VMOBA_STAGE_SCORES = 0,
+  VMOBA_STAGE_SELECT = 1,
+  VMOBA_STAGE_ATTN_FWD = 2,
+  VMOBA_STAGE_ATTN_BWD = 3,
+  VMOBA_STAGE_FULL_FWD = 4,
+  VMOBA_STAGE_FULL_BWD = 5
+} vmoba_stage;
+
+typedef struct {
+  int32_t B, heads, head_dim; /* head_dim: 64 or 128                                            */
+  int32_t T, H, W;            /* latent grid, S = T*H*W                                         */
+  int32_t bT, bH, bW;         /* block shape in tokens; must divide T, H, W                     */
+  int32_t dtype;              /* vmoba_dtype of q, k, v, o and the gradients                    */
+  float softmax_scale;        /* attention scale and selection temperature; 0 => head_dim^-1/2 */
+} vmoba_shape;
+
+const char* vmoba_status_string(int status);
+
+/* Bytes of scratch `ws` a stage needs.  `capacity` is the number of (query, key-block) pairs
+ * the work lists can hold (the q_idx_capacity given to vmoba_select); stages that do not
+ * depend on it ignore it.  Returns 0 for an invalid shape or stage. */
+size_t vmoba_workspace_bytes(const vmoba_shape* shape, int stage, int64_t capacity);
+
+/*
+ * Step 1, Eq. 1: reorder tokens into blocks (inverse = 0) or back (inverse = 1).
+ *   raster : [B, S, heads, head_dim] addressed by element strides raster_strides_bsh =
+ *            {batch, token, head}; head_dim is contiguous; strides must keep rows 16-byte aligned.
+ *   bm     : block-major [B, heads, S, head_dim], contiguous.
+ * inverse = 0 reads raster and writes bm; inverse = 1 reads bm and writes raster.
+ * perm_or_null / inv_perm_or_null: optional int32 [S] outputs, perm[p] = raster index of the
+ * token at block-major position p, inv_perm its inverse.
+ */
+int vmoba_partition(const vmoba_shape* shape, int inverse, const void* src, void* dst,
+                    const int64_t raster_strides_bsh[3], int32_t* perm_or_null,
+                    int32_t* inv_perm_or_null, void* stream);
+
+/*
+ * Step 1 + Step 2a, Eq. 2 and the similarity map of Section 3.3:
+ *   centroids [B, heads, N_b, head_dim] fp32 = mean of each key block,
+ *   scores    [B, heads, S, N_b]       fp32 = q . centroid, unscaled.
+ * q_bm, k_bm are block-major.
+ */
+int vmoba_block_scores(const vmoba_shape* shape, const void* q_bm, const void* k_bm,
+                       float* centroids, float* scores, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Step 2b, Eq. 3 + Eq. 4: global threshold selection per (batch, head).
+ * The head's S*N_b scores are normalised with a softmax at temperature softmax_scale over the
+ * whole pool; pairs are taken in descending score order until the cumulative mass is >= tau
+ * (tau >= 1 selects everything).  Every pair whose score is >= the score of the last pair
+ * taken is selected (exact ties at the cutoff are all kept).
+ * Outputs
+ *   mask_bits        uint32 [B*heads*S, ceil(N_b/32)]  bit j of a row = block j selected by that query
+ *   kb_ptr           int32  [B*heads*N_b + 1]          CSR offsets by (batch, head, key block) into q_idx
+ *   q_idx            int32  [capacity]                 per key block: the in-head positions p (ascending) of
+ *                                                      the queries that selected it
+ *   q_ptr            int32  [B*heads*S + 1]            CSR offsets by flat query G into q_pairs
+ *   q_pairs          int32  [capacity]                 per query: positions in q_idx of its pairs, by ascending block
+ *   k_per_head       int64  [B*heads]                  number of selected pairs
+ *   cutoff_per_head  float  [B*heads]                  score of the last pair taken
+ * dev_status gets VMOBA_ERR_CAPACITY if the total exceeds `capacity` (lists are then truncated).
+ */
+int vmoba_select(const vmoba_shape* shape, const float* scores, float tau, uint32_t* mask_bits,
+                 int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr, int32_t* q_pairs,
+                 int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
+                 int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Step 3: attention of every query over the keys of its selected blocks.
+ *   o_bm [B, heads, S, head_dim] (dtype), lse [B*heads*S] fp32 natural-log sum-exp of the scaled logits.
+ * A query with no selected block gets o = 0 and lse = -inf.
+ * o_resid_or_null (bf16 only, same shape as o_bm): if given, receives the rounding residual
+ * bf16(o_exact - o_bm).  The backward needs rowsum(dO * O) to better than bf16 accuracy of O
+ * (taken from the rounded output alone, dQ loses about 6e-3 relative accuracy); training
+ * callers keep this tensor with o_bm and lse for vmoba_attn_bwd.
+ * `capacity` is the one given to vmoba_select (bounds the per-pair partial results in ws).
+ */
+int vmoba_attn_fwd(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
+                   const int32_t* kb_ptr, const int32_t* q_idx, const int32_t* q_ptr,
+                   const int32_t* q_pairs, int64_t capacity, void* o_bm, void* o_resid_or_null,
+                   float* lse, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Training backward of Step 3 with the selection held constant (TopkMask has zero gradient):
+ * dq, dk, dv [B, heads, S, head_dim] (dtype) from do_bm, the forward's o_bm (+ o_resid) and lse.
+ * Queries without a selected block get dq = 0.  The paper states no gradient formula; this is
+ * the softmax-attention gradient restricted to the selected pairs.  `capacity` is the one given
+ * to vmoba_select (list positions at or beyond it are never read).
+ */
+int vmoba_attn_bwd(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
+                   const void* o_bm, const void* o_resid_or_null, const float* lse, const void* do_bm,
+                   const int32_t* kb_ptr,
+                   const int32_t* q_idx, const int32_t* q_ptr, int64_t capacity, void* dq_bm, void* dk_bm,
+                   void* dv_bm, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Dense softmax attention over all S keys: the tau = 1 limit of the layer and the speed-up
+ * denominator (the "Full Attention" baseline of Section 4.1).  Tensors are [B, heads, S, head_dim]
+ * in any one token order.  If do_or_null is given, also computes dq, dk, dv.
+ */
+int vmoba_full_attn(const vmoba_shape* shape, const void* q, const void* k, const void* v, void* o,
+                    float* lse, const void* do_or_null, void* dq, void* dk, void* dv,
+                    int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VMOBA_H_ */

@@ -1,0 +1,174 @@
+"""ctypes binding of ``libvmoba.so``: the same entry points as ``include/vmoba.h``, taking torch
+CUDA tensors and passing their device pointers through.  Argument marshalling only -- every
+step of the layer runs in the library's kernels.  There is no CPU fallback: if the library is
+missing, or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+
+from . import build as _build
+
+OK, ERR_ARG, ERR_SHAPE, ERR_WORKSPACE, ERR_CAPACITY, ERR_TIMEOUT, ERR_CUDA, ERR_NOT_IMPLEMENTED = range(8)
+F32, BF16 = 0, 1
+STAGE_SCORES, STAGE_SELECT, STAGE_ATTN_FWD, STAGE_ATTN_BWD, STAGE_FULL_FWD, STAGE_FULL_BWD = range(6)
+
+EXPORTS = (
+    "vmoba_status_string", "vmoba_workspace_bytes", "vmoba_partition", "vmoba_block_scores",
+    "vmoba_select", "vmoba_attn_fwd", "vmoba_attn_bwd", "vmoba_full_attn",
+)
+
+
+class VmobaError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: status {code} ({status_string(code)})")
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("B", "heads", "head_dim", "T", "H", "W", "bT", "bH", "bW", "dtype")] + [
+        ("softmax_scale", ctypes.c_float)]
+
+    @property
+    def S(self):
+        return self.T * self.H * self.W
+
+    @property
+    def n_blocks(self):
+        return (self.T // self.bT) * (self.H // self.bH) * (self.W // self.bW)
+
+    @property
+    def block_tokens(self):
+        return self.bT * self.bH * self.bW
+
+    @property
+    def mask_words(self):
+        return (self.n_blocks + 31) // 32
+
+    @property
+    def scale(self):
+        return self.softmax_scale if self.softmax_scale > 0 else 1.0 / math.sqrt(self.head_dim)
+
+
+def make_shape(B, heads, head_dim, grid, block, dtype, softmax_scale=0.0) -> Shape:
+    code = {"f32": F32, "bf16": BF16}[dtype] if isinstance(dtype, str) else int(dtype)
+    return Shape(B, heads, head_dim, grid[0], grid[1], grid[2], block[0], block[1], block[2], code, softmax_scale)
+
+
+def shape_of(w) -> Shape:
+    """Shape of an ``inputs.Workload``."""
+    return make_shape(w.B, w.heads, w.head_dim, (w.T, w.H, w.W), w.block, w.dtype)
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB_PATH
+
+
+def lib():
+    """Loads the C-ABI library (built in-tree by ``build.py``); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = lib_path()
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: run `python -m paper_2506_23858_b200.build` (no CPU fallback exists)")
+    L = ctypes.CDLL(path)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    sp = ctypes.POINTER(Shape)
+    L.vmoba_status_string.restype = ctypes.c_char_p
+    L.vmoba_status_string.argtypes = [ctypes.c_int]
+    L.vmoba_workspace_bytes.restype = sz
+    L.vmoba_workspace_bytes.argtypes = [sp, ctypes.c_int, i64]
+    L.vmoba_partition.restype = ctypes.c_int
+    L.vmoba_partition.argtypes = [sp, ctypes.c_int, vp, vp, ctypes.POINTER(i64), vp, vp, vp]
+    L.vmoba_block_scores.restype = ctypes.c_int
+    L.vmoba_block_scores.argtypes = [sp, vp, vp, vp, vp, vp, sz, vp]
+    L.vmoba_select.restype = ctypes.c_int
+    L.vmoba_select.argtypes = [sp, vp, ctypes.c_float, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp]
+    L.vmoba_attn_fwd.restype = ctypes.c_int
+    L.vmoba_attn_fwd.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
+    L.vmoba_attn_bwd.restype = ctypes.c_int
+    L.vmoba_attn_bwd.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
+    L.vmoba_full_attn.restype = ctypes.c_int
+    L.vmoba_full_attn.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    _lib = L
+    return L
+
+
+def status_string(code: int) -> str:
+    return lib().vmoba_status_string(int(code)).decode()
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(code, where):
+    if code != OK:
+        raise VmobaError(code, where)
+
+
+def workspace_bytes(shape: Shape, stage: int, capacity: int = 0) -> int:
+    return int(lib().vmoba_workspace_bytes(ctypes.byref(shape), stage, capacity))
+
+
+def _ws_args(ws):
+    if ws is None:
+        return None, 0
+    return _ptr(ws), ws.numel() * ws.element_size()
+
+
+def vmoba_partition(shape, inverse, src, dst, raster_strides_bsh, perm=None, inv_perm=None, stream=None):
+    strides = (ctypes.c_int64 * 3)(*[int(x) for x in raster_strides_bsh])
+    _check(lib().vmoba_partition(ctypes.byref(shape), int(inverse), _ptr(src), _ptr(dst), strides, _ptr(perm),
+                                 _ptr(inv_perm), _stream(stream)), "vmoba_partition")
+
+
+def vmoba_block_scores(shape, q_bm, k_bm, centroids, scores, ws=None, stream=None):
+    p, n = _ws_args(ws)
+    _check(lib().vmoba_block_scores(ctypes.byref(shape), _ptr(q_bm), _ptr(k_bm), _ptr(centroids), _ptr(scores), p, n,
+                                    _stream(stream)), "vmoba_block_scores")
+
+
+def vmoba_select(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity, k_per_head,
+                 cutoff_per_head, dev_status, ws, stream=None):
+    p, n = _ws_args(ws)
+    _check(lib().vmoba_select(ctypes.byref(shape), _ptr(scores), float(tau), _ptr(mask_bits), _ptr(kb_ptr),
+                              _ptr(q_idx), _ptr(q_ptr), _ptr(q_pairs), int(capacity), _ptr(k_per_head),
+                              _ptr(cutoff_per_head), _ptr(dev_status), p, n, _stream(stream)), "vmoba_select")
+
+
+def vmoba_attn_fwd(shape, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid, lse, dev_status,
+                   ws, stream=None):
+    p, n = _ws_args(ws)
+    _check(lib().vmoba_attn_fwd(ctypes.byref(shape), _ptr(q_bm), _ptr(k_bm), _ptr(v_bm), _ptr(kb_ptr), _ptr(q_idx),
+                                _ptr(q_ptr), _ptr(q_pairs), int(capacity), _ptr(o_bm), _ptr(o_resid), _ptr(lse),
+                                _ptr(dev_status), p, n, _stream(stream)), "vmoba_attn_fwd")
+
+
+def vmoba_attn_bwd(shape, q_bm, k_bm, v_bm, o_bm, o_resid, lse, do_bm, kb_ptr, q_idx, q_ptr, capacity, dq_bm, dk_bm,
+                   dv_bm, dev_status, ws, stream=None):
+    p, n = _ws_args(ws)
+    _check(lib().vmoba_attn_bwd(ctypes.byref(shape), _ptr(q_bm), _ptr(k_bm), _ptr(v_bm), _ptr(o_bm), _ptr(o_resid),
+                                _ptr(lse),
+                                _ptr(do_bm), _ptr(kb_ptr), _ptr(q_idx), _ptr(q_ptr), int(capacity), _ptr(dq_bm),
+                                _ptr(dk_bm), _ptr(dv_bm), _ptr(dev_status), p, n, _stream(stream)), "vmoba_attn_bwd")
+
+
+def vmoba_full_attn(shape, q, k, v, o, lse, do=None, dq=None, dk=None, dv=None, dev_status=None, ws=None,
+                    stream=None):
+    p, n = _ws_args(ws)
+    _check(lib().vmoba_full_attn(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(do),
+                                 _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dev_status), p, n, _stream(stream)),
+           "vmoba_full_attn")

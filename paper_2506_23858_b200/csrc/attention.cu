@@ -1,0 +1,206 @@
+// Entry points of Step 3 of VMoBA (attention over the selected blocks), its training
+// backward and the dense tau = 1 path: argument checks, workspace carving and kernel dispatch.
+#include <algorithm>
+
+#include "attn_simt.cuh"
+#include "common.cuh"
+
+namespace vmoba {
+
+size_t select_ws_bytes(const Dims& D);   // select.cu
+
+struct FwdWs { int* item_ptr; float* part_o; float* part_lse; size_t bytes; };
+static FwdWs carve_fwd(const Dims& D, long long cap, void* ws) {
+  Carver c(ws);
+  FwdWs w;
+  w.item_ptr = c.take<int>((size_t)D.BH * D.Nb + 1);
+  w.part_lse = c.take<float>((size_t)cap);
+  w.part_o = c.take<float>((size_t)cap * D.d);
+  w.bytes = c.total();
+  return w;
+}
+
+struct BwdWs { int* item_ptr; float* Dv; float* dq_acc; void* o_resid; size_t bytes; };
+static BwdWs carve_bwd(const Dims& D, bool dense, void* ws) {
+  Carver c(ws);
+  BwdWs w;
+  w.item_ptr = c.take<int>((size_t)D.BH * D.Nb + 1);
+  w.Dv = c.take<float>((size_t)D.BH * D.S);
+  w.dq_acc = dense ? nullptr : c.take<float>((size_t)D.BH * D.S * D.d);
+  w.o_resid = (dense && D.dtype == VMOBA_BF16) ? c.take<__nv_bfloat16>((size_t)D.BH * D.S * D.d) : nullptr;
+  w.bytes = c.total();
+  return w;
+}
+
+static int grid_for(long long items, int per_sm) {
+  long long g = std::min<long long>(items, 148ll * per_sm);
+  return (int)std::max<long long>(g, 1);
+}
+
+template <typename T, int DH>
+static int simt_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr,
+                           const int* q_idx, const int* q_ptr, const int* q_pairs, long long cap, void* o,
+                           void* o_resid, float* lse, void* ws, cudaStream_t st) {
+  FwdWs w = carve_fwd(D, cap, ws);
+  const long long n_kb = (long long)D.BH * D.Nb;
+  simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, simt::kRows, cap, w.item_ptr);
+  long long max_items = cap / simt::kRows + n_kb;
+  simt::attn_fwd_kernel<T, DH, false><<<grid_for(max_items, 8), simt::kThreads, 0, st>>>(
+      (const T*)q, (const T*)k, (const T*)v, kb_ptr, q_idx, q_ptr, w.item_ptr, (int)n_kb, D.S, D.Nb, D.sb, D.BH,
+      D.scale, (T*)o, (T*)o_resid, lse, w.part_o, w.part_lse, cap);
+  long long nq = (long long)D.BH * D.S;
+  simt::merge_kernel<T, DH, float><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(
+      q_ptr, q_pairs, nq, w.part_o, w.part_lse, cap, (T*)o, (T*)o_resid, lse);
+  VMOBA_LAUNCH_OK();
+  return VMOBA_OK;
+}
+
+template <typename T, int DH>
+static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* o,
+                           const void* o_resid, const float* lse, const void* d_o, const int* kb_ptr, const int* q_idx, long long cap,
+                           void* dq, void* dk, void* dv, void* ws, cudaStream_t st) {
+  BwdWs w = carve_bwd(D, false, ws);
+  const long long n_kb = (long long)D.BH * D.Nb;
+  const long long nq = (long long)D.BH * D.S;
+  VMOBA_CUDA_OK(cudaMemsetAsync(w.dq_acc, 0, (size_t)nq * DH * sizeof(float), st));
+  simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>((const T*)o, (const T*)o_resid,
+                                                                        (const T*)d_o, nq, w.Dv);
+  simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, simt::kRows, cap, w.item_ptr);
+  long long tiles = (D.sb + simt::kRows - 1) / simt::kRows;
+  simt::attn_bwd_dkdv_kernel<T, DH, false><<<grid_for(n_kb * tiles, 4), simt::kThreads, 0, st>>>(
+      (const T*)q, (const T*)k, (const T*)v, (const T*)d_o, lse, w.Dv, kb_ptr, q_idx, D.S, D.Nb, D.sb, D.BH,
+      D.scale, cap, (T*)dk, (T*)dv);
+  simt::attn_bwd_dq_kernel<T, DH, false><<<grid_for(nq / simt::kRows * D.Nb + n_kb, 4), simt::kThreads, 0, st>>>(
+      (const T*)q, (const T*)k, (const T*)v, (const T*)d_o, lse, w.Dv, kb_ptr, q_idx, w.item_ptr, (int)n_kb, D.S,
+      D.Nb, D.sb, D.BH, D.scale, cap, w.dq_acc, (T*)dq);
+  simt::cast_kernel<T><<<grid_for((nq * DH / 4 + 255) / 256, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, nq * DH / 4);
+  VMOBA_LAUNCH_OK();
+  return VMOBA_OK;
+}
+
+template <typename T, int DH>
+static int simt_dense(const Dims& D, const void* q, const void* k, const void* v, void* o, float* lse,
+                      const void* d_o, void* dq, void* dk, void* dv, void* ws, cudaStream_t st) {
+  const long long nq = (long long)D.BH * D.S;
+  const long long tiles = (D.S + simt::kRows - 1) / simt::kRows;
+  BwdWs w = carve_bwd(D, true, d_o ? ws : nullptr);
+  simt::attn_fwd_kernel<T, DH, true><<<grid_for(D.BH * tiles, 8), simt::kThreads, 0, st>>>(
+      (const T*)q, (const T*)k, (const T*)v, nullptr, nullptr, nullptr, nullptr, 0, D.S, 1, D.S, D.BH, D.scale,
+      (T*)o, d_o ? (T*)w.o_resid : nullptr, lse, nullptr, nullptr, 0);
+  if (d_o) {
+    simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>((const T*)o, (const T*)w.o_resid,
+                                                                          (const T*)d_o, nq, w.Dv);
+    simt::attn_bwd_dkdv_kernel<T, DH, true><<<grid_for(D.BH * tiles, 4), simt::kThreads, 0, st>>>(
+        (const T*)q, (const T*)k, (const T*)v, (const T*)d_o, lse, w.Dv, nullptr, nullptr, D.S, 1, D.S, D.BH,
+        D.scale, 0, (T*)dk, (T*)dv);
+    simt::attn_bwd_dq_kernel<T, DH, true><<<grid_for(D.BH * tiles, 4), simt::kThreads, 0, st>>>(
+        (const T*)q, (const T*)k, (const T*)v, (const T*)d_o, lse, w.Dv, nullptr, nullptr, nullptr, 0, D.S, 1, D.S,
+        D.BH, D.scale, 0, nullptr, (T*)dq);
+  }
+  VMOBA_LAUNCH_OK();
+  return VMOBA_OK;
+}
+
+#define VMOBA_DISPATCH(FN, ...)                                                        \
+  do {                                                                                 \
+    if (D.dtype == VMOBA_BF16) {                                                       \
+      if (D.d == 128) return FN<__nv_bfloat16, 128>(__VA_ARGS__);                      \
+      return FN<__nv_bfloat16, 64>(__VA_ARGS__);                                       \
+    }                                                                                  \
+    if (D.d == 128) return FN<float, 128>(__VA_ARGS__);                                \
+    return FN<float, 64>(__VA_ARGS__);                                                 \
+  } while (0)
+
+}  // namespace vmoba
+
+using namespace vmoba;
+
+extern "C" const char* vmoba_status_string(int status) {
+  switch (status) {
+    case VMOBA_OK: return "ok";
+    case VMOBA_ERR_ARG: return "invalid argument";
+    case VMOBA_ERR_SHAPE: return "invalid shape";
+    case VMOBA_ERR_WORKSPACE: return "workspace too small";
+    case VMOBA_ERR_CAPACITY: return "work-list capacity exceeded";
+    case VMOBA_ERR_TIMEOUT: return "device-side wait timed out";
+    case VMOBA_ERR_CUDA: return "CUDA error";
+    case VMOBA_ERR_NOT_IMPLEMENTED: return "not implemented";
+    default: return "unknown status";
+  }
+}
+
+extern "C" size_t vmoba_workspace_bytes(const vmoba_shape* shape, int stage, int64_t capacity) {
+  Dims D;
+  if (make_dims(shape, &D)) return 0;
+  if (capacity < 0) return 0;
+  switch (stage) {
+    case VMOBA_STAGE_SCORES: return 256;
+    case VMOBA_STAGE_SELECT: return select_ws_bytes(D);
+    case VMOBA_STAGE_ATTN_FWD: return carve_fwd(D, capacity, nullptr).bytes;
+    case VMOBA_STAGE_ATTN_BWD: return carve_bwd(D, false, nullptr).bytes;
+    case VMOBA_STAGE_FULL_FWD: return 256;
+    case VMOBA_STAGE_FULL_BWD: return carve_bwd(D, true, nullptr).bytes;
+    default: return 0;
+  }
+}
+
+extern "C" int vmoba_attn_fwd(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
+                              const int32_t* kb_ptr, const int32_t* q_idx, const int32_t* q_ptr,
+                              const int32_t* q_pairs, int64_t capacity, void* o_bm, void* o_resid_or_null,
+                              float* lse, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  Dims D;
+  int rc = make_dims(shape, &D);
+  if (rc) return rc;
+  if (!q_bm || !k_bm || !v_bm || !kb_ptr || !q_idx || !q_ptr || !q_pairs || !o_bm || !lse || !dev_status || !ws)
+    return VMOBA_ERR_ARG;
+  if (!aligned16(q_bm) || !aligned16(k_bm) || !aligned16(v_bm) || !aligned16(o_bm) || !aligned16(ws) ||
+      !aligned16(o_resid_or_null))
+    return VMOBA_ERR_ARG;
+  if (capacity <= 0 || capacity > (int64_t)INT32_MAX) return VMOBA_ERR_ARG;
+  if (ws_bytes < carve_fwd(D, capacity, nullptr).bytes) return VMOBA_ERR_WORKSPACE;
+  if (D.dtype != VMOBA_BF16) o_resid_or_null = nullptr;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  VMOBA_DISPATCH(simt_sparse_fwd, D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null,
+                 lse, ws, st);
+}
+
+extern "C" int vmoba_attn_bwd(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
+                              const void* o_bm, const void* o_resid_or_null, const float* lse, const void* do_bm,
+                              const int32_t* kb_ptr,
+                              const int32_t* q_idx, const int32_t* q_ptr, int64_t capacity, void* dq_bm, void* dk_bm,
+                              void* dv_bm, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  Dims D;
+  int rc = make_dims(shape, &D);
+  if (rc) return rc;
+  if (!q_bm || !k_bm || !v_bm || !o_bm || !lse || !do_bm || !kb_ptr || !q_idx || !q_ptr || !dq_bm || !dk_bm ||
+      !dv_bm || !dev_status || !ws)
+    return VMOBA_ERR_ARG;
+  if (!aligned16(q_bm) || !aligned16(k_bm) || !aligned16(v_bm) || !aligned16(o_bm) || !aligned16(do_bm) ||
+      !aligned16(dq_bm) || !aligned16(dk_bm) || !aligned16(dv_bm) || !aligned16(ws))
+    return VMOBA_ERR_ARG;
+  if (capacity <= 0 || capacity > (int64_t)INT32_MAX) return VMOBA_ERR_ARG;
+  if (ws_bytes < carve_bwd(D, false, nullptr).bytes) return VMOBA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (D.dtype != VMOBA_BF16) o_resid_or_null = nullptr;
+  if (!aligned16(o_resid_or_null)) return VMOBA_ERR_ARG;
+  VMOBA_DISPATCH(simt_sparse_bwd, D, q_bm, k_bm, v_bm, o_bm, o_resid_or_null, lse, do_bm, kb_ptr, q_idx, capacity, dq_bm, dk_bm, dv_bm,
+                 ws, st);
+}
+
+extern "C" int vmoba_full_attn(const vmoba_shape* shape, const void* q, const void* k, const void* v, void* o,
+                               float* lse, const void* do_or_null, void* dq, void* dk, void* dv,
+                               int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  Dims D;
+  int rc = make_dims(shape, &D);
+  if (rc) return rc;
+  if (!q || !k || !v || !o || !lse || !dev_status) return VMOBA_ERR_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return VMOBA_ERR_ARG;
+  if (do_or_null) {
+    if (!dq || !dk || !dv || !ws) return VMOBA_ERR_ARG;
+    if (!aligned16(do_or_null) || !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
+      return VMOBA_ERR_ARG;
+    if (ws_bytes < carve_bwd(D, true, nullptr).bytes) return VMOBA_ERR_WORKSPACE;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  VMOBA_DISPATCH(simt_dense, D, q, k, v, o, lse, do_or_null, dq, dk, dv, ws, st);
+}

@@ -1,0 +1,140 @@
+// Step 1b + Step 2a of VMoBA: mean key-block centroids (Eq. 2) and the query x centroid
+// similarity map S_hat = q b^T (Section 3.3), both in fp32.
+//
+// Both kernels are bound by HBM traffic: K is read once for the centroids, Q once for the
+// scores, and the [S, N_b] fp32 score matrix is written once.  The contraction itself
+// (2 * S * N_b * d flops) is small next to that and runs on the fp32 FMA pipe so that the
+// scores carry fp32 accuracy (the selection cutoff is compared in fp32).
+#include "common.cuh"
+
+namespace vmoba {
+
+// One CTA per (batch, head, block): 256 threads = (256 / V) row lanes x V float4-column lanes.
+template <typename T, int DH>
+__global__ void __launch_bounds__(256)
+centroid_kernel(const T* __restrict__ k_bm, float* __restrict__ cent, int sb) {
+  constexpr int V = DH / 4;            // float4 columns per row
+  constexpr int RL = 256 / V;          // row lanes
+  __shared__ float4 red[RL][V];
+  const long long blk = blockIdx.x;    // (b*heads + head) * Nb + j : blocks are contiguous in block-major order
+  const T* base = k_bm + blk * (long long)sb * DH;
+  const int col = threadIdx.x % V, rl = threadIdx.x / V;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int r = rl; r < sb; r += RL) {
+    float4 x = load4(base + (long long)r * DH + col * 4);
+    acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+  }
+  red[rl][col] = acc;
+  __syncthreads();
+  if (rl == 0) {
+    float4 s = red[0][col];
+    for (int i = 1; i < RL; ++i) {
+      float4 x = red[i][col];
+      s.x += x.x; s.y += x.y; s.z += x.z; s.w += x.w;
+    }
+    float inv = 1.0f / (float)sb;
+    s.x *= inv; s.y *= inv; s.z *= inv; s.w *= inv;
+    store4(cent + blk * DH + col * 4, s);
+  }
+}
+
+// fp32 tile GEMM: a CTA computes 64 queries x 64 blocks with the whole head_dim in shared
+// memory (operands stored transposed so that each thread reads its 4x4 micro-tile as float4).
+template <typename T, int DH>
+__global__ void __launch_bounds__(256)
+scores_kernel(const T* __restrict__ q_bm, const float* __restrict__ cent, float* __restrict__ scores,
+              int S, int Nb) {
+  extern __shared__ float smem[];
+  constexpr int LD = 64 + 4;
+  float* qT = smem;                 // [DH][LD]
+  float* bT = smem + DH * LD;       // [DH][LD]
+  const int bh = blockIdx.z;
+  const int q0 = blockIdx.x * 64;
+  const int tid = threadIdx.x;
+  const T* qh = q_bm + ((long long)bh * S + q0) * DH;
+  // Load the query tile once: thread t reads float4 #(t % (DH/4)) of row (t / (DH/4)) + k * rows_per_pass.
+  constexpr int V = DH / 4;
+  for (int i = tid; i < 64 * V; i += 256) {
+    int r = i / V, c4 = i % V;
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (q0 + r < S) x = load4(qh + (long long)r * DH + c4 * 4);
+    qT[(c4 * 4 + 0) * LD + r] = x.x;
+    qT[(c4 * 4 + 1) * LD + r] = x.y;
+    qT[(c4 * 4 + 2) * LD + r] = x.z;
+    qT[(c4 * 4 + 3) * LD + r] = x.w;
+  }
+  const int ty = tid / 16, tx = tid % 16;
+  const float* ch = cent + (long long)bh * Nb * DH;
+  float* out = scores + ((long long)bh * S + q0) * Nb;
+  for (int j0 = 0; j0 < Nb; j0 += 64) {
+    __syncthreads();
+    for (int i = tid; i < 64 * V; i += 256) {
+      int r = i / V, c4 = i % V;
+      float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (j0 + r < Nb) x = *reinterpret_cast<const float4*>(ch + (long long)(j0 + r) * DH + c4 * 4);
+      bT[(c4 * 4 + 0) * LD + r] = x.x;
+      bT[(c4 * 4 + 1) * LD + r] = x.y;
+      bT[(c4 * 4 + 2) * LD + r] = x.z;
+      bT[(c4 * 4 + 3) * LD + r] = x.w;
+    }
+    __syncthreads();
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 8
+    for (int c = 0; c < DH; ++c) {
+      float4 a = *reinterpret_cast<const float4*>(qT + c * LD + ty * 4);
+      float4 b = *reinterpret_cast<const float4*>(bT + c * LD + tx * 4);
+      float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      int r = ty * 4 + i;
+      if (q0 + r >= S) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        int col = j0 + tx * 4 + j;
+        if (col < Nb) out[(long long)r * Nb + col] = acc[i][j];
+      }
+    }
+  }
+}
+
+template <typename T, int DH>
+static int run_scores(const Dims& D, const void* q, const void* k, float* cent, float* scores, cudaStream_t st) {
+  centroid_kernel<T, DH><<<D.BH * D.Nb, 256, 0, st>>>(static_cast<const T*>(k), cent, D.sb);
+  VMOBA_LAUNCH_OK();
+  size_t smem = 2 * DH * (64 + 4) * sizeof(float);
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(scores_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  dim3 grid((D.S + 63) / 64, 1, D.BH);
+  scores_kernel<T, DH><<<grid, 256, smem, st>>>(static_cast<const T*>(q), cent, scores, D.S, D.Nb);
+  VMOBA_LAUNCH_OK();
+  return VMOBA_OK;
+}
+
+}  // namespace vmoba
+
+using namespace vmoba;
+
+extern "C" int vmoba_block_scores(const vmoba_shape* shape, const void* q_bm, const void* k_bm,
+                                  float* centroids, float* scores, void* ws, size_t ws_bytes, void* stream) {
+  (void)ws; (void)ws_bytes;
+  Dims D;
+  int rc = make_dims(shape, &D);
+  if (rc) return rc;
+  if (!q_bm || !k_bm || !centroids || !scores) return VMOBA_ERR_ARG;
+  if (!aligned16(q_bm) || !aligned16(k_bm) || !aligned16(centroids) || !aligned16(scores)) return VMOBA_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (D.dtype == VMOBA_BF16) {
+    if (D.d == 128) return run_scores<__nv_bfloat16, 128>(D, q_bm, k_bm, centroids, scores, st);
+    return run_scores<__nv_bfloat16, 64>(D, q_bm, k_bm, centroids, scores, st);
+  }
+  if (D.d == 128) return run_scores<float, 128>(D, q_bm, k_bm, centroids, scores, st);
+  return run_scores<float, 64>(D, q_bm, k_bm, centroids, scores, st);
+}

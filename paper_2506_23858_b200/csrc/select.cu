@@ -1,0 +1,499 @@
+// Step 2b of VMoBA: global (per head) threshold selection of (query, key-block) pairs
+// (Eq. 3 TopkMask, Eq. 4 threshold k), and emission of the work lists the attention
+// kernels consume.
+//
+// Sorting the head's pool and accumulating normalised similarity until tau is reached is
+// equivalent to finding the weighted quantile of the scores under the softmax weights:
+// the cutoff is the largest score c with mass{score >= c} >= tau * Z.  That is found without
+// a sort by three histogram refinements (2048 bins each, linear in the score, fp64 bin
+// masses), after which the mask is one comparison per pair.  Every kernel streams the score
+// matrix with 16-byte loads; the stage is bound by HBM bandwidth.
+//
+//   minmax  -> hist level 0 -> scan -> hist level 1 -> scan -> hist level 2 -> scan (cutoff)
+//   mark    : mask bits + per (segment, block) counts + per-segment pair totals
+//   offsets : CSR offsets by key block (kb_ptr) and by query (q_ptr)
+//   fill    : q_idx (queries of each key block, ascending) and q_pairs (pairs of each query)
+#include <algorithm>
+
+#include "common.cuh"
+
+namespace vmoba {
+
+constexpr int kBins = 2048;
+constexpr int kSegThreads = 512;
+
+struct HeadState {
+  uint32_t min_key, max_key;   // order-preserving keys of the head's extreme scores
+  float anchor[3];             // lower edge of the interval refined at each level
+  float inv[3];                // bins per unit score at each level
+  int bin[3];                  // crossing bin found at each level
+  int level_ok;
+  double Z;                    // sum of all weights
+  double target;               // tau * Z
+  double mass_above;           // weight of everything above the crossing bin so far
+  unsigned long long cnt_above;
+  uint32_t cutoff_key;
+  uint32_t pad;
+};
+
+// bin of a score at refinement level L given the state; monotone non-decreasing in s.
+__device__ __forceinline__ int bin_at(const HeadState& hs, int L, float s) {
+  float t = (s - hs.anchor[L]) * hs.inv[L];
+  int b = t > 0.f ? (int)fminf(t, (float)(kBins - 1)) : 0;
+  return b;
+}
+
+// Streams the P scores of one head through f(value); blockIdx.x strides over chunks.
+template <typename F>
+__device__ __forceinline__ void for_each_score(const float* __restrict__ base, long long P, F f) {
+  const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long nth = (long long)gridDim.x * blockDim.x;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) == 0) {
+    long long P4 = P >> 2;
+    const float4* b4 = reinterpret_cast<const float4*>(base);
+    for (long long i = tid; i < P4; i += nth) {
+      float4 x = __ldg(b4 + i);
+      f(x.x); f(x.y); f(x.z); f(x.w);
+    }
+    for (long long i = (P4 << 2) + tid; i < P; i += nth) f(__ldg(base + i));
+  } else {
+    for (long long i = tid; i < P; i += nth) f(__ldg(base + i));
+  }
+}
+
+__global__ void __launch_bounds__(256)
+minmax_kernel(const float* __restrict__ scores, long long P, HeadState* __restrict__ st) {
+  const int bh = blockIdx.y;
+  uint32_t kmin = 0xffffffffu, kmax = 0u;
+  for_each_score(scores + (long long)bh * P, P, [&](float s) {
+    uint32_t k = float_key(s);
+    kmin = min(kmin, k);
+    kmax = max(kmax, k);
+  });
+  kmin = __reduce_min_sync(0xffffffffu, kmin);
+  kmax = __reduce_max_sync(0xffffffffu, kmax);
+  if ((threadIdx.x & 31) == 0) {
+    atomicMin(&st[bh].min_key, kmin);
+    atomicMax(&st[bh].max_key, kmax);
+  }
+}
+
+__global__ void init_state_kernel(HeadState* st, int BH) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= BH) return;
+  HeadState h;
+  memset(&h, 0, sizeof(h));
+  h.min_key = 0xffffffffu;
+  h.max_key = 0u;
+  st[i] = h;
+}
+
+// Level L histogram: pairs that fall in the crossing bins of all earlier levels add
+// (1, exp(sigma * (s - max))) to their level-L bin.  At the last level the smallest key of
+// each bin is tracked too, which turns the crossing bin into an exact fp32 cutoff.
+template <int L>
+__global__ void __launch_bounds__(256)
+hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __restrict__ st, float sigma,
+            unsigned int* __restrict__ g_cnt, double* __restrict__ g_w, uint32_t* __restrict__ g_minkey) {
+  __shared__ unsigned int s_cnt[kBins];
+  __shared__ float s_w[kBins];
+  __shared__ uint32_t s_min[L == 2 ? kBins : 1];
+  const int bh = blockIdx.y;
+  const HeadState hs = st[bh];
+  for (int i = threadIdx.x; i < kBins; i += blockDim.x) {
+    s_cnt[i] = 0; s_w[i] = 0.f;
+    if (L == 2) s_min[i] = 0xffffffffu;
+  }
+  __syncthreads();
+  const float smax = key_float(hs.max_key);
+  for_each_score(scores + (long long)bh * P, P, [&](float s) {
+    if (L >= 1 && bin_at(hs, 0, s) != hs.bin[0]) return;
+    if (L >= 2 && bin_at(hs, 1, s) != hs.bin[1]) return;
+    int b = bin_at(hs, L, s);
+    atomicAdd(&s_cnt[b], 1u);
+    atomicAdd(&s_w[b], expf(sigma * (s - smax)));
+    if (L == 2) atomicMin(&s_min[b], float_key(s));
+  });
+  __syncthreads();
+  for (int i = threadIdx.x; i < kBins; i += blockDim.x) {
+    unsigned int c = s_cnt[i];
+    if (c) {
+      atomicAdd(&g_cnt[(long long)bh * kBins + i], c);
+      atomicAdd(&g_w[(long long)bh * kBins + i], (double)s_w[i]);
+      if (L == 2) atomicMin(&g_minkey[(long long)bh * kBins + i], s_min[i]);
+    }
+  }
+}
+
+// One CTA (1024 threads, two bins each) per head: walk the bins from the top, find the bin in
+// which the cumulative mass first reaches the target, record it and clear the histogram.
+template <int L>
+__global__ void __launch_bounds__(1024)
+scan_kernel(HeadState* __restrict__ st, float tau, unsigned int* __restrict__ g_cnt, double* __restrict__ g_w,
+            uint32_t* __restrict__ g_minkey, int64_t* __restrict__ k_per_head, float* __restrict__ cutoff_per_head) {
+  __shared__ double s_wsum[32];
+  __shared__ unsigned long long s_csum[32];
+  __shared__ int s_cross;
+  __shared__ int s_lowest;
+  __shared__ uint32_t s_minkey;
+  const int bh = blockIdx.x;
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  HeadState hs = st[bh];
+  // element e = 0..2047 walks bins from the top: bin = 2047 - e; thread t owns e = 2t, 2t+1
+  const long long hb = (long long)bh * kBins;
+  double w0 = g_w[hb + (kBins - 1 - 2 * t)], w1 = g_w[hb + (kBins - 2 - 2 * t)];
+  unsigned long long c0 = g_cnt[hb + (kBins - 1 - 2 * t)], c1 = g_cnt[hb + (kBins - 2 - 2 * t)];
+  uint32_t mk0 = 0xffffffffu, mk1 = 0xffffffffu;
+  if (L == 2) { mk0 = g_minkey[hb + (kBins - 1 - 2 * t)]; mk1 = g_minkey[hb + (kBins - 2 - 2 * t)]; }
+  // clear for the next level / next call
+  g_w[hb + (kBins - 1 - 2 * t)] = 0.0; g_w[hb + (kBins - 2 - 2 * t)] = 0.0;
+  g_cnt[hb + (kBins - 1 - 2 * t)] = 0u; g_cnt[hb + (kBins - 2 - 2 * t)] = 0u;
+  if (L == 2) { g_minkey[hb + (kBins - 1 - 2 * t)] = 0xffffffffu; g_minkey[hb + (kBins - 2 - 2 * t)] = 0xffffffffu; }
+  double wl = w0 + w1;
+  unsigned long long cl = c0 + c1;
+  // inclusive warp scan
+  double wi = wl; unsigned long long ci = cl;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    double wv = __shfl_up_sync(0xffffffffu, wi, o);
+    unsigned long long cv = __shfl_up_sync(0xffffffffu, ci, o);
+    if (lane >= o) { wi += wv; ci += cv; }
+  }
+  if (lane == 31) { s_wsum[warp] = wi; s_csum[warp] = ci; }
+  if (t == 0) { s_cross = -1; s_lowest = -1; s_minkey = 0xffffffffu; }
+  __syncthreads();
+  if (warp == 0) {
+    double wv = s_wsum[lane]; unsigned long long cv = s_csum[lane];
+    double wi2 = wv; unsigned long long ci2 = cv;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      double a = __shfl_up_sync(0xffffffffu, wi2, o);
+      unsigned long long b = __shfl_up_sync(0xffffffffu, ci2, o);
+      if (lane >= o) { wi2 += a; ci2 += b; }
+    }
+    s_wsum[lane] = wi2 - wv;    // exclusive
+    s_csum[lane] = ci2 - cv;
+  }
+  __syncthreads();
+  const double w_excl = s_wsum[warp] + (wi - wl);            // mass of all elements before e = 2t
+  const unsigned long long c_excl = s_csum[warp] + (ci - cl);
+  __shared__ double s_total;
+  if (t == 1023) s_total = w_excl + wl;
+  __syncthreads();
+  if (L == 0) { hs.Z = s_total; hs.target = (double)tau * s_total; hs.mass_above = 0.0; hs.cnt_above = 0ull; }
+  const double need = hs.target - hs.mass_above;    // mass still to be covered inside this level
+  // crossing element: first e with inclusive mass >= need (and a non-empty bin)
+  int my_cross = -1;
+  if (c0 && w_excl < need && w_excl + w0 >= need) my_cross = 2 * t;
+  else if (c1 && w_excl + w0 < need && w_excl + w0 + w1 >= need) my_cross = 2 * t + 1;
+  if (my_cross >= 0) atomicMax(&s_cross, kBins - 1 - my_cross);      // as a bin index
+  // lowest non-empty bin = fallback when rounding keeps the sum below `need`
+  if (c1) atomicMax(&s_lowest, 2 * t + 1);
+  else if (c0) atomicMax(&s_lowest, 2 * t);
+  __syncthreads();
+  int cross_bin = s_cross;
+  if (cross_bin < 0) cross_bin = s_lowest >= 0 ? kBins - 1 - s_lowest : 0;
+  // mass / count strictly above the crossing bin
+  const int e_cross = kBins - 1 - cross_bin;
+  __shared__ double s_above_w;
+  __shared__ unsigned long long s_above_c;
+  if (2 * t == e_cross) { s_above_w = w_excl; s_above_c = c_excl; }
+  if (2 * t + 1 == e_cross) { s_above_w = w_excl + w0; s_above_c = c_excl + c0; }
+  if (L == 2) {
+    // exact cutoff: smallest key among the bins at or above the crossing bin
+    uint32_t mk = 0xffffffffu;
+    if (2 * t <= e_cross) mk = min(mk, mk0);
+    if (2 * t + 1 <= e_cross) mk = min(mk, mk1);
+    mk = __reduce_min_sync(0xffffffffu, mk);
+    if (lane == 0) atomicMin(&s_minkey, mk);
+  }
+  __syncthreads();
+  if (t == 0) {
+    hs.bin[L] = cross_bin;
+    hs.mass_above += s_above_w;
+    hs.cnt_above += s_above_c;
+    if (L < 2) {
+      hs.anchor[L + 1] = hs.inv[L] > 0.f ? hs.anchor[L] + (float)cross_bin / hs.inv[L] : hs.anchor[L];
+      hs.inv[L + 1] = fminf(hs.inv[L] * (float)kBins, 1e30f);
+    } else {
+      hs.cutoff_key = s_minkey;
+      if (tau >= 1.0f) hs.cutoff_key = hs.min_key;
+      cutoff_per_head[bh] = key_float(hs.cutoff_key);
+    }
+    st[bh] = hs;
+  }
+}
+
+// After minmax: level-0 anchors.
+__global__ void setup_level0_kernel(HeadState* st, int BH) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= BH) return;
+  float lo = key_float(st[i].min_key), hi = key_float(st[i].max_key);
+  float range = hi - lo;
+  st[i].anchor[0] = lo;
+  st[i].inv[0] = range > 0.f ? (float)kBins / range : 0.f;
+}
+
+// mark: a CTA takes a segment of QSEG consecutive queries of one head (a contiguous run of
+// QSEG * Nb scores), sets the mask bits in shared memory, counts selections per key block,
+// then writes mask words, per-(segment, block) counts and the segment's pair total.
+__global__ void __launch_bounds__(kSegThreads)
+mark_kernel(const float* __restrict__ scores, const HeadState* __restrict__ st, int S, int Nb, int mw, int QSEG,
+            int nseg, uint32_t* __restrict__ mask_bits, int* __restrict__ seg_cnt, int* __restrict__ seg_total) {
+  extern __shared__ uint32_t sm[];
+  uint32_t* s_mask = sm;                              // [QSEG][mw]
+  int* s_cnt = reinterpret_cast<int*>(sm + QSEG * mw);  // [Nb]
+  __shared__ int s_total;
+  const int seg = blockIdx.x, bh = blockIdx.y;
+  const int q0 = seg * QSEG;
+  const int nq = min(QSEG, S - q0);
+  const uint32_t cutoff = st[bh].cutoff_key;
+  for (int i = threadIdx.x; i < QSEG * mw; i += blockDim.x) s_mask[i] = 0u;
+  for (int i = threadIdx.x; i < Nb; i += blockDim.x) s_cnt[i] = 0;
+  if (threadIdx.x == 0) s_total = 0;
+  __syncthreads();
+  const float* base = scores + ((long long)bh * S + q0) * Nb;
+  const long long n = (long long)nq * Nb;
+  auto mark = [&](long long i, float s) {
+    if (float_key(s) >= cutoff) {
+      int ii = (int)i;
+      int ql = ii / Nb, j = ii - ql * Nb;
+      atomicOr(&s_mask[ql * mw + (j >> 5)], 1u << (j & 31));
+      atomicAdd(&s_cnt[j], 1);
+    }
+  };
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) == 0) {
+    const float4* b4 = reinterpret_cast<const float4*>(base);
+    long long n4 = n >> 2;
+    for (long long i = threadIdx.x; i < n4; i += blockDim.x) {
+      float4 x = __ldg(b4 + i);
+      mark(4 * i, x.x); mark(4 * i + 1, x.y); mark(4 * i + 2, x.z); mark(4 * i + 3, x.w);
+    }
+    for (long long i = (n4 << 2) + threadIdx.x; i < n; i += blockDim.x) mark(i, __ldg(base + i));
+  } else {
+    for (long long i = threadIdx.x; i < n; i += blockDim.x) mark(i, __ldg(base + i));
+  }
+  __syncthreads();
+  uint32_t* gm = mask_bits + ((long long)bh * S + q0) * mw;
+  int local = 0;
+  for (int i = threadIdx.x; i < nq * mw; i += blockDim.x) {
+    uint32_t wv = s_mask[i];
+    gm[i] = wv;
+    local += __popc(wv);
+  }
+  local = __reduce_add_sync(0xffffffffu, local);
+  if ((threadIdx.x & 31) == 0 && local) atomicAdd(&s_total, local);
+  int* sc = seg_cnt + ((long long)bh * nseg + seg) * Nb;
+  for (int i = threadIdx.x; i < Nb; i += blockDim.x) sc[i] = s_cnt[i];
+  __syncthreads();
+  if (threadIdx.x == 0) seg_total[bh * nseg + seg] = s_total;
+}
+
+// offsets A: per (head, block) turn the per-segment counts into exclusive prefixes along the
+// segments and record the block's total.
+__global__ void seg_prefix_kernel(int* __restrict__ seg_cnt, int* __restrict__ kb_total, int BH, int Nb, int nseg) {
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long long)BH * Nb) return;
+  int bh = (int)(i / Nb), j = (int)(i % Nb);
+  int run = 0;
+  for (int s = 0; s < nseg; ++s) {
+    int* p = seg_cnt + ((long long)bh * nseg + s) * Nb + j;
+    int c = *p;
+    *p = run;
+    run += c;
+  }
+  kb_total[i] = run;
+}
+
+__global__ void __launch_bounds__(1024)
+offsets_kernel(const int* __restrict__ kb_total, int* __restrict__ kb_ptr, long long n_kb,
+               const int* __restrict__ seg_total, int* __restrict__ seg_qoff, long long n_seg,
+               int BH, int Nb, int64_t* __restrict__ k_per_head, long long capacity,
+               int* __restrict__ q_ptr_last, int32_t* __restrict__ dev_status) {
+  __shared__ long long total_a, total_b;
+  block_exclusive_scan([&](long long i) { return kb_total[i]; }, kb_ptr, n_kb, &total_a);
+  block_exclusive_scan([&](long long i) { return seg_total[i]; }, seg_qoff, n_seg, &total_b);
+  __syncthreads();
+  for (int bh = threadIdx.x; bh < BH; bh += blockDim.x) {
+    long long a = 0;
+    for (int j = 0; j < Nb; ++j) a += kb_total[(long long)bh * Nb + j];
+    k_per_head[bh] = a;
+  }
+  if (threadIdx.x == 0) {
+    *q_ptr_last = (int)min(total_a, (long long)INT32_MAX);
+    if (total_a > capacity) set_status(dev_status, VMOBA_ERR_CAPACITY);
+  }
+}
+
+// fill: a CTA re-reads its segment's mask words, derives q_ptr for its queries and, one warp
+// per key block, ranks the selecting queries in ascending order to place them in q_idx; the
+// same position is recorded in the query-major list q_pairs.
+__global__ void __launch_bounds__(kSegThreads)
+fill_kernel(const uint32_t* __restrict__ mask_bits, int S, int Nb, int mw, int QSEG, int nseg,
+            const int* __restrict__ kb_ptr, const int* __restrict__ seg_cnt, const int* __restrict__ seg_qoff,
+            int* __restrict__ q_idx, int* __restrict__ q_ptr, int* __restrict__ q_pairs, long long capacity) {
+  extern __shared__ uint32_t sm[];
+  uint32_t* s_mask = sm;                                   // [QSEG][mw]
+  int* s_qoff = reinterpret_cast<int*>(sm + QSEG * mw);    // [QSEG] exclusive pair offset inside the segment
+  __shared__ int s_warp[kSegThreads / 32];
+  const int seg = blockIdx.x, bh = blockIdx.y;
+  const int q0 = seg * QSEG;
+  const int nq = min(QSEG, S - q0);
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5, nwarps = blockDim.x >> 5;
+  const uint32_t* gm = mask_bits + ((long long)bh * S + q0) * mw;
+  for (int i = t; i < QSEG * mw; i += blockDim.x) s_mask[i] = i < nq * mw ? gm[i] : 0u;
+  __syncthreads();
+  const int qbase = seg_qoff[bh * nseg + seg];
+  // exclusive scan of per-query pair counts (QSEG <= blockDim.x)
+  int cnt = 0;
+  if (t < nq)
+    for (int w = 0; w < mw; ++w) cnt += __popc(s_mask[t * mw + w]);
+  int inc = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int x = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += x;
+  }
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int x = lane < nwarps ? s_warp[lane] : 0;
+    int xi = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, xi, o);
+      if (lane >= o) xi += y;
+    }
+    if (lane < nwarps) s_warp[lane] = xi - x;
+  }
+  __syncthreads();
+  if (t < QSEG) {
+    int excl = s_warp[warp] + inc - cnt;
+    s_qoff[t] = excl;
+    if (t < nq) q_ptr[(long long)bh * S + q0 + t] = (int)min((long long)qbase + excl, (long long)INT32_MAX);
+  }
+  __syncthreads();
+  const int* sc = seg_cnt + ((long long)bh * nseg + seg) * Nb;
+  for (int j = warp; j < Nb; j += nwarps) {
+    long long base = (long long)kb_ptr[(long long)bh * Nb + j] + sc[j];
+    const int wj = j >> 5;
+    const uint32_t bit = 1u << (j & 31);
+    int run = 0;
+    for (int qs = 0; qs < nq; qs += 32) {
+      int ql = qs + lane;
+      uint32_t word = ql < nq ? s_mask[ql * mw + wj] : 0u;
+      bool sel = (word & bit) != 0;
+      unsigned ball = __ballot_sync(0xffffffffu, sel);
+      if (sel) {
+        long long pos = base + run + __popc(ball & ((1u << lane) - 1u));
+        if (pos < capacity) {
+          q_idx[pos] = q0 + ql;
+          int within = __popc(word & (bit - 1u));
+          for (int w = 0; w < wj; ++w) within += __popc(s_mask[ql * mw + w]);
+          long long qp = (long long)qbase + s_qoff[ql] + within;
+          if (qp < capacity) q_pairs[qp] = (int)pos;
+        }
+      }
+      run += __popc(ball);
+    }
+  }
+}
+
+static int seg_queries(int mw) {
+  int q = 4096 / mw;            // keep the shared mask tile <= 16 KB
+  q = q / 32 * 32;
+  if (q > kSegThreads) q = kSegThreads;
+  if (q < 32) q = 32;
+  return q;
+}
+
+struct SelectWs {
+  HeadState* state;
+  unsigned int* g_cnt;
+  double* g_w;
+  uint32_t* g_minkey;
+  int* seg_cnt;
+  int* seg_total;
+  int* seg_qoff;
+  int* kb_total;
+  size_t bytes;
+};
+
+static SelectWs carve_select(const Dims& D, void* ws) {
+  SelectWs w;
+  Carver c(ws);
+  int QSEG = seg_queries(D.mask_words);
+  long long nseg = (D.S + QSEG - 1) / QSEG;
+  w.state = c.take<HeadState>(D.BH);
+  w.g_cnt = c.take<unsigned int>((size_t)D.BH * kBins);
+  w.g_w = c.take<double>((size_t)D.BH * kBins);
+  w.g_minkey = c.take<uint32_t>((size_t)D.BH * kBins);
+  w.seg_cnt = c.take<int>((size_t)D.BH * nseg * D.Nb);
+  w.seg_total = c.take<int>((size_t)D.BH * nseg);
+  w.seg_qoff = c.take<int>((size_t)D.BH * nseg + 1);
+  w.kb_total = c.take<int>((size_t)D.BH * D.Nb);
+  w.bytes = c.total();
+  return w;
+}
+
+size_t select_ws_bytes(const Dims& D) { return carve_select(D, nullptr).bytes; }
+
+}  // namespace vmoba
+
+using namespace vmoba;
+
+extern "C" int vmoba_select(const vmoba_shape* shape, const float* scores, float tau, uint32_t* mask_bits,
+                            int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr, int32_t* q_pairs,
+                            int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
+                            int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  Dims D;
+  int rc = make_dims(shape, &D);
+  if (rc) return rc;
+  if (!(tau > 0.0f) || tau > 1.0f) return VMOBA_ERR_ARG;
+  if (!scores || !mask_bits || !kb_ptr || !q_idx || !q_ptr || !q_pairs || !k_per_head || !cutoff_per_head ||
+      !dev_status || !ws)
+    return VMOBA_ERR_ARG;
+  if (!aligned16(scores) || !aligned16(ws)) return VMOBA_ERR_ARG;
+  if (capacity <= 0 || capacity > (int64_t)INT32_MAX) return VMOBA_ERR_ARG;
+  if (D.Nb > 8192) return VMOBA_ERR_SHAPE;
+  SelectWs w = carve_select(D, ws);
+  if (ws_bytes < w.bytes) return VMOBA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const long long P = (long long)D.S * D.Nb;
+  const int QSEG = seg_queries(D.mask_words);
+  const int nseg = (D.S + QSEG - 1) / QSEG;
+
+  init_state_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH);
+  VMOBA_CUDA_OK(cudaMemsetAsync(w.g_cnt, 0, (size_t)D.BH * kBins * sizeof(unsigned int), st));
+  VMOBA_CUDA_OK(cudaMemsetAsync(w.g_w, 0, (size_t)D.BH * kBins * sizeof(double), st));
+  VMOBA_CUDA_OK(cudaMemsetAsync(w.g_minkey, 0xff, (size_t)D.BH * kBins * sizeof(uint32_t), st));
+
+  // enough CTAs per head to fill the machine, few enough that the per-CTA flush stays small
+  long long per_head = (P / 4 + 255) / 256;
+  int gx = (int)std::min<long long>(std::max<long long>(per_head / 8, 1), std::max(1, 148 * 8 / D.BH));
+  dim3 grid(gx, D.BH);
+  minmax_kernel<<<grid, 256, 0, st>>>(scores, P, w.state);
+  setup_level0_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH);
+  hist_kernel<0><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey);
+  scan_kernel<0><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, k_per_head, cutoff_per_head);
+  hist_kernel<1><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey);
+  scan_kernel<1><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, k_per_head, cutoff_per_head);
+  hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey);
+  scan_kernel<2><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, k_per_head, cutoff_per_head);
+  VMOBA_LAUNCH_OK();
+
+  size_t smem = (size_t)QSEG * D.mask_words * 4 + (size_t)std::max(D.Nb, QSEG) * 4;
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(mark_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  dim3 sgrid(nseg, D.BH);
+  mark_kernel<<<sgrid, kSegThreads, smem, st>>>(scores, w.state, D.S, D.Nb, D.mask_words, QSEG, nseg, mask_bits,
+                                                w.seg_cnt, w.seg_total);
+  long long nkb = (long long)D.BH * D.Nb;
+  seg_prefix_kernel<<<(unsigned)((nkb + 255) / 256), 256, 0, st>>>(w.seg_cnt, w.kb_total, D.BH, D.Nb, nseg);
+  offsets_kernel<<<1, 1024, 0, st>>>(w.kb_total, kb_ptr, nkb, w.seg_total, w.seg_qoff, (long long)D.BH * nseg,
+                                     D.BH, D.Nb, k_per_head, capacity, q_ptr + (long long)D.BH * D.S, dev_status);
+  fill_kernel<<<sgrid, kSegThreads, smem, st>>>(mask_bits, D.S, D.Nb, D.mask_words, QSEG, nseg, kb_ptr, w.seg_cnt,
+                                                w.seg_qoff, q_idx, q_ptr, q_pairs, capacity);
+  VMOBA_LAUNCH_OK();
+  return VMOBA_OK;
+}

@@ -15,8 +15,8 @@ Two recipes:
 * ``smooth``: x = N(0,1) + f, where f is, per (batch, head), one white N(0,1)
               field of shape [T,H,W,head_dim] blurred along T, H and W (not along
               channels) with a separable Gaussian (sigma = 2 tokens, radius 8,
-              periodic wrap, taps normalised) and then rescaled to unit standard
-              deviation.  f is shared by q, k and v; the N(0,1) noise is independent.
+              periodic wrap, taps normalised; scipy.ndimage.correlate1d) and then
+              rescaled to unit standard deviation.  f is shared by q, k and v; the N(0,1) noise is independent.
 
 Draw order per (batch, head), from numpy's PCG64 ``default_rng(seed)`` spawned
 per (batch, head) so that any subset of heads can be generated alone:
@@ -89,15 +89,12 @@ def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
 def _gauss_taps(sigma: float, radius: int) -> np.ndarray:
     x = np.arange(-radius, radius + 1, dtype=np.float64)
     w = np.exp(-0.5 * (x / sigma) ** 2)
-    return (w / w.sum()).astype(np.float32)
+    return w / w.sum()
 
 
 def _blur_wrap(f: np.ndarray, axis: int, taps: np.ndarray) -> np.ndarray:
-    r = (len(taps) - 1) // 2
-    out = np.zeros_like(f)
-    for i, w in enumerate(taps):
-        out += w * np.roll(f, i - r, axis=axis)
-    return out
+    from scipy.ndimage import correlate1d
+    return correlate1d(f, taps, axis=axis, mode="wrap")
 
 
 def _unit_rng(seed: int, b: int, head: int) -> np.random.Generator:
@@ -142,13 +139,20 @@ def make_inputs(w: Workload, with_do: bool = True, heads=None):
     restricts generation to a list of head indices (the per-head streams are
     independent, so a subset reproduces the same values).
     """
+    from concurrent.futures import ThreadPoolExecutor
+    import os
     head_list = list(range(w.heads)) if heads is None else list(heads)
     names = ["q", "k", "v"] + (["do"] if with_do else [])
     arrs = {n: np.empty((w.B, w.S, len(head_list), w.head_dim), dtype=np.float32) for n in names}
-    for b in range(w.B):
-        for hi, head in enumerate(head_list):
-            for n, x in zip(names, make_head(w, b, head, with_do)):
-                arrs[n][b, :, hi, :] = x
+
+    def one(unit):
+        b, hi, head = unit
+        for n, x in zip(names, make_head(w, b, head, with_do)):
+            arrs[n][b, :, hi, :] = x
+
+    units = [(b, hi, head) for b in range(w.B) for hi, head in enumerate(head_list)]
+    with ThreadPoolExecutor(max_workers=min(len(units), os.cpu_count() or 1, 32)) as pool:
+        list(pool.map(one, units))
     out = {}
     for n in names:
         if w.dtype == "bf16":

@@ -1,0 +1,145 @@
+"""Buffer management and stage sequencing for one VMoBA attention layer on one GPU.
+
+Everything numerical happens inside the C-ABI library; this module only allocates torch
+tensors (device memory), passes their pointers to the entry points in order, and exposes the
+intermediate buffers so that tests can compare each stage with the oracle.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as vb
+
+
+def torch_dtype(shape):
+    return torch.bfloat16 if shape.dtype == vb.BF16 else torch.float32
+
+
+def default_capacity(shape, tau: float, slack: float = 0.02) -> int:
+    """Upper bound on the number of selected pairs: the threshold rule keeps at most ceil(tau*P)
+    pairs per head (the kept fraction never exceeds tau, Section 4.1), plus exact ties."""
+    P = shape.S * shape.n_blocks
+    per_head = int(min(P, tau * P * (1.0 + slack) + 1024))
+    return min(per_head * shape.B * shape.heads, 2 ** 31 - 1)
+
+
+class VmobaLayer:
+    """Owns the device buffers of one layer shape and runs the stages on the current stream."""
+
+    def __init__(self, shape, capacity: int, device="cuda", with_backward: bool = False):
+        self.shape = shape
+        self.capacity = int(capacity)
+        self.device = torch.device(device)
+        s = shape
+        dt = torch_dtype(s)
+        dev = self.device
+        BH, S, d, Nb = s.B * s.heads, s.S, s.head_dim, s.n_blocks
+        self.BH, self.S, self.d, self.Nb = BH, S, d, Nb
+        bm = lambda: torch.empty((s.B, s.heads, S, d), dtype=dt, device=dev)
+        self.q_bm, self.k_bm, self.v_bm, self.o_bm = bm(), bm(), bm(), bm()
+        self.centroids = torch.empty((s.B, s.heads, Nb, d), dtype=torch.float32, device=dev)
+        self.scores = torch.empty((s.B, s.heads, S, Nb), dtype=torch.float32, device=dev)
+        self.mask_bits = torch.empty((BH * S, s.mask_words), dtype=torch.int32, device=dev)
+        self.kb_ptr = torch.empty(BH * Nb + 1, dtype=torch.int32, device=dev)
+        self.q_idx = torch.empty(self.capacity, dtype=torch.int32, device=dev)
+        self.q_ptr = torch.empty(BH * S + 1, dtype=torch.int32, device=dev)
+        self.q_pairs = torch.empty(self.capacity, dtype=torch.int32, device=dev)
+        self.k_per_head = torch.empty(BH, dtype=torch.int64, device=dev)
+        self.cutoff = torch.empty(BH, dtype=torch.float32, device=dev)
+        self.lse = torch.empty(BH * S, dtype=torch.float32, device=dev)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
+        stages = [vb.STAGE_SCORES, vb.STAGE_SELECT, vb.STAGE_ATTN_FWD]
+        if with_backward:
+            stages.append(vb.STAGE_ATTN_BWD)
+            self.do_bm, self.dq_bm, self.dk_bm, self.dv_bm = bm(), bm(), bm(), bm()
+        # rounding residual of o, kept for the backward's rowsum(dO * O) (bf16 training only)
+        self.o_resid = bm() if (with_backward and s.dtype == vb.BF16) else None
+        ws_bytes = max(vb.workspace_bytes(s, st, self.capacity) for st in stages)
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        self.with_backward = with_backward
+
+    # ---- stage wrappers -----------------------------------------------------------------
+    @staticmethod
+    def raster_strides(x):
+        """Element strides (batch, token, head) of a [B, S, heads, d] tensor."""
+        assert x.stride(3) == 1
+        return (x.stride(0), x.stride(1), x.stride(2))
+
+    def partition(self, raster, bm, inverse=False, perm=None, inv_perm=None):
+        src, dst = (bm, raster) if inverse else (raster, bm)
+        vb.vmoba_partition(self.shape, int(inverse), src, dst, self.raster_strides(raster), perm, inv_perm)
+
+    def block_scores(self):
+        vb.vmoba_block_scores(self.shape, self.q_bm, self.k_bm, self.centroids, self.scores, self.ws)
+
+    def select(self, tau, scores=None):
+        vb.vmoba_select(self.shape, self.scores if scores is None else scores, tau, self.mask_bits, self.kb_ptr,
+                        self.q_idx, self.q_ptr, self.q_pairs, self.capacity, self.k_per_head, self.cutoff,
+                        self.dev_status, self.ws)
+
+    def attn_fwd(self):
+        vb.vmoba_attn_fwd(self.shape, self.q_bm, self.k_bm, self.v_bm, self.kb_ptr, self.q_idx, self.q_ptr,
+                          self.q_pairs, self.capacity, self.o_bm, self.o_resid, self.lse, self.dev_status, self.ws)
+
+    def attn_bwd(self):
+        vb.vmoba_attn_bwd(self.shape, self.q_bm, self.k_bm, self.v_bm, self.o_bm, self.o_resid, self.lse, self.do_bm,
+                          self.kb_ptr, self.q_idx, self.q_ptr, self.capacity, self.dq_bm, self.dk_bm, self.dv_bm,
+                          self.dev_status, self.ws)
+
+    # ---- whole layer --------------------------------------------------------------------
+    def forward(self, q, k, v, tau, o_out):
+        """q, k, v, o_out: [B, S, heads, d] raster-order tensors on the device."""
+        self.partition(q, self.q_bm)
+        self.partition(k, self.k_bm)
+        self.partition(v, self.v_bm)
+        self.block_scores()
+        self.select(tau)
+        self.attn_fwd()
+        self.partition(o_out, self.o_bm, inverse=True)
+
+    def backward(self, do, dq_out, dk_out, dv_out):
+        """Gradients of the last forward(); do and the outputs are raster-order [B, S, heads, d]."""
+        self.partition(do, self.do_bm)
+        self.attn_bwd()
+        self.partition(dq_out, self.dq_bm, inverse=True)
+        self.partition(dk_out, self.dk_bm, inverse=True)
+        self.partition(dv_out, self.dv_bm, inverse=True)
+
+    def check_status(self):
+        code = int(self.dev_status.item())
+        if code != vb.OK:
+            raise vb.VmobaError(code, "device status")
+
+    def n_selected(self) -> int:
+        return int(self.k_per_head.sum().item())
+
+
+def lists_from_mask(mask_bh, capacity=None, device="cuda"):
+    """Builds kb_ptr / q_idx / q_ptr / q_pairs on the host from a boolean mask [BH, S, Nb]
+    (used by tests to feed the attention kernels a selection that did not come from
+    vmoba_select).  Pure index bookkeeping."""
+    import numpy as np
+    BH, S, Nb = mask_bh.shape
+    kb_ptr = [0]
+    q_idx = []
+    pos_of = {}
+    for bh in range(BH):
+        for j in range(Nb):
+            qs = np.nonzero(mask_bh[bh, :, j])[0]
+            base = len(q_idx)
+            for n, qq in enumerate(qs):
+                pos_of[(bh, int(qq), j)] = base + n
+            q_idx.extend(qs.tolist())
+            kb_ptr.append(len(q_idx))
+    q_ptr = [0]
+    q_pairs = []
+    for bh in range(BH):
+        for qq in range(S):
+            for j in np.nonzero(mask_bh[bh, qq])[0]:
+                q_pairs.append(pos_of[(bh, qq, int(j))])
+            q_ptr.append(len(q_pairs))
+    n = len(q_idx)
+    cap = max(n, 1) if capacity is None else capacity
+    pad = lambda a: a + [0] * (cap - len(a))
+    mk = lambda a: torch.tensor(a, dtype=torch.int32, device=device)
+    return mk(kb_ptr), mk(pad(q_idx)), mk(q_ptr), mk(pad(q_pairs)), n

@@ -1,0 +1,70 @@
+"""Helpers shared by the GPU parity tests: moving generated inputs to the device and comparing
+device results with oracle results.  No method arithmetic lives here."""
+import numpy as np
+import torch
+
+from paper_2506_23858_b200 import inputs as gen
+
+# Tolerances: bf16 outputs and gradients within max-abs 2e-2 and relative-L2 1e-2 (the
+# contract of this build); fp32 path 1e-4 / 1e-5 (fp32 FMA arithmetic against fp64).
+TOL = {"bf16": (2e-2, 1e-2), "f32": (1e-4, 1e-5)}
+SCORE_BAND = 1e-3       # pairs whose fp32 score is this close to the cutoff may differ
+SCORE_TOL = 1e-4        # |GPU score - oracle score| for |score| <= 32, growing in proportion beyond (fp32 accumulation)
+
+
+def assert_scores_close(got, ref):
+    err = np.abs(np.asarray(got, dtype=np.float64) - np.asarray(ref, dtype=np.float64))
+    allow = SCORE_TOL * np.maximum(1.0, np.abs(ref) / 32.0)
+    assert np.all(err <= allow), f"score error {err.max():.3e}"
+
+
+def to_device(w, data, name, device="cuda"):
+    """[B, S, heads, d] tensor of the workload's dtype from generated data."""
+    if w.dtype == "bf16":
+        bits = torch.from_numpy(data[name + "_bits"].view(np.int16)).to(device)
+        return bits.view(torch.bfloat16)
+    return torch.from_numpy(data[name]).to(device)
+
+
+def to_numpy_f32(t):
+    return t.detach().float().cpu().numpy()
+
+
+def block_major(w, data, name, perm):
+    """fp32 [B, heads, S, d] block-major copy of a generated raster tensor (index bookkeeping only)."""
+    return np.ascontiguousarray(data[name][:, perm].transpose(0, 2, 1, 3))
+
+
+def bm_to_device(w, x_bm, device="cuda"):
+    """Block-major fp32 numpy values (already representable in the workload dtype) -> device tensor."""
+    t = torch.from_numpy(np.ascontiguousarray(x_bm)).to(device)
+    return t.to(torch.bfloat16) if w.dtype == "bf16" else t
+
+
+def max_abs(a, b):
+    return float(np.max(np.abs(np.asarray(a, dtype=np.float64) - np.asarray(b, dtype=np.float64)))) if np.size(a) else 0.0
+
+
+def rel_l2(a, b):
+    a = np.asarray(a, dtype=np.float64); b = np.asarray(b, dtype=np.float64)
+    den = float(np.sqrt((b * b).sum()))
+    return float(np.sqrt(((a - b) ** 2).sum())) / den if den > 0 else float(np.sqrt(((a - b) ** 2).sum()))
+
+
+def assert_close(got, ref, dtype, what=""):
+    """max-abs and relative-L2 bounds.  A bf16 result cannot be closer to the exact value than half
+    a bf16 ulp (2^-9 |ref|), which alone exceeds 2e-2 once |ref| >= 8; the max-abs bound is therefore
+    taken on top of that unavoidable rounding of the stored result."""
+    ma, rl = TOL[dtype]
+    got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
+    allow = ma + (2.0 ** -9) * np.abs(ref) if dtype == "bf16" else ma
+    excess = float(np.max(np.abs(got - ref) - allow)) if got.size else -1.0
+    e1, e2 = max_abs(got, ref), rel_l2(got, ref)
+    assert excess <= 0 and e2 <= rl, f"{what}: max-abs {e1:.3e} (tol {ma} + half ulp), rel-L2 {e2:.3e} (tol {rl})"
+
+
+def unpack_mask(mask_bits, BH, S, Nb):
+    """uint32 words [BH*S, mw] -> bool [BH, S, Nb]."""
+    wds = mask_bits.cpu().numpy().view(np.uint32).reshape(BH, S, -1)
+    bits = (wds[..., None] >> np.arange(32, dtype=np.uint32)) & 1
+    return bits.reshape(BH, S, -1)[..., :Nb].astype(bool)

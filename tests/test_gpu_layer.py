@@ -1,0 +1,189 @@
+"""End-to-end parity of the whole layer (raster order in, raster order out) against the oracle,
+on the tiny config in full and on the benchmark configurations at full size with sampled
+heads / rows / key blocks (rows of attention are independent, so sampled rows are exact).
+
+Mask parity rule: the GPU mask must equal the oracle's on every pair whose oracle fp32 score
+is farther than 1e-3 from the oracle's cutoff.  Output rows that own a pair inside that band
+are left out of the O / dQ comparison; dK / dV are compared against the oracle re-run on the
+GPU's (validated) mask."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import vmoba_oracle as orc
+from paper_2506_23858_b200 import binding as vb
+from paper_2506_23858_b200 import inputs as gen
+from paper_2506_23858_b200.layer import VmobaLayer, default_capacity
+from tests import _util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_layer(w, data, with_bwd, capacity=None):
+    shape = vb.shape_of(w)
+    cap = capacity or default_capacity(shape, w.tau)
+    L = VmobaLayer(shape, capacity=cap, with_backward=with_bwd)
+    q, k, v = (U.to_device(w, data, n) for n in "qkv")
+    o = torch.empty_like(q)
+    L.forward(q, k, v, w.tau, o)
+    out = dict(L=L, o=o)
+    if with_bwd:
+        do = U.to_device(w, data, "do")
+        out["dq"], out["dk"], out["dv"] = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+        L.backward(do, out["dq"], out["dk"], out["dv"])
+    torch.cuda.synchronize()
+    L.check_status()
+    return out
+
+
+def _check_head(w, data, res, b, h, rng, n_rows, n_blocks, with_bwd):
+    """Oracle for one (batch, head); compares mask (band rule), O/LSE/dQ on sampled clean rows and
+    dK/dV on sampled key blocks."""
+    L = res["L"]
+    scale = w.head_dim ** -0.5
+    perm, inv = orc.partition_perm(w.T, w.H, w.W, *w.block)
+    q, k, v = (data[n][b, :, h][perm] for n in "qkv")
+    cent = orc.centroids(k, w.n_blocks)
+    sc = orc.block_scores(q, cent)
+    m_ref, k_ref, c_ref = orc.select(sc, w.tau, scale)
+    bh = b * w.heads + h
+    S, Nb = w.S, w.n_blocks
+    words = L.mask_bits[bh * S:(bh + 1) * S].cpu().numpy().view(np.uint32)
+    m_gpu = (((words[:, :, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(S, -1)[:, :Nb]).astype(bool)
+    sc_gpu = L.scores.view(-1, S, Nb)[bh].cpu().numpy()
+    U.assert_scores_close(sc_gpu, sc)
+    decided = np.abs(sc - c_ref) > U.SCORE_BAND
+    assert np.array_equal(m_gpu[decided], m_ref[decided]), f"mask mismatch outside the band, head {bh}"
+    assert int(L.k_per_head[bh].item()) == int(m_gpu.sum())
+    clean = decided.all(axis=1)
+    assert clean.mean() > 0.5
+    rows = rng.choice(np.nonzero(clean)[0], size=min(n_rows, int(clean.sum())), replace=False)
+    # make sure both empty and non-empty rows are sampled when they exist
+    o_ref, lse_ref = orc.sparse_attn_fwd(q, k, v, m_ref, scale, rows=rows)
+    raster_rows = torch.from_numpy(perm[rows].astype(np.int64)).cuda()
+    o_gpu = U.to_numpy_f32(res["o"][b, raster_rows, h])
+    U.assert_close(o_gpu, o_ref, w.dtype, f"o head {bh}")
+    lse_gpu = L.lse[bh * S:(bh + 1) * S].cpu().numpy()[rows]
+    ne = np.isfinite(lse_ref)
+    assert np.all(np.isneginf(lse_gpu[~ne])) and np.all(o_gpu[~ne] == 0)
+    assert U.max_abs(lse_gpu[ne], lse_ref[ne]) <= (2e-2 if w.dtype == "bf16" else 1e-4)
+    if with_bwd:
+        do = data["do"][b, :, h][perm]
+        dq_ref, _, _ = orc.sparse_attn_bwd(q, k, v, m_ref, scale, do, rows=rows)
+        U.assert_close(U.to_numpy_f32(res["dq"][b, raster_rows, h]), dq_ref, w.dtype, f"dq head {bh}")
+        # properties that hold at any size: softmax rows sum to 1, so sum_t dV_t = sum of dO over the
+        # non-empty queries; shifting all keys by one vector changes nothing, so sum_t dK_t = 0.
+        all_tok = torch.from_numpy(perm.astype(np.int64)).cuda()
+        dv_all = res["dv"][b, :, h].float()
+        dk_all = res["dk"][b, :, h].float()
+        nonempty = m_gpu.any(axis=1)
+        want = do[nonempty].astype(np.float64).sum(axis=0)
+        eps = 2.0 ** -9 if w.dtype == "bf16" else 1e-6
+        tol_v = 6.0 * np.sqrt(S) * eps * float(dv_all.pow(2).mean().sqrt()) + 1e-3 * np.abs(want).max() + 1e-4
+        assert U.max_abs(dv_all.double().sum(dim=0).cpu().numpy(), want) <= tol_v
+        # D = dO.o is taken from the stored (rounded) output, as in any FlashAttention-style backward, so
+        # each query leaves a residual of order eps * sqrt(d) in sum_t dS_qt; these add up over the queries.
+        tol_k = (6.0 * np.sqrt(S) * eps * float(dk_all.pow(2).mean().sqrt()) + 1e-4
+                 + 3.0 * scale * np.sqrt(S) * eps * np.sqrt(w.head_dim))
+        assert float(dk_all.double().sum(dim=0).abs().max()) <= tol_k
+        # exact dK / dV rows of sampled key blocks, where the oracle can afford the block's queries
+        for j in rng.choice(Nb, size=min(n_blocks, Nb), replace=False):
+            n_q = int(m_gpu[:, j].sum())
+            keys_per_q = float(m_gpu[m_gpu[:, j]].sum(axis=1).mean()) * w.block_tokens if n_q else 0.0
+            if n_q * keys_per_q > 6e7:
+                continue
+            dk_ref, dv_ref = orc.sparse_attn_bwd_key_block(q, k, v, m_gpu, scale, do, int(j))
+            tok = torch.from_numpy(perm[j * w.block_tokens:(j + 1) * w.block_tokens].astype(np.int64)).cuda()
+            U.assert_close(U.to_numpy_f32(res["dk"][b, tok, h]), dk_ref, w.dtype, f"dk head {bh} block {j}")
+            U.assert_close(U.to_numpy_f32(res["dv"][b, tok, h]), dv_ref, w.dtype, f"dv head {bh} block {j}")
+    return float(m_gpu.mean())
+
+
+def test_tiny_config_forward_full_comparison():
+    """Config 1: fp32, 256 tokens, 1D partition, tau 0.25, every row of both heads."""
+    w = gen.C1
+    data = gen.make_inputs(w)
+    res = _run_layer(w, data, with_bwd=True)
+    rng = np.random.default_rng(0)
+    for h in range(w.heads):
+        dens = _check_head(w, data, res, 0, h, rng, n_rows=w.S, n_blocks=w.n_blocks, with_bwd=True)
+        assert 0 < dens <= w.tau + 1e-3
+
+
+MID = gen.Workload("mid", 2, 3, 128, 6, 12, 26, (3, 6, 13), 0.25, "bf16", "smooth", 9)
+
+
+@pytest.mark.parametrize("block", [(1, 12, 26), (6, 6, 13), (3, 6, 13), (1, 3, 13)], ids=["1d", "2d", "3d", "48blk"])
+def test_mid_size_layer_forward_backward(block):
+    w = MID.with_(block=block)
+    data = gen.make_inputs(w)
+    res = _run_layer(w, data, with_bwd=True)
+    rng = np.random.default_rng(1)
+    for b in range(w.B):
+        for h in range(w.heads):
+            _check_head(w, data, res, b, h, rng, n_rows=400, n_blocks=3, with_bwd=True)
+
+
+def test_mid_size_threshold_one_equals_dense_path():
+    """tau = 1.0 through the sparse pipeline must equal the library's dense path and the oracle's dense attention."""
+    w = MID.with_(tau=1.0, B=1, heads=2)
+    data = gen.make_inputs(w)
+    res = _run_layer(w, data, with_bwd=False, capacity=w.B * w.heads * w.S * w.n_blocks)
+    shape = vb.shape_of(w)
+    q, k, v = (U.to_device(w, data, n).permute(0, 2, 1, 3).contiguous() for n in "qkv")     # [B, heads, S, d] raster order
+    o = torch.empty_like(q)
+    lse = torch.empty(w.B * w.heads * w.S, dtype=torch.float32, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    vb.vmoba_full_attn(shape, q, k, v, o, lse, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    sparse = U.to_numpy_f32(res["o"].permute(0, 2, 1, 3))
+    dense = U.to_numpy_f32(o)
+    U.assert_close(sparse, dense, w.dtype, "sparse(tau=1) vs dense path")
+    for h in range(w.heads):
+        od, _ = orc.dense_attn_fwd(data["q"][0, :, h], data["k"][0, :, h], data["v"][0, :, h], w.head_dim ** -0.5,
+                                   rows=np.arange(0, w.S, 7))
+        U.assert_close(dense[0, h][::7], od, w.dtype, "dense path vs oracle")
+
+
+# ---- the benchmark configurations at full size, sampled -----------------------------------
+def _full_size(w, with_bwd, heads_checked, n_rows=96, n_blocks=2, capacity=None):
+    data = gen.make_inputs(w, with_do=with_bwd)
+    res = _run_layer(w, data, with_bwd, capacity=capacity)
+    rng = np.random.default_rng(2)
+    dens = []
+    for (b, h) in heads_checked:
+        dens.append(_check_head(w, data, res, b, h, rng, n_rows, n_blocks, with_bwd))
+    return res, dens
+
+
+def test_config2_wan_layer_3d_forward():
+    res, dens = _full_size(gen.C2, False, [(0, 0), (0, 7)])
+    assert all(0 < d <= 0.25 for d in dens)
+
+
+@pytest.mark.parametrize("name", ["1d", "2d"])
+def test_config3_partitions_forward(name):
+    w = gen.C2.with_(name="c3_" + name, block=gen.C3_BLOCKS[name])
+    _full_size(w, False, [(0, 3)])
+
+
+@pytest.mark.parametrize("tau", [0.1, 0.5])
+def test_config3_threshold_sweep_3d(tau):
+    w = gen.C2.with_(name=f"c3_tau{tau}", tau=tau, heads=4)
+    res, dens = _full_size(w, False, [(0, 1)])
+    assert dens[0] <= tau
+
+
+def test_config4_training_step():
+    res, dens = _full_size(gen.C4, True, [(1, 5)])
+
+
+@pytest.mark.parametrize("name", ["1d", "2d", "3d"])
+def test_config5_720p_shape_forward_backward(name):
+    """Config 5's grid and block shapes with 4 of its 40 heads (per-head work is independent;
+    the input generator is the bottleneck of this test, not the GPU)."""
+    w = gen.C5.with_(name="c5_" + name, block=gen.C5_BLOCKS[name], heads=4)
+    shape = vb.shape_of(w)
+    cap = int(0.3 * default_capacity(shape, w.tau)) if name == "3d" else None
+    _full_size(w, True, [(0, 2)], n_rows=48, n_blocks=1, capacity=cap)

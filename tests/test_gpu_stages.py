@@ -1,0 +1,260 @@
+"""Stage-isolated parity: each CUDA stage is fed the ORACLE's output of the previous stage and
+compared element by element with the oracle's output of that stage.  All calls go through the
+C-ABI library."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import vmoba_oracle as orc
+from paper_2506_23858_b200 import binding as vb
+from paper_2506_23858_b200 import inputs as gen
+from paper_2506_23858_b200.layer import VmobaLayer, lists_from_mask
+from tests import _util as U
+
+pytestmark = pytest.mark.gpu
+
+# Mid-size cases: 1872 tokens (29.25 tiles of 64, 14.6 tiles of 128), several block geometries
+# (1 to 15 mask words), both dtypes, both head dims, batch 2.
+MID = gen.Workload("mid", 1, 2, 128, 6, 12, 26, (3, 6, 13), 0.25, "bf16", "smooth", 5)
+CASES = [
+    gen.C1,
+    gen.C1.with_(name="c1_3d", block=(2, 4, 2)),
+    gen.C1.with_(name="c1_d128", head_dim=128, block=(4, 2, 4)),
+    MID,
+    MID.with_(name="mid_1d", block=(1, 12, 26)),
+    MID.with_(name="mid_2d", block=(6, 6, 13), B=2),
+    MID.with_(name="mid_48blk", block=(1, 3, 13)),
+    MID.with_(name="mid_468blk", block=(1, 2, 2), tau=0.1),
+    MID.with_(name="mid_f32", dtype="f32", head_dim=64, block=(2, 6, 13)),
+    MID.with_(name="mid_bf16_d64", head_dim=64, block=(3, 4, 13)),
+]
+IDS = [c.name for c in CASES]
+
+
+def _oracle_front(w, data):
+    """Oracle partition, centroids, scores, selection for every (b, head)."""
+    perm, inv = orc.partition_perm(w.T, w.H, w.W, *w.block)
+    scale = w.head_dim ** -0.5
+    out = dict(perm=perm, inv=inv, scale=scale, heads=[])
+    for b in range(w.B):
+        for h in range(w.heads):
+            q, k, v = (data[n][b, :, h][perm] for n in "qkv")
+            cent = orc.centroids(k, w.n_blocks)
+            sc = orc.block_scores(q, cent)
+            mask, kk, cutoff = orc.select(sc, w.tau, scale)
+            out["heads"].append(dict(q=q, k=k, v=v, cent=cent, scores=sc, mask=mask, k_sel=kk, cutoff=cutoff))
+    return out
+
+
+_cache = {}
+
+
+def _prep(w):
+    if w.name not in _cache:
+        data = gen.make_inputs(w)
+        _cache[w.name] = (data, _oracle_front(w, data))
+    return _cache[w.name]
+
+
+@pytest.mark.parametrize("w", CASES, ids=IDS)
+def test_partition_bit_exact_and_inverse(w):
+    data, ora = _prep(w)
+    shape = vb.shape_of(w)
+    L = VmobaLayer(shape, capacity=1024)
+    x = U.to_device(w, data, "q")
+    perm = torch.empty(w.S, dtype=torch.int32, device="cuda")
+    inv = torch.empty(w.S, dtype=torch.int32, device="cuda")
+    L.partition(x, L.q_bm, perm=perm, inv_perm=inv)
+    assert np.array_equal(perm.cpu().numpy(), ora["perm"])
+    assert np.array_equal(inv.cpu().numpy(), ora["inv"])
+    got = L.q_bm.view(torch.int16 if w.dtype == "bf16" else torch.int32).cpu().numpy()
+    src = x.view(torch.int16 if w.dtype == "bf16" else torch.int32).cpu().numpy()
+    ref = np.ascontiguousarray(src[:, ora["perm"]].transpose(0, 2, 1, 3))
+    assert np.array_equal(got, ref)
+    back = torch.zeros_like(x)
+    L.partition(back, L.q_bm, inverse=True)
+    assert torch.equal(back.view(torch.int16 if w.dtype == "bf16" else torch.int32),
+                       x.view(torch.int16 if w.dtype == "bf16" else torch.int32))
+
+
+def test_partition_strided_raster_view():
+    """q, k, v often live interleaved in one [B, S, 3, heads, d] projection output."""
+    w = MID
+    data, ora = _prep(w)
+    shape = vb.shape_of(w)
+    L = VmobaLayer(shape, capacity=1024)
+    qkv = torch.stack([U.to_device(w, data, n) for n in "qkv"], dim=2)      # [B, S, 3, heads, d]
+    kview = qkv[:, :, 1]
+    L.partition(kview, L.k_bm)
+    ref = np.ascontiguousarray(data["k"][:, ora["perm"]].transpose(0, 2, 1, 3))
+    assert np.array_equal(U.to_numpy_f32(L.k_bm), ref)
+
+
+@pytest.mark.parametrize("w", CASES, ids=IDS)
+def test_centroids_and_scores(w):
+    data, ora = _prep(w)
+    shape = vb.shape_of(w)
+    L = VmobaLayer(shape, capacity=1024)
+    L.q_bm.copy_(U.bm_to_device(w, U.block_major(w, data, "q", ora["perm"])))
+    L.k_bm.copy_(U.bm_to_device(w, U.block_major(w, data, "k", ora["perm"])))
+    L.block_scores()
+    cent = L.centroids.cpu().numpy().reshape(w.B * w.heads, w.n_blocks, w.head_dim)
+    sc = L.scores.cpu().numpy().reshape(w.B * w.heads, w.S, w.n_blocks)
+    for i, hd in enumerate(ora["heads"]):
+        assert U.max_abs(cent[i], hd["cent"]) <= 2e-6
+        U.assert_scores_close(sc[i], hd["scores"])
+
+
+def _check_lists(L, w, mask):
+    """kb_ptr/q_idx/q_ptr/q_pairs must be exactly the CSR forms of `mask` [BH, S, Nb]."""
+    BH, S, Nb = mask.shape
+    kb_ptr = L.kb_ptr.cpu().numpy(); q_idx = L.q_idx.cpu().numpy()
+    q_ptr = L.q_ptr.cpu().numpy(); q_pairs = L.q_pairs.cpu().numpy()
+    counts = mask.sum(axis=1).reshape(-1)
+    assert np.array_equal(np.diff(kb_ptr), counts) and kb_ptr[0] == 0
+    assert np.array_equal(np.diff(q_ptr), mask.sum(axis=2).reshape(-1)) and q_ptr[0] == 0
+    n = int(mask.sum())
+    assert kb_ptr[-1] == n and q_ptr[-1] == n
+    for bh in range(BH):
+        for j in range(Nb):
+            lo, hi = kb_ptr[bh * Nb + j], kb_ptr[bh * Nb + j + 1]
+            assert np.array_equal(q_idx[lo:hi], np.nonzero(mask[bh, :, j])[0])
+    # q_pairs: for query G its pairs in ascending block order point back at (block j list, entry == q)
+    block_of_pos = np.repeat(np.arange(BH * Nb), counts)
+    for G in np.random.default_rng(0).choice(BH * S, size=min(BH * S, 600), replace=False):
+        bh, qq = divmod(int(G), S)
+        pp = q_pairs[q_ptr[G]:q_ptr[G + 1]]
+        assert np.array_equal(block_of_pos[pp] - bh * Nb, np.nonzero(mask[bh, qq])[0])
+        assert np.all(q_idx[pp] == qq)
+
+
+@pytest.mark.parametrize("w", CASES, ids=IDS)
+def test_select_matches_oracle_outside_the_cutoff_band(w):
+    data, ora = _prep(w)
+    shape = vb.shape_of(w)
+    cap = w.B * w.heads * w.S * w.n_blocks
+    L = VmobaLayer(shape, capacity=cap)
+    sc = np.stack([hd["scores"] for hd in ora["heads"]]).reshape(w.B, w.heads, w.S, w.n_blocks)
+    L.scores.copy_(torch.from_numpy(sc))
+    for tau in (w.tau, 0.6, 1.0):
+        L.dev_status.zero_()
+        L.select(tau)
+        L.check_status()
+        got = U.unpack_mask(L.mask_bits, w.B * w.heads, w.S, w.n_blocks)
+        kph = L.k_per_head.cpu().numpy(); cut = L.cutoff.cpu().numpy()
+        for i, hd in enumerate(ora["heads"]):
+            m_ref, k_ref, c_ref = orc.select(hd["scores"], tau, ora["scale"])
+            decided = np.abs(hd["scores"] - c_ref) > U.SCORE_BAND
+            assert np.array_equal(got[i][decided], m_ref[decided]), (tau, i)
+            assert kph[i] == got[i].sum()
+            # same scores in, so the GPU may only differ by exact ties and fp64 summation order
+            assert abs(float(cut[i]) - float(c_ref)) <= U.SCORE_BAND
+            assert abs(int(kph[i]) - k_ref) <= max(8, int(1e-4 * k_ref)), (tau, i, kph[i], k_ref)
+            assert np.all(hd["scores"][got[i]] >= cut[i]) and np.all(hd["scores"][~got[i]] < cut[i])
+        _check_lists(L, w, got)
+    assert got.all()          # tau = 1 selects every pair
+
+
+def test_select_reports_capacity_overflow():
+    w = MID
+    data, ora = _prep(w)
+    shape = vb.shape_of(w)
+    L = VmobaLayer(shape, capacity=256)
+    sc = np.stack([hd["scores"] for hd in ora["heads"]]).reshape(w.B, w.heads, w.S, w.n_blocks)
+    L.scores.copy_(torch.from_numpy(sc))
+    L.select(0.25)
+    torch.cuda.synchronize()
+    assert int(L.dev_status.item()) == vb.ERR_CAPACITY
+    # the truncated lists must still be usable without leaving the buffers
+    L.q_bm.normal_(); L.k_bm.normal_(); L.v_bm.normal_()
+    L.attn_fwd()
+    torch.cuda.synchronize()
+
+
+def _oracle_attention(w, ora, data, masks, with_bwd):
+    res = []
+    for i, hd in enumerate(ora["heads"]):
+        o, lse = orc.sparse_attn_fwd(hd["q"], hd["k"], hd["v"], masks[i], ora["scale"])
+        r = dict(o=o, lse=lse)
+        if with_bwd:
+            b, h = divmod(i, w.heads)
+            do = data["do"][b, :, h][ora["perm"]]
+            r["dq"], r["dk"], r["dv"] = orc.sparse_attn_bwd(hd["q"], hd["k"], hd["v"], masks[i], ora["scale"], do)
+        res.append(r)
+    return res
+
+
+@pytest.mark.parametrize("w", CASES, ids=IDS)
+def test_sparse_attention_forward_backward(w):
+    data, ora = _prep(w)
+    shape = vb.shape_of(w)
+    masks = np.stack([hd["mask"] for hd in ora["heads"]])
+    kb_ptr, q_idx, q_ptr, q_pairs, n = lists_from_mask(masks)
+    L = VmobaLayer(shape, capacity=max(n, 1), with_backward=True)
+    for name, buf in (("q", L.q_bm), ("k", L.k_bm), ("v", L.v_bm), ("do", L.do_bm)):
+        buf.copy_(U.bm_to_device(w, U.block_major(w, data, name, ora["perm"])))
+    L.kb_ptr.copy_(kb_ptr); L.q_idx.copy_(q_idx); L.q_ptr.copy_(q_ptr); L.q_pairs.copy_(q_pairs)
+    L.o_bm.fill_(7.0); L.lse.fill_(7.0)
+    L.attn_fwd()
+    L.attn_bwd()
+    L.check_status()
+    ref = _oracle_attention(w, ora, data, masks, True)
+    BH = w.B * w.heads
+    o = U.to_numpy_f32(L.o_bm).reshape(BH, w.S, w.head_dim)
+    lse = L.lse.cpu().numpy().reshape(BH, w.S)
+    dq, dk, dv = (U.to_numpy_f32(t).reshape(BH, w.S, w.head_dim) for t in (L.dq_bm, L.dk_bm, L.dv_bm))
+    for i, r in enumerate(ref):
+        empty = ~masks[i].any(axis=1)
+        assert np.all(o[i][empty] == 0) and np.all(np.isneginf(lse[i][empty])) and np.all(dq[i][empty] == 0)
+        U.assert_close(o[i], r["o"], w.dtype, f"o head {i}")
+        assert U.max_abs(lse[i][~empty], r["lse"][~empty]) <= (2e-2 if w.dtype == "bf16" else 1e-4)
+        U.assert_close(dq[i], r["dq"], w.dtype, f"dq head {i}")
+        U.assert_close(dk[i], r["dk"], w.dtype, f"dk head {i}")
+        U.assert_close(dv[i], r["dv"], w.dtype, f"dv head {i}")
+
+
+@pytest.mark.parametrize("w", [CASES[0], CASES[3], CASES[8]], ids=[IDS[0], IDS[3], IDS[8]])
+def test_sparse_attention_full_mask_equals_dense_oracle(w):
+    """tau = 1: the sparse path over every pair must reproduce dense softmax attention."""
+    data, ora = _prep(w)
+    shape = vb.shape_of(w)
+    BH = w.B * w.heads
+    masks = np.ones((BH, w.S, w.n_blocks), dtype=bool)
+    kb_ptr, q_idx, q_ptr, q_pairs, n = lists_from_mask(masks)
+    L = VmobaLayer(shape, capacity=n)
+    for name, buf in (("q", L.q_bm), ("k", L.k_bm), ("v", L.v_bm)):
+        buf.copy_(U.bm_to_device(w, U.block_major(w, data, name, ora["perm"])))
+    L.kb_ptr.copy_(kb_ptr); L.q_idx.copy_(q_idx); L.q_ptr.copy_(q_ptr); L.q_pairs.copy_(q_pairs)
+    L.attn_fwd()
+    L.check_status()
+    o = U.to_numpy_f32(L.o_bm).reshape(BH, w.S, w.head_dim)
+    for i, hd in enumerate(ora["heads"]):
+        od, _ = orc.dense_attn_fwd(hd["q"], hd["k"], hd["v"], ora["scale"])
+        U.assert_close(o[i], od, w.dtype, f"head {i}")
+
+
+@pytest.mark.parametrize("w", [CASES[0], CASES[3], CASES[8], CASES[9]], ids=[IDS[0], IDS[3], IDS[8], IDS[9]])
+def test_dense_attention_forward_backward(w):
+    data, ora = _prep(w)
+    shape = vb.shape_of(w)
+    BH = w.B * w.heads
+    dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    mk = lambda name: U.bm_to_device(w, U.block_major(w, data, name, ora["perm"]))
+    q, k, v, do = mk("q"), mk("k"), mk("v"), mk("do")
+    o = torch.empty_like(q); dq = torch.empty_like(q); dk = torch.empty_like(q); dv = torch.empty_like(q)
+    lse = torch.empty(BH * w.S, dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(vb.workspace_bytes(shape, vb.STAGE_FULL_BWD), dtype=torch.uint8, device="cuda")
+    vb.vmoba_full_attn(shape, q, k, v, o, lse, do, dq, dk, dv, status, ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    on = U.to_numpy_f32(o).reshape(BH, w.S, -1)
+    g = [U.to_numpy_f32(t).reshape(BH, w.S, -1) for t in (dq, dk, dv)]
+    for i, hd in enumerate(ora["heads"]):
+        b, h = divmod(i, w.heads)
+        od, lsed = orc.dense_attn_fwd(hd["q"], hd["k"], hd["v"], ora["scale"])
+        U.assert_close(on[i], od, w.dtype, "o")
+        assert U.max_abs(lse.cpu().numpy().reshape(BH, w.S)[i], lsed) <= (2e-2 if w.dtype == "bf16" else 1e-4)
+        ref = orc.dense_attn_bwd(hd["q"], hd["k"], hd["v"], ora["scale"], data["do"][b, :, h][ora["perm"]])
+        for name, got, want in zip(("dq", "dk", "dv"), g, ref):
+            U.assert_close(got[i], want, w.dtype, name)
