@@ -75,6 +75,10 @@ typedef struct {
 
 const char* vmoba_status_string(int status);
 
+/* Number of CUDA kernels this library has launched in this process since it was loaded
+ * (bookkeeping for benchmarks; the paper has no counterpart). */
+uint64_t vmoba_kernel_launches(void);
+
 /* Bytes of scratch `ws` a stage needs.  `capacity` is the number of (query, key-block) pairs
  * the work lists can hold (the q_idx_capacity given to vmoba_select); stages that do not
  * depend on it ignore it.  Returns 0 for an invalid shape or stage. */

@@ -16,7 +16,7 @@ F32, BF16 = 0, 1
 STAGE_SCORES, STAGE_SELECT, STAGE_ATTN_FWD, STAGE_ATTN_BWD, STAGE_FULL_FWD, STAGE_FULL_BWD = range(6)
 
 EXPORTS = (
-    "vmoba_status_string", "vmoba_workspace_bytes", "vmoba_partition", "vmoba_block_scores",
+    "vmoba_status_string", "vmoba_kernel_launches", "vmoba_workspace_bytes", "vmoba_partition", "vmoba_block_scores",
     "vmoba_select", "vmoba_attn_fwd", "vmoba_attn_bwd", "vmoba_full_attn",
 )
 
@@ -76,12 +76,16 @@ def lib():
         return _lib
     path = lib_path()
     if not os.path.exists(path):
+        _build.build()          # needs nvcc; raises if the build fails -- there is no CPU fallback
+    if not os.path.exists(path):
         raise RuntimeError(f"{path} is missing: run `python -m paper_2506_23858_b200.build` (no CPU fallback exists)")
     L = ctypes.CDLL(path)
     vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
     sp = ctypes.POINTER(Shape)
     L.vmoba_status_string.restype = ctypes.c_char_p
     L.vmoba_status_string.argtypes = [ctypes.c_int]
+    L.vmoba_kernel_launches.restype = ctypes.c_uint64
+    L.vmoba_kernel_launches.argtypes = []
     L.vmoba_workspace_bytes.restype = sz
     L.vmoba_workspace_bytes.argtypes = [sp, ctypes.c_int, i64]
     L.vmoba_partition.restype = ctypes.c_int
@@ -117,6 +121,10 @@ def _stream(stream=None):
 def _check(code, where):
     if code != OK:
         raise VmobaError(code, where)
+
+
+def kernel_launches() -> int:
+    return int(lib().vmoba_kernel_launches())
 
 
 def workspace_bytes(shape: Shape, stage: int, capacity: int = 0) -> int:

@@ -51,7 +51,7 @@ static int simt_sparse_fwd(const Dims& D, const void* q, const void* k, const vo
   long long nq = (long long)D.BH * D.S;
   simt::merge_kernel<T, DH, float><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(
       q_ptr, q_pairs, nq, w.part_o, w.part_lse, cap, (T*)o, (T*)o_resid, lse);
-  VMOBA_LAUNCH_OK();
+  VMOBA_LAUNCH_OK(3);
   return VMOBA_OK;
 }
 
@@ -74,7 +74,7 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
       (const T*)q, (const T*)k, (const T*)v, (const T*)d_o, lse, w.Dv, kb_ptr, q_idx, w.item_ptr, (int)n_kb, D.S,
       D.Nb, D.sb, D.BH, D.scale, cap, w.dq_acc, (T*)dq);
   simt::cast_kernel<T><<<grid_for((nq * DH / 4 + 255) / 256, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, nq * DH / 4);
-  VMOBA_LAUNCH_OK();
+  VMOBA_LAUNCH_OK(5);
   return VMOBA_OK;
 }
 
@@ -97,7 +97,7 @@ static int simt_dense(const Dims& D, const void* q, const void* k, const void* v
         (const T*)q, (const T*)k, (const T*)v, (const T*)d_o, lse, w.Dv, nullptr, nullptr, nullptr, 0, D.S, 1, D.S,
         D.BH, D.scale, 0, nullptr, (T*)dq);
   }
-  VMOBA_LAUNCH_OK();
+  VMOBA_LAUNCH_OK(d_o ? 4 : 1);
   return VMOBA_OK;
 }
 
@@ -128,6 +128,8 @@ extern "C" const char* vmoba_status_string(int status) {
     default: return "unknown status";
   }
 }
+
+extern "C" uint64_t vmoba_kernel_launches(void) { return g_kernel_launches.load(std::memory_order_relaxed); }
 
 extern "C" size_t vmoba_workspace_bytes(const vmoba_shape* shape, int stage, int64_t capacity) {
   Dims D;

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/vmoba.h"
 
 namespace vmoba {
@@ -77,12 +79,19 @@ struct Carver {
     if (e__ != cudaSuccess) return VMOBA_ERR_CUDA; \
   } while (0)
 
-#define VMOBA_LAUNCH_OK()                                   \
+// Number of kernels this library has launched since it was loaded (reported by
+// vmoba_kernel_launches(); benchmarks use it to show that the CUDA path did the work).
+inline std::atomic<unsigned long long> g_kernel_launches{0};
+inline void count_launches(int n) { g_kernel_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+// Checks the launches issued since the last check; n = how many kernels those were.
+#define VMOBA_LAUNCH_OK(n)                                  \
   do {                                                      \
     if (cudaPeekAtLastError() != cudaSuccess) {             \
       cudaGetLastError();                                   \
       return VMOBA_ERR_CUDA;                                \
     }                                                       \
+    ::vmoba::count_launches(n);                             \
   } while (0)
 
 // ---------------------------------------------------------------- device helpers

@@ -88,7 +88,7 @@ static int launch_partition(const Dims& D, const PermGeom& g, int inverse, const
   partition_kernel<V><<<(unsigned)blocks, 256, 0, st>>>(
       g, D.S, D.heads, n_rows, inverse, static_cast<const uint4*>(src), static_cast<uint4*>(dst),
       rs[0] / per_vec, rs[1] / per_vec, rs[2] / per_vec);
-  VMOBA_LAUNCH_OK();
+  VMOBA_LAUNCH_OK(1);
   return VMOBA_OK;
 }
 
@@ -111,7 +111,7 @@ extern "C" int vmoba_partition(const vmoba_shape* shape, int inverse, const void
   PermGeom g{D.H, D.W, D.bT, D.bH, D.bW, D.nH, D.nW, D.sb};
   if (perm_or_null || inv_perm_or_null) {
     perm_table_kernel<<<(D.S + 255) / 256, 256, 0, st>>>(g, D.S, perm_or_null, inv_perm_or_null);
-    VMOBA_LAUNCH_OK();
+    VMOBA_LAUNCH_OK(1);
   }
   int V = D.d * D.es / 16;
   switch (V) {

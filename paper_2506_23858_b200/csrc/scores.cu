@@ -109,12 +109,12 @@ scores_kernel(const T* __restrict__ q_bm, const float* __restrict__ cent, float*
 template <typename T, int DH>
 static int run_scores(const Dims& D, const void* q, const void* k, float* cent, float* scores, cudaStream_t st) {
   centroid_kernel<T, DH><<<D.BH * D.Nb, 256, 0, st>>>(static_cast<const T*>(k), cent, D.sb);
-  VMOBA_LAUNCH_OK();
+  VMOBA_LAUNCH_OK(1);
   size_t smem = 2 * DH * (64 + 4) * sizeof(float);
   VMOBA_CUDA_OK(cudaFuncSetAttribute(scores_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid((D.S + 63) / 64, 1, D.BH);
   scores_kernel<T, DH><<<grid, 256, smem, st>>>(static_cast<const T*>(q), cent, scores, D.S, D.Nb);
-  VMOBA_LAUNCH_OK();
+  VMOBA_LAUNCH_OK(1);
   return VMOBA_OK;
 }
 

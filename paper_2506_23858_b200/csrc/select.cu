@@ -480,7 +480,7 @@ extern "C" int vmoba_select(const vmoba_shape* shape, const float* scores, float
   scan_kernel<1><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, k_per_head, cutoff_per_head);
   hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey);
   scan_kernel<2><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, k_per_head, cutoff_per_head);
-  VMOBA_LAUNCH_OK();
+  VMOBA_LAUNCH_OK(9);
 
   size_t smem = (size_t)QSEG * D.mask_words * 4 + (size_t)std::max(D.Nb, QSEG) * 4;
   VMOBA_CUDA_OK(cudaFuncSetAttribute(mark_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -494,6 +494,6 @@ extern "C" int vmoba_select(const vmoba_shape* shape, const float* scores, float
                                      D.BH, D.Nb, k_per_head, capacity, q_ptr + (long long)D.BH * D.S, dev_status);
   fill_kernel<<<sgrid, kSegThreads, smem, st>>>(mask_bits, D.S, D.Nb, D.mask_words, QSEG, nseg, kb_ptr, w.seg_cnt,
                                                 w.seg_qoff, q_idx, q_ptr, q_pairs, capacity);
-  VMOBA_LAUNCH_OK();
+  VMOBA_LAUNCH_OK(4);
   return VMOBA_OK;
 }
