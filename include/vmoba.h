@@ -129,6 +129,32 @@ int vmoba_select(const vmoba_shape* shape, const float* scores, float tau, uint3
                  int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * vmoba_select for callers that cannot hand over scratch memory.  (The paper has no counterpart:
+ * this is a packaging variant of the selection stage, not a step of the method.)
+ *
+ * Who needs it: code that runs where allocating device memory is not possible or not allowed --
+ * a plug-in inside a memory-planned inference engine that only receives its input and output
+ * buffers, or a serving loop in which cudaMalloc (it synchronises the whole device) is banned.
+ * Same arguments and results as vmoba_select minus `ws`: the scratch is a fixed
+ * vmoba_select_static_scratch_bytes() = 16 MiB array inside the library image, which every GPU
+ * that loads the library keeps resident until the process exits.
+ *   - Shapes whose vmoba_workspace_bytes(shape, VMOBA_STAGE_SELECT, 0) exceeds that size are
+ *     rejected with VMOBA_ERR_WORKSPACE; use vmoba_select with your own buffer for those.
+ *   - The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ *   - The first call on each device looks up the array's device address (one
+ *     cudaGetSymbolAddress, with that device current); make that first call outside of any stream
+ *     capture.  Later calls on the device reuse the address.
+ *   - All calls on one device share the one array.  Every call re-initialises what it needs, so
+ *     stale contents are harmless, but two calls whose kernels can overlap on the GPU (different
+ *     streams, no ordering between them) race on it: serialise them.
+ */
+size_t vmoba_select_static_scratch_bytes(void);
+int vmoba_select_static(const vmoba_shape* shape, const float* scores, float tau, uint32_t* mask_bits,
+                        int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr, int32_t* q_pairs,
+                        int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
+                        int32_t* dev_status, void* stream);
+
+/*
  * Step 3: attention of every query over the keys of its selected blocks.
  *   o_bm [B, heads, S, head_dim] (dtype), lse [B*heads*S] fp32 natural-log sum-exp of the scaled logits.
  * A query with no selected block gets o = 0 and lse = -inf.

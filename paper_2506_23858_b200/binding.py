@@ -17,7 +17,7 @@ STAGE_SCORES, STAGE_SELECT, STAGE_ATTN_FWD, STAGE_ATTN_BWD, STAGE_FULL_FWD, STAG
 
 EXPORTS = (
     "vmoba_status_string", "vmoba_kernel_launches", "vmoba_workspace_bytes", "vmoba_partition", "vmoba_block_scores",
-    "vmoba_select", "vmoba_attn_fwd", "vmoba_attn_bwd", "vmoba_full_attn",
+    "vmoba_select", "vmoba_select_static", "vmoba_select_static_scratch_bytes", "vmoba_attn_fwd", "vmoba_attn_bwd", "vmoba_full_attn",
 )
 
 
@@ -94,6 +94,10 @@ def lib():
     L.vmoba_block_scores.argtypes = [sp, vp, vp, vp, vp, vp, sz, vp]
     L.vmoba_select.restype = ctypes.c_int
     L.vmoba_select.argtypes = [sp, vp, ctypes.c_float, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp]
+    L.vmoba_select_static.restype = ctypes.c_int
+    L.vmoba_select_static.argtypes = [sp, vp, ctypes.c_float, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp]
+    L.vmoba_select_static_scratch_bytes.restype = sz
+    L.vmoba_select_static_scratch_bytes.argtypes = []
     L.vmoba_attn_fwd.restype = ctypes.c_int
     L.vmoba_attn_fwd.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
     L.vmoba_attn_bwd.restype = ctypes.c_int
@@ -155,6 +159,19 @@ def vmoba_select(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, c
     _check(lib().vmoba_select(ctypes.byref(shape), _ptr(scores), float(tau), _ptr(mask_bits), _ptr(kb_ptr),
                               _ptr(q_idx), _ptr(q_ptr), _ptr(q_pairs), int(capacity), _ptr(k_per_head),
                               _ptr(cutoff_per_head), _ptr(dev_status), p, n, _stream(stream)), "vmoba_select")
+
+
+def vmoba_select_static(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity, k_per_head,
+                        cutoff_per_head, dev_status, stream=None):
+    """vmoba_select with the library's built-in 16 MiB scratch array instead of a caller workspace: for callers
+    that may not allocate device memory.  Calls on one device share that array and must not overlap."""
+    _check(lib().vmoba_select_static(ctypes.byref(shape), _ptr(scores), float(tau), _ptr(mask_bits), _ptr(kb_ptr),
+                                     _ptr(q_idx), _ptr(q_ptr), _ptr(q_pairs), int(capacity), _ptr(k_per_head),
+                                     _ptr(cutoff_per_head), _ptr(dev_status), _stream(stream)), "vmoba_select_static")
+
+
+def select_static_scratch_bytes() -> int:
+    return int(lib().vmoba_select_static_scratch_bytes())
 
 
 def vmoba_attn_fwd(shape, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid, lse, dev_status,

@@ -497,3 +497,51 @@ extern "C" int vmoba_select(const vmoba_shape* shape, const float* scores, float
   VMOBA_LAUNCH_OK(4);
   return VMOBA_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// Selection without a caller-provided workspace.
+//
+// Some callers of this library are not allowed to allocate device memory at the point where
+// they run the layer: code running inside a memory-planned inference engine or a framework
+// plug-in that was handed fixed input/output buffers and nothing else, or a latency-critical
+// loop in which cudaMalloc (which synchronises the device) is forbidden.  For them the scratch
+// of the selection stage lives in the array below, which is part of the library image: every
+// GPU that loads the library holds these bytes until the process exits.
+namespace vmoba {
+constexpr size_t kStaticSelectScratchBytes = 16u << 20;   // 16 MiB
+static __device__ __align__(256) unsigned char g_select_scratch[kStaticSelectScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static void* g_select_scratch_addr[kMaxDevices] = {nullptr};
+}  // namespace vmoba
+
+extern "C" size_t vmoba_select_static_scratch_bytes(void) { return vmoba::kStaticSelectScratchBytes; }
+
+extern "C" int vmoba_select_static(const vmoba_shape* shape, const float* scores, float tau, uint32_t* mask_bits,
+                                   int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr, int32_t* q_pairs,
+                                   int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
+                                   int32_t* dev_status, void* stream) {
+  Dims D;
+  int rc = make_dims(shape, &D);
+  if (rc) return rc;
+  if (D.Nb > 8192) return VMOBA_ERR_SHAPE;
+  // The shape's scratch need must fit the fixed array; larger problems have to use vmoba_select.
+  if (select_ws_bytes(D) > kStaticSelectScratchBytes) return VMOBA_ERR_WORKSPACE;
+  int dev = -1;
+  VMOBA_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return VMOBA_ERR_CUDA;
+  if (!g_select_scratch_addr[dev]) {
+    // In host code the array's name is only a handle for the symbol, not a device address: ask the
+    // runtime for the address on the current device, once per device.
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return VMOBA_ERR_CUDA;
+    }
+    g_select_scratch_addr[dev] = p;
+  }
+  // vmoba_select clears everything in its scratch that has to start at zero, so the contents
+  // left by an earlier call do not matter.
+  return vmoba_select(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity, k_per_head,
+                      cutoff_per_head, dev_status, g_select_scratch_addr[dev], kStaticSelectScratchBytes, stream);
+}
