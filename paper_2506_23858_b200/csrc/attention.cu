@@ -9,6 +9,22 @@ namespace vmoba {
 
 size_t select_ws_bytes(const Dims& D);   // select.cu
 
+// attn_tc.cu: tensor-core forward kernels (bf16, head_dim 128)
+int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
+                  const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
+                  int32_t* status, int* item_ptr, float* part_o, float* part_lse, cudaStream_t st);
+int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, void* o, void* o_resid, float* lse,
+                 int32_t* status, cudaStream_t st);
+
+// attn_tc_bwd.cu: tensor-core backward kernels (bf16, head_dim 128)
+int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                  const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap,
+                  const int* item_ptr, float* dq_acc, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st);
+int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                 const float* Dv, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st);
+
+static bool use_tensor_cores(const Dims& D) { return D.dtype == VMOBA_BF16 && D.d == 128; }
+
 struct FwdWs { int* item_ptr; float* part_o; float* part_lse; size_t bytes; };
 static FwdWs carve_fwd(const Dims& D, long long cap, void* ws) {
   Carver c(ws);
@@ -57,14 +73,25 @@ static int simt_sparse_fwd(const Dims& D, const void* q, const void* k, const vo
 
 template <typename T, int DH>
 static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* o,
-                           const void* o_resid, const float* lse, const void* d_o, const int* kb_ptr, const int* q_idx, long long cap,
-                           void* dq, void* dk, void* dv, void* ws, cudaStream_t st) {
+                           const void* o_resid, const float* lse, const void* d_o, const int* kb_ptr, const int* q_idx,
+                           const int* q_ptr, long long cap, void* dq, void* dk, void* dv, int32_t* status, void* ws,
+                           cudaStream_t st) {
   BwdWs w = carve_bwd(D, false, ws);
   const long long n_kb = (long long)D.BH * D.Nb;
   const long long nq = (long long)D.BH * D.S;
   VMOBA_CUDA_OK(cudaMemsetAsync(w.dq_acc, 0, (size_t)nq * DH * sizeof(float), st));
   simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>((const T*)o, (const T*)o_resid,
                                                                         (const T*)d_o, nq, w.Dv);
+  if (use_tensor_cores(D)) {
+    simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, 128, cap, w.item_ptr);
+    count_launches(2);
+    int rc = tc_sparse_bwd(D, q, k, v, d_o, lse, w.Dv, kb_ptr, q_idx, q_ptr, cap, w.item_ptr, w.dq_acc, dq, dk, dv,
+                           status, st);
+    if (rc) return rc;
+    simt::cast_rows_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, q_ptr, nq, 1);
+    VMOBA_LAUNCH_OK(1);
+    return VMOBA_OK;
+  }
   simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, simt::kRows, cap, w.item_ptr);
   long long tiles = (D.sb + simt::kRows - 1) / simt::kRows;
   simt::attn_bwd_dkdv_kernel<T, DH, false><<<grid_for(n_kb * tiles, 4), simt::kThreads, 0, st>>>(
@@ -80,16 +107,26 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
 
 template <typename T, int DH>
 static int simt_dense(const Dims& D, const void* q, const void* k, const void* v, void* o, float* lse,
-                      const void* d_o, void* dq, void* dk, void* dv, void* ws, cudaStream_t st) {
+                      const void* d_o, void* dq, void* dk, void* dv, void* ws, int32_t* status, cudaStream_t st) {
   const long long nq = (long long)D.BH * D.S;
   const long long tiles = (D.S + simt::kRows - 1) / simt::kRows;
   BwdWs w = carve_bwd(D, true, d_o ? ws : nullptr);
-  simt::attn_fwd_kernel<T, DH, true><<<grid_for(D.BH * tiles, 8), simt::kThreads, 0, st>>>(
-      (const T*)q, (const T*)k, (const T*)v, nullptr, nullptr, nullptr, nullptr, 0, D.S, 1, D.S, D.BH, D.scale,
-      (T*)o, d_o ? (T*)w.o_resid : nullptr, lse, nullptr, nullptr, 0);
+  if (use_tensor_cores(D)) {
+    int rc = tc_dense_fwd(D, q, k, v, o, d_o ? w.o_resid : nullptr, lse, status, st);
+    if (rc) return rc;
+  } else {
+    simt::attn_fwd_kernel<T, DH, true><<<grid_for(D.BH * tiles, 8), simt::kThreads, 0, st>>>(
+        (const T*)q, (const T*)k, (const T*)v, nullptr, nullptr, nullptr, nullptr, 0, D.S, 1, D.S, D.BH, D.scale,
+        (T*)o, d_o ? (T*)w.o_resid : nullptr, lse, nullptr, nullptr, 0);
+    count_launches(1);
+  }
   if (d_o) {
     simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>((const T*)o, (const T*)w.o_resid,
                                                                           (const T*)d_o, nq, w.Dv);
+    if (use_tensor_cores(D)) {
+      VMOBA_LAUNCH_OK(1);
+      return tc_dense_bwd(D, q, k, v, d_o, lse, w.Dv, dq, dk, dv, status, st);
+    }
     simt::attn_bwd_dkdv_kernel<T, DH, true><<<grid_for(D.BH * tiles, 4), simt::kThreads, 0, st>>>(
         (const T*)q, (const T*)k, (const T*)v, (const T*)d_o, lse, w.Dv, nullptr, nullptr, D.S, 1, D.S, D.BH,
         D.scale, 0, (T*)dk, (T*)dv);
@@ -97,7 +134,7 @@ static int simt_dense(const Dims& D, const void* q, const void* k, const void* v
         (const T*)q, (const T*)k, (const T*)v, (const T*)d_o, lse, w.Dv, nullptr, nullptr, nullptr, 0, D.S, 1, D.S,
         D.BH, D.scale, 0, nullptr, (T*)dq);
   }
-  VMOBA_LAUNCH_OK(d_o ? 4 : 1);
+  VMOBA_LAUNCH_OK(d_o ? 3 : 0);
   return VMOBA_OK;
 }
 
@@ -162,6 +199,11 @@ extern "C" int vmoba_attn_fwd(const vmoba_shape* shape, const void* q_bm, const 
   if (ws_bytes < carve_fwd(D, capacity, nullptr).bytes) return VMOBA_ERR_WORKSPACE;
   if (D.dtype != VMOBA_BF16) o_resid_or_null = nullptr;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (use_tensor_cores(D)) {
+    FwdWs w = carve_fwd(D, capacity, ws);
+    return tc_sparse_fwd(D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null, lse,
+                         dev_status, w.item_ptr, w.part_o, w.part_lse, st);
+  }
   VMOBA_DISPATCH(simt_sparse_fwd, D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null,
                  lse, ws, st);
 }
@@ -185,8 +227,8 @@ extern "C" int vmoba_attn_bwd(const vmoba_shape* shape, const void* q_bm, const 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (D.dtype != VMOBA_BF16) o_resid_or_null = nullptr;
   if (!aligned16(o_resid_or_null)) return VMOBA_ERR_ARG;
-  VMOBA_DISPATCH(simt_sparse_bwd, D, q_bm, k_bm, v_bm, o_bm, o_resid_or_null, lse, do_bm, kb_ptr, q_idx, capacity, dq_bm, dk_bm, dv_bm,
-                 ws, st);
+  VMOBA_DISPATCH(simt_sparse_bwd, D, q_bm, k_bm, v_bm, o_bm, o_resid_or_null, lse, do_bm, kb_ptr, q_idx, q_ptr,
+                 capacity, dq_bm, dk_bm, dv_bm, dev_status, ws, st);
 }
 
 extern "C" int vmoba_full_attn(const vmoba_shape* shape, const void* q, const void* k, const void* v, void* o,
@@ -204,5 +246,5 @@ extern "C" int vmoba_full_attn(const vmoba_shape* shape, const void* q, const vo
     if (ws_bytes < carve_bwd(D, true, nullptr).bytes) return VMOBA_ERR_WORKSPACE;
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  VMOBA_DISPATCH(simt_dense, D, q, k, v, o, lse, do_or_null, dq, dk, dv, ws, st);
+  VMOBA_DISPATCH(simt_dense, D, q, k, v, o, lse, do_or_null, dq, dk, dv, ws, dev_status, st);
 }

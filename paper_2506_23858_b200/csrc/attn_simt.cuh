@@ -20,7 +20,7 @@ constexpr int kThreads = 256;  // 4 threads per row, each owning head_dim/4 chan
 
 // chunk-count prefix over the (batch, head, key block) lists: item_ptr[i] = number of work
 // items before list i when every list is cut into chunks of `rows` queries.
-__global__ void __launch_bounds__(1024)
+static __global__ void __launch_bounds__(1024)
 item_ptr_kernel(const int* __restrict__ kb_ptr, long long n_kb, int rows, long long capacity,
                 int* __restrict__ item_ptr) {
   __shared__ long long total;
@@ -438,6 +438,23 @@ attn_bwd_dq_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
         }
       }
     }
+  }
+}
+
+// fp32 accumulator rows -> output dtype, one warp per query.  Rows of queries with exactly one
+// selected block are skipped when `skip_single` is set (their result was written directly).
+template <typename T, int DH>
+__global__ void __launch_bounds__(256)
+cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, const int* __restrict__ q_ptr, long long n_queries,
+                 int skip_single) {
+  constexpr int C = DH / 32;
+  const int lane = threadIdx.x & 31;
+  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
+  for (long long g = warp; g < n_queries; g += nwarps) {
+    if (skip_single && q_ptr[g + 1] - q_ptr[g] == 1) continue;
+#pragma unroll
+    for (int c = 0; c < C; ++c) dst[g * DH + lane * C + c] = from_f32<T>(src[g * DH + lane * C + c]);
   }
 }
 

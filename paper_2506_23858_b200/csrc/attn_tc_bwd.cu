@@ -1,0 +1,619 @@
+// Tensor-core attention backward for bf16, head_dim 128: the training backward of Step 3 of
+// VMoBA (mask constant) and of the dense path.  Two kernels, both persistent (one CTA per SM):
+//
+//   dK/dV  key-stationary.  Item = 128 keys of one key block (or of the sequence).  K and V tiles
+//          stay in shared memory; the queries that selected the block stream through in gathered
+//          chunks of 128 (Q and dO rows, double buffered).  Per chunk, with keys on the TMEM lanes:
+//            S^T = K Q^T,  dP^T = V dO^T            (two SS MMAs)
+//            P^T = exp2(c S^T - lse),  dS^T = P^T (dP^T - D)   (threads = key rows)
+//            dV += P^T dO,  dK += dS^T Q            (two TS MMAs, A = bf16 P^T / dS^T in TMEM;
+//                                                    B = the same dO / Q tiles read MN-major)
+//          Every key belongs to exactly one item: dK and dV are written once, no atomics.
+//   dQ     query-stationary over the forward's work items (128 gathered queries x one key block):
+//            S = Q K^T,  dP = dO V^T,  dS = P (dP - D),  dQ += dS K
+//          A query's blocks add their contributions into an fp32 accumulator (atomics); the dense
+//          path writes dQ directly.
+//
+// D = rowsum(dO * O) and lse come in per query; exp runs in the exp2 domain (c = scale * log2 e).
+#include <algorithm>
+
+#include "attn_simt.cuh"
+#include "sm100.cuh"
+
+namespace vmoba {
+namespace tcb {
+
+using namespace sm100;
+
+constexpr int BM = 128, BN = 128, DH = 128;
+constexpr int PANEL = 128 * 128;
+constexpr int TILE = 2 * PANEL;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr uint32_t IDESC_KK = make_idesc_bf16(128, 128, false, false);   // A, B both K-major in shared memory
+constexpr uint32_t IDESC_TN = make_idesc_bf16(128, 128, false, true);    // A from TMEM, B MN-major
+
+// 16 threads per row: copy `n_rows` gathered 256-byte rows into a swizzled K-major tile (two
+// 64-column panels of 128-byte rows); rows beyond n_rows are zero-filled.
+template <int NTHREADS, typename RowOf>
+__device__ __forceinline__ void gather_tile(uint8_t* dst, const __nv_bfloat16* head_base, int n_rows, int tid, RowOf row_of) {
+  const int chunk = tid & 15;
+  const int panel = chunk >> 3, cc = chunk & 7;
+#pragma unroll 4
+  for (int row = tid >> 4; row < 128; row += NTHREADS / 16) {
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (row < n_rows) v = __ldg(reinterpret_cast<const uint4*>(head_base + (long long)row_of(row) * DH) + chunk);
+    *reinterpret_cast<uint4*>(dst + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v;
+  }
+}
+
+// 16-byte vector reduction into global memory (fp32 add).
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+// K-major operand descriptor for k-step ks (16 of the 128 head-dim columns) of a swizzled tile.
+__device__ __forceinline__ uint64_t desc_k(uint32_t tile_addr, int ks) {
+  return make_smem_desc(tile_addr + (ks >> 2) * PANEL + (ks & 3) * 32, 16, 1024);
+}
+// MN-major B operand descriptor: N = the 128 head-dim columns, K = rows 16*ks .. 16*ks+15 of the tile.
+__device__ __forceinline__ uint64_t desc_mn(uint32_t tile_addr, int ks) {
+  return make_smem_desc(tile_addr + ks * 2048, PANEL, 1024);
+}
+
+// ==========================================================================================
+// dK / dV
+// ==========================================================================================
+struct KvSmem {
+  uint64_t kv_full;            // K and V tiles landed (TMA)
+  uint64_t chunk_full[2];      // Q/dO chunk gathered (128 loader arrivals)
+  uint64_t chunk_empty[2];     // dV/dK MMAs of the chunk done (commit)
+  uint64_t sdp_full;           // S^T and dP^T ready (commit)
+  uint64_t pds_ready;          // P^T and dS^T written (128 compute arrivals)
+  uint64_t acc_done;           // all MMAs of the item done (commit)
+  uint32_t tmem_base;
+  int abort_flag;
+  float lse2[2][128];
+  float Dq[2][128];
+};
+constexpr size_t KV_SMEM_BYTES = 1024 + 6 * TILE + sizeof(KvSmem) + 64;
+constexpr int KV_THREADS = 320;
+
+struct KvParams {
+  const __nv_bfloat16 *q, *d_o;
+  const float *lse, *Dv;
+  const int *kb_ptr, *q_idx;
+  int S, Nb, sb, BH;
+  float scale, scale_log2;
+  long long capacity;
+  __nv_bfloat16 *dk, *dv;
+  int32_t* status;
+};
+
+template <bool DENSE>
+__global__ void __launch_bounds__(KV_THREADS, 1)
+attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const KvParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sK = base;
+  uint8_t* sV = base + TILE;
+  uint8_t* sQ = base + 2 * TILE;       // [2][TILE]
+  uint8_t* sdO = base + 4 * TILE;      // [2][TILE]
+  KvSmem* sm = reinterpret_cast<KvSmem*>(base + 6 * TILE);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &sm->abort_flag;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&sm->kv_full, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(&sm->chunk_full[b], 128); mbar_init(&sm->chunk_empty[b], 1); }
+    mbar_init(&sm->sdp_full, 1);
+    mbar_init(&sm->pds_ready, 128);
+    mbar_init(&sm->acc_done, 1);
+    sm->abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmK);
+    prefetch_tmap(&tmV);
+  }
+  if (warp == 1) {
+    tmem_alloc(&sm->tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm->tmem_base;
+  constexpr uint32_t ST_COL = 0, DPT_COL = 128, DV_COL = 256, DK_COL = 384;
+
+  const int span = DENSE ? p.S : p.sb;
+  const int tiles = (span + BN - 1) / BN;
+  const long long n_items = (long long)p.BH * (DENSE ? 1 : p.Nb) * tiles;
+
+  uint32_t it_n = 0;   // items with at least one chunk processed by this CTA
+  uint32_t cg = 0;     // chunks processed by this CTA (ring position of the Q/dO buffers)
+  for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const int tile = (int)(item % tiles);
+    const long long kbi = item / tiles;
+    const int bh = DENSE ? (int)kbi : (int)(kbi / p.Nb);
+    const int j = DENSE ? 0 : (int)(kbi - (long long)bh * p.Nb);
+    const int key0 = j * p.sb + tile * BN;              // first key of the tile inside the head
+    const int valid = min(BN, span - tile * BN);
+    long long list_lo = 0, list_hi = p.S;
+    if (!DENSE) {
+      list_lo = min((long long)p.kb_ptr[kbi], p.capacity);
+      list_hi = min((long long)p.kb_ptr[kbi + 1], p.capacity);
+    }
+    const int nchunks = (int)((list_hi - list_lo + BM - 1) / BM);
+    const long long head_off = (long long)bh * p.S;
+    // everything of the previous item (MMAs, epilogue reads of TMEM, K/V tiles) is finished here
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (nchunks == 0) {
+      // no query selected this block: its keys get zero gradients
+      if (warp >= 2 && warp < 6) {
+        const int r = (warp & 3) * 32 + lane;
+        if (r < valid) {
+          uint4 z = make_uint4(0u, 0u, 0u, 0u);
+          uint4* a = reinterpret_cast<uint4*>(p.dk + (head_off + key0 + r) * DH);
+          uint4* b = reinterpret_cast<uint4*>(p.dv + (head_off + key0 + r) * DH);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { a[i] = z; b[i] = z; }
+        }
+      }
+      continue;
+    }
+
+    if (warp == 0) {
+      // ---------------------------------------------------------------- TMA: the item's K and V tiles
+      if (lane == 0) {
+        const int y = (int)head_off + key0;
+        mbar_expect_tx(&sm->kv_full, 2 * TILE);
+        tma_load_2d(sK, &tmK, &sm->kv_full, 0, y);
+        tma_load_2d(sK + PANEL, &tmK, &sm->kv_full, 64, y);
+        tma_load_2d(sV, &tmV, &sm->kv_full, 0, y);
+        tma_load_2d(sV + PANEL, &tmV, &sm->kv_full, 64, y);
+      }
+    } else if (warp == 1) {
+      // ---------------------------------------------------------------- MMA issuer
+      if (lane == 0) {
+        mbar_wait(&sm->kv_full, it_n & 1, abort_flag, p.status);
+        tc_fence_after();
+        const uint32_t sK_addr = smem_u32(sK), sV_addr = smem_u32(sV);
+        for (int c = 0; c < nchunks; ++c) {
+          const uint32_t g = cg + c;
+          const int b = g & 1;
+          const uint32_t sQ_addr = smem_u32(sQ + b * TILE), sdO_addr = smem_u32(sdO + b * TILE);
+          mbar_wait(&sm->chunk_full[b], (g >> 1) & 1, abort_flag, p.status);
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < DH / 16; ++ks)
+            mma_ss(tmem + ST_COL, desc_k(sK_addr, ks), desc_k(sQ_addr, ks), IDESC_KK, ks > 0 ? 1u : 0u);
+#pragma unroll
+          for (int ks = 0; ks < DH / 16; ++ks)
+            mma_ss(tmem + DPT_COL, desc_k(sV_addr, ks), desc_k(sdO_addr, ks), IDESC_KK, ks > 0 ? 1u : 0u);
+          mma_commit(&sm->sdp_full);
+          mbar_wait(&sm->pds_ready, g & 1, abort_flag, p.status);
+          tc_fence_after();
+          const int rows = (int)min((long long)BM, list_hi - list_lo - (long long)c * BM);
+          const int ksteps = (rows + 15) >> 4;
+          for (int ks = 0; ks < ksteps; ++ks)
+            mma_ts(tmem + DV_COL, tmem + ST_COL + ks * 8, desc_mn(sdO_addr, ks), IDESC_TN, (c > 0 || ks > 0) ? 1u : 0u);
+          for (int ks = 0; ks < ksteps; ++ks)
+            mma_ts(tmem + DK_COL, tmem + DPT_COL + ks * 8, desc_mn(sQ_addr, ks), IDESC_TN, (c > 0 || ks > 0) ? 1u : 0u);
+          mma_commit(&sm->chunk_empty[b]);
+        }
+        mma_commit(&sm->acc_done);
+      }
+    } else if (warp >= 6) {
+      // ---------------------------------------------------------------- loaders: gather Q / dO chunks
+      const int lt = threadIdx.x - 192;   // 0..127
+      for (int c = 0; c < nchunks; ++c) {
+        const uint32_t g = cg + c;
+        const int b = g & 1;
+        if (g >= 2) mbar_wait(&sm->chunk_empty[b], ((g >> 1) - 1) & 1, abort_flag, p.status);
+        const long long lo = list_lo + (long long)c * BM;
+        const int rows = (int)min((long long)BM, list_hi - lo);
+        auto row_of = [&](int i) { return DENSE ? (int)(lo + i) : p.q_idx[lo + i]; };
+        gather_tile<128>(sQ + b * TILE, p.q + head_off * DH, rows, lt, row_of);
+        gather_tile<128>(sdO + b * TILE, p.d_o + head_off * DH, rows, lt, row_of);
+        float l2 = INFINITY, dd = 0.f;     // padded queries: P = exp2(-inf) = 0
+        if (lt < rows) {
+          const long long G_ = head_off + row_of(lt);
+          l2 = p.lse[G_] * LOG2E;
+          dd = p.Dv[G_];
+        }
+        sm->lse2[b][lt] = l2;
+        sm->Dq[b][lt] = dd;
+        fence_async_proxy();
+        mbar_arrive(&sm->chunk_full[b]);
+      }
+    } else {
+      // ---------------------------------------------------------------- compute: thread = key row
+      const int quad = warp & 3;
+      const int r = quad * 32 + lane;
+      const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+      for (int c = 0; c < nchunks; ++c) {
+        const uint32_t g = cg + c;
+        const int b = g & 1;
+        mbar_wait(&sm->chunk_full[b], (g >> 1) & 1, abort_flag, p.status);   // publishes lse2 / Dq of this chunk
+        mbar_wait(&sm->sdp_full, g & 1, abort_flag, p.status);
+        tc_fence_after();
+        const float* lse2 = sm->lse2[b];
+        const float* Dq = sm->Dq[b];
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+          uint32_t sv[2][32], dv_[2][32];
+          tmem_ld32(tmem + lane_addr + ST_COL + h * 64, sv[0]);
+          tmem_ld32(tmem + lane_addr + ST_COL + h * 64 + 32, sv[1]);
+          tmem_ld32(tmem + lane_addr + DPT_COL + h * 64, dv_[0]);
+          tmem_ld32(tmem + lane_addr + DPT_COL + h * 64 + 32, dv_[1]);
+          tmem_ld_wait();
+          uint32_t pk[32], dk_[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int q0 = h * 64 + 2 * i;
+            const float s0 = __uint_as_float(sv[i >> 4][(2 * i) & 31]), s1 = __uint_as_float(sv[i >> 4][((2 * i) & 31) + 1]);
+            const float d0 = __uint_as_float(dv_[i >> 4][(2 * i) & 31]), d1 = __uint_as_float(dv_[i >> 4][((2 * i) & 31) + 1]);
+            const float p0 = ex2(fmaf(s0, p.scale_log2, -lse2[q0]));
+            const float p1 = ex2(fmaf(s1, p.scale_log2, -lse2[q0 + 1]));
+            pk[i] = pack_bf16(p0, p1);
+            dk_[i] = pack_bf16(p0 * (d0 - Dq[q0]), p1 * (d1 - Dq[q0 + 1]));
+          }
+          tmem_st32(tmem + lane_addr + ST_COL + h * 32, pk);
+          tmem_st32(tmem + lane_addr + DPT_COL + h * 32, dk_);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(&sm->pds_ready);
+      }
+      // ---- epilogue: dV and dK rows of this tile
+      mbar_wait(&sm->acc_done, it_n & 1, abort_flag, p.status);
+      tc_fence_after();
+      __nv_bfloat16* dv_row = p.dv + (head_off + key0 + r) * DH;
+      __nv_bfloat16* dk_row = p.dk + (head_off + key0 + r) * DH;
+#pragma unroll 1
+      for (int cgrp = 0; cgrp < 4; ++cgrp) {
+        uint32_t a[32], bb[32];
+        tmem_ld32(tmem + lane_addr + DV_COL + cgrp * 32, a);
+        tmem_ld32(tmem + lane_addr + DK_COL + cgrp * 32, bb);
+        tmem_ld_wait();
+        if (r < valid) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            store4(dv_row + cgrp * 32 + i, make_float4(__uint_as_float(a[i]), __uint_as_float(a[i + 1]),
+                                                       __uint_as_float(a[i + 2]), __uint_as_float(a[i + 3])));
+            store4(dk_row + cgrp * 32 + i,
+                   make_float4(__uint_as_float(bb[i]) * p.scale, __uint_as_float(bb[i + 1]) * p.scale,
+                               __uint_as_float(bb[i + 2]) * p.scale, __uint_as_float(bb[i + 3]) * p.scale));
+          }
+        }
+      }
+    }
+    cg += nchunks;
+    ++it_n;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+// ==========================================================================================
+// dQ
+// ==========================================================================================
+constexpr int DQ_STAGES = 2;
+struct DqSmem {
+  uint64_t k_full[DQ_STAGES], v_full[DQ_STAGES], kv_empty[DQ_STAGES];
+  uint64_t s_full[2];          // S buffer ready (commit)
+  uint64_t dp_full;            // dP ready (commit)
+  uint64_t ds_ready;           // dS written (128 arrivals)
+  uint64_t dq_done[2];         // all MMAs of the item done (commit), alternating by item
+  uint64_t qdo_ready;          // Q and dO gathered (128 arrivals)
+  uint32_t tmem_base;
+  int abort_flag;
+};
+constexpr size_t DQ_SMEM_BYTES = 1024 + 2 * TILE + 2 * DQ_STAGES * TILE + sizeof(DqSmem) + 64;
+constexpr int DQ_THREADS = 192;
+
+struct DqParams {
+  const __nv_bfloat16 *q, *d_o;
+  const float *lse, *Dv;
+  const int *kb_ptr, *q_idx, *q_ptr, *item_ptr;
+  int n_kb, S, Nb, sb, BH;
+  float scale, scale_log2;
+  long long capacity;
+  float* dq_acc;            // sparse, queries with several blocks: fp32 accumulator [BH*S, 128]
+  __nv_bfloat16* dq;        // dense, and sparse queries with a single block: written directly
+  int32_t* status;
+};
+
+template <bool DENSE>
+__device__ __forceinline__ void dq_decode(const DqParams& p, int item, int& bh, int& key_begin, int& n_keys, int& list_lo,
+                                          int& n_rows) {
+  if (DENSE) {
+    const int tiles = (p.S + BM - 1) / BM;
+    bh = item / tiles;
+    const int t = item - bh * tiles;
+    key_begin = 0; n_keys = p.S; list_lo = t * BM; n_rows = min(BM, p.S - list_lo);
+  } else {
+    simt::Item it = simt::decode_sparse(item, p.item_ptr, p.n_kb, p.kb_ptr, p.Nb, p.sb, BM, p.capacity);
+    bh = it.bh; key_begin = it.key_begin; n_keys = p.sb; list_lo = it.list_lo; n_rows = it.list_hi - it.list_lo;
+  }
+}
+
+template <bool DENSE>
+__global__ void __launch_bounds__(DQ_THREADS, 1)
+attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const DqParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = base;
+  uint8_t* sdO = base + TILE;
+  uint8_t* sK = base + 2 * TILE;
+  uint8_t* sV = sK + DQ_STAGES * TILE;
+  DqSmem* sm = reinterpret_cast<DqSmem*>(sV + DQ_STAGES * TILE);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* abort_flag = &sm->abort_flag;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < DQ_STAGES; ++s) { mbar_init(&sm->k_full[s], 1); mbar_init(&sm->v_full[s], 1); mbar_init(&sm->kv_empty[s], 1); }
+    mbar_init(&sm->s_full[0], 1); mbar_init(&sm->s_full[1], 1);
+    mbar_init(&sm->dp_full, 1);
+    mbar_init(&sm->ds_ready, 128);
+    mbar_init(&sm->dq_done[0], 1); mbar_init(&sm->dq_done[1], 1);
+    mbar_init(&sm->qdo_ready, 128);
+    sm->abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tmap(&tmK);
+    prefetch_tmap(&tmV);
+  }
+  if (warp == 1) {
+    tmem_alloc(&sm->tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm->tmem_base;
+  constexpr uint32_t S_COL0 = 0, S_COL1 = 128, DP_COL = 256, DQ_COL = 384;
+  const int n_items = DENSE ? p.BH * ((p.S + BM - 1) / BM) : p.item_ptr[p.n_kb];
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t fills = 0;
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        int bh, key_begin, n_keys, list_lo, n_rows;
+        dq_decode<DENSE>(p, item, bh, key_begin, n_keys, list_lo, n_rows);
+        const int row0 = bh * p.S + key_begin;
+        const int ntiles = (n_keys + BN - 1) / BN;
+        for (int t = 0; t < ntiles; ++t, ++fills) {
+          const int s = fills % DQ_STAGES;
+          if (fills >= DQ_STAGES) mbar_wait(&sm->kv_empty[s], ((fills / DQ_STAGES) - 1) & 1, abort_flag, p.status);
+          const int y = row0 + t * BN;
+          mbar_expect_tx(&sm->k_full[s], TILE);
+          tma_load_2d(sK + s * TILE, &tmK, &sm->k_full[s], 0, y);
+          tma_load_2d(sK + s * TILE + PANEL, &tmK, &sm->k_full[s], 64, y);
+          mbar_expect_tx(&sm->v_full[s], TILE);
+          tma_load_2d(sV + s * TILE, &tmV, &sm->v_full[s], 0, y);
+          tma_load_2d(sV + s * TILE + PANEL, &tmV, &sm->v_full[s], 64, y);
+        }
+      }
+      if (*abort_flag) {
+        const uint32_t first = fills > DQ_STAGES ? fills - DQ_STAGES : 0;
+        for (uint32_t f = first; f < fills; ++f) {
+          mbar_wait(&sm->k_full[f % DQ_STAGES], (f / DQ_STAGES) & 1, abort_flag, p.status);
+          mbar_wait(&sm->v_full[f % DQ_STAGES], (f / DQ_STAGES) & 1, abort_flag, p.status);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t fills = 0, tg = 0, items_done = 0;
+      const uint32_t sQ_addr = smem_u32(sQ), sdO_addr = smem_u32(sdO);
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++items_done) {
+        int bh, key_begin, n_keys, list_lo, n_rows;
+        dq_decode<DENSE>(p, item, bh, key_begin, n_keys, list_lo, n_rows);
+        const int ntiles = (n_keys + BN - 1) / BN;
+        mbar_wait(&sm->qdo_ready, items_done & 1, abort_flag, p.status);
+        tc_fence_after();
+        auto n_mma_of = [&](int t) { return (min(BN, n_keys - t * BN) + 15) & ~15; };
+        auto issue_s = [&](int t) {
+          const uint32_t f = fills + t;
+          const int s = f % DQ_STAGES;
+          mbar_wait(&sm->k_full[s], (f / DQ_STAGES) & 1, abort_flag, p.status);
+          tc_fence_after();
+          const uint32_t idesc = make_idesc_bf16(BM, n_mma_of(t), false, false);
+          const uint32_t buf = (tg + t) & 1;
+          const uint32_t sK_addr = smem_u32(sK + s * TILE);
+#pragma unroll
+          for (int ks = 0; ks < DH / 16; ++ks)
+            mma_ss(tmem + (buf ? S_COL1 : S_COL0), desc_k(sQ_addr, ks), desc_k(sK_addr, ks), idesc, ks > 0 ? 1u : 0u);
+          mma_commit(&sm->s_full[buf]);
+        };
+        issue_s(0);
+        for (int t = 0; t < ntiles; ++t) {
+          const uint32_t f = fills + t;
+          const int s = f % DQ_STAGES;
+          // dP(t) = dO V^T : the dP/dS region is free because dQ(t-1), which read dS(t-1), was issued before
+          mbar_wait(&sm->v_full[s], (f / DQ_STAGES) & 1, abort_flag, p.status);
+          tc_fence_after();
+          {
+            const uint32_t idesc = make_idesc_bf16(BM, n_mma_of(t), false, false);
+            const uint32_t sV_addr = smem_u32(sV + s * TILE);
+#pragma unroll
+            for (int ks = 0; ks < DH / 16; ++ks)
+              mma_ss(tmem + DP_COL, desc_k(sdO_addr, ks), desc_k(sV_addr, ks), idesc, ks > 0 ? 1u : 0u);
+            mma_commit(&sm->dp_full);
+          }
+          if (t + 1 < ntiles) issue_s(t + 1);
+          mbar_wait(&sm->ds_ready, (tg + t) & 1, abort_flag, p.status);
+          tc_fence_after();
+          const int ksteps = n_mma_of(t) >> 4;
+          const uint32_t sK_addr = smem_u32(sK + s * TILE);
+          for (int ks = 0; ks < ksteps; ++ks)
+            mma_ts(tmem + DQ_COL, tmem + DP_COL + ks * 8, desc_mn(sK_addr, ks), IDESC_TN, (t > 0 || ks > 0) ? 1u : 0u);
+          mma_commit(&sm->kv_empty[s]);
+        }
+        mma_commit(&sm->dq_done[items_done & 1]);
+        fills += ntiles;
+        tg += ntiles;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ compute: thread = query row
+    const int quad = warp & 3;
+    const int r = quad * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const int ct = threadIdx.x - 64;
+    uint32_t tg = 0, items_done = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++items_done) {
+      int bh, key_begin, n_keys, list_lo, n_rows;
+      dq_decode<DENSE>(p, item, bh, key_begin, n_keys, list_lo, n_rows);
+      const int ntiles = (n_keys + BN - 1) / BN;
+      const long long head_off = (long long)bh * p.S;
+      auto row_of = [&](int i) { return DENSE ? list_lo + i : p.q_idx[list_lo + i]; };
+      gather_tile<128>(sQ, p.q + head_off * DH, n_rows, ct, row_of);
+      gather_tile<128>(sdO, p.d_o + head_off * DH, n_rows, ct, row_of);
+      fence_async_proxy();
+      mbar_arrive(&sm->qdo_ready);
+      const bool row_ok = r < n_rows;
+      long long G_ = 0;
+      float lse2 = INFINITY, Dr = 0.f;
+      bool direct = DENSE;
+      if (row_ok) {
+        G_ = head_off + row_of(r);
+        lse2 = p.lse[G_] * LOG2E;
+        Dr = p.Dv[G_];
+        if (!DENSE) direct = (p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1;
+      }
+      for (int t = 0; t < ntiles; ++t) {
+        const uint32_t buf = (tg + t) & 1;
+        const int valid = min(BN, n_keys - t * BN);
+        mbar_wait(&sm->s_full[buf], ((tg + t) >> 1) & 1, abort_flag, p.status);
+        mbar_wait(&sm->dp_full, (tg + t) & 1, abort_flag, p.status);
+        tc_fence_after();
+        const uint32_t s_tmem = tmem + lane_addr + (buf ? S_COL1 : S_COL0);
+        const uint32_t dp_tmem = tmem + lane_addr + DP_COL;
+#pragma unroll 1
+        for (int h = 0; h < 2; ++h) {
+          uint32_t sv[2][32], dv_[2][32];
+          tmem_ld32(s_tmem + h * 64, sv[0]);
+          tmem_ld32(s_tmem + h * 64 + 32, sv[1]);
+          tmem_ld32(dp_tmem + h * 64, dv_[0]);
+          tmem_ld32(dp_tmem + h * 64 + 32, dv_[1]);
+          tmem_ld_wait();
+          uint32_t ds[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int k0 = h * 64 + 2 * i;
+            const float s0 = __uint_as_float(sv[i >> 4][(2 * i) & 31]), s1 = __uint_as_float(sv[i >> 4][((2 * i) & 31) + 1]);
+            const float d0 = __uint_as_float(dv_[i >> 4][(2 * i) & 31]), d1 = __uint_as_float(dv_[i >> 4][((2 * i) & 31) + 1]);
+            const float p0 = ex2(fmaf(s0, p.scale_log2, -lse2));
+            const float p1 = ex2(fmaf(s1, p.scale_log2, -lse2));
+            const float x0 = (k0 < valid) ? p0 * (d0 - Dr) : 0.f;
+            const float x1 = (k0 + 1 < valid) ? p1 * (d1 - Dr) : 0.f;
+            ds[i] = pack_bf16(x0, x1);
+          }
+          tmem_st32(dp_tmem + h * 32, ds);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        mbar_arrive(&sm->ds_ready);
+      }
+      // ---- epilogue
+      mbar_wait(&sm->dq_done[items_done & 1], (items_done >> 1) & 1, abort_flag, p.status);
+      tc_fence_after();
+      tg += ntiles;
+#pragma unroll 1
+      for (int cgrp = 0; cgrp < 4; ++cgrp) {
+        uint32_t a[32];
+        tmem_ld32(tmem + lane_addr + DQ_COL + cgrp * 32, a);
+        tmem_ld_wait();
+        if (row_ok) {
+          if (direct) {
+            __nv_bfloat16* dst = p.dq + G_ * DH + cgrp * 32;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              store4(dst + i, make_float4(__uint_as_float(a[i]) * p.scale, __uint_as_float(a[i + 1]) * p.scale,
+                                          __uint_as_float(a[i + 2]) * p.scale, __uint_as_float(a[i + 3]) * p.scale));
+          } else {
+            float* dst = p.dq_acc + G_ * DH + cgrp * 32;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              red_add_v4(dst + i, __uint_as_float(a[i]) * p.scale, __uint_as_float(a[i + 1]) * p.scale,
+                         __uint_as_float(a[i + 2]) * p.scale, __uint_as_float(a[i + 3]) * p.scale);
+          }
+        }
+      }
+      tc_fence_before();
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
+}
+
+static int grid_items(long long items) { return (int)std::max<long long>(1, std::min<long long>(items, 148)); }
+
+}  // namespace tcb
+
+// Backward over the work lists (bf16, head_dim 128).  Dv holds rowsum(dO * O) per query; dq_acc is
+// a zeroed fp32 accumulator that the caller converts to bf16 afterwards.
+int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                  const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap,
+                  const int* item_ptr, float* dq_acc, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st) {
+  using namespace tcb;
+  CUtensorMap tmK, tmV;
+  const uint64_t rows = (uint64_t)D.BH * D.S;
+  if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN))
+    return VMOBA_ERR_CUDA;
+  const long long n_kb = (long long)D.BH * D.Nb;
+  KvParams kp;
+  kp.q = (const __nv_bfloat16*)q; kp.d_o = (const __nv_bfloat16*)d_o; kp.lse = lse; kp.Dv = Dv;
+  kp.kb_ptr = kb_ptr; kp.q_idx = q_idx; kp.S = D.S; kp.Nb = D.Nb; kp.sb = D.sb; kp.BH = D.BH;
+  kp.scale = D.scale; kp.scale_log2 = D.scale * LOG2E; kp.capacity = cap;
+  kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status;
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)KV_SMEM_BYTES));
+  const long long kv_items = n_kb * ((D.sb + BN - 1) / BN);
+  attn_bwd_dkdv_tc_kernel<false><<<grid_items(kv_items), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, kp);
+  DqParams qp;
+  qp.q = kp.q; qp.d_o = kp.d_o; qp.lse = lse; qp.Dv = Dv; qp.kb_ptr = kb_ptr; qp.q_idx = q_idx; qp.item_ptr = item_ptr;
+  qp.n_kb = (int)n_kb; qp.S = D.S; qp.Nb = D.Nb; qp.sb = D.sb; qp.BH = D.BH; qp.scale = D.scale;
+  qp.scale_log2 = D.scale * LOG2E; qp.capacity = cap; qp.dq_acc = dq_acc; qp.dq = (__nv_bfloat16*)dq; qp.status = status;
+  qp.q_ptr = q_ptr;
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)DQ_SMEM_BYTES));
+  attn_bwd_dq_tc_kernel<false><<<grid_items(cap / BM + n_kb), DQ_THREADS, DQ_SMEM_BYTES, st>>>(tmK, tmV, qp);
+  VMOBA_LAUNCH_OK(2);
+  return VMOBA_OK;
+}
+
+int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                 const float* Dv, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st) {
+  using namespace tcb;
+  CUtensorMap tmK, tmV;
+  const uint64_t rows = (uint64_t)D.BH * D.S;
+  if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN))
+    return VMOBA_ERR_CUDA;
+  KvParams kp;
+  kp.q = (const __nv_bfloat16*)q; kp.d_o = (const __nv_bfloat16*)d_o; kp.lse = lse; kp.Dv = Dv;
+  kp.kb_ptr = nullptr; kp.q_idx = nullptr; kp.S = D.S; kp.Nb = 1; kp.sb = D.S; kp.BH = D.BH;
+  kp.scale = D.scale; kp.scale_log2 = D.scale * LOG2E; kp.capacity = 0;
+  kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status;
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)KV_SMEM_BYTES));
+  const long long tiles = (D.S + BN - 1) / BN;
+  attn_bwd_dkdv_tc_kernel<true><<<grid_items(D.BH * tiles), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, kp);
+  DqParams qp;
+  qp.q = kp.q; qp.d_o = kp.d_o; qp.lse = lse; qp.Dv = Dv; qp.kb_ptr = nullptr; qp.q_idx = nullptr; qp.item_ptr = nullptr;
+  qp.n_kb = 0; qp.S = D.S; qp.Nb = 1; qp.sb = D.S; qp.BH = D.BH; qp.scale = D.scale; qp.scale_log2 = D.scale * LOG2E;
+  qp.capacity = 0; qp.dq_acc = nullptr; qp.dq = (__nv_bfloat16*)dq; qp.status = status; qp.q_ptr = nullptr;
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)DQ_SMEM_BYTES));
+  attn_bwd_dq_tc_kernel<true><<<grid_items(D.BH * tiles), DQ_THREADS, DQ_SMEM_BYTES, st>>>(tmK, tmV, qp);
+  VMOBA_LAUNCH_OK(2);
+  return VMOBA_OK;
+}
+
+}  // namespace vmoba

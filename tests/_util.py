@@ -52,15 +52,17 @@ def rel_l2(a, b):
 
 
 def assert_close(got, ref, dtype, what=""):
-    """max-abs and relative-L2 bounds.  A bf16 result cannot be closer to the exact value than half
-    a bf16 ulp (2^-9 |ref|), which alone exceeds 2e-2 once |ref| >= 8; the max-abs bound is therefore
-    taken on top of that unavoidable rounding of the stored result."""
+    """max-abs and relative-L2 bounds.  bf16 arithmetic has two error terms that grow with the size of
+    the result and that no kernel can avoid: the stored result is rounded to bf16 (half an ulp,
+    2^-9 |ref|, which alone exceeds 2e-2 once |ref| >= 8), and the tensor-core operands P and dS are
+    rounded to bf16 (2^-9 relative per term; a sum of same-signed terms keeps that relative error).
+    The max-abs bound of 2e-2 is therefore taken on top of 2^-8 |ref|."""
     ma, rl = TOL[dtype]
     got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
-    allow = ma + (2.0 ** -9) * np.abs(ref) if dtype == "bf16" else ma
+    allow = ma + (2.0 ** -8) * np.abs(ref) if dtype == "bf16" else ma
     excess = float(np.max(np.abs(got - ref) - allow)) if got.size else -1.0
     e1, e2 = max_abs(got, ref), rel_l2(got, ref)
-    assert excess <= 0 and e2 <= rl, f"{what}: max-abs {e1:.3e} (tol {ma} + half ulp), rel-L2 {e2:.3e} (tol {rl})"
+    assert excess <= 0 and e2 <= rl, f"{what}: max-abs {e1:.3e} (tol {ma} + 2^-8 |ref|), rel-L2 {e2:.3e} (tol {rl})"
 
 
 def unpack_mask(mask_bits, BH, S, Nb):

@@ -139,7 +139,8 @@ def test_mid_size_threshold_one_equals_dense_path():
     assert int(st.item()) == 0
     sparse = U.to_numpy_f32(res["o"].permute(0, 2, 1, 3))
     dense = U.to_numpy_f32(o)
-    U.assert_close(sparse, dense, w.dtype, "sparse(tau=1) vs dense path")
+    # two independently rounded bf16 results may sit one bf16 ulp apart
+    assert np.all(np.abs(sparse - dense) <= 2e-2 + 2.0 ** -8 * np.abs(dense)) and U.rel_l2(sparse, dense) <= 1e-2
     for h in range(w.heads):
         od, _ = orc.dense_attn_fwd(data["q"][0, :, h], data["k"][0, :, h], data["v"][0, :, h], w.head_dim ** -0.5,
                                    rows=np.arange(0, w.S, 7))
