@@ -221,14 +221,20 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
       {
         const int chunk = st & 15;                 // 16-byte chunk of the 256-byte row
         const int panel = chunk >> 3, cc = chunk & 7;
-#pragma unroll 4
-        for (int row = st >> 4; row < BM; row += 8) {
-          uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        uint4 v[16];                               // all loads in flight before the first store
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int row = (st >> 4) + 8 * i;
+          v[i] = make_uint4(0u, 0u, 0u, 0u);
           if (row < n_rows) {
             const int qpos = DENSE ? list_lo + row : p.q_idx[list_lo + row];
-            v = __ldg(reinterpret_cast<const uint4*>(p.q + (head_off + qpos) * DH) + chunk);
+            v[i] = __ldg(reinterpret_cast<const uint4*>(p.q + (head_off + qpos) * DH) + chunk);
           }
-          *reinterpret_cast<uint4*>(sQ + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v;
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int row = (st >> 4) + 8 * i;
+          *reinterpret_cast<uint4*>(sQ + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v[i];
         }
       }
       fence_async_proxy();

@@ -37,13 +37,21 @@ constexpr uint32_t IDESC_TN = make_idesc_bf16(128, 128, false, true);    // A fr
 // 64-column panels of 128-byte rows); rows beyond n_rows are zero-filled.
 template <int NTHREADS, typename RowOf>
 __device__ __forceinline__ void gather_tile(uint8_t* dst, const __nv_bfloat16* head_base, int n_rows, int tid, RowOf row_of) {
+  constexpr int PASSES = 128 / (NTHREADS / 16);
   const int chunk = tid & 15;
   const int panel = chunk >> 3, cc = chunk & 7;
-#pragma unroll 4
-  for (int row = tid >> 4; row < 128; row += NTHREADS / 16) {
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (row < n_rows) v = __ldg(reinterpret_cast<const uint4*>(head_base + (long long)row_of(row) * DH) + chunk);
-    *reinterpret_cast<uint4*>(dst + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v;
+  // issue every load of this thread before the first store: the gather is latency-bound otherwise
+  uint4 v[PASSES];
+#pragma unroll
+  for (int i = 0; i < PASSES; ++i) {
+    const int row = (tid >> 4) + i * (NTHREADS / 16);
+    v[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (row < n_rows) v[i] = __ldg(reinterpret_cast<const uint4*>(head_base + (long long)row_of(row) * DH) + chunk);
+  }
+#pragma unroll
+  for (int i = 0; i < PASSES; ++i) {
+    const int row = (tid >> 4) + i * (NTHREADS / 16);
+    *reinterpret_cast<uint4*>(dst + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v[i];
   }
 }
 
