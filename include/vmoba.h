@@ -104,7 +104,8 @@ int vmoba_partition(const vmoba_shape* shape, int inverse, const void* src, void
  * q_bm, k_bm are block-major.
  */
 int vmoba_block_scores(const vmoba_shape* shape, const void* q_bm, const void* k_bm,
-                       float* centroids, float* scores, void* ws, size_t ws_bytes, void* stream);
+                       float* centroids, float* scores, int32_t* dev_status, void* ws, size_t ws_bytes,
+                       void* stream);
 
 /*
  * Step 2b, Eq. 3 + Eq. 4: global threshold selection per (batch, head).

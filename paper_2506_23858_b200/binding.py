@@ -91,7 +91,7 @@ def lib():
     L.vmoba_partition.restype = ctypes.c_int
     L.vmoba_partition.argtypes = [sp, ctypes.c_int, vp, vp, ctypes.POINTER(i64), vp, vp, vp]
     L.vmoba_block_scores.restype = ctypes.c_int
-    L.vmoba_block_scores.argtypes = [sp, vp, vp, vp, vp, vp, sz, vp]
+    L.vmoba_block_scores.argtypes = [sp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.vmoba_select.restype = ctypes.c_int
     L.vmoba_select.argtypes = [sp, vp, ctypes.c_float, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp]
     L.vmoba_select_static.restype = ctypes.c_int
@@ -147,10 +147,10 @@ def vmoba_partition(shape, inverse, src, dst, raster_strides_bsh, perm=None, inv
                                  _ptr(inv_perm), _stream(stream)), "vmoba_partition")
 
 
-def vmoba_block_scores(shape, q_bm, k_bm, centroids, scores, ws=None, stream=None):
+def vmoba_block_scores(shape, q_bm, k_bm, centroids, scores, dev_status, ws, stream=None):
     p, n = _ws_args(ws)
-    _check(lib().vmoba_block_scores(ctypes.byref(shape), _ptr(q_bm), _ptr(k_bm), _ptr(centroids), _ptr(scores), p, n,
-                                    _stream(stream)), "vmoba_block_scores")
+    _check(lib().vmoba_block_scores(ctypes.byref(shape), _ptr(q_bm), _ptr(k_bm), _ptr(centroids), _ptr(scores),
+                                    _ptr(dev_status), p, n, _stream(stream)), "vmoba_block_scores")
 
 
 def vmoba_select(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity, k_per_head,

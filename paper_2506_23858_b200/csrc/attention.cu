@@ -8,6 +8,7 @@
 namespace vmoba {
 
 size_t select_ws_bytes(const Dims& D);   // select.cu
+size_t scores_ws_bytes(const Dims& D);   // scores.cu
 
 // attn_tc.cu: tensor-core forward kernels (bf16, head_dim 128)
 int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
@@ -173,7 +174,7 @@ extern "C" size_t vmoba_workspace_bytes(const vmoba_shape* shape, int stage, int
   if (make_dims(shape, &D)) return 0;
   if (capacity < 0) return 0;
   switch (stage) {
-    case VMOBA_STAGE_SCORES: return 256;
+    case VMOBA_STAGE_SCORES: return scores_ws_bytes(D);
     case VMOBA_STAGE_SELECT: return select_ws_bytes(D);
     case VMOBA_STAGE_ATTN_FWD: return carve_fwd(D, capacity, nullptr).bytes;
     case VMOBA_STAGE_ATTN_BWD: return carve_bwd(D, false, nullptr).bytes;

@@ -9,6 +9,15 @@
 
 namespace vmoba {
 
+// scores_tc.cu: tensor-core scores for bf16 / head_dim 128
+size_t scores_tc_ws_bytes(const Dims& D);
+int scores_tc(const Dims& D, const void* q_bm, const float* cent, float* scores, void* ws, int32_t* status,
+              cudaStream_t st);
+
+size_t scores_ws_bytes(const Dims& D) {
+  return (D.dtype == VMOBA_BF16 && D.d == 128) ? scores_tc_ws_bytes(D) : 256;
+}
+
 // One CTA per (batch, head, block): 256 threads = (256 / V) row lanes x V float4-column lanes.
 template <typename T, int DH>
 __global__ void __launch_bounds__(256)
@@ -107,9 +116,11 @@ scores_kernel(const T* __restrict__ q_bm, const float* __restrict__ cent, float*
 }
 
 template <typename T, int DH>
-static int run_scores(const Dims& D, const void* q, const void* k, float* cent, float* scores, cudaStream_t st) {
+static int run_scores(const Dims& D, const void* q, const void* k, float* cent, float* scores, void* ws,
+                      int32_t* status, cudaStream_t st) {
   centroid_kernel<T, DH><<<D.BH * D.Nb, 256, 0, st>>>(static_cast<const T*>(k), cent, D.sb);
   VMOBA_LAUNCH_OK(1);
+  if (D.dtype == VMOBA_BF16 && DH == 128) return scores_tc(D, q, cent, scores, ws, status, st);
   size_t smem = 2 * DH * (64 + 4) * sizeof(float);
   VMOBA_CUDA_OK(cudaFuncSetAttribute(scores_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid((D.S + 63) / 64, 1, D.BH);
@@ -123,18 +134,20 @@ static int run_scores(const Dims& D, const void* q, const void* k, float* cent, 
 using namespace vmoba;
 
 extern "C" int vmoba_block_scores(const vmoba_shape* shape, const void* q_bm, const void* k_bm,
-                                  float* centroids, float* scores, void* ws, size_t ws_bytes, void* stream) {
-  (void)ws; (void)ws_bytes;
+                                  float* centroids, float* scores, int32_t* dev_status, void* ws,
+                                  size_t ws_bytes, void* stream) {
   Dims D;
   int rc = make_dims(shape, &D);
   if (rc) return rc;
-  if (!q_bm || !k_bm || !centroids || !scores) return VMOBA_ERR_ARG;
-  if (!aligned16(q_bm) || !aligned16(k_bm) || !aligned16(centroids) || !aligned16(scores)) return VMOBA_ERR_ARG;
+  if (!q_bm || !k_bm || !centroids || !scores || !dev_status || !ws) return VMOBA_ERR_ARG;
+  if (!aligned16(q_bm) || !aligned16(k_bm) || !aligned16(centroids) || !aligned16(scores) || !aligned16(ws))
+    return VMOBA_ERR_ARG;
+  if (ws_bytes < scores_ws_bytes(D)) return VMOBA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (D.dtype == VMOBA_BF16) {
-    if (D.d == 128) return run_scores<__nv_bfloat16, 128>(D, q_bm, k_bm, centroids, scores, st);
-    return run_scores<__nv_bfloat16, 64>(D, q_bm, k_bm, centroids, scores, st);
+    if (D.d == 128) return run_scores<__nv_bfloat16, 128>(D, q_bm, k_bm, centroids, scores, ws, dev_status, st);
+    return run_scores<__nv_bfloat16, 64>(D, q_bm, k_bm, centroids, scores, ws, dev_status, st);
   }
-  if (D.d == 128) return run_scores<float, 128>(D, q_bm, k_bm, centroids, scores, st);
-  return run_scores<float, 64>(D, q_bm, k_bm, centroids, scores, st);
+  if (D.d == 128) return run_scores<float, 128>(D, q_bm, k_bm, centroids, scores, ws, dev_status, st);
+  return run_scores<float, 64>(D, q_bm, k_bm, centroids, scores, ws, dev_status, st);
 }

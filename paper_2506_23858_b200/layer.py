@@ -70,7 +70,7 @@ class VmobaLayer:
         vb.vmoba_partition(self.shape, int(inverse), src, dst, self.raster_strides(raster), perm, inv_perm)
 
     def block_scores(self):
-        vb.vmoba_block_scores(self.shape, self.q_bm, self.k_bm, self.centroids, self.scores, self.ws)
+        vb.vmoba_block_scores(self.shape, self.q_bm, self.k_bm, self.centroids, self.scores, self.dev_status, self.ws)
 
     def select(self, tau, scores=None):
         vb.vmoba_select(self.shape, self.scores if scores is None else scores, tau, self.mask_bits, self.kb_ptr,
