@@ -3,7 +3,7 @@
 //
 //   dK/dV  key-stationary.  Item = 128 keys of one key block (or of the sequence).  K and V tiles
 //          stay in shared memory; the queries that selected the block stream through in gathered
-//          chunks of 128 (Q and dO rows, double buffered).  Per chunk, with keys on the TMEM lanes:
+//          chunks of 64 (Q and dO rows, 3-deep ring).  Per chunk, with keys on the TMEM lanes:
 //            S^T = K Q^T,  dP^T = V dO^T            (two SS MMAs)
 //            P^T = exp2(c S^T - lse),  dS^T = P^T (dP^T - D)   (threads = key rows)
 //            dV += P^T dO,  dK += dS^T Q            (two TS MMAs, A = bf16 P^T / dS^T in TMEM;
@@ -72,20 +72,29 @@ __device__ __forceinline__ uint64_t desc_mn(uint32_t tile_addr, int ks) {
 // ==========================================================================================
 // dK / dV
 // ==========================================================================================
+// Units of 64 queries flow through a 3-deep ring of gathered (Q, dO) chunks; S^T / dP^T are double
+// buffered in TMEM (64 columns each), so the tensor pipe computes unit u+1 while the compute warps
+// turn unit u into P^T / dS^T.  K and V tiles are double buffered across items, and the loader and
+// TMA warps run ahead of the MMA warp across item boundaries.
+constexpr int QC = 64;                       // queries per unit
+constexpr int CPANEL = QC * 128;             // bytes of one 64-column panel of a 64-row chunk (8 KB)
+constexpr int CTILE = 2 * CPANEL;            // [64 x 128] bf16 (16 KB)
+constexpr int NQ = 3;                        // chunk ring depth
 struct KvSmem {
-  uint64_t kv_full;            // K and V tiles landed (TMA)
-  uint64_t chunk_full[2];      // Q/dO chunk gathered (128 loader arrivals)
-  uint64_t chunk_empty[2];     // dV/dK MMAs of the chunk done (commit)
-  uint64_t sdp_full;           // S^T and dP^T ready (commit)
-  uint64_t pds_ready;          // P^T and dS^T written (128 compute arrivals)
-  uint64_t acc_done;           // all MMAs of the item done (commit)
+  uint64_t kv_full[2], kv_empty[2];          // K+V tiles of an item (TMA / commit)
+  uint64_t chunk_full[NQ], chunk_empty[NQ];  // gathered Q/dO chunk (128 loader arrivals / commit)
+  uint64_t sdp_full[2];                      // S^T and dP^T of a unit ready (commit)
+  uint64_t pds_ready[2];                     // P^T and dS^T written (128 compute arrivals)
+  uint64_t acc_done;                         // all MMAs of the item done (commit)
+  uint64_t acc_free;                         // epilogue has read dV / dK (128 compute arrivals)
   uint32_t tmem_base;
   int abort_flag;
-  float lse2[2][128];
-  float Dq[2][128];
+  float lse2[NQ][QC];
+  float Dq[NQ][QC];
 };
-constexpr size_t KV_SMEM_BYTES = 1024 + 6 * TILE + sizeof(KvSmem) + 64;
+constexpr size_t KV_SMEM_BYTES = 1024 + 4 * TILE + NQ * 2 * CTILE + sizeof(KvSmem) + 32;
 constexpr int KV_THREADS = 320;
+constexpr uint32_t IDESC_K64 = make_idesc_bf16(128, QC, false, false);   // S^T, dP^T: N = 64 queries
 
 struct KvParams {
   const __nv_bfloat16 *q, *d_o;
@@ -98,25 +107,81 @@ struct KvParams {
   int32_t* status;
 };
 
+// 16 threads per row: gather `n_rows` (<= 64) 256-byte rows into a swizzled [64 x 128] chunk tile.
+template <typename RowOf>
+__device__ __forceinline__ void gather_chunk64(uint8_t* dst, const __nv_bfloat16* head_base, int n_rows, int tid, RowOf row_of,
+                                               uint4 (&v)[8]) {
+  const int chunk = tid & 15;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = (tid >> 4) + i * 8;
+    v[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (row < n_rows) v[i] = __ldg(reinterpret_cast<const uint4*>(head_base + (long long)row_of(row) * DH) + chunk);
+  }
+  (void)dst;
+}
+__device__ __forceinline__ void store_chunk64(uint8_t* dst, int tid, const uint4 (&v)[8]) {
+  const int chunk = tid & 15;
+  const int panel = chunk >> 3, cc = chunk & 7;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = (tid >> 4) + i * 8;
+    *reinterpret_cast<uint4*>(dst + panel * CPANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v[i];
+  }
+}
+// chunk tile as K-major B operand (N = 64 queries, K = head dim), k-step ks of 8
+__device__ __forceinline__ uint64_t cdesc_k(uint32_t tile_addr, int ks) {
+  return make_smem_desc(tile_addr + (ks >> 2) * CPANEL + (ks & 3) * 32, 16, 1024);
+}
+// chunk tile as MN-major B operand (N = head dim, K = 16 queries of k-step ks of 4)
+__device__ __forceinline__ uint64_t cdesc_mn(uint32_t tile_addr, int ks) {
+  return make_smem_desc(tile_addr + ks * 2048, CPANEL, 1024);
+}
+
+struct KvItem {
+  int bh, key0, valid, n_units;
+  long long list_lo, list_hi, head_off;
+};
+
+template <bool DENSE>
+__device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, int tiles, int span) {
+  KvItem it;
+  const int tile = (int)(item % tiles);
+  const long long kbi = item / tiles;
+  it.bh = DENSE ? (int)kbi : (int)(kbi / p.Nb);
+  const int j = DENSE ? 0 : (int)(kbi - (long long)it.bh * p.Nb);
+  it.key0 = j * p.sb + tile * BN;
+  it.valid = min(BN, span - tile * BN);
+  it.list_lo = 0; it.list_hi = p.S;
+  if (!DENSE) {
+    it.list_lo = min((long long)p.kb_ptr[kbi], p.capacity);
+    it.list_hi = min((long long)p.kb_ptr[kbi + 1], p.capacity);
+  }
+  it.n_units = (int)((it.list_hi - it.list_lo + QC - 1) / QC);
+  it.head_off = (long long)it.bh * p.S;
+  return it;
+}
+
 template <bool DENSE>
 __global__ void __launch_bounds__(KV_THREADS, 1)
 attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const KvParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sK = base;
-  uint8_t* sV = base + TILE;
-  uint8_t* sQ = base + 2 * TILE;       // [2][TILE]
-  uint8_t* sdO = base + 4 * TILE;      // [2][TILE]
-  KvSmem* sm = reinterpret_cast<KvSmem*>(base + 6 * TILE);
+  uint8_t* sK = base;                  // [2][TILE]
+  uint8_t* sV = base + 2 * TILE;       // [2][TILE]
+  uint8_t* sC = base + 4 * TILE;       // [NQ][Q chunk | dO chunk]
+  KvSmem* sm = reinterpret_cast<KvSmem*>(sC + NQ * 2 * CTILE);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm->abort_flag;
 
   if (threadIdx.x == 0) {
-    mbar_init(&sm->kv_full, 1);
-    for (int b = 0; b < 2; ++b) { mbar_init(&sm->chunk_full[b], 128); mbar_init(&sm->chunk_empty[b], 1); }
-    mbar_init(&sm->sdp_full, 1);
-    mbar_init(&sm->pds_ready, 128);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sm->kv_full[b], 1); mbar_init(&sm->kv_empty[b], 1);
+      mbar_init(&sm->sdp_full[b], 1); mbar_init(&sm->pds_ready[b], 128);
+    }
+    for (int b = 0; b < NQ; ++b) { mbar_init(&sm->chunk_full[b], 128); mbar_init(&sm->chunk_empty[b], 1); }
     mbar_init(&sm->acc_done, 1);
+    mbar_init(&sm->acc_free, 128);
     sm->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmK);
@@ -130,162 +195,173 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm->tmem_base;
-  constexpr uint32_t ST_COL = 0, DPT_COL = 128, DV_COL = 256, DK_COL = 384;
+  constexpr uint32_t ST_COL = 0, DPT_COL = 128, DV_COL = 256, DK_COL = 384;   // ST/DPT: two 64-column buffers each
 
   const int span = DENSE ? p.S : p.sb;
   const int tiles = (span + BN - 1) / BN;
   const long long n_items = (long long)p.BH * (DENSE ? 1 : p.Nb) * tiles;
 
-  uint32_t it_n = 0;   // items with at least one chunk processed by this CTA
-  uint32_t cg = 0;     // chunks processed by this CTA (ring position of the Q/dO buffers)
-  for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const int tile = (int)(item % tiles);
-    const long long kbi = item / tiles;
-    const int bh = DENSE ? (int)kbi : (int)(kbi / p.Nb);
-    const int j = DENSE ? 0 : (int)(kbi - (long long)bh * p.Nb);
-    const int key0 = j * p.sb + tile * BN;              // first key of the tile inside the head
-    const int valid = min(BN, span - tile * BN);
-    long long list_lo = 0, list_hi = p.S;
-    if (!DENSE) {
-      list_lo = min((long long)p.kb_ptr[kbi], p.capacity);
-      list_hi = min((long long)p.kb_ptr[kbi + 1], p.capacity);
-    }
-    const int nchunks = (int)((list_hi - list_lo + BM - 1) / BM);
-    const long long head_off = (long long)bh * p.S;
-    // everything of the previous item (MMAs, epilogue reads of TMEM, K/V tiles) is finished here
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    if (nchunks == 0) {
-      // no query selected this block: its keys get zero gradients
-      if (warp >= 2 && warp < 6) {
-        const int r = (warp & 3) * 32 + lane;
-        if (r < valid) {
-          uint4 z = make_uint4(0u, 0u, 0u, 0u);
-          uint4* a = reinterpret_cast<uint4*>(p.dk + (head_off + key0 + r) * DH);
-          uint4* b = reinterpret_cast<uint4*>(p.dv + (head_off + key0 + r) * DH);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) { a[i] = z; b[i] = z; }
-        }
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA: K and V tiles, one pair per item
+    if (lane == 0) {
+      uint32_t n = 0;
+      for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+        if (it.n_units == 0) continue;
+        const int b = n & 1;
+        if (n >= 2) mbar_wait(&sm->kv_empty[b], ((n >> 1) - 1) & 1, abort_flag, p.status);
+        const int y = (int)it.head_off + it.key0;
+        mbar_expect_tx(&sm->kv_full[b], 2 * TILE);
+        tma_load_2d(sK + b * TILE, &tmK, &sm->kv_full[b], 0, y);
+        tma_load_2d(sK + b * TILE + PANEL, &tmK, &sm->kv_full[b], 64, y);
+        tma_load_2d(sV + b * TILE, &tmV, &sm->kv_full[b], 0, y);
+        tma_load_2d(sV + b * TILE + PANEL, &tmV, &sm->kv_full[b], 64, y);
+        ++n;
       }
-      continue;
+      if (*abort_flag)
+        for (uint32_t f = n > 2 ? n - 2 : 0; f < n; ++f) mbar_wait(&sm->kv_full[f & 1], (f >> 1) & 1, abort_flag, p.status);
     }
-
-    if (warp == 0) {
-      // ---------------------------------------------------------------- TMA: the item's K and V tiles
-      if (lane == 0) {
-        const int y = (int)head_off + key0;
-        mbar_expect_tx(&sm->kv_full, 2 * TILE);
-        tma_load_2d(sK, &tmK, &sm->kv_full, 0, y);
-        tma_load_2d(sK + PANEL, &tmK, &sm->kv_full, 64, y);
-        tma_load_2d(sV, &tmV, &sm->kv_full, 0, y);
-        tma_load_2d(sV + PANEL, &tmV, &sm->kv_full, 64, y);
-      }
-    } else if (warp == 1) {
-      // ---------------------------------------------------------------- MMA issuer
-      if (lane == 0) {
-        mbar_wait(&sm->kv_full, it_n & 1, abort_flag, p.status);
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t n = 0, u0 = 0;      // items and units done so far
+      for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+        if (it.n_units == 0) continue;
+        const int b = n & 1;
+        mbar_wait(&sm->kv_full[b], (n >> 1) & 1, abort_flag, p.status);
         tc_fence_after();
-        const uint32_t sK_addr = smem_u32(sK), sV_addr = smem_u32(sV);
-        for (int c = 0; c < nchunks; ++c) {
-          const uint32_t g = cg + c;
-          const int b = g & 1;
-          const uint32_t sQ_addr = smem_u32(sQ + b * TILE), sdO_addr = smem_u32(sdO + b * TILE);
-          mbar_wait(&sm->chunk_full[b], (g >> 1) & 1, abort_flag, p.status);
+        const uint32_t sK_addr = smem_u32(sK + b * TILE), sV_addr = smem_u32(sV + b * TILE);
+        auto issue_sdp = [&](int i) {
+          const uint32_t u = u0 + i;
+          const int cb = u % NQ, tb = u & 1;
+          mbar_wait(&sm->chunk_full[cb], (u / NQ) & 1, abort_flag, p.status);
           tc_fence_after();
+          const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE), sdO_addr = sQ_addr + CTILE;
 #pragma unroll
           for (int ks = 0; ks < DH / 16; ++ks)
-            mma_ss(tmem + ST_COL, desc_k(sK_addr, ks), desc_k(sQ_addr, ks), IDESC_KK, ks > 0 ? 1u : 0u);
+            mma_ss(tmem + ST_COL + tb * QC, desc_k(sK_addr, ks), cdesc_k(sQ_addr, ks), IDESC_K64, ks > 0 ? 1u : 0u);
 #pragma unroll
           for (int ks = 0; ks < DH / 16; ++ks)
-            mma_ss(tmem + DPT_COL, desc_k(sV_addr, ks), desc_k(sdO_addr, ks), IDESC_KK, ks > 0 ? 1u : 0u);
-          mma_commit(&sm->sdp_full);
-          mbar_wait(&sm->pds_ready, g & 1, abort_flag, p.status);
+            mma_ss(tmem + DPT_COL + tb * QC, desc_k(sV_addr, ks), cdesc_k(sdO_addr, ks), IDESC_K64, ks > 0 ? 1u : 0u);
+          mma_commit(&sm->sdp_full[tb]);
+        };
+        issue_sdp(0);
+        for (int i = 0; i < it.n_units; ++i) {
+          if (i + 1 < it.n_units) issue_sdp(i + 1);
+          const uint32_t u = u0 + i;
+          const int cb = u % NQ, tb = u & 1;
+          mbar_wait(&sm->pds_ready[tb], (u >> 1) & 1, abort_flag, p.status);
+          // dV / dK still hold the previous item until its epilogue has read them
+          if (i == 0 && n > 0) mbar_wait(&sm->acc_free, (n - 1) & 1, abort_flag, p.status);
           tc_fence_after();
-          const int rows = (int)min((long long)BM, list_hi - list_lo - (long long)c * BM);
+          const int rows = (int)min((long long)QC, it.list_hi - it.list_lo - (long long)i * QC);
           const int ksteps = (rows + 15) >> 4;
+          const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE), sdO_addr = sQ_addr + CTILE;
           for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(tmem + DV_COL, tmem + ST_COL + ks * 8, desc_mn(sdO_addr, ks), IDESC_TN, (c > 0 || ks > 0) ? 1u : 0u);
+            mma_ts(tmem + DV_COL, tmem + ST_COL + tb * QC + ks * 8, cdesc_mn(sdO_addr, ks), IDESC_TN, (i > 0 || ks > 0) ? 1u : 0u);
           for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(tmem + DK_COL, tmem + DPT_COL + ks * 8, desc_mn(sQ_addr, ks), IDESC_TN, (c > 0 || ks > 0) ? 1u : 0u);
-          mma_commit(&sm->chunk_empty[b]);
+            mma_ts(tmem + DK_COL, tmem + DPT_COL + tb * QC + ks * 8, cdesc_mn(sQ_addr, ks), IDESC_TN, (i > 0 || ks > 0) ? 1u : 0u);
+          mma_commit(&sm->chunk_empty[cb]);
         }
+        mma_commit(&sm->kv_empty[b]);
         mma_commit(&sm->acc_done);
+        u0 += it.n_units;
+        ++n;
       }
-    } else if (warp >= 6) {
-      // ---------------------------------------------------------------- loaders: gather Q / dO chunks
-      const int lt = threadIdx.x - 192;   // 0..127
-      for (int c = 0; c < nchunks; ++c) {
-        const uint32_t g = cg + c;
-        const int b = g & 1;
-        if (g >= 2) mbar_wait(&sm->chunk_empty[b], ((g >> 1) - 1) & 1, abort_flag, p.status);
-        const long long lo = list_lo + (long long)c * BM;
-        const int rows = (int)min((long long)BM, list_hi - lo);
-        auto row_of = [&](int i) { return DENSE ? (int)(lo + i) : p.q_idx[lo + i]; };
-        gather_tile<128>(sQ + b * TILE, p.q + head_off * DH, rows, lt, row_of);
-        gather_tile<128>(sdO + b * TILE, p.d_o + head_off * DH, rows, lt, row_of);
+    }
+  } else if (warp >= 6) {
+    // ------------------------------------------------------------------ loaders: gather Q / dO chunks (run ahead)
+    const int lt = threadIdx.x - 192;   // 0..127
+    uint32_t u0 = 0;
+    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+      const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+      for (int i = 0; i < it.n_units; ++i) {
+        const uint32_t u = u0 + i;
+        const int cb = u % NQ;
+        const long long lo = it.list_lo + (long long)i * QC;
+        const int rows = (int)min((long long)QC, it.list_hi - lo);
+        auto row_of = [&](int r) { return DENSE ? (int)(lo + r) : __ldg(p.q_idx + lo + r); };
+        uint4 vq[8], vo[8];
+        gather_chunk64(nullptr, p.q + it.head_off * DH, rows, lt, row_of, vq);
+        gather_chunk64(nullptr, p.d_o + it.head_off * DH, rows, lt, row_of, vo);
         float l2 = INFINITY, dd = 0.f;     // padded queries: P = exp2(-inf) = 0
         if (lt < rows) {
-          const long long G_ = head_off + row_of(lt);
+          const long long G_ = it.head_off + row_of(lt);
           l2 = p.lse[G_] * LOG2E;
           dd = p.Dv[G_];
         }
-        sm->lse2[b][lt] = l2;
-        sm->Dq[b][lt] = dd;
+        if (u >= NQ) mbar_wait(&sm->chunk_empty[cb], ((u / NQ) - 1) & 1, abort_flag, p.status);
+        uint8_t* dst = sC + cb * 2 * CTILE;
+        store_chunk64(dst, lt, vq);
+        store_chunk64(dst + CTILE, lt, vo);
+        if (lt < QC) { sm->lse2[cb][lt] = l2; sm->Dq[cb][lt] = dd; }
         fence_async_proxy();
-        mbar_arrive(&sm->chunk_full[b]);
+        mbar_arrive(&sm->chunk_full[cb]);
       }
-    } else {
-      // ---------------------------------------------------------------- compute: thread = key row
-      const int quad = warp & 3;
-      const int r = quad * 32 + lane;
-      const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-      for (int c = 0; c < nchunks; ++c) {
-        const uint32_t g = cg + c;
-        const int b = g & 1;
-        mbar_wait(&sm->chunk_full[b], (g >> 1) & 1, abort_flag, p.status);   // publishes lse2 / Dq of this chunk
-        mbar_wait(&sm->sdp_full, g & 1, abort_flag, p.status);
-        tc_fence_after();
-        const float* lse2 = sm->lse2[b];
-        const float* Dq = sm->Dq[b];
-#pragma unroll 1
-        for (int h = 0; h < 2; ++h) {
-          uint32_t sv[2][32], dv_[2][32];
-          tmem_ld32(tmem + lane_addr + ST_COL + h * 64, sv[0]);
-          tmem_ld32(tmem + lane_addr + ST_COL + h * 64 + 32, sv[1]);
-          tmem_ld32(tmem + lane_addr + DPT_COL + h * 64, dv_[0]);
-          tmem_ld32(tmem + lane_addr + DPT_COL + h * 64 + 32, dv_[1]);
-          tmem_ld_wait();
-          uint32_t pk[32], dk_[32];
+      u0 += it.n_units;
+    }
+  } else {
+    // ------------------------------------------------------------------ compute: thread = key row
+    const int quad = warp & 3;
+    const int r = quad * 32 + lane;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    uint32_t n = 0, u0 = 0;
+    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+      const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+      __nv_bfloat16* dv_row = p.dv + (it.head_off + it.key0 + r) * DH;
+      __nv_bfloat16* dk_row = p.dk + (it.head_off + it.key0 + r) * DH;
+      if (it.n_units == 0) {
+        // no query selected this block: its keys get zero gradients
+        if (r < it.valid) {
+          const uint4 z = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int q0 = h * 64 + 2 * i;
-            const float s0 = __uint_as_float(sv[i >> 4][(2 * i) & 31]), s1 = __uint_as_float(sv[i >> 4][((2 * i) & 31) + 1]);
-            const float d0 = __uint_as_float(dv_[i >> 4][(2 * i) & 31]), d1 = __uint_as_float(dv_[i >> 4][((2 * i) & 31) + 1]);
-            const float p0 = ex2(fmaf(s0, p.scale_log2, -lse2[q0]));
-            const float p1 = ex2(fmaf(s1, p.scale_log2, -lse2[q0 + 1]));
-            pk[i] = pack_bf16(p0, p1);
-            dk_[i] = pack_bf16(p0 * (d0 - Dq[q0]), p1 * (d1 - Dq[q0 + 1]));
-          }
-          tmem_st32(tmem + lane_addr + ST_COL + h * 32, pk);
-          tmem_st32(tmem + lane_addr + DPT_COL + h * 32, dk_);
+          for (int i = 0; i < 16; ++i) { reinterpret_cast<uint4*>(dk_row)[i] = z; reinterpret_cast<uint4*>(dv_row)[i] = z; }
         }
+        continue;
+      }
+      for (int i = 0; i < it.n_units; ++i) {
+        const uint32_t u = u0 + i;
+        const int cb = u % NQ, tb = u & 1;
+        mbar_wait(&sm->chunk_full[cb], (u / NQ) & 1, abort_flag, p.status);   // publishes lse2 / Dq of this unit
+        mbar_wait(&sm->sdp_full[tb], (u >> 1) & 1, abort_flag, p.status);
+        tc_fence_after();
+        const float* lse2 = sm->lse2[cb];
+        const float* Dq = sm->Dq[cb];
+        const uint32_t st_t = tmem + lane_addr + ST_COL + tb * QC, dp_t = tmem + lane_addr + DPT_COL + tb * QC;
+        uint32_t sv[2][32], dv_[2][32];
+        tmem_ld32(st_t, sv[0]);
+        tmem_ld32(st_t + 32, sv[1]);
+        tmem_ld32(dp_t, dv_[0]);
+        tmem_ld32(dp_t + 32, dv_[1]);
+        tmem_ld_wait();
+        uint32_t pk[32], dk_[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int q0 = 2 * e;
+          const float s0 = __uint_as_float(sv[e >> 4][(2 * e) & 31]), s1 = __uint_as_float(sv[e >> 4][((2 * e) & 31) + 1]);
+          const float d0 = __uint_as_float(dv_[e >> 4][(2 * e) & 31]), d1 = __uint_as_float(dv_[e >> 4][((2 * e) & 31) + 1]);
+          const float p0 = ex2(fmaf(s0, p.scale_log2, -lse2[q0]));
+          const float p1 = ex2(fmaf(s1, p.scale_log2, -lse2[q0 + 1]));
+          pk[e] = pack_bf16(p0, p1);
+          dk_[e] = pack_bf16(p0 * (d0 - Dq[q0]), p1 * (d1 - Dq[q0 + 1]));
+        }
+        tmem_st32(st_t, pk);       // P^T (bf16 pairs) over the first 32 columns of this S^T buffer
+        tmem_st32(dp_t, dk_);      // dS^T over the first 32 columns of this dP^T buffer
         tmem_st_wait();
         tc_fence_before();
-        mbar_arrive(&sm->pds_ready);
+        mbar_arrive(&sm->pds_ready[tb]);
       }
       // ---- epilogue: dV and dK rows of this tile
-      mbar_wait(&sm->acc_done, it_n & 1, abort_flag, p.status);
+      mbar_wait(&sm->acc_done, n & 1, abort_flag, p.status);
       tc_fence_after();
-      __nv_bfloat16* dv_row = p.dv + (head_off + key0 + r) * DH;
-      __nv_bfloat16* dk_row = p.dk + (head_off + key0 + r) * DH;
 #pragma unroll 1
       for (int cgrp = 0; cgrp < 4; ++cgrp) {
         uint32_t a[32], bb[32];
         tmem_ld32(tmem + lane_addr + DV_COL + cgrp * 32, a);
         tmem_ld32(tmem + lane_addr + DK_COL + cgrp * 32, bb);
         tmem_ld_wait();
-        if (r < valid) {
+        if (r < it.valid) {
 #pragma unroll
           for (int i = 0; i < 32; i += 4) {
             store4(dv_row + cgrp * 32 + i, make_float4(__uint_as_float(a[i]), __uint_as_float(a[i + 1]),
@@ -296,9 +372,11 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           }
         }
       }
+      tc_fence_before();
+      mbar_arrive(&sm->acc_free);
+      u0 += it.n_units;
+      ++n;
     }
-    cg += nchunks;
-    ++it_n;
   }
   tc_fence_before();
   __syncthreads();
