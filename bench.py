@@ -222,6 +222,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dense", action="store_true", help="also time the dense vmoba_full_attn path on the same inputs")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small profiling runs)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -246,6 +247,8 @@ def main():
     pk = peaks()
 
     layers, with_bwd = workloads(args.workload)
+    if args.heads > 0:
+        layers = [w.with_(heads=args.heads) for w in layers]
     layers = rank_workloads(layers, rank)
     w0 = layers[0]
     data = gen.make_inputs(w0, with_do=with_bwd)

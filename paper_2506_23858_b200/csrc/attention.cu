@@ -20,7 +20,8 @@ int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, voi
 // attn_tc_bwd.cu: tensor-core backward kernels (bf16, head_dim 128)
 int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                   const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap,
-                  const int* item_ptr, float* dq_acc, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st);
+                  const int* item_ptr, const int* item_tab, float* dq_acc, void* dq, void* dk, void* dv,
+                  int32_t* status, cudaStream_t st);
 int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* Dv, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st);
 
@@ -37,11 +38,14 @@ static FwdWs carve_fwd(const Dims& D, long long cap, void* ws) {
   return w;
 }
 
-struct BwdWs { int* item_ptr; float* Dv; float* dq_acc; void* o_resid; size_t bytes; };
-static BwdWs carve_bwd(const Dims& D, bool dense, void* ws) {
+static long long max_items_128(const Dims& D, long long cap) { return cap / 128 + (long long)D.BH * D.Nb + 1; }
+
+struct BwdWs { int* item_ptr; int* item_tab; float* Dv; float* dq_acc; void* o_resid; size_t bytes; };
+static BwdWs carve_bwd(const Dims& D, bool dense, void* ws, long long cap = 0) {
   Carver c(ws);
   BwdWs w;
   w.item_ptr = c.take<int>((size_t)D.BH * D.Nb + 1);
+  w.item_tab = dense ? nullptr : c.take<int>((size_t)max_items_128(D, cap));
   w.Dv = c.take<float>((size_t)D.BH * D.S);
   w.dq_acc = dense ? nullptr : c.take<float>((size_t)D.BH * D.S * D.d);
   w.o_resid = (dense && D.dtype == VMOBA_BF16) ? c.take<__nv_bfloat16>((size_t)D.BH * D.S * D.d) : nullptr;
@@ -77,7 +81,7 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
                            const void* o_resid, const float* lse, const void* d_o, const int* kb_ptr, const int* q_idx,
                            const int* q_ptr, long long cap, void* dq, void* dk, void* dv, int32_t* status, void* ws,
                            cudaStream_t st) {
-  BwdWs w = carve_bwd(D, false, ws);
+  BwdWs w = carve_bwd(D, false, ws, cap);
   const long long n_kb = (long long)D.BH * D.Nb;
   const long long nq = (long long)D.BH * D.S;
   VMOBA_CUDA_OK(cudaMemsetAsync(w.dq_acc, 0, (size_t)nq * DH * sizeof(float), st));
@@ -85,9 +89,11 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
                                                                         (const T*)d_o, nq, w.Dv);
   if (use_tensor_cores(D)) {
     simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, 128, cap, w.item_ptr);
-    count_launches(2);
-    int rc = tc_sparse_bwd(D, q, k, v, d_o, lse, w.Dv, kb_ptr, q_idx, q_ptr, cap, w.item_ptr, w.dq_acc, dq, dk, dv,
-                           status, st);
+    simt::item_tab_kernel<<<(int)std::min<long long>((n_kb + 255) / 256, 148 * 4), 256, 0, st>>>(
+        w.item_ptr, n_kb, max_items_128(D, cap), w.item_tab);
+    count_launches(3);
+    int rc = tc_sparse_bwd(D, q, k, v, d_o, lse, w.Dv, kb_ptr, q_idx, q_ptr, cap, w.item_ptr, w.item_tab, w.dq_acc, dq,
+                           dk, dv, status, st);
     if (rc) return rc;
     simt::cast_rows_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, q_ptr, nq, 1);
     VMOBA_LAUNCH_OK(1);
@@ -177,7 +183,7 @@ extern "C" size_t vmoba_workspace_bytes(const vmoba_shape* shape, int stage, int
     case VMOBA_STAGE_SCORES: return scores_ws_bytes(D);
     case VMOBA_STAGE_SELECT: return select_ws_bytes(D);
     case VMOBA_STAGE_ATTN_FWD: return carve_fwd(D, capacity, nullptr).bytes;
-    case VMOBA_STAGE_ATTN_BWD: return carve_bwd(D, false, nullptr).bytes;
+    case VMOBA_STAGE_ATTN_BWD: return carve_bwd(D, false, nullptr, capacity).bytes;
     case VMOBA_STAGE_FULL_FWD: return 256;
     case VMOBA_STAGE_FULL_BWD: return carve_bwd(D, true, nullptr).bytes;
     default: return 0;
@@ -224,7 +230,7 @@ extern "C" int vmoba_attn_bwd(const vmoba_shape* shape, const void* q_bm, const 
       !aligned16(dq_bm) || !aligned16(dk_bm) || !aligned16(dv_bm) || !aligned16(ws))
     return VMOBA_ERR_ARG;
   if (capacity <= 0 || capacity > (int64_t)INT32_MAX) return VMOBA_ERR_ARG;
-  if (ws_bytes < carve_bwd(D, false, nullptr).bytes) return VMOBA_ERR_WORKSPACE;
+  if (ws_bytes < carve_bwd(D, false, nullptr, capacity).bytes) return VMOBA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (D.dtype != VMOBA_BF16) o_resid_or_null = nullptr;
   if (!aligned16(o_resid_or_null)) return VMOBA_ERR_ARG;

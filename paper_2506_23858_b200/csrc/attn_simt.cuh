@@ -32,6 +32,15 @@ item_ptr_kernel(const int* __restrict__ kb_ptr, long long n_kb, int rows, long l
       item_ptr, n_kb, &total);
 }
 
+// item_tab[item] = index of the (batch, head, key block) list the item belongs to.
+static __global__ void __launch_bounds__(256)
+item_tab_kernel(const int* __restrict__ item_ptr, long long n_kb, long long max_items, int* __restrict__ item_tab) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n_kb; i += (long long)gridDim.x * blockDim.x) {
+    const long long lo = item_ptr[i], hi = min((long long)item_ptr[i + 1], max_items);
+    for (long long t = lo; t < hi; ++t) item_tab[t] = (int)i;
+  }
+}
+
 struct Item {
   int bh;          // batch * heads + head
   int key_begin;   // key range inside the head (block-major positions)

@@ -55,6 +55,28 @@ __device__ __forceinline__ void gather_tile(uint8_t* dst, const __nv_bfloat16* h
   }
 }
 
+// The same gather split in two, so that a wait can sit between the loads and the stores
+// (128 threads, 16 rows per thread).
+template <typename RowOf>
+__device__ __forceinline__ void gather_load128(const __nv_bfloat16* head_base, int n_rows, int tid, RowOf row_of, uint4 (&v)[16]) {
+  const int chunk = tid & 15;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int row = (tid >> 4) + i * 8;
+    v[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (row < n_rows) v[i] = __ldg(reinterpret_cast<const uint4*>(head_base + (long long)row_of(row) * DH) + chunk);
+  }
+}
+__device__ __forceinline__ void gather_store128(uint8_t* dst, int tid, const uint4 (&v)[16]) {
+  const int chunk = tid & 15;
+  const int panel = chunk >> 3, cc = chunk & 7;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int row = (tid >> 4) + i * 8;
+    *reinterpret_cast<uint4*>(dst + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v[i];
+  }
+}
+
 // 16-byte vector reduction into global memory (fp32 add).
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
@@ -386,24 +408,36 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
 // ==========================================================================================
 // dQ
 // ==========================================================================================
-constexpr int DQ_STAGES = 2;
+// Item = 128 gathered queries x one key block (the forward's work items).  Keys stream in units of
+// 64 through a 2-stage TMA ring; S and dP are double buffered in TMEM (64 columns each) and the dQ
+// accumulator is double buffered across items, so the epilogue of one item overlaps the MMAs of
+// the next.  Loader warps gather Q / dO rows (and lse, D, output row) of the NEXT item meanwhile.
+constexpr int KU = 64;                       // keys per unit
+// Two shared-memory splits: short key blocks (few units per item) double buffer the gathered
+// Q / dO tiles across items and keep a 2-deep K/V ring; long blocks keep one Q / dO tile and a
+// 4-deep K/V ring, because there the ring depth hides the TMA latency.
+constexpr int DQ_NS_MAX = 4;
 struct DqSmem {
-  uint64_t k_full[DQ_STAGES], v_full[DQ_STAGES], kv_empty[DQ_STAGES];
-  uint64_t s_full[2];          // S buffer ready (commit)
-  uint64_t dp_full;            // dP ready (commit)
-  uint64_t ds_ready;           // dS written (128 arrivals)
-  uint64_t dq_done[2];         // all MMAs of the item done (commit), alternating by item
-  uint64_t qdo_ready;          // Q and dO gathered (128 arrivals)
+  uint64_t kv_full[DQ_NS_MAX], kv_empty[DQ_NS_MAX];  // K+V unit (TMA / commit)
+  uint64_t qdo_full[2], qdo_empty[2];        // gathered Q/dO of an item (128 loader arrivals / commit)
+  uint64_t sdp_full[2];                      // S and dP of a unit ready (commit)
+  uint64_t ds_ready[2];                      // dS written (128 compute arrivals)
+  uint64_t dq_done[2];                       // all MMAs of the item done (commit)
+  uint64_t dq_free[2];                       // epilogue has read the accumulator (128 compute arrivals)
   uint32_t tmem_base;
   int abort_flag;
+  float lse2[2][128];
+  float Dr[2][128];
+  long long G[2][128];                       // flat output row of each query, -1 for padding rows
+  int direct[2][128];                        // query has a single block: write bf16 directly
 };
-constexpr size_t DQ_SMEM_BYTES = 1024 + 2 * TILE + 2 * DQ_STAGES * TILE + sizeof(DqSmem) + 64;
-constexpr int DQ_THREADS = 192;
+constexpr size_t dq_smem_bytes(int QB, int NS) { return 1024 + QB * 2 * TILE + NS * 2 * CTILE + sizeof(DqSmem) + 32; }
+constexpr int DQ_THREADS = 320;
 
 struct DqParams {
   const __nv_bfloat16 *q, *d_o;
   const float *lse, *Dv;
-  const int *kb_ptr, *q_idx, *q_ptr, *item_ptr;
+  const int *kb_ptr, *q_idx, *q_ptr, *item_ptr, *item_tab;
   int n_kb, S, Nb, sb, BH;
   float scale, scale_log2;
   long long capacity;
@@ -412,40 +446,52 @@ struct DqParams {
   int32_t* status;
 };
 
-template <bool DENSE>
-__device__ __forceinline__ void dq_decode(const DqParams& p, int item, int& bh, int& key_begin, int& n_keys, int& list_lo,
-                                          int& n_rows) {
-  if (DENSE) {
-    const int tiles = (p.S + BM - 1) / BM;
-    bh = item / tiles;
-    const int t = item - bh * tiles;
-    key_begin = 0; n_keys = p.S; list_lo = t * BM; n_rows = min(BM, p.S - list_lo);
-  } else {
-    simt::Item it = simt::decode_sparse(item, p.item_ptr, p.n_kb, p.kb_ptr, p.Nb, p.sb, BM, p.capacity);
-    bh = it.bh; key_begin = it.key_begin; n_keys = p.sb; list_lo = it.list_lo; n_rows = it.list_hi - it.list_lo;
-  }
-}
+struct DqItem {
+  int bh, key_begin, n_keys, list_lo, n_rows, n_units;
+  long long head_off;
+};
 
 template <bool DENSE>
+__device__ __forceinline__ DqItem dq_decode(const DqParams& p, int item) {
+  DqItem it;
+  if (DENSE) {
+    const int tiles = (p.S + BM - 1) / BM;
+    it.bh = item / tiles;
+    const int t = item - it.bh * tiles;
+    it.key_begin = 0; it.n_keys = p.S; it.list_lo = t * BM; it.n_rows = min(BM, p.S - it.list_lo);
+  } else {
+    const int kbi = __ldg(p.item_tab + item);
+    const int chunk = item - __ldg(p.item_ptr + kbi);
+    it.bh = kbi / p.Nb;
+    const int j = kbi - it.bh * p.Nb;
+    it.key_begin = j * p.sb; it.n_keys = p.sb;
+    const long long end = min((long long)__ldg(p.kb_ptr + kbi + 1), p.capacity);
+    it.list_lo = __ldg(p.kb_ptr + kbi) + chunk * BM;
+    it.n_rows = (int)min((long long)BM, end - it.list_lo);
+  }
+  it.n_units = (it.n_keys + KU - 1) / KU;
+  it.head_off = (long long)it.bh * p.S;
+  return it;
+}
+
+template <bool DENSE, int QB, int DQ_NS>
 __global__ void __launch_bounds__(DQ_THREADS, 1)
 attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const DqParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = base;
-  uint8_t* sdO = base + TILE;
-  uint8_t* sK = base + 2 * TILE;
-  uint8_t* sV = sK + DQ_STAGES * TILE;
-  DqSmem* sm = reinterpret_cast<DqSmem*>(sV + DQ_STAGES * TILE);
+  uint8_t* sQdO = base;                    // [QB][Q tile | dO tile]
+  uint8_t* sKV = base + QB * 2 * TILE;     // [DQ_NS][K unit | V unit]
+  DqSmem* sm = reinterpret_cast<DqSmem*>(sKV + DQ_NS * 2 * CTILE);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm->abort_flag;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < DQ_STAGES; ++s) { mbar_init(&sm->k_full[s], 1); mbar_init(&sm->v_full[s], 1); mbar_init(&sm->kv_empty[s], 1); }
-    mbar_init(&sm->s_full[0], 1); mbar_init(&sm->s_full[1], 1);
-    mbar_init(&sm->dp_full, 1);
-    mbar_init(&sm->ds_ready, 128);
-    mbar_init(&sm->dq_done[0], 1); mbar_init(&sm->dq_done[1], 1);
-    mbar_init(&sm->qdo_ready, 128);
+    for (int s = 0; s < DQ_NS; ++s) { mbar_init(&sm->kv_full[s], 1); mbar_init(&sm->kv_empty[s], 1); }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sm->qdo_full[b], 128); mbar_init(&sm->qdo_empty[b], 1);
+      mbar_init(&sm->sdp_full[b], 1); mbar_init(&sm->ds_ready[b], 128);
+      mbar_init(&sm->dq_done[b], 1); mbar_init(&sm->dq_free[b], 128);
+    }
     sm->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmK);
@@ -459,163 +505,164 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm->tmem_base;
-  constexpr uint32_t S_COL0 = 0, S_COL1 = 128, DP_COL = 256, DQ_COL = 384;
+  constexpr uint32_t S_COL = 0, DP_COL = 128, DQ_COL = 256;   // S, dP: two 64-column buffers; dQ: two 128-column buffers
   const int n_items = DENSE ? p.BH * ((p.S + BM - 1) / BM) : p.item_ptr[p.n_kb];
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer: K and V units
     if (lane == 0) {
-      uint32_t fills = 0;
+      uint32_t f = 0;
       for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-        int bh, key_begin, n_keys, list_lo, n_rows;
-        dq_decode<DENSE>(p, item, bh, key_begin, n_keys, list_lo, n_rows);
-        const int row0 = bh * p.S + key_begin;
-        const int ntiles = (n_keys + BN - 1) / BN;
-        for (int t = 0; t < ntiles; ++t, ++fills) {
-          const int s = fills % DQ_STAGES;
-          if (fills >= DQ_STAGES) mbar_wait(&sm->kv_empty[s], ((fills / DQ_STAGES) - 1) & 1, abort_flag, p.status);
-          const int y = row0 + t * BN;
-          mbar_expect_tx(&sm->k_full[s], TILE);
-          tma_load_2d(sK + s * TILE, &tmK, &sm->k_full[s], 0, y);
-          tma_load_2d(sK + s * TILE + PANEL, &tmK, &sm->k_full[s], 64, y);
-          mbar_expect_tx(&sm->v_full[s], TILE);
-          tma_load_2d(sV + s * TILE, &tmV, &sm->v_full[s], 0, y);
-          tma_load_2d(sV + s * TILE + PANEL, &tmV, &sm->v_full[s], 64, y);
+        const DqItem it = dq_decode<DENSE>(p, item);
+        const int row0 = (int)it.head_off + it.key_begin;
+        for (int i = 0; i < it.n_units; ++i, ++f) {
+          const int s = f % DQ_NS;
+          if (f >= DQ_NS) mbar_wait(&sm->kv_empty[s], ((f / DQ_NS) - 1) & 1, abort_flag, p.status);
+          uint8_t* dst = sKV + s * 2 * CTILE;
+          const int y = row0 + i * KU;
+          mbar_expect_tx(&sm->kv_full[s], 2 * CTILE);
+          tma_load_2d(dst, &tmK, &sm->kv_full[s], 0, y);
+          tma_load_2d(dst + CPANEL, &tmK, &sm->kv_full[s], 64, y);
+          tma_load_2d(dst + CTILE, &tmV, &sm->kv_full[s], 0, y);
+          tma_load_2d(dst + CTILE + CPANEL, &tmV, &sm->kv_full[s], 64, y);
         }
       }
-      if (*abort_flag) {
-        const uint32_t first = fills > DQ_STAGES ? fills - DQ_STAGES : 0;
-        for (uint32_t f = first; f < fills; ++f) {
-          mbar_wait(&sm->k_full[f % DQ_STAGES], (f / DQ_STAGES) & 1, abort_flag, p.status);
-          mbar_wait(&sm->v_full[f % DQ_STAGES], (f / DQ_STAGES) & 1, abort_flag, p.status);
-        }
-      }
+      if (*abort_flag)
+        for (uint32_t g = f > DQ_NS ? f - DQ_NS : 0; g < f; ++g)
+          mbar_wait(&sm->kv_full[g % DQ_NS], (g / DQ_NS) & 1, abort_flag, p.status);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      uint32_t fills = 0, tg = 0, items_done = 0;
-      const uint32_t sQ_addr = smem_u32(sQ), sdO_addr = smem_u32(sdO);
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++items_done) {
-        int bh, key_begin, n_keys, list_lo, n_rows;
-        dq_decode<DENSE>(p, item, bh, key_begin, n_keys, list_lo, n_rows);
-        const int ntiles = (n_keys + BN - 1) / BN;
-        mbar_wait(&sm->qdo_ready, items_done & 1, abort_flag, p.status);
+      uint32_t n = 0, u0 = 0;
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+        const DqItem it = dq_decode<DENSE>(p, item);
+        const int qb = n & 1;                 // accumulator / scalar slot
+        const int qs = n % QB;                // Q / dO tile slot
+        mbar_wait(&sm->qdo_full[qs], (n / QB) & 1, abort_flag, p.status);
         tc_fence_after();
-        auto n_mma_of = [&](int t) { return (min(BN, n_keys - t * BN) + 15) & ~15; };
-        auto issue_s = [&](int t) {
-          const uint32_t f = fills + t;
-          const int s = f % DQ_STAGES;
-          mbar_wait(&sm->k_full[s], (f / DQ_STAGES) & 1, abort_flag, p.status);
+        const uint32_t sQ_addr = smem_u32(sQdO + qs * 2 * TILE), sdO_addr = sQ_addr + TILE;
+        auto n_mma_of = [&](int i) { return (min(KU, it.n_keys - i * KU) + 15) & ~15; };
+        auto issue_sdp = [&](int i) {
+          const uint32_t u = u0 + i;
+          const int s = u % DQ_NS, tb = u & 1;
+          mbar_wait(&sm->kv_full[s], (u / DQ_NS) & 1, abort_flag, p.status);
           tc_fence_after();
-          const uint32_t idesc = make_idesc_bf16(BM, n_mma_of(t), false, false);
-          const uint32_t buf = (tg + t) & 1;
-          const uint32_t sK_addr = smem_u32(sK + s * TILE);
+          const uint32_t idesc = make_idesc_bf16(BM, n_mma_of(i), false, false);
+          const uint32_t sK_addr = smem_u32(sKV + s * 2 * CTILE), sV_addr = sK_addr + CTILE;
 #pragma unroll
           for (int ks = 0; ks < DH / 16; ++ks)
-            mma_ss(tmem + (buf ? S_COL1 : S_COL0), desc_k(sQ_addr, ks), desc_k(sK_addr, ks), idesc, ks > 0 ? 1u : 0u);
-          mma_commit(&sm->s_full[buf]);
-        };
-        issue_s(0);
-        for (int t = 0; t < ntiles; ++t) {
-          const uint32_t f = fills + t;
-          const int s = f % DQ_STAGES;
-          // dP(t) = dO V^T : the dP/dS region is free because dQ(t-1), which read dS(t-1), was issued before
-          mbar_wait(&sm->v_full[s], (f / DQ_STAGES) & 1, abort_flag, p.status);
-          tc_fence_after();
-          {
-            const uint32_t idesc = make_idesc_bf16(BM, n_mma_of(t), false, false);
-            const uint32_t sV_addr = smem_u32(sV + s * TILE);
+            mma_ss(tmem + S_COL + tb * KU, desc_k(sQ_addr, ks), cdesc_k(sK_addr, ks), idesc, ks > 0 ? 1u : 0u);
 #pragma unroll
-            for (int ks = 0; ks < DH / 16; ++ks)
-              mma_ss(tmem + DP_COL, desc_k(sdO_addr, ks), desc_k(sV_addr, ks), idesc, ks > 0 ? 1u : 0u);
-            mma_commit(&sm->dp_full);
-          }
-          if (t + 1 < ntiles) issue_s(t + 1);
-          mbar_wait(&sm->ds_ready, (tg + t) & 1, abort_flag, p.status);
+          for (int ks = 0; ks < DH / 16; ++ks)
+            mma_ss(tmem + DP_COL + tb * KU, desc_k(sdO_addr, ks), cdesc_k(sV_addr, ks), idesc, ks > 0 ? 1u : 0u);
+          mma_commit(&sm->sdp_full[tb]);
+        };
+        issue_sdp(0);
+        for (int i = 0; i < it.n_units; ++i) {
+          if (i + 1 < it.n_units) issue_sdp(i + 1);
+          const uint32_t u = u0 + i;
+          const int s = u % DQ_NS, tb = u & 1;
+          mbar_wait(&sm->ds_ready[tb], (u >> 1) & 1, abort_flag, p.status);
+          // this accumulator was last used two items ago: its epilogue must have read it
+          if (i == 0 && n >= 2) mbar_wait(&sm->dq_free[qb], ((n >> 1) - 1) & 1, abort_flag, p.status);
           tc_fence_after();
-          const int ksteps = n_mma_of(t) >> 4;
-          const uint32_t sK_addr = smem_u32(sK + s * TILE);
+          const int ksteps = n_mma_of(i) >> 4;
+          const uint32_t sK_addr = smem_u32(sKV + s * 2 * CTILE);
           for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(tmem + DQ_COL, tmem + DP_COL + ks * 8, desc_mn(sK_addr, ks), IDESC_TN, (t > 0 || ks > 0) ? 1u : 0u);
+            mma_ts(tmem + DQ_COL + qb * 128, tmem + DP_COL + tb * KU + ks * 8, cdesc_mn(sK_addr, ks), IDESC_TN,
+                   (i > 0 || ks > 0) ? 1u : 0u);
           mma_commit(&sm->kv_empty[s]);
         }
-        mma_commit(&sm->dq_done[items_done & 1]);
-        fills += ntiles;
-        tg += ntiles;
+        mma_commit(&sm->qdo_empty[qs]);
+        mma_commit(&sm->dq_done[qb]);
+        u0 += it.n_units;
       }
+    }
+  } else if (warp >= 6) {
+    // ------------------------------------------------------------------ loaders: Q / dO rows of the next items
+    const int lt = threadIdx.x - 192;   // 0..127
+    uint32_t n = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+      const DqItem it = dq_decode<DENSE>(p, item);
+      const int qb = n & 1, qs = n % QB;
+      auto row_of = [&](int r) { return DENSE ? it.list_lo + r : __ldg(p.q_idx + it.list_lo + r); };
+      // this thread's own row (lt) for the per-row scalars; issue before the big gathers
+      long long G_ = -1;
+      float l2 = INFINITY, dd = 0.f;
+      int direct = DENSE ? 1 : 0;
+      if (lt < it.n_rows) {
+        G_ = it.head_off + row_of(lt);
+        l2 = p.lse[G_] * LOG2E;
+        dd = p.Dv[G_];
+        if (!DENSE) direct = (p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1;
+      }
+      uint4 vq[16], vo[16];
+      gather_load128(p.q + it.head_off * DH, it.n_rows, lt, row_of, vq);
+      gather_load128(p.d_o + it.head_off * DH, it.n_rows, lt, row_of, vo);
+      if (n >= QB) mbar_wait(&sm->qdo_empty[qs], ((n / QB) - 1) & 1, abort_flag, p.status);
+      // the scalar slots alternate by item; with a single Q / dO tile the compute warps may still be
+      // reading slot qb of item n-2 only if they lag two items behind, which qdo_empty(n-1) excludes
+      uint8_t* dst = sQdO + qs * 2 * TILE;
+      gather_store128(dst, lt, vq);
+      gather_store128(dst + TILE, lt, vo);
+      sm->lse2[qb][lt] = l2; sm->Dr[qb][lt] = dd; sm->G[qb][lt] = G_; sm->direct[qb][lt] = direct;
+      fence_async_proxy();
+      mbar_arrive(&sm->qdo_full[qs]);
     }
   } else {
     // ------------------------------------------------------------------ compute: thread = query row
     const int quad = warp & 3;
     const int r = quad * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const int ct = threadIdx.x - 64;
-    uint32_t tg = 0, items_done = 0;
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++items_done) {
-      int bh, key_begin, n_keys, list_lo, n_rows;
-      dq_decode<DENSE>(p, item, bh, key_begin, n_keys, list_lo, n_rows);
-      const int ntiles = (n_keys + BN - 1) / BN;
-      const long long head_off = (long long)bh * p.S;
-      auto row_of = [&](int i) { return DENSE ? list_lo + i : p.q_idx[list_lo + i]; };
-      gather_tile<128>(sQ, p.q + head_off * DH, n_rows, ct, row_of);
-      gather_tile<128>(sdO, p.d_o + head_off * DH, n_rows, ct, row_of);
-      fence_async_proxy();
-      mbar_arrive(&sm->qdo_ready);
-      const bool row_ok = r < n_rows;
-      long long G_ = 0;
-      float lse2 = INFINITY, Dr = 0.f;
-      bool direct = DENSE;
-      if (row_ok) {
-        G_ = head_off + row_of(r);
-        lse2 = p.lse[G_] * LOG2E;
-        Dr = p.Dv[G_];
-        if (!DENSE) direct = (p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1;
-      }
-      for (int t = 0; t < ntiles; ++t) {
-        const uint32_t buf = (tg + t) & 1;
-        const int valid = min(BN, n_keys - t * BN);
-        mbar_wait(&sm->s_full[buf], ((tg + t) >> 1) & 1, abort_flag, p.status);
-        mbar_wait(&sm->dp_full, (tg + t) & 1, abort_flag, p.status);
+    uint32_t n = 0, u0 = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+      const DqItem it = dq_decode<DENSE>(p, item);
+      const int qb = n & 1, qs = n % QB;
+      mbar_wait(&sm->qdo_full[qs], (n / QB) & 1, abort_flag, p.status);   // publishes the per-row scalars
+      const float lse2 = sm->lse2[qb][r], Dr = sm->Dr[qb][r];
+      const long long G_ = sm->G[qb][r];
+      const int direct = sm->direct[qb][r];
+      for (int i = 0; i < it.n_units; ++i) {
+        const uint32_t u = u0 + i;
+        const int tb = u & 1;
+        const int valid = min(KU, it.n_keys - i * KU);
+        mbar_wait(&sm->sdp_full[tb], (u >> 1) & 1, abort_flag, p.status);
         tc_fence_after();
-        const uint32_t s_tmem = tmem + lane_addr + (buf ? S_COL1 : S_COL0);
-        const uint32_t dp_tmem = tmem + lane_addr + DP_COL;
-#pragma unroll 1
-        for (int h = 0; h < 2; ++h) {
-          uint32_t sv[2][32], dv_[2][32];
-          tmem_ld32(s_tmem + h * 64, sv[0]);
-          tmem_ld32(s_tmem + h * 64 + 32, sv[1]);
-          tmem_ld32(dp_tmem + h * 64, dv_[0]);
-          tmem_ld32(dp_tmem + h * 64 + 32, dv_[1]);
-          tmem_ld_wait();
-          uint32_t ds[32];
+        const uint32_t s_t = tmem + lane_addr + S_COL + tb * KU, dp_t = tmem + lane_addr + DP_COL + tb * KU;
+        uint32_t sv[2][32], dv_[2][32];
+        tmem_ld32(s_t, sv[0]);
+        tmem_ld32(s_t + 32, sv[1]);
+        tmem_ld32(dp_t, dv_[0]);
+        tmem_ld32(dp_t + 32, dv_[1]);
+        tmem_ld_wait();
+        uint32_t ds[32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int k0 = h * 64 + 2 * i;
-            const float s0 = __uint_as_float(sv[i >> 4][(2 * i) & 31]), s1 = __uint_as_float(sv[i >> 4][((2 * i) & 31) + 1]);
-            const float d0 = __uint_as_float(dv_[i >> 4][(2 * i) & 31]), d1 = __uint_as_float(dv_[i >> 4][((2 * i) & 31) + 1]);
-            const float p0 = ex2(fmaf(s0, p.scale_log2, -lse2));
-            const float p1 = ex2(fmaf(s1, p.scale_log2, -lse2));
-            const float x0 = (k0 < valid) ? p0 * (d0 - Dr) : 0.f;
-            const float x1 = (k0 + 1 < valid) ? p1 * (d1 - Dr) : 0.f;
-            ds[i] = pack_bf16(x0, x1);
-          }
-          tmem_st32(dp_tmem + h * 32, ds);
+        for (int e = 0; e < 32; ++e) {
+          const int k0 = 2 * e;
+          const float s0 = __uint_as_float(sv[e >> 4][(2 * e) & 31]), s1 = __uint_as_float(sv[e >> 4][((2 * e) & 31) + 1]);
+          const float d0 = __uint_as_float(dv_[e >> 4][(2 * e) & 31]), d1 = __uint_as_float(dv_[e >> 4][((2 * e) & 31) + 1]);
+          const float p0 = ex2(fmaf(s0, p.scale_log2, -lse2));
+          const float p1 = ex2(fmaf(s1, p.scale_log2, -lse2));
+          const float x0 = (k0 < valid) ? p0 * (d0 - Dr) : 0.f;
+          const float x1 = (k0 + 1 < valid) ? p1 * (d1 - Dr) : 0.f;
+          ds[e] = pack_bf16(x0, x1);
         }
+        tmem_st32(dp_t, ds);      // dS (bf16 pairs) over the first 32 columns of this dP buffer
         tmem_st_wait();
         tc_fence_before();
-        mbar_arrive(&sm->ds_ready);
+        mbar_arrive(&sm->ds_ready[tb]);
       }
+      u0 += it.n_units;
       // ---- epilogue
-      mbar_wait(&sm->dq_done[items_done & 1], (items_done >> 1) & 1, abort_flag, p.status);
+      mbar_wait(&sm->dq_done[qb], (n >> 1) & 1, abort_flag, p.status);
       tc_fence_after();
-      tg += ntiles;
 #pragma unroll 1
       for (int cgrp = 0; cgrp < 4; ++cgrp) {
         uint32_t a[32];
-        tmem_ld32(tmem + lane_addr + DQ_COL + cgrp * 32, a);
+        tmem_ld32(tmem + lane_addr + DQ_COL + qb * 128 + cgrp * 32, a);
         tmem_ld_wait();
-        if (row_ok) {
+        if (G_ >= 0) {
           if (direct) {
             __nv_bfloat16* dst = p.dq + G_ * DH + cgrp * 32;
 #pragma unroll
@@ -632,6 +679,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         }
       }
       tc_fence_before();
+      mbar_arrive(&sm->dq_free[qb]);
     }
   }
   tc_fence_before();
@@ -647,11 +695,13 @@ static int grid_items(long long items) { return (int)std::max<long long>(1, std:
 // a zeroed fp32 accumulator that the caller converts to bf16 afterwards.
 int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                   const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap,
-                  const int* item_ptr, float* dq_acc, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st) {
+                  const int* item_ptr, const int* item_tab, float* dq_acc, void* dq, void* dk, void* dv,
+                  int32_t* status, cudaStream_t st) {
   using namespace tcb;
-  CUtensorMap tmK, tmV;
+  CUtensorMap tmK, tmV, tmK64, tmV64;
   const uint64_t rows = (uint64_t)D.BH * D.S;
-  if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN))
+  if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN) ||
+      !sm100::make_tmap_bf16_rows(&tmK64, k, rows, DH, KU) || !sm100::make_tmap_bf16_rows(&tmV64, v, rows, DH, KU))
     return VMOBA_ERR_CUDA;
   const long long n_kb = (long long)D.BH * D.Nb;
   KvParams kp;
@@ -665,12 +715,19 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
   attn_bwd_dkdv_tc_kernel<false><<<grid_items(kv_items), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, kp);
   DqParams qp;
   qp.q = kp.q; qp.d_o = kp.d_o; qp.lse = lse; qp.Dv = Dv; qp.kb_ptr = kb_ptr; qp.q_idx = q_idx; qp.item_ptr = item_ptr;
+  qp.item_tab = item_tab;
   qp.n_kb = (int)n_kb; qp.S = D.S; qp.Nb = D.Nb; qp.sb = D.sb; qp.BH = D.BH; qp.scale = D.scale;
   qp.scale_log2 = D.scale * LOG2E; qp.capacity = cap; qp.dq_acc = dq_acc; qp.dq = (__nv_bfloat16*)dq; qp.status = status;
   qp.q_ptr = q_ptr;
-  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)DQ_SMEM_BYTES));
-  attn_bwd_dq_tc_kernel<false><<<grid_items(cap / BM + n_kb), DQ_THREADS, DQ_SMEM_BYTES, st>>>(tmK, tmV, qp);
+  if (D.sb >= 1024) {
+    constexpr size_t SM = dq_smem_bytes(1, 4);
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<false, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM));
+    attn_bwd_dq_tc_kernel<false, 1, 4><<<grid_items(cap / BM + n_kb), DQ_THREADS, SM, st>>>(tmK64, tmV64, qp);
+  } else {
+    constexpr size_t SM = dq_smem_bytes(2, 2);
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<false, 2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM));
+    attn_bwd_dq_tc_kernel<false, 2, 2><<<grid_items(cap / BM + n_kb), DQ_THREADS, SM, st>>>(tmK64, tmV64, qp);
+  }
   VMOBA_LAUNCH_OK(2);
   return VMOBA_OK;
 }
@@ -678,9 +735,10 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
 int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* Dv, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st) {
   using namespace tcb;
-  CUtensorMap tmK, tmV;
+  CUtensorMap tmK, tmV, tmK64, tmV64;
   const uint64_t rows = (uint64_t)D.BH * D.S;
-  if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN))
+  if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN) ||
+      !sm100::make_tmap_bf16_rows(&tmK64, k, rows, DH, KU) || !sm100::make_tmap_bf16_rows(&tmV64, v, rows, DH, KU))
     return VMOBA_ERR_CUDA;
   KvParams kp;
   kp.q = (const __nv_bfloat16*)q; kp.d_o = (const __nv_bfloat16*)d_o; kp.lse = lse; kp.Dv = Dv;
@@ -693,11 +751,14 @@ int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, con
   attn_bwd_dkdv_tc_kernel<true><<<grid_items(D.BH * tiles), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, kp);
   DqParams qp;
   qp.q = kp.q; qp.d_o = kp.d_o; qp.lse = lse; qp.Dv = Dv; qp.kb_ptr = nullptr; qp.q_idx = nullptr; qp.item_ptr = nullptr;
+  qp.item_tab = nullptr;
   qp.n_kb = 0; qp.S = D.S; qp.Nb = 1; qp.sb = D.S; qp.BH = D.BH; qp.scale = D.scale; qp.scale_log2 = D.scale * LOG2E;
   qp.capacity = 0; qp.dq_acc = nullptr; qp.dq = (__nv_bfloat16*)dq; qp.status = status; qp.q_ptr = nullptr;
-  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)DQ_SMEM_BYTES));
-  attn_bwd_dq_tc_kernel<true><<<grid_items(D.BH * tiles), DQ_THREADS, DQ_SMEM_BYTES, st>>>(tmK, tmV, qp);
+  {
+    constexpr size_t SM = dq_smem_bytes(1, 4);
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<true, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM));
+    attn_bwd_dq_tc_kernel<true, 1, 4><<<grid_items(D.BH * tiles), DQ_THREADS, SM, st>>>(tmK64, tmV64, qp);
+  }
   VMOBA_LAUNCH_OK(2);
   return VMOBA_OK;
 }
