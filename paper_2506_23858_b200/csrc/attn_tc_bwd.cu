@@ -111,11 +111,11 @@ struct KvSmem {
   uint64_t acc_free;                         // epilogue has read dV / dK (128 compute arrivals)
   uint32_t tmem_base;
   int abort_flag;
-  float lse2[NQ][QC];
-  float Dq[NQ][QC];
+  alignas(16) float lse2[NQ][QC];
+  alignas(16) float Dq[NQ][QC];
 };
 constexpr size_t KV_SMEM_BYTES = 1024 + 4 * TILE + NQ * 2 * CTILE + sizeof(KvSmem) + 32;
-constexpr int KV_THREADS = 320;
+constexpr int KV_THREADS = 448;   // TMA, MMA, 8 compute warps, 4 loader warps
 constexpr uint32_t IDESC_K64 = make_idesc_bf16(128, QC, false, false);   // S^T, dP^T: N = 64 queries
 
 struct KvParams {
@@ -199,11 +199,11 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   if (threadIdx.x == 0) {
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sm->kv_full[b], 1); mbar_init(&sm->kv_empty[b], 1);
-      mbar_init(&sm->sdp_full[b], 1); mbar_init(&sm->pds_ready[b], 128);
+      mbar_init(&sm->sdp_full[b], 1); mbar_init(&sm->pds_ready[b], 256);
     }
     for (int b = 0; b < NQ; ++b) { mbar_init(&sm->chunk_full[b], 128); mbar_init(&sm->chunk_empty[b], 1); }
     mbar_init(&sm->acc_done, 1);
-    mbar_init(&sm->acc_free, 128);
+    mbar_init(&sm->acc_free, 256);
     sm->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmK);
@@ -280,10 +280,13 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           const int rows = (int)min((long long)QC, it.list_hi - it.list_lo - (long long)i * QC);
           const int ksteps = (rows + 15) >> 4;
           const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE), sdO_addr = sQ_addr + CTILE;
+          // P^T / dS^T of queries 32h .. 32h+31 sit in columns 32h .. 32h+15 of their buffer
           for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(tmem + DV_COL, tmem + ST_COL + tb * QC + ks * 8, cdesc_mn(sdO_addr, ks), IDESC_TN, (i > 0 || ks > 0) ? 1u : 0u);
+            mma_ts(tmem + DV_COL, tmem + ST_COL + tb * QC + (ks >> 1) * 32 + (ks & 1) * 8, cdesc_mn(sdO_addr, ks), IDESC_TN,
+                   (i > 0 || ks > 0) ? 1u : 0u);
           for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(tmem + DK_COL, tmem + DPT_COL + tb * QC + ks * 8, cdesc_mn(sQ_addr, ks), IDESC_TN, (i > 0 || ks > 0) ? 1u : 0u);
+            mma_ts(tmem + DK_COL, tmem + DPT_COL + tb * QC + (ks >> 1) * 32 + (ks & 1) * 8, cdesc_mn(sQ_addr, ks), IDESC_TN,
+                   (i > 0 || ks > 0) ? 1u : 0u);
           mma_commit(&sm->chunk_empty[cb]);
         }
         mma_commit(&sm->kv_empty[b]);
@@ -292,9 +295,9 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         ++n;
       }
     }
-  } else if (warp >= 6) {
+  } else if (warp >= 10) {
     // ------------------------------------------------------------------ loaders: gather Q / dO chunks (run ahead)
-    const int lt = threadIdx.x - 192;   // 0..127
+    const int lt = threadIdx.x - 320;   // 0..127
     uint32_t u0 = 0;
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
       const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
@@ -324,8 +327,9 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       u0 += it.n_units;
     }
   } else {
-    // ------------------------------------------------------------------ compute: thread = key row
+    // ------------------------------------------------------------------ compute: thread = (key row, half of the unit's queries)
     const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;                 // warps 2-5: queries 0-31 of a unit, warps 6-9: queries 32-63
     const int r = quad * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     uint32_t n = 0, u0 = 0;
@@ -338,7 +342,10 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         if (r < it.valid) {
           const uint4 z = make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-          for (int i = 0; i < 16; ++i) { reinterpret_cast<uint4*>(dk_row)[i] = z; reinterpret_cast<uint4*>(dv_row)[i] = z; }
+          for (int i = 0; i < 8; ++i) {
+            reinterpret_cast<uint4*>(dk_row)[half * 8 + i] = z;
+            reinterpret_cast<uint4*>(dv_row)[half * 8 + i] = z;
+          }
         }
         continue;
       }
@@ -348,37 +355,39 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         mbar_wait(&sm->chunk_full[cb], (u / NQ) & 1, abort_flag, p.status);   // publishes lse2 / Dq of this unit
         mbar_wait(&sm->sdp_full[tb], (u >> 1) & 1, abort_flag, p.status);
         tc_fence_after();
-        const float* lse2 = sm->lse2[cb];
-        const float* Dq = sm->Dq[cb];
-        const uint32_t st_t = tmem + lane_addr + ST_COL + tb * QC, dp_t = tmem + lane_addr + DPT_COL + tb * QC;
-        uint32_t sv[2][32], dv_[2][32];
-        tmem_ld32(st_t, sv[0]);
-        tmem_ld32(st_t + 32, sv[1]);
-        tmem_ld32(dp_t, dv_[0]);
-        tmem_ld32(dp_t + 32, dv_[1]);
+        const float4* lse2 = reinterpret_cast<const float4*>(sm->lse2[cb] + 32 * half);
+        const float4* Dq = reinterpret_cast<const float4*>(sm->Dq[cb] + 32 * half);
+        const uint32_t st_t = tmem + lane_addr + ST_COL + tb * QC + 32 * half;
+        const uint32_t dp_t = tmem + lane_addr + DPT_COL + tb * QC + 32 * half;
+        uint32_t sv[32], dv_[32];
+        tmem_ld32(st_t, sv);
+        tmem_ld32(dp_t, dv_);
         tmem_ld_wait();
-        uint32_t pk[32], dk_[32];
+        uint32_t pk[16], dk_[16];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int q0 = 2 * e;
-          const float s0 = __uint_as_float(sv[e >> 4][(2 * e) & 31]), s1 = __uint_as_float(sv[e >> 4][((2 * e) & 31) + 1]);
-          const float d0 = __uint_as_float(dv_[e >> 4][(2 * e) & 31]), d1 = __uint_as_float(dv_[e >> 4][((2 * e) & 31) + 1]);
-          const float p0 = ex2(fmaf(s0, p.scale_log2, -lse2[q0]));
-          const float p1 = ex2(fmaf(s1, p.scale_log2, -lse2[q0 + 1]));
-          pk[e] = pack_bf16(p0, p1);
-          dk_[e] = pack_bf16(p0 * (d0 - Dq[q0]), p1 * (d1 - Dq[q0 + 1]));
+        for (int e = 0; e < 8; ++e) {
+          const float4 l4 = lse2[e], d4 = Dq[e];
+          const float p0 = ex2(fmaf(__uint_as_float(sv[4 * e]), p.scale_log2, -l4.x));
+          const float p1 = ex2(fmaf(__uint_as_float(sv[4 * e + 1]), p.scale_log2, -l4.y));
+          const float p2 = ex2(fmaf(__uint_as_float(sv[4 * e + 2]), p.scale_log2, -l4.z));
+          const float p3 = ex2(fmaf(__uint_as_float(sv[4 * e + 3]), p.scale_log2, -l4.w));
+          pk[2 * e] = pack_bf16(p0, p1);
+          pk[2 * e + 1] = pack_bf16(p2, p3);
+          dk_[2 * e] = pack_bf16(p0 * (__uint_as_float(dv_[4 * e]) - d4.x), p1 * (__uint_as_float(dv_[4 * e + 1]) - d4.y));
+          dk_[2 * e + 1] = pack_bf16(p2 * (__uint_as_float(dv_[4 * e + 2]) - d4.z), p3 * (__uint_as_float(dv_[4 * e + 3]) - d4.w));
         }
-        tmem_st32(st_t, pk);       // P^T (bf16 pairs) over the first 32 columns of this S^T buffer
-        tmem_st32(dp_t, dk_);      // dS^T over the first 32 columns of this dP^T buffer
+        tmem_st16(st_t, pk);       // P^T (bf16 pairs) over the first 16 of this thread's 32 S^T columns
+        tmem_st16(dp_t, dk_);      // dS^T likewise over its dP^T columns
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(&sm->pds_ready[tb]);
       }
-      // ---- epilogue: dV and dK rows of this tile
+      // ---- epilogue: each half writes 64 of the 128 dV / dK columns of its key row
       mbar_wait(&sm->acc_done, n & 1, abort_flag, p.status);
       tc_fence_after();
 #pragma unroll 1
-      for (int cgrp = 0; cgrp < 4; ++cgrp) {
+      for (int cg2 = 0; cg2 < 2; ++cg2) {
+        const int cgrp = half * 2 + cg2;
         uint32_t a[32], bb[32];
         tmem_ld32(tmem + lane_addr + DV_COL + cgrp * 32, a);
         tmem_ld32(tmem + lane_addr + DK_COL + cgrp * 32, bb);
@@ -432,7 +441,7 @@ struct DqSmem {
   int direct[2][128];                        // query has a single block: write bf16 directly
 };
 constexpr size_t dq_smem_bytes(int QB, int NS) { return 1024 + QB * 2 * TILE + NS * 2 * CTILE + sizeof(DqSmem) + 32; }
-constexpr int DQ_THREADS = 320;
+constexpr int DQ_THREADS = 448;   // TMA, MMA, 8 compute warps, 4 loader warps
 
 struct DqParams {
   const __nv_bfloat16 *q, *d_o;
@@ -489,8 +498,8 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
     for (int s = 0; s < DQ_NS; ++s) { mbar_init(&sm->kv_full[s], 1); mbar_init(&sm->kv_empty[s], 1); }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sm->qdo_full[b], 128); mbar_init(&sm->qdo_empty[b], 1);
-      mbar_init(&sm->sdp_full[b], 1); mbar_init(&sm->ds_ready[b], 128);
-      mbar_init(&sm->dq_done[b], 1); mbar_init(&sm->dq_free[b], 128);
+      mbar_init(&sm->sdp_full[b], 1); mbar_init(&sm->ds_ready[b], 256);
+      mbar_init(&sm->dq_done[b], 1); mbar_init(&sm->dq_free[b], 256);
     }
     sm->abort_flag = 0;
     fence_barrier_init();
@@ -569,9 +578,10 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
           tc_fence_after();
           const int ksteps = n_mma_of(i) >> 4;
           const uint32_t sK_addr = smem_u32(sKV + s * 2 * CTILE);
+          // dS of keys 32h .. 32h+31 sits in columns 32h .. 32h+15 of the dP buffer
           for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(tmem + DQ_COL + qb * 128, tmem + DP_COL + tb * KU + ks * 8, cdesc_mn(sK_addr, ks), IDESC_TN,
-                   (i > 0 || ks > 0) ? 1u : 0u);
+            mma_ts(tmem + DQ_COL + qb * 128, tmem + DP_COL + tb * KU + (ks >> 1) * 32 + (ks & 1) * 8, cdesc_mn(sK_addr, ks),
+                   IDESC_TN, (i > 0 || ks > 0) ? 1u : 0u);
           mma_commit(&sm->kv_empty[s]);
         }
         mma_commit(&sm->qdo_empty[qs]);
@@ -579,9 +589,9 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         u0 += it.n_units;
       }
     }
-  } else if (warp >= 6) {
+  } else if (warp >= 10) {
     // ------------------------------------------------------------------ loaders: Q / dO rows of the next items
-    const int lt = threadIdx.x - 192;   // 0..127
+    const int lt = threadIdx.x - 320;   // 0..127
     uint32_t n = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
       const DqItem it = dq_decode<DENSE>(p, item);
@@ -597,22 +607,23 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
         dd = p.Dv[G_];
         if (!DENSE) direct = (p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1;
       }
-      uint4 vq[16], vo[16];
+      uint4 vq[16];
       gather_load128(p.q + it.head_off * DH, it.n_rows, lt, row_of, vq);
-      gather_load128(p.d_o + it.head_off * DH, it.n_rows, lt, row_of, vo);
       if (n >= QB) mbar_wait(&sm->qdo_empty[qs], ((n / QB) - 1) & 1, abort_flag, p.status);
       // the scalar slots alternate by item; with a single Q / dO tile the compute warps may still be
       // reading slot qb of item n-2 only if they lag two items behind, which qdo_empty(n-1) excludes
       uint8_t* dst = sQdO + qs * 2 * TILE;
       gather_store128(dst, lt, vq);
-      gather_store128(dst + TILE, lt, vo);
+      gather_load128(p.d_o + it.head_off * DH, it.n_rows, lt, row_of, vq);
+      gather_store128(dst + TILE, lt, vq);
       sm->lse2[qb][lt] = l2; sm->Dr[qb][lt] = dd; sm->G[qb][lt] = G_; sm->direct[qb][lt] = direct;
       fence_async_proxy();
       mbar_arrive(&sm->qdo_full[qs]);
     }
   } else {
-    // ------------------------------------------------------------------ compute: thread = query row
+    // ------------------------------------------------------------------ compute: thread = (query row, half of the unit's keys)
     const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;                 // warps 2-5: keys 0-31 of a unit, warps 6-9: keys 32-63
     const int r = quad * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     uint32_t n = 0, u0 = 0;
@@ -626,39 +637,36 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
       for (int i = 0; i < it.n_units; ++i) {
         const uint32_t u = u0 + i;
         const int tb = u & 1;
-        const int valid = min(KU, it.n_keys - i * KU);
+        const int valid = min(KU, it.n_keys - i * KU) - 32 * half;     // valid keys among this thread's 32
         mbar_wait(&sm->sdp_full[tb], (u >> 1) & 1, abort_flag, p.status);
         tc_fence_after();
-        const uint32_t s_t = tmem + lane_addr + S_COL + tb * KU, dp_t = tmem + lane_addr + DP_COL + tb * KU;
-        uint32_t sv[2][32], dv_[2][32];
-        tmem_ld32(s_t, sv[0]);
-        tmem_ld32(s_t + 32, sv[1]);
-        tmem_ld32(dp_t, dv_[0]);
-        tmem_ld32(dp_t + 32, dv_[1]);
+        const uint32_t s_t = tmem + lane_addr + S_COL + tb * KU + 32 * half;
+        const uint32_t dp_t = tmem + lane_addr + DP_COL + tb * KU + 32 * half;
+        uint32_t sv[32], dv_[32];
+        tmem_ld32(s_t, sv);
+        tmem_ld32(dp_t, dv_);
         tmem_ld_wait();
-        uint32_t ds[32];
+        uint32_t ds[16];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int k0 = 2 * e;
-          const float s0 = __uint_as_float(sv[e >> 4][(2 * e) & 31]), s1 = __uint_as_float(sv[e >> 4][((2 * e) & 31) + 1]);
-          const float d0 = __uint_as_float(dv_[e >> 4][(2 * e) & 31]), d1 = __uint_as_float(dv_[e >> 4][((2 * e) & 31) + 1]);
-          const float p0 = ex2(fmaf(s0, p.scale_log2, -lse2));
-          const float p1 = ex2(fmaf(s1, p.scale_log2, -lse2));
-          const float x0 = (k0 < valid) ? p0 * (d0 - Dr) : 0.f;
-          const float x1 = (k0 + 1 < valid) ? p1 * (d1 - Dr) : 0.f;
+        for (int e = 0; e < 16; ++e) {
+          const float p0 = ex2(fmaf(__uint_as_float(sv[2 * e]), p.scale_log2, -lse2));
+          const float p1 = ex2(fmaf(__uint_as_float(sv[2 * e + 1]), p.scale_log2, -lse2));
+          const float x0 = (2 * e < valid) ? p0 * (__uint_as_float(dv_[2 * e]) - Dr) : 0.f;
+          const float x1 = (2 * e + 1 < valid) ? p1 * (__uint_as_float(dv_[2 * e + 1]) - Dr) : 0.f;
           ds[e] = pack_bf16(x0, x1);
         }
-        tmem_st32(dp_t, ds);      // dS (bf16 pairs) over the first 32 columns of this dP buffer
+        tmem_st16(dp_t, ds);      // dS (bf16 pairs) over the first 16 of this thread's 32 dP columns
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(&sm->ds_ready[tb]);
       }
       u0 += it.n_units;
-      // ---- epilogue
+      // ---- epilogue: each half writes 64 of the 128 dQ columns of its row
       mbar_wait(&sm->dq_done[qb], (n >> 1) & 1, abort_flag, p.status);
       tc_fence_after();
 #pragma unroll 1
-      for (int cgrp = 0; cgrp < 4; ++cgrp) {
+      for (int cg2 = 0; cg2 < 2; ++cg2) {
+        const int cgrp = half * 2 + cg2;
         uint32_t a[32];
         tmem_ld32(tmem + lane_addr + DQ_COL + qb * 128 + cgrp * 32, a);
         tmem_ld_wait();
