@@ -82,6 +82,12 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
+// Descriptor arithmetic: the start-address field sits in the low 14 bits (in 16-byte units), so a
+// byte offset inside the tile is a plain add on the descriptor (the MMA-issuing thread must not
+// rebuild descriptors per instruction: it is the serial bottleneck of these kernels).
+__device__ __forceinline__ constexpr uint32_t koff(int ks, int panel_bytes) { return (uint32_t)(((ks >> 2) * panel_bytes + (ks & 3) * 32) >> 4); }
+__device__ __forceinline__ constexpr uint32_t mnoff(int ks) { return (uint32_t)((ks * 2048) >> 4); }
+
 // K-major operand descriptor for k-step ks (16 of the 128 head-dim columns) of a swizzled tile.
 __device__ __forceinline__ uint64_t desc_k(uint32_t tile_addr, int ks) {
   return make_smem_desc(tile_addr + (ks >> 2) * PANEL + (ks & 3) * 32, 16, 1024);
@@ -127,6 +133,7 @@ struct KvParams {
   long long capacity;
   __nv_bfloat16 *dk, *dv;
   int32_t* status;
+  unsigned long long* prof;    // optional wait-time counters (diagnostics), or null
 };
 
 // 16 threads per row: gather `n_rows` (<= 64) 256-byte rows into a swizzled [64 x 128] chunk tile.
@@ -195,6 +202,24 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   KvSmem* sm = reinterpret_cast<KvSmem*>(sC + NQ * 2 * CTILE);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm->abort_flag;
+  // diagnostics: cycles spent in each wait site by one representative thread per role
+  unsigned long long wp[4] = {0, 0, 0, 0};
+  const long long t_begin = clock64();
+  auto twait = [&](int site, uint64_t* bar, uint32_t parity) {
+    if (p.prof) {
+      const long long t0 = clock64();
+      mbar_wait(bar, parity, abort_flag, p.status);
+      wp[site] += (unsigned long long)(clock64() - t0);
+    } else {
+      mbar_wait(bar, parity, abort_flag, p.status);
+    }
+  };
+  auto tflush = [&](int base_site, int nsites) {
+    if (p.prof) {
+      for (int i = 0; i < nsites; ++i) atomicAdd(p.prof + base_site + i, wp[i]);
+      atomicAdd(p.prof + base_site + nsites, (unsigned long long)(clock64() - t_begin));
+    }
+  };
 
   if (threadIdx.x == 0) {
     for (int b = 0; b < 2; ++b) {
@@ -231,7 +256,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
         if (it.n_units == 0) continue;
         const int b = n & 1;
-        if (n >= 2) mbar_wait(&sm->kv_empty[b], ((n >> 1) - 1) & 1, abort_flag, p.status);
+        if (n >= 2) twait(0, &sm->kv_empty[b], ((n >> 1) - 1) & 1);
         const int y = (int)it.head_off + it.key0;
         mbar_expect_tx(&sm->kv_full[b], 2 * TILE);
         tma_load_2d(sK + b * TILE, &tmK, &sm->kv_full[b], 0, y);
@@ -242,6 +267,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       }
       if (*abort_flag)
         for (uint32_t f = n > 2 ? n - 2 : 0; f < n; ++f) mbar_wait(&sm->kv_full[f & 1], (f >> 1) & 1, abort_flag, p.status);
+      tflush(0, 1);      // [0] kv_empty, [1] total
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -251,21 +277,23 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
         if (it.n_units == 0) continue;
         const int b = n & 1;
-        mbar_wait(&sm->kv_full[b], (n >> 1) & 1, abort_flag, p.status);
+        twait(0, &sm->kv_full[b], (n >> 1) & 1);
         tc_fence_after();
-        const uint32_t sK_addr = smem_u32(sK + b * TILE), sV_addr = smem_u32(sV + b * TILE);
+        const uint64_t dK0 = desc_k(smem_u32(sK + b * TILE), 0), dV0 = desc_k(smem_u32(sV + b * TILE), 0);
         auto issue_sdp = [&](int i) {
           const uint32_t u = u0 + i;
           const int cb = u % NQ, tb = u & 1;
-          mbar_wait(&sm->chunk_full[cb], (u / NQ) & 1, abort_flag, p.status);
+          twait(1, &sm->chunk_full[cb], (u / NQ) & 1);
           tc_fence_after();
-          const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE), sdO_addr = sQ_addr + CTILE;
+          const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE);
+          const uint64_t dQ0 = cdesc_k(sQ_addr, 0), dO0 = cdesc_k(sQ_addr + CTILE, 0);
+          const uint32_t st = tmem + ST_COL + tb * QC, dp = tmem + DPT_COL + tb * QC;
+          // the two accumulation chains are independent: interleave them
 #pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks)
-            mma_ss(tmem + ST_COL + tb * QC, desc_k(sK_addr, ks), cdesc_k(sQ_addr, ks), IDESC_K64, ks > 0 ? 1u : 0u);
-#pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks)
-            mma_ss(tmem + DPT_COL + tb * QC, desc_k(sV_addr, ks), cdesc_k(sdO_addr, ks), IDESC_K64, ks > 0 ? 1u : 0u);
+          for (int ks = 0; ks < DH / 16; ++ks) {
+            mma_ss(st, dK0 + koff(ks, PANEL), dQ0 + koff(ks, CPANEL), IDESC_K64, ks > 0 ? 1u : 0u);
+            mma_ss(dp, dV0 + koff(ks, PANEL), dO0 + koff(ks, CPANEL), IDESC_K64, ks > 0 ? 1u : 0u);
+          }
           mma_commit(&sm->sdp_full[tb]);
         };
         issue_sdp(0);
@@ -273,20 +301,23 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           if (i + 1 < it.n_units) issue_sdp(i + 1);
           const uint32_t u = u0 + i;
           const int cb = u % NQ, tb = u & 1;
-          mbar_wait(&sm->pds_ready[tb], (u >> 1) & 1, abort_flag, p.status);
+          twait(2, &sm->pds_ready[tb], (u >> 1) & 1);
           // dV / dK still hold the previous item until its epilogue has read them
-          if (i == 0 && n > 0) mbar_wait(&sm->acc_free, (n - 1) & 1, abort_flag, p.status);
+          if (i == 0 && n > 0) twait(3, &sm->acc_free, (n - 1) & 1);
           tc_fence_after();
           const int rows = (int)min((long long)QC, it.list_hi - it.list_lo - (long long)i * QC);
           const int ksteps = (rows + 15) >> 4;
-          const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE), sdO_addr = sQ_addr + CTILE;
+          const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE);
+          const uint64_t mQ0 = cdesc_mn(sQ_addr, 0), mO0 = cdesc_mn(sQ_addr + CTILE, 0);
+          const uint32_t pt = tmem + ST_COL + tb * QC, dst_ = tmem + DPT_COL + tb * QC;
+          const uint32_t acc0 = i > 0 ? 1u : 0u;
           // P^T / dS^T of queries 32h .. 32h+31 sit in columns 32h .. 32h+15 of their buffer
-          for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(tmem + DV_COL, tmem + ST_COL + tb * QC + (ks >> 1) * 32 + (ks & 1) * 8, cdesc_mn(sdO_addr, ks), IDESC_TN,
-                   (i > 0 || ks > 0) ? 1u : 0u);
-          for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(tmem + DK_COL, tmem + DPT_COL + tb * QC + (ks >> 1) * 32 + (ks & 1) * 8, cdesc_mn(sQ_addr, ks), IDESC_TN,
-                   (i > 0 || ks > 0) ? 1u : 0u);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            if (ks < ksteps) {
+              mma_ts(tmem + DV_COL, pt + (ks >> 1) * 32 + (ks & 1) * 8, mO0 + mnoff(ks), IDESC_TN, ks > 0 ? 1u : acc0);
+              mma_ts(tmem + DK_COL, dst_ + (ks >> 1) * 32 + (ks & 1) * 8, mQ0 + mnoff(ks), IDESC_TN, ks > 0 ? 1u : acc0);
+            }
           mma_commit(&sm->chunk_empty[cb]);
         }
         mma_commit(&sm->kv_empty[b]);
@@ -294,6 +325,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         u0 += it.n_units;
         ++n;
       }
+      tflush(2, 4);      // [2] kv_full, [3] chunk_full, [4] pds_ready, [5] acc_free, [6] total
     }
   } else if (warp >= 10) {
     // ------------------------------------------------------------------ loaders: gather Q / dO chunks (run ahead)
@@ -316,7 +348,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           l2 = p.lse[G_] * LOG2E;
           dd = p.Dv[G_];
         }
-        if (u >= NQ) mbar_wait(&sm->chunk_empty[cb], ((u / NQ) - 1) & 1, abort_flag, p.status);
+        if (u >= NQ) twait(0, &sm->chunk_empty[cb], ((u / NQ) - 1) & 1);
         uint8_t* dst = sC + cb * 2 * CTILE;
         store_chunk64(dst, lt, vq);
         store_chunk64(dst + CTILE, lt, vo);
@@ -326,6 +358,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       }
       u0 += it.n_units;
     }
+    if (lt == 0) tflush(7, 1);     // [7] chunk_empty, [8] total
   } else {
     // ------------------------------------------------------------------ compute: thread = (key row, half of the unit's queries)
     const int quad = warp & 3;
@@ -352,8 +385,8 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       for (int i = 0; i < it.n_units; ++i) {
         const uint32_t u = u0 + i;
         const int cb = u % NQ, tb = u & 1;
-        mbar_wait(&sm->chunk_full[cb], (u / NQ) & 1, abort_flag, p.status);   // publishes lse2 / Dq of this unit
-        mbar_wait(&sm->sdp_full[tb], (u >> 1) & 1, abort_flag, p.status);
+        twait(0, &sm->chunk_full[cb], (u / NQ) & 1);   // publishes lse2 / Dq of this unit
+        twait(1, &sm->sdp_full[tb], (u >> 1) & 1);
         tc_fence_after();
         const float4* lse2 = reinterpret_cast<const float4*>(sm->lse2[cb] + 32 * half);
         const float4* Dq = reinterpret_cast<const float4*>(sm->Dq[cb] + 32 * half);
@@ -383,7 +416,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         mbar_arrive(&sm->pds_ready[tb]);
       }
       // ---- epilogue: each half writes 64 of the 128 dV / dK columns of its key row
-      mbar_wait(&sm->acc_done, n & 1, abort_flag, p.status);
+      twait(2, &sm->acc_done, n & 1);
       tc_fence_after();
 #pragma unroll 1
       for (int cg2 = 0; cg2 < 2; ++cg2) {
@@ -408,6 +441,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       u0 += it.n_units;
       ++n;
     }
+    if (threadIdx.x == 64) tflush(10, 3);   // [10] chunk_full, [11] sdp_full, [12] acc_done, [13] total
   }
   tc_fence_before();
   __syncthreads();
@@ -695,6 +729,10 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
+// Diagnostics: when a device buffer of 16 counters is registered, the dK/dV kernel adds the cycles
+// its roles spend in each wait (one representative thread per role and CTA).
+static unsigned long long* g_wait_profile = nullptr;
+
 static int grid_items(long long items) { return (int)std::max<long long>(1, std::min<long long>(items, 148)); }
 
 }  // namespace tcb
@@ -716,7 +754,7 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
   kp.q = (const __nv_bfloat16*)q; kp.d_o = (const __nv_bfloat16*)d_o; kp.lse = lse; kp.Dv = Dv;
   kp.kb_ptr = kb_ptr; kp.q_idx = q_idx; kp.S = D.S; kp.Nb = D.Nb; kp.sb = D.sb; kp.BH = D.BH;
   kp.scale = D.scale; kp.scale_log2 = D.scale * LOG2E; kp.capacity = cap;
-  kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status;
+  kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status; kp.prof = tcb::g_wait_profile;
   VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)KV_SMEM_BYTES));
   const long long kv_items = n_kb * ((D.sb + BN - 1) / BN);
@@ -752,7 +790,7 @@ int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, con
   kp.q = (const __nv_bfloat16*)q; kp.d_o = (const __nv_bfloat16*)d_o; kp.lse = lse; kp.Dv = Dv;
   kp.kb_ptr = nullptr; kp.q_idx = nullptr; kp.S = D.S; kp.Nb = 1; kp.sb = D.S; kp.BH = D.BH;
   kp.scale = D.scale; kp.scale_log2 = D.scale * LOG2E; kp.capacity = 0;
-  kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status;
+  kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status; kp.prof = tcb::g_wait_profile;
   VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)KV_SMEM_BYTES));
   const long long tiles = (D.S + BN - 1) / BN;
@@ -772,3 +810,9 @@ int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, con
 }
 
 }  // namespace vmoba
+
+// Registers (or clears, with null) a device buffer of 16 uint64 counters for the dK/dV kernel's
+// wait-time diagnostics.  Not part of the method; see the kernel for the counter layout.
+extern "C" void vmoba_debug_wait_profile(void* dev_counters16) {
+  vmoba::tcb::g_wait_profile = static_cast<unsigned long long*>(dev_counters16);
+}
