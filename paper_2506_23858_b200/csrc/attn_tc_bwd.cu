@@ -30,6 +30,9 @@ constexpr int PANEL = 128 * 128;
 constexpr int TILE = 2 * PANEL;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr float LOG2E = 1.4426950408889634f;
+// Diagnostics: when a device buffer of 16 counters is registered, the dK/dV kernels add the cycles
+// their roles spend in each wait (one representative thread per role and CTA).
+static unsigned long long* g_wait_profile = nullptr;
 constexpr uint32_t IDESC_KK = make_idesc_bf16(128, 128, false, false);   // A, B both K-major in shared memory
 constexpr uint32_t IDESC_TN = make_idesc_bf16(128, 128, false, true);    // A from TMEM, B MN-major
 
@@ -729,13 +732,18 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_cons
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-// Diagnostics: when a device buffer of 16 counters is registered, the dK/dV kernel adds the cycles
-// its roles spend in each wait (one representative thread per role and CTA).
-static unsigned long long* g_wait_profile = nullptr;
-
 static int grid_items(long long items) { return (int)std::max<long long>(1, std::min<long long>(items, 148)); }
 
 }  // namespace tcb
+
+// attn_tc_bwd_long.cu
+int tc_long_dkdv(const Dims& D, bool dense, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                 const float* Dv, const int* kb_ptr, const int* q_idx, long long cap, void* dk, void* dv, int32_t* status,
+                 unsigned long long* prof, cudaStream_t st);
+int tc_long_dq(const Dims& D, bool dense, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+               const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap, const int* item_ptr,
+               const int* item_tab, float* dq_acc, void* dq, int32_t* status, cudaStream_t st);
+static bool use_long_kernels(const Dims& D) { (void)D; return false; }   // measured slower than the 64-column unit kernels on every sparse workload tried
 
 // Backward over the work lists (bf16, head_dim 128).  Dv holds rowsum(dO * O) per query; dq_acc is
 // a zeroed fp32 accumulator that the caller converts to bf16 afterwards.
@@ -743,6 +751,11 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
                   const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap,
                   const int* item_ptr, const int* item_tab, float* dq_acc, void* dq, void* dk, void* dv,
                   int32_t* status, cudaStream_t st) {
+  if (use_long_kernels(D)) {
+    int rc = tc_long_dkdv(D, false, q, k, v, d_o, lse, Dv, kb_ptr, q_idx, cap, dk, dv, status, tcb::g_wait_profile, st);
+    if (rc) return rc;
+    return tc_long_dq(D, false, q, k, v, d_o, lse, Dv, kb_ptr, q_idx, q_ptr, cap, item_ptr, item_tab, dq_acc, dq, status, st);
+  }
   using namespace tcb;
   CUtensorMap tmK, tmV, tmK64, tmV64;
   const uint64_t rows = (uint64_t)D.BH * D.S;
@@ -780,6 +793,11 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
 
 int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* Dv, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st) {
+  {
+    int rc = tc_long_dkdv(D, true, q, k, v, d_o, lse, Dv, nullptr, nullptr, 0, dk, dv, status, tcb::g_wait_profile, st);
+    if (rc) return rc;
+    return tc_long_dq(D, true, q, k, v, d_o, lse, Dv, nullptr, nullptr, nullptr, 0, nullptr, nullptr, nullptr, dq, status, st);
+  }
   using namespace tcb;
   CUtensorMap tmK, tmV, tmK64, tmV64;
   const uint64_t rows = (uint64_t)D.BH * D.S;

@@ -67,6 +67,24 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
       : "memory");
 }
+// Row gather: four rows (given by their row coordinates) of a 2D tensor whose map has a one-row
+// box of 64 columns; the rows land in four consecutive 128-byte rows at smem_dst with the same
+// 128-byte swizzle a tiled load produces, so a 128-row operand tile is 32 of these per panel.
+__device__ __forceinline__ void tma_gather4(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int col, int r0, int r1,
+                                            int r2, int r3) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, "
+      "%6, %7}], [%2];" ::"r"(smem_u32(smem_dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+      : "memory");
+}
+// One warp gathers a [128 x 128] bf16 tile (two 64-column panels of 16 KB): lane l fetches tile rows
+// 4l .. 4l+3.  rows[k] are absolute row coordinates of this lane's four rows.
+__device__ __forceinline__ void tma_gather_tile128(uint8_t* tile, const CUtensorMap* map, uint64_t* bar, int lane,
+                                                   const int (&rows)[4]) {
+  tma_gather4(tile + lane * 512, map, bar, 0, rows[0], rows[1], rows[2], rows[3]);
+  tma_gather4(tile + 16384 + lane * 512, map, bar, 64, rows[0], rows[1], rows[2], rows[3]);
+}
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
