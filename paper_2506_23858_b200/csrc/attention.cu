@@ -13,7 +13,8 @@ size_t scores_ws_bytes(const Dims& D);   // scores.cu
 // attn_tc.cu: tensor-core forward kernels (bf16, head_dim 128)
 int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                   const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
-                  int32_t* status, int* item_ptr, float* part_o, float* part_lse, cudaStream_t st);
+                  int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o, float* part_lse,
+                  cudaStream_t st);
 int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, void* o, void* o_resid, float* lse,
                  int32_t* status, cudaStream_t st);
 
@@ -27,18 +28,19 @@ int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, con
 
 static bool use_tensor_cores(const Dims& D) { return D.dtype == VMOBA_BF16 && D.d == 128; }
 
-struct FwdWs { int* item_ptr; float* part_o; float* part_lse; size_t bytes; };
+static long long max_items_128(const Dims& D, long long cap) { return cap / 128 + (long long)D.BH * D.Nb + 1; }
+
+struct FwdWs { int* item_ptr; int* item_tab; float* part_o; float* part_lse; size_t bytes; };
 static FwdWs carve_fwd(const Dims& D, long long cap, void* ws) {
   Carver c(ws);
   FwdWs w;
   w.item_ptr = c.take<int>((size_t)D.BH * D.Nb + 1);
+  w.item_tab = c.take<int>((size_t)max_items_128(D, cap));
   w.part_lse = c.take<float>((size_t)cap);
   w.part_o = c.take<float>((size_t)cap * D.d);
   w.bytes = c.total();
   return w;
 }
-
-static long long max_items_128(const Dims& D, long long cap) { return cap / 128 + (long long)D.BH * D.Nb + 1; }
 
 struct BwdWs { int* item_ptr; int* item_tab; float* Dv; float* dq_acc; void* o_resid; size_t bytes; };
 static BwdWs carve_bwd(const Dims& D, bool dense, void* ws, long long cap = 0) {
@@ -209,7 +211,7 @@ extern "C" int vmoba_attn_fwd(const vmoba_shape* shape, const void* q_bm, const 
   if (use_tensor_cores(D)) {
     FwdWs w = carve_fwd(D, capacity, ws);
     return tc_sparse_fwd(D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null, lse,
-                         dev_status, w.item_ptr, w.part_o, w.part_lse, st);
+                         dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse, st);
   }
   VMOBA_DISPATCH(simt_sparse_fwd, D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null,
                  lse, ws, st);

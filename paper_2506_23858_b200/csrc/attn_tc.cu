@@ -4,17 +4,19 @@
 // the queries that selected key block j, gathered by index; dense: 128 consecutive rows) against
 // a contiguous key range (the block, or the whole sequence), streamed in tiles of 128 keys:
 //
-//   warp 0      TMA producer: K and V tiles (two 64-column panels each, 128-byte swizzle) into a
-//               3-stage ring, completion on mbarriers
-//   warp 1      MMA issuer (one thread): S = Q K^T into one of two TMEM score buffers, then
-//               O += P V with P read from TMEM; tcgen05.commit signals the other roles
-//   warps 2-5   softmax: thread = query row.  Reads S from TMEM, online softmax in the exp2
-//               domain, writes P (bf16) over S in TMEM, rescales O in TMEM only when the running
-//               max moved by more than 2^8, and runs the epilogue (normalise, write O / partials)
+//   warp 0       TMA producer: K and V tiles (two 64-column panels each, 128-byte swizzle) into a
+//                2-stage ring
+//   warp 1       MMA issuer (one thread): S = Q K^T into one of two TMEM score buffers, then
+//                O += P V with P read from TMEM; tcgen05.commit signals the other roles
+//   warps 2-9    softmax: thread = (query row, 64 of the tile's 128 keys).  The two threads of a row
+//                exchange their maxima through shared memory, run the online softmax in the exp2
+//                domain, write P (bf16) over their own score columns, rescale O only when the
+//                running max moved by more than 2^8, and run the epilogue
+//   warps 10-13  loaders: gather the Q rows (and the per-row output bookkeeping) of the NEXT item
 //
-// QK^T of tile t+1 is issued before P V of tile t, so the tensor pipe works on the next scores
-// while the softmax warps process the current ones.  TMEM: 2 x 128 columns of scores (P aliases the
-// first 64 columns of its score buffer) + 128 columns of O.
+// Q tiles and the O accumulator are double buffered across items, so gather, MMAs and epilogue of
+// neighbouring items overlap; QK^T of tile t+1 is issued before P V of tile t.
+// TMEM: 2 x 128 columns of scores (P aliases them) + 2 x 128 columns of O.
 #include <algorithm>
 
 #include "attn_simt.cuh"
@@ -28,22 +30,28 @@ using namespace sm100;
 constexpr int BM = 128;              // query rows per item
 constexpr int BN = 128;              // keys per tile
 constexpr int DH = 128;              // head dim
-constexpr int STAGES = 3;            // K/V ring depth
+constexpr int STAGES = 2;            // K/V ring depth
 constexpr int PANEL = BM * 128;      // bytes of one 64-column panel of a 128-row tile (16 KB)
 constexpr int TILE = 2 * PANEL;      // bytes of a [128 x 128] bf16 tile (32 KB)
-constexpr int THREADS = 192;
+constexpr int THREADS = 448;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t S_COL0 = 0, S_COL1 = 128, O_COL = 256;
+constexpr uint32_t S_COL = 0, O_COL = 256;     // S: two 128-column buffers; O: two 128-column accumulators
 constexpr float RESCALE_LOG2 = 8.0f;
 
 struct Smem {
   uint64_t k_full[STAGES], v_full[STAGES], kv_empty[STAGES];
   uint64_t s_full[2], p_ready[2];
-  uint64_t o_done[2], q_ready;
+  uint64_t o_done[2];                // P V of a tile complete (commit), alternating by tile
+  uint64_t q_full[2], q_empty[2];    // gathered Q tile of an item (128 loader arrivals / commit)
+  uint64_t o_free[2];                // epilogue has read the accumulator (256 arrivals)
   uint32_t tmem_base;
   int abort_flag;
+  float xmax[2][2][128];             // [score buffer][half][row]: row maxima exchanged between the halves
+  float xsum[2][2][128];             // [half][l, l_r][row]: row sums exchanged in the epilogue
+  int qpos[4][128];                  // [item % 4][row]: in-head position of the query, -1 for padding rows
+  int direct[4][128];                // [item % 4][row]: query has a single block -> final result
 };
-constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + TILE /*Q*/ + 2 * STAGES * TILE + sizeof(Smem) + 64;
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + 2 * TILE /*Q*/ + 2 * STAGES * TILE + sizeof(Smem) + 32;
 
 struct Params {
   const __nv_bfloat16* q;
@@ -51,6 +59,7 @@ struct Params {
   const int* q_idx;
   const int* q_ptr;
   const int* item_ptr;
+  const int* item_tab;
   int n_kb, S, Nb, sb, BH;
   float scale_log2;      // softmax scale * log2(e)
   __nv_bfloat16* o;
@@ -62,45 +71,60 @@ struct Params {
   int32_t* status;
 };
 
+struct FwdItem {
+  int bh, key_begin, n_keys, list_lo, n_rows, ntiles;
+  long long head_off;
+};
+
 template <bool DENSE>
-__device__ __forceinline__ void decode_item(const Params& p, int item, int& bh, int& key_begin, int& n_keys, int& list_lo,
-                                            int& n_rows) {
+__device__ __forceinline__ FwdItem decode_item(const Params& p, int item) {
+  FwdItem it;
   if (DENSE) {
     const int tiles = (p.S + BM - 1) / BM;
-    bh = item / tiles;
-    const int t = item - bh * tiles;
-    key_begin = 0;
-    n_keys = p.S;
-    list_lo = t * BM;
-    n_rows = min(BM, p.S - list_lo);
+    it.bh = item / tiles;
+    const int t = item - it.bh * tiles;
+    it.key_begin = 0; it.n_keys = p.S; it.list_lo = t * BM; it.n_rows = min(BM, p.S - it.list_lo);
   } else {
-    simt::Item it = simt::decode_sparse(item, p.item_ptr, p.n_kb, p.kb_ptr, p.Nb, p.sb, BM, p.capacity);
-    bh = it.bh;
-    key_begin = it.key_begin;
-    n_keys = p.sb;
-    list_lo = it.list_lo;
-    n_rows = it.list_hi - it.list_lo;
+    const int kbi = __ldg(p.item_tab + item);
+    const int chunk = item - __ldg(p.item_ptr + kbi);
+    it.bh = kbi / p.Nb;
+    const int j = kbi - it.bh * p.Nb;
+    it.key_begin = j * p.sb; it.n_keys = p.sb;
+    const long long end = min((long long)__ldg(p.kb_ptr + kbi + 1), p.capacity);
+    it.list_lo = __ldg(p.kb_ptr + kbi) + chunk * BM;
+    it.n_rows = (int)min((long long)BM, end - it.list_lo);
   }
+  it.ntiles = (it.n_keys + BN - 1) / BN;
+  it.head_off = (long long)it.bh * p.S;
+  return it;
 }
+
+__device__ __forceinline__ constexpr uint32_t koff(int ks) { return (uint32_t)(((ks >> 2) * PANEL + (ks & 3) * 32) >> 4); }
+__device__ __forceinline__ constexpr uint32_t mnoff(int ks) { return (uint32_t)((ks * 2048) >> 4); }
+
+// named barrier shared by the two softmax warps of one TMEM lane quarter (64 threads)
+__device__ __forceinline__ void pair_sync(int quad) { asm volatile("bar.sync %0, 64;" ::"r"(quad + 1) : "memory"); }
 
 template <bool DENSE>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = base;
-  uint8_t* sK = base + TILE;
-  uint8_t* sV = sK + STAGES * TILE;
+  uint8_t* sQ = base;                      // [2][TILE]
+  uint8_t* sK = base + 2 * TILE;           // [STAGES][TILE]
+  uint8_t* sV = sK + STAGES * TILE;        // [STAGES][TILE]
   Smem* sm = reinterpret_cast<Smem*>(sV + STAGES * TILE);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm->abort_flag;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sm->k_full[s], 1); mbar_init(&sm->v_full[s], 1); mbar_init(&sm->kv_empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&sm->s_full[b], 1); mbar_init(&sm->p_ready[b], 128); }
-    mbar_init(&sm->o_done[0], 1);
-    mbar_init(&sm->o_done[1], 1);
-    mbar_init(&sm->q_ready, 128);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&sm->s_full[b], 1); mbar_init(&sm->p_ready[b], 256);
+      mbar_init(&sm->o_done[b], 1);
+      mbar_init(&sm->q_full[b], 128); mbar_init(&sm->q_empty[b], 1);
+      mbar_init(&sm->o_free[b], 256);
+    }
     sm->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmK);
@@ -114,9 +138,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm->tmem_base;
-
   const int n_items = DENSE ? p.BH * ((p.S + BM - 1) / BM) : p.item_ptr[p.n_kb];
-  constexpr uint32_t IDESC_QK_FULL = make_idesc_bf16(BM, BN, false, false);
   constexpr uint32_t IDESC_PV = make_idesc_bf16(BM, DH, false, true);
 
   if (warp == 0) {
@@ -124,11 +146,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     if (lane == 0) {
       uint32_t fills = 0;
       for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-        int bh, key_begin, n_keys, list_lo, n_rows;
-        decode_item<DENSE>(p, item, bh, key_begin, n_keys, list_lo, n_rows);
-        const int row0 = bh * p.S + key_begin;
-        const int ntiles = (n_keys + BN - 1) / BN;
-        for (int t = 0; t < ntiles; ++t, ++fills) {
+        const FwdItem it = decode_item<DENSE>(p, item);
+        const int row0 = (int)it.head_off + it.key_begin;
+        for (int t = 0; t < it.ntiles; ++t, ++fills) {
           const int s = fills % STAGES;
           if (fills >= STAGES) mbar_wait(&sm->kv_empty[s], ((fills / STAGES) - 1) & 1, abort_flag, p.status);
           const int y = row0 + t * BN;
@@ -152,124 +172,145 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      uint32_t fills = 0;        // K/V tiles consumed so far (global ring position)
-      uint32_t tiles_done = 0;   // score buffers used so far (global): buffer = count & 1
-      uint32_t items_done = 0;
-      const uint32_t sQ_addr = smem_u32(sQ);
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++items_done) {
-        int bh, key_begin, n_keys, list_lo, n_rows;
-        decode_item<DENSE>(p, item, bh, key_begin, n_keys, list_lo, n_rows);
-        const int ntiles = (n_keys + BN - 1) / BN;
-        mbar_wait(&sm->q_ready, items_done & 1, abort_flag, p.status);
+      uint32_t fills = 0;        // K/V tiles consumed so far (ring position)
+      uint32_t tg = 0;           // tiles done so far: score buffer and o_done slot = count & 1
+      uint32_t n = 0;            // items done so far: Q slot and O accumulator = count & 1
+      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+        const FwdItem it = decode_item<DENSE>(p, item);
+        const int qb = n & 1;
+        mbar_wait(&sm->q_full[qb], (n >> 1) & 1, abort_flag, p.status);
         tc_fence_after();
+        const uint64_t dQ0 = make_smem_desc(smem_u32(sQ + qb * TILE), 16, 1024);
         auto issue_qk = [&](int t) {
           const uint32_t f = fills + t;
           const int s = f % STAGES;
           mbar_wait(&sm->k_full[s], (f / STAGES) & 1, abort_flag, p.status);
           tc_fence_after();
-          const int valid = min(BN, n_keys - t * BN);
-          const int n_mma = (valid + 15) & ~15;
-          const uint32_t idesc = (n_mma == BN) ? IDESC_QK_FULL : make_idesc_bf16(BM, n_mma, false, false);
-          const uint32_t buf = (tiles_done + t) & 1;
-          const uint32_t d_tmem = tmem + (buf ? S_COL1 : S_COL0);
-          const uint32_t sK_addr = smem_u32(sK + s * TILE);
+          const int n_mma = (min(BN, it.n_keys - t * BN) + 15) & ~15;
+          const uint32_t idesc = make_idesc_bf16(BM, n_mma, false, false);
+          const uint32_t buf = (tg + t) & 1;
+          const uint64_t dK0 = make_smem_desc(smem_u32(sK + s * TILE), 16, 1024);
 #pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks) {
-            const uint32_t off = (ks >> 2) * PANEL + (ks & 3) * 32;
-            mma_ss(d_tmem, make_smem_desc(sQ_addr + off, 16, 1024), make_smem_desc(sK_addr + off, 16, 1024), idesc,
-                   ks > 0 ? 1u : 0u);
-          }
+          for (int ks = 0; ks < DH / 16; ++ks)
+            mma_ss(tmem + S_COL + buf * 128, dQ0 + koff(ks), dK0 + koff(ks), idesc, ks > 0 ? 1u : 0u);
           mma_commit(&sm->s_full[buf]);
         };
         issue_qk(0);
-        for (int t = 0; t < ntiles; ++t) {
-          if (t + 1 < ntiles) issue_qk(t + 1);
+        for (int t = 0; t < it.ntiles; ++t) {
+          if (t + 1 < it.ntiles) issue_qk(t + 1);
           const uint32_t f = fills + t;
           const int s = f % STAGES;
-          const uint32_t buf = (tiles_done + t) & 1;
-          mbar_wait(&sm->p_ready[buf], ((tiles_done + t) >> 1) & 1, abort_flag, p.status);
+          const uint32_t buf = (tg + t) & 1;
+          mbar_wait(&sm->p_ready[buf], ((tg + t) >> 1) & 1, abort_flag, p.status);
           mbar_wait(&sm->v_full[s], (f / STAGES) & 1, abort_flag, p.status);
+          // this accumulator was last used two items ago: its epilogue must have read it
+          if (t == 0 && n >= 2) mbar_wait(&sm->o_free[qb], ((n >> 1) - 1) & 1, abort_flag, p.status);
           tc_fence_after();
-          const int valid = min(BN, n_keys - t * BN);
-          const int ksteps = (valid + 15) >> 4;
-          const uint32_t p_tmem = tmem + (buf ? S_COL1 : S_COL0);
-          const uint32_t sV_addr = smem_u32(sV + s * TILE);
-          for (int ks = 0; ks < ksteps; ++ks) {
-            mma_ts(tmem + O_COL, p_tmem + ks * 8, make_smem_desc(sV_addr + ks * 2048, PANEL, 1024), IDESC_PV,
-                   (t > 0 || ks > 0) ? 1u : 0u);
-          }
+          const int ksteps = (min(BN, it.n_keys - t * BN) + 15) >> 4;
+          const uint32_t p_tmem = tmem + S_COL + buf * 128;
+          const uint64_t mV0 = make_smem_desc(smem_u32(sV + s * TILE), PANEL, 1024);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+            if (ks < ksteps)   // P of keys 64h + 16kk .. sits in columns 64h + 8kk .. of the score buffer
+              mma_ts(tmem + O_COL + qb * 128, p_tmem + (ks >> 2) * 64 + (ks & 3) * 8, mV0 + mnoff(ks), IDESC_PV,
+                     (t > 0 || ks > 0) ? 1u : 0u);
           mma_commit(&sm->kv_empty[s]);
-          mma_commit(&sm->o_done[(tiles_done + t) & 1]);
+          mma_commit(&sm->o_done[buf]);
         }
-        fills += ntiles;
-        tiles_done += ntiles;
+        // Release the Q slot only after the item's last P V: that MMA needed the softmax warps' P, so
+        // every waiter of this q_full phase has passed it before the loaders can complete the next one.
+        mma_commit(&sm->q_empty[qb]);
+        fills += it.ntiles;
+        tg += it.ntiles;
       }
     }
+  } else if (warp >= 10) {
+    // ------------------------------------------------------------------ loaders: Q rows of the next items
+    const int lt = threadIdx.x - 320;   // 0..127
+    const int chunk = lt & 15, panel = chunk >> 3, cc = chunk & 7;
+    uint32_t n = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+      const FwdItem it = decode_item<DENSE>(p, item);
+      const int qb = n & 1;
+      const __nv_bfloat16* qh = p.q + it.head_off * DH;
+      uint4 v[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int row = (lt >> 4) + 8 * i;
+        v[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (row < it.n_rows) {
+          const int qp = DENSE ? it.list_lo + row : __ldg(p.q_idx + it.list_lo + row);
+          v[i] = __ldg(reinterpret_cast<const uint4*>(qh + (long long)qp * DH) + chunk);
+        }
+      }
+      int my_qpos = -1, my_direct = DENSE ? 1 : 0;
+      if (lt < it.n_rows) {
+        my_qpos = DENSE ? it.list_lo + lt : __ldg(p.q_idx + it.list_lo + lt);
+        if (!DENSE) {
+          const long long G_ = it.head_off + my_qpos;
+          my_direct = (p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1;
+        }
+      }
+      if (n >= 2) mbar_wait(&sm->q_empty[qb], ((n >> 1) - 1) & 1, abort_flag, p.status);
+      uint8_t* dst = sQ + qb * TILE;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int row = (lt >> 4) + 8 * i;
+        *reinterpret_cast<uint4*>(dst + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v[i];
+      }
+      // Four slots: q_empty(n - 2) has fired, so the softmax warps finished item n - 2's tiles and copied
+      // its bookkeeping (and that of item n - 4, the previous user of this slot) to registers long ago.
+      sm->qpos[n & 3][lt] = my_qpos;
+      sm->direct[n & 3][lt] = my_direct;
+      fence_async_proxy();
+      mbar_arrive(&sm->q_full[qb]);
+    }
   } else {
-    // ------------------------------------------------------------------ softmax + epilogue (128 threads)
+    // ------------------------------------------------------------------ softmax + epilogue (8 warps)
     const int quad = warp & 3;                      // TMEM lane quarter this warp may access
+    const int half = (warp - 2) >> 2;               // which 64 of the tile's 128 keys / of the 128 output columns
     const int r = quad * 32 + lane;                 // query row of this thread
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const int st = threadIdx.x - 64;                // 0..127
-    uint32_t tiles_done = 0, pv_done = 0;
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-      int bh, key_begin, n_keys, list_lo, n_rows;
-      decode_item<DENSE>(p, item, bh, key_begin, n_keys, list_lo, n_rows);
-      const int ntiles = (n_keys + BN - 1) / BN;
-      const long long head_off = (long long)bh * p.S;
-      // ---- gather Q rows into the swizzled K-major tile: 16 threads per row, 8 rows per pass
-      {
-        const int chunk = st & 15;                 // 16-byte chunk of the 256-byte row
-        const int panel = chunk >> 3, cc = chunk & 7;
-        uint4 v[16];                               // all loads in flight before the first store
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int row = (st >> 4) + 8 * i;
-          v[i] = make_uint4(0u, 0u, 0u, 0u);
-          if (row < n_rows) {
-            const int qpos = DENSE ? list_lo + row : p.q_idx[list_lo + row];
-            v[i] = __ldg(reinterpret_cast<const uint4*>(p.q + (head_off + qpos) * DH) + chunk);
-          }
-        }
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int row = (st >> 4) + 8 * i;
-          *reinterpret_cast<uint4*>(sQ + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v[i];
-        }
-      }
-      fence_async_proxy();
-      mbar_arrive(&sm->q_ready);
-
-      const bool row_ok = r < n_rows;
-      int qpos = 0;
-      long long pos = 0;
-      if (row_ok) {
-        pos = (long long)list_lo + r;
-        qpos = DENSE ? list_lo + r : p.q_idx[pos];
-      }
+    uint32_t tg = 0, n = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+      const FwdItem it = decode_item<DENSE>(p, item);
+      const int qb = n & 1;
+      mbar_wait(&sm->q_full[qb], (n >> 1) & 1, abort_flag, p.status);     // publishes qpos / direct
+      const int qpos = sm->qpos[n & 3][r];
+      const bool direct = sm->direct[n & 3][r] != 0;
+      const uint32_t o_tmem = tmem + lane_addr + O_COL + qb * 128 + 64 * half;
       float m_used = -INFINITY, l = 0.f, l_r = 0.f;   // l: exact sum (for LSE); l_r: sum of the bf16-rounded weights
-      for (int t = 0; t < ntiles; ++t) {
-        const uint32_t buf = (tiles_done + t) & 1;
-        const uint32_t s_tmem = tmem + lane_addr + (buf ? S_COL1 : S_COL0);
-        mbar_wait(&sm->s_full[buf], ((tiles_done + t) >> 1) & 1, abort_flag, p.status);
+      for (int t = 0; t < it.ntiles; ++t) {
+        const uint32_t gt = tg + t;
+        const uint32_t buf = gt & 1;
+        const uint32_t s_tmem = tmem + lane_addr + S_COL + buf * 128 + 64 * half;
+        mbar_wait(&sm->s_full[buf], (gt >> 1) & 1, abort_flag, p.status);
         tc_fence_after();
-        const int valid = min(BN, n_keys - t * BN);
-        uint32_t sv[4][32];
-        tmem_ld32(s_tmem + 0, sv[0]);
+        const int valid = min(BN, it.n_keys - t * BN) - 64 * half;      // valid keys among this thread's 64
+        uint32_t sv[2][32];
+        tmem_ld32(s_tmem, sv[0]);
         tmem_ld32(s_tmem + 32, sv[1]);
-        tmem_ld32(s_tmem + 64, sv[2]);
-        tmem_ld32(s_tmem + 96, sv[3]);
         tmem_ld_wait();
-        float mx = -INFINITY;
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < 2; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            float x = __uint_as_float(sv[c][i]) * p.scale_log2;
-            x = (c * 32 + i < valid) ? x : -INFINITY;
-            sv[c][i] = __float_as_uint(x);
-            mx = fmaxf(mx, x);
+          for (int i = 0; i < 32; i += 4) {
+            float x0 = __uint_as_float(sv[c][i]) * p.scale_log2, x1 = __uint_as_float(sv[c][i + 1]) * p.scale_log2;
+            float x2 = __uint_as_float(sv[c][i + 2]) * p.scale_log2, x3 = __uint_as_float(sv[c][i + 3]) * p.scale_log2;
+            x0 = (c * 32 + i < valid) ? x0 : -INFINITY;
+            x1 = (c * 32 + i + 1 < valid) ? x1 : -INFINITY;
+            x2 = (c * 32 + i + 2 < valid) ? x2 : -INFINITY;
+            x3 = (c * 32 + i + 3 < valid) ? x3 : -INFINITY;
+            sv[c][i] = __float_as_uint(x0); sv[c][i + 1] = __float_as_uint(x1);
+            sv[c][i + 2] = __float_as_uint(x2); sv[c][i + 3] = __float_as_uint(x3);
+            mx0 = fmaxf(mx0, x0); mx1 = fmaxf(mx1, x1); mx2 = fmaxf(mx2, x2); mx3 = fmaxf(mx3, x3);
           }
+        float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+        // the row's other 64 keys belong to the thread with the same lane in the partner warp
+        sm->xmax[buf][half][r] = mx;
+        pair_sync(quad);
+        mx = fmaxf(mx, sm->xmax[buf][half ^ 1][r]);
         // lazy rescale: keep the old reference max unless the new one is more than 2^8 larger
         float factor = 1.0f;
         bool need = false;
@@ -282,11 +323,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         }
         if (t > 0 && __any_sync(0xffffffffu, need)) {
           // O of the previous tiles must be complete before it is rescaled
-          mbar_wait(&sm->o_done[(pv_done + t - 1) & 1], ((pv_done + t - 1) >> 1) & 1, abort_flag, p.status);
+          mbar_wait(&sm->o_done[(gt - 1) & 1], ((gt - 1) >> 1) & 1, abort_flag, p.status);
           tc_fence_after();
-          const uint32_t o_tmem = tmem + lane_addr + O_COL;
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 2; ++c) {
             uint32_t ov[32];
             tmem_ld32(o_tmem + c * 32, ov);
             tmem_ld_wait();
@@ -297,56 +337,59 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
           l *= factor;
           l_r *= factor;
         }
-        float sum = 0.f, sum_r = 0.f;
-        // P (bf16 pairs) goes over the first 64 columns of this score buffer: keys 2i, 2i+1 -> column i
+        // P (bf16 pairs) goes over the first 32 of this thread's 64 score columns: keys 2i, 2i+1 -> column i
+        float s0 = 0.f, s1 = 0.f, r0 = 0.f, r1 = 0.f;
+        uint32_t pk[32];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          uint32_t pk[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float p0 = ex2(__uint_as_float(sv[2 * h + (i >> 4)][(2 * i) & 31]) - m_used);
-            const float p1 = ex2(__uint_as_float(sv[2 * h + (i >> 4)][((2 * i) & 31) + 1]) - m_used);
-            sum += p0 + p1;
-            pk[i] = pack_bf16(p0, p1);
-            // the tensor core multiplies the ROUNDED weights: normalise O by their sum, so that the
-            // rounding of P perturbs the weights but never their total
-            sum_r += __uint_as_float(pk[i] << 16) + __uint_as_float(pk[i] & 0xffff0000u);
-          }
-          tmem_st32(s_tmem + h * 32, pk);
+        for (int i = 0; i < 32; ++i) {
+          const float p0 = ex2(__uint_as_float(sv[i >> 4][(2 * i) & 31]) - m_used);
+          const float p1 = ex2(__uint_as_float(sv[i >> 4][((2 * i) & 31) + 1]) - m_used);
+          s0 += p0; s1 += p1;
+          pk[i] = pack_bf16(p0, p1);
+          // the tensor core multiplies the ROUNDED weights: normalise O by their sum, so that the
+          // rounding of P perturbs the weights but never their total
+          r0 += __uint_as_float(pk[i] << 16);
+          r1 += __uint_as_float(pk[i] & 0xffff0000u);
         }
-        l += sum;
-        l_r += sum_r;
+        tmem_st32(s_tmem, pk);
+        l += s0 + s1;
+        l_r += r0 + r1;
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(&sm->p_ready[buf]);
       }
-      // ---- epilogue: wait for the last P V, normalise, write
-      mbar_wait(&sm->o_done[(pv_done + ntiles - 1) & 1], ((pv_done + ntiles - 1) >> 1) & 1, abort_flag, p.status);
+      // ---- epilogue: wait for the last P V, combine the two halves' sums, normalise, write 64 columns
+      const uint32_t gl = tg + it.ntiles - 1;
+      sm->xsum[half][0][r] = l;
+      sm->xsum[half][1][r] = l_r;
+      pair_sync(quad);
+      l += sm->xsum[half ^ 1][0][r];
+      l_r += sm->xsum[half ^ 1][1][r];
+      mbar_wait(&sm->o_done[gl & 1], (gl >> 1) & 1, abort_flag, p.status);
       tc_fence_after();
-      pv_done += ntiles;
-      tiles_done += ntiles;
+      tg += it.ntiles;
       const float inv = 1.0f / l_r;
       const float row_lse = (m_used + log2f(l)) * 0.6931471805599453f;
-      const long long G_ = head_off + qpos;
-      bool direct = DENSE;
-      if (!DENSE && row_ok) direct = (p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1;
-      const uint32_t o_tmem = tmem + lane_addr + O_COL;
+      const bool row_ok = qpos >= 0;
+      const long long G_ = it.head_off + (row_ok ? qpos : 0);
+      const long long pos = (long long)it.list_lo + r;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t ov[32];
         tmem_ld32(o_tmem + c * 32, ov);
         tmem_ld_wait();
         if (row_ok) {
+          const int col = 64 * half + 32 * c;
           if (direct) {
-            __nv_bfloat16* dst = p.o + G_ * DH + c * 32;
-            __nv_bfloat16* rdst = p.o_resid ? p.o_resid + G_ * DH + c * 32 : nullptr;
+            __nv_bfloat16* dst = p.o + G_ * DH + col;
+            __nv_bfloat16* rdst = p.o_resid ? p.o_resid + G_ * DH + col : nullptr;
 #pragma unroll
             for (int i = 0; i < 32; i += 4)
               store4_resid(dst + i, rdst ? rdst + i : nullptr,
                            make_float4(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
                                        __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv));
           } else {
-            float* dst = p.part_o + pos * DH + c * 32;
+            float* dst = p.part_o + pos * DH + col;
 #pragma unroll
             for (int i = 0; i < 32; i += 4)
               *reinterpret_cast<float4*>(dst + i) =
@@ -355,11 +398,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
           }
         }
       }
-      if (row_ok) {
+      if (row_ok && half == 0) {
         if (direct) p.lse[G_] = row_lse; else p.part_lse[pos] = row_lse;
       }
-      // the next item's first P V overwrites O: order our TMEM reads before the q_ready arrival
       tc_fence_before();
+      mbar_arrive(&sm->o_free[qb]);
     }
   }
   tc_fence_before();
@@ -375,7 +418,8 @@ static int grid_items(long long items) { return (int)std::max<long long>(1, std:
 // the launch fail.
 int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                   const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
-                  int32_t* status, int* item_ptr, float* part_o, float* part_lse, cudaStream_t st) {
+                  int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o, float* part_lse,
+                  cudaStream_t st) {
   using namespace tc;
   CUtensorMap tmK, tmV;
   const uint64_t rows = (uint64_t)D.BH * D.S;
@@ -383,8 +427,11 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
     return VMOBA_ERR_CUDA;
   const long long n_kb = (long long)D.BH * D.Nb;
   simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, BM, cap, item_ptr);
+  simt::item_tab_kernel<<<(int)std::min<long long>((n_kb + 255) / 256, 148 * 4), 256, 0, st>>>(item_ptr, n_kb, max_items,
+                                                                                               item_tab);
   Params p;
   p.q = (const __nv_bfloat16*)q; p.kb_ptr = kb_ptr; p.q_idx = q_idx; p.q_ptr = q_ptr; p.item_ptr = item_ptr;
+  p.item_tab = item_tab;
   p.n_kb = (int)n_kb; p.S = D.S; p.Nb = D.Nb; p.sb = D.sb; p.BH = D.BH;
   p.scale_log2 = D.scale * 1.4426950408889634f;
   p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
@@ -395,7 +442,7 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
   const long long nq = (long long)D.BH * D.S;
   simt::merge_kernel<__nv_bfloat16, 128, float><<<(int)std::min<long long>((nq + 7) / 8, 148 * 16), 256, 0, st>>>(
       q_ptr, q_pairs, nq, part_o, part_lse, cap, (__nv_bfloat16*)o, (__nv_bfloat16*)o_resid, lse);
-  VMOBA_LAUNCH_OK(3);
+  VMOBA_LAUNCH_OK(4);
   return VMOBA_OK;
 }
 
@@ -408,6 +455,7 @@ int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, voi
     return VMOBA_ERR_CUDA;
   Params p;
   p.q = (const __nv_bfloat16*)q; p.kb_ptr = nullptr; p.q_idx = nullptr; p.q_ptr = nullptr; p.item_ptr = nullptr;
+  p.item_tab = nullptr;
   p.n_kb = 0; p.S = D.S; p.Nb = 1; p.sb = D.S; p.BH = D.BH;
   p.scale_log2 = D.scale * 1.4426950408889634f;
   p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = nullptr; p.part_lse = nullptr;
