@@ -86,10 +86,11 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
   BwdWs w = carve_bwd(D, false, ws, cap);
   const long long n_kb = (long long)D.BH * D.Nb;
   const long long nq = (long long)D.BH * D.S;
-  VMOBA_CUDA_OK(cudaMemsetAsync(w.dq_acc, 0, (size_t)nq * DH * sizeof(float), st));
   simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>((const T*)o, (const T*)o_resid,
                                                                         (const T*)d_o, nq, w.Dv);
   if (use_tensor_cores(D)) {
+    simt::zero_multi_rows_kernel<DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, q_ptr, nq);
+    count_launches(1);
     simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, 128, cap, w.item_ptr);
     simt::item_tab_kernel<<<(int)std::min<long long>((n_kb + 255) / 256, 148 * 4), 256, 0, st>>>(
         w.item_ptr, n_kb, max_items_128(D, cap), w.item_tab);
@@ -101,6 +102,7 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
     VMOBA_LAUNCH_OK(1);
     return VMOBA_OK;
   }
+  VMOBA_CUDA_OK(cudaMemsetAsync(w.dq_acc, 0, (size_t)nq * DH * sizeof(float), st));
   simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, simt::kRows, cap, w.item_ptr);
   long long tiles = (D.sb + simt::kRows - 1) / simt::kRows;
   simt::attn_bwd_dkdv_kernel<T, DH, false><<<grid_for(n_kb * tiles, 4), simt::kThreads, 0, st>>>(
