@@ -4,8 +4,8 @@
 // the queries that selected key block j, gathered by index; dense: 128 consecutive rows) against
 // a contiguous key range (the block, or the whole sequence), streamed in tiles of 128 keys:
 //
-//   warp 0       TMA producer: K and V tiles (two 64-column panels each, 128-byte swizzle) into a
-//                2-stage ring
+//   warp 0       TMA producer: K and V tiles (two 64-column panels each, 128-byte swizzle) into two
+//                2-stage rings (a K stage is released by the tile's Q K^T, a V stage by its P V)
 //   warp 1       MMA issuer (one thread): S = Q K^T into one of two TMEM score buffers, then
 //                O += P V with P read from TMEM; tcgen05.commit signals the other roles
 //   warps 2-9    softmax: thread = (query row, 64 of the tile's 128 keys).  The two threads of a row
@@ -39,13 +39,14 @@ constexpr uint32_t S_COL = 0, O_COL = 256;     // S: two 128-column buffers; O: 
 constexpr float RESCALE_LOG2 = 8.0f;
 
 struct Smem {
-  uint64_t k_full[STAGES], v_full[STAGES], kv_empty[STAGES];
+  uint64_t k_full[STAGES], v_full[STAGES], k_empty[STAGES], v_empty[STAGES];
   uint64_t s_full[2], p_ready[2];
   uint64_t o_done[2];                // P V of a tile complete (commit), alternating by tile
   uint64_t q_full[2], q_empty[2];    // gathered Q tile of an item (128 loader arrivals / commit)
   uint64_t o_free[2];                // epilogue has read the accumulator (256 arrivals)
   uint32_t tmem_base;
   int abort_flag;
+  long long t_issue[STAGES];        // diagnostics: when the K tile of a stage was requested
   float xmax[2][2][128];             // [score buffer][half][row]: row maxima exchanged between the halves
   float xsum[2][2][128];             // [half][l, l_r][row]: row sums exchanged in the epilogue
   int qpos[4][128];                  // [item % 4][row]: in-head position of the query, -1 for padding rows
@@ -69,6 +70,7 @@ struct Params {
   float* part_lse;
   long long capacity;
   int32_t* status;
+  unsigned long long* prof;   // optional per-site cycle counters (diagnostics), or null
 };
 
 struct FwdItem {
@@ -116,9 +118,26 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   Smem* sm = reinterpret_cast<Smem*>(sV + STAGES * TILE);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm->abort_flag;
+  // diagnostics: cycles one representative thread per role spends in each section
+  unsigned long long wp[6] = {0, 0, 0, 0, 0, 0};
+  long long t_mark = clock64();
+  const long long t_begin = t_mark;
+  auto lap = [&](int site) {
+    if (p.prof) {
+      const long long now = clock64();
+      wp[site] += (unsigned long long)(now - t_mark);
+      t_mark = now;
+    }
+  };
+  auto tflush = [&](int base_site) {
+    if (p.prof) {
+      for (int i = 0; i < 6; ++i) atomicAdd(p.prof + base_site + i, wp[i]);
+      atomicAdd(p.prof + base_site + 6, (unsigned long long)(clock64() - t_begin));
+    }
+  };
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sm->k_full[s], 1); mbar_init(&sm->v_full[s], 1); mbar_init(&sm->kv_empty[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sm->k_full[s], 1); mbar_init(&sm->v_full[s], 1); mbar_init(&sm->k_empty[s], 1); mbar_init(&sm->v_empty[s], 1); }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sm->s_full[b], 1); mbar_init(&sm->p_ready[b], 256);
       mbar_init(&sm->o_done[b], 1);
@@ -150,11 +169,15 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         const int row0 = (int)it.head_off + it.key_begin;
         for (int t = 0; t < it.ntiles; ++t, ++fills) {
           const int s = fills % STAGES;
-          if (fills >= STAGES) mbar_wait(&sm->kv_empty[s], ((fills / STAGES) - 1) & 1, abort_flag, p.status);
+          // a K stage is free once the tile's Q K^T has run, a V stage only after its P V: separate
+          // rings, so that the next K tile is already on its way while the softmax of this one runs
+          if (fills >= STAGES) mbar_wait(&sm->k_empty[s], ((fills / STAGES) - 1) & 1, abort_flag, p.status);
           const int y = row0 + t * BN;
+          if (p.prof) sm->t_issue[s] = clock64();
           mbar_expect_tx(&sm->k_full[s], TILE);
           tma_load_2d(sK + s * TILE, &tmK, &sm->k_full[s], 0, y);
           tma_load_2d(sK + s * TILE + PANEL, &tmK, &sm->k_full[s], 64, y);
+          if (fills >= STAGES) mbar_wait(&sm->v_empty[s], ((fills / STAGES) - 1) & 1, abort_flag, p.status);
           mbar_expect_tx(&sm->v_full[s], TILE);
           tma_load_2d(sV + s * TILE, &tmV, &sm->v_full[s], 0, y);
           tma_load_2d(sV + s * TILE + PANEL, &tmV, &sm->v_full[s], 64, y);
@@ -172,19 +195,28 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
+      unsigned long long lat_sum = 0, lat_cnt = 0;
       uint32_t fills = 0;        // K/V tiles consumed so far (ring position)
       uint32_t tg = 0;           // tiles done so far: score buffer and o_done slot = count & 1
       uint32_t n = 0;            // items done so far: Q slot and O accumulator = count & 1
       for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
         const FwdItem it = decode_item<DENSE>(p, item);
         const int qb = n & 1;
+        lap(5);
         mbar_wait(&sm->q_full[qb], (n >> 1) & 1, abort_flag, p.status);
+        lap(0);
         tc_fence_after();
         const uint64_t dQ0 = make_smem_desc(smem_u32(sQ + qb * TILE), 16, 1024);
         auto issue_qk = [&](int t) {
           const uint32_t f = fills + t;
           const int s = f % STAGES;
+          lap(5);
           mbar_wait(&sm->k_full[s], (f / STAGES) & 1, abort_flag, p.status);
+          if (p.prof) {
+            const long long now = clock64();
+            if (now - t_mark > 100) { lat_sum += (unsigned long long)(now - sm->t_issue[s]); lat_cnt += 1; }
+          }
+          lap(1);
           tc_fence_after();
           const int n_mma = (min(BN, it.n_keys - t * BN) + 15) & ~15;
           const uint32_t idesc = make_idesc_bf16(BM, n_mma, false, false);
@@ -194,6 +226,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
           for (int ks = 0; ks < DH / 16; ++ks)
             mma_ss(tmem + S_COL + buf * 128, dQ0 + koff(ks), dK0 + koff(ks), idesc, ks > 0 ? 1u : 0u);
           mma_commit(&sm->s_full[buf]);
+          mma_commit(&sm->k_empty[s]);
         };
         issue_qk(0);
         for (int t = 0; t < it.ntiles; ++t) {
@@ -201,10 +234,14 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
           const uint32_t f = fills + t;
           const int s = f % STAGES;
           const uint32_t buf = (tg + t) & 1;
+          lap(5);
           mbar_wait(&sm->p_ready[buf], ((tg + t) >> 1) & 1, abort_flag, p.status);
+          lap(2);
           mbar_wait(&sm->v_full[s], (f / STAGES) & 1, abort_flag, p.status);
+          lap(3);
           // this accumulator was last used two items ago: its epilogue must have read it
           if (t == 0 && n >= 2) mbar_wait(&sm->o_free[qb], ((n >> 1) - 1) & 1, abort_flag, p.status);
+          lap(4);
           tc_fence_after();
           const int ksteps = (min(BN, it.n_keys - t * BN) + 15) >> 4;
           const uint32_t p_tmem = tmem + S_COL + buf * 128;
@@ -214,7 +251,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
             if (ks < ksteps)   // P of keys 64h + 16kk .. sits in columns 64h + 8kk .. of the score buffer
               mma_ts(tmem + O_COL + qb * 128, p_tmem + (ks >> 2) * 64 + (ks & 3) * 8, mV0 + mnoff(ks), IDESC_PV,
                      (t > 0 || ks > 0) ? 1u : 0u);
-          mma_commit(&sm->kv_empty[s]);
+          mma_commit(&sm->v_empty[s]);
           mma_commit(&sm->o_done[buf]);
         }
         // Release the Q slot only after the item's last P V: that MMA needed the softmax warps' P, so
@@ -223,6 +260,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         fills += it.ntiles;
         tg += it.ntiles;
       }
+      lap(5);
+      tflush(8);
+      if (p.prof) { atomicAdd(p.prof + 7, lat_sum); atomicAdd(p.prof + 15, lat_cnt); }
     }
   } else if (warp >= 10) {
     // ------------------------------------------------------------------ loaders: Q rows of the next items
@@ -275,7 +315,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
       const FwdItem it = decode_item<DENSE>(p, item);
       const int qb = n & 1;
+      lap(4);
       mbar_wait(&sm->q_full[qb], (n >> 1) & 1, abort_flag, p.status);     // publishes qpos / direct
+      lap(5);
       const int qpos = sm->qpos[n & 3][r];
       const bool direct = sm->direct[n & 3][r] != 0;
       const uint32_t o_tmem = tmem + lane_addr + O_COL + qb * 128 + 64 * half;
@@ -284,33 +326,40 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         const uint32_t gt = tg + t;
         const uint32_t buf = gt & 1;
         const uint32_t s_tmem = tmem + lane_addr + S_COL + buf * 128 + 64 * half;
+        lap(3);
         mbar_wait(&sm->s_full[buf], (gt >> 1) & 1, abort_flag, p.status);
+        lap(0);
         tc_fence_after();
         const int valid = min(BN, it.n_keys - t * BN) - 64 * half;      // valid keys among this thread's 64
         uint32_t sv[2][32];
         tmem_ld32(s_tmem, sv[0]);
         tmem_ld32(s_tmem + 32, sv[1]);
         tmem_ld_wait();
+        if (valid < 64) {    // ragged last tile of the key range: keys beyond it get weight zero
+#pragma unroll
+          for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c * 32 + i >= valid) sv[c][i] = 0xff800000u;
+        }
+        // row maximum of the raw scores (the softmax scale is positive, so it commutes with the max)
         float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
         for (int c = 0; c < 2; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; i += 4) {
-            float x0 = __uint_as_float(sv[c][i]) * p.scale_log2, x1 = __uint_as_float(sv[c][i + 1]) * p.scale_log2;
-            float x2 = __uint_as_float(sv[c][i + 2]) * p.scale_log2, x3 = __uint_as_float(sv[c][i + 3]) * p.scale_log2;
-            x0 = (c * 32 + i < valid) ? x0 : -INFINITY;
-            x1 = (c * 32 + i + 1 < valid) ? x1 : -INFINITY;
-            x2 = (c * 32 + i + 2 < valid) ? x2 : -INFINITY;
-            x3 = (c * 32 + i + 3 < valid) ? x3 : -INFINITY;
-            sv[c][i] = __float_as_uint(x0); sv[c][i + 1] = __float_as_uint(x1);
-            sv[c][i + 2] = __float_as_uint(x2); sv[c][i + 3] = __float_as_uint(x3);
-            mx0 = fmaxf(mx0, x0); mx1 = fmaxf(mx1, x1); mx2 = fmaxf(mx2, x2); mx3 = fmaxf(mx3, x3);
+          for (int i = 0; i < 32; i += 8) {
+            mx0 = max3(mx0, __uint_as_float(sv[c][i]), __uint_as_float(sv[c][i + 1]));
+            mx1 = max3(mx1, __uint_as_float(sv[c][i + 2]), __uint_as_float(sv[c][i + 3]));
+            mx2 = max3(mx2, __uint_as_float(sv[c][i + 4]), __uint_as_float(sv[c][i + 5]));
+            mx3 = max3(mx3, __uint_as_float(sv[c][i + 6]), __uint_as_float(sv[c][i + 7]));
           }
         float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
         // the row's other 64 keys belong to the thread with the same lane in the partner warp
         sm->xmax[buf][half][r] = mx;
+        lap(1);
         pair_sync(quad);
-        mx = fmaxf(mx, sm->xmax[buf][half ^ 1][r]);
+        lap(2);
+        mx = fmaxf(mx, sm->xmax[buf][half ^ 1][r]) * p.scale_log2;   // exp2 domain from here on
         // lazy rescale: keep the old reference max unless the new one is more than 2^8 larger
         float factor = 1.0f;
         bool need = false;
@@ -340,16 +389,19 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         // P (bf16 pairs) goes over the first 32 of this thread's 64 score columns: keys 2i, 2i+1 -> column i
         float s0 = 0.f, s1 = 0.f, r0 = 0.f, r1 = 0.f;
         uint32_t pk[32];
+        const float neg_m = -m_used;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          const float p0 = ex2(__uint_as_float(sv[i >> 4][(2 * i) & 31]) - m_used);
-          const float p1 = ex2(__uint_as_float(sv[i >> 4][((2 * i) & 31) + 1]) - m_used);
-          s0 += p0; s1 += p1;
+          float p0, p1;
+          fma2(p0, p1, __uint_as_float(sv[i >> 4][(2 * i) & 31]), __uint_as_float(sv[i >> 4][((2 * i) & 31) + 1]),
+               p.scale_log2, p.scale_log2, neg_m, neg_m);
+          p0 = ex2(p0);
+          p1 = ex2(p1);
+          add2(s0, s1, s0, s1, p0, p1);
           pk[i] = pack_bf16(p0, p1);
           // the tensor core multiplies the ROUNDED weights: normalise O by their sum, so that the
           // rounding of P perturbs the weights but never their total
-          r0 += __uint_as_float(pk[i] << 16);
-          r1 += __uint_as_float(pk[i] & 0xffff0000u);
+          add2(r0, r1, r0, r1, __uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u));
         }
         tmem_st32(s_tmem, pk);
         l += s0 + s1;
@@ -359,6 +411,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
         mbar_arrive(&sm->p_ready[buf]);
       }
       // ---- epilogue: wait for the last P V, combine the two halves' sums, normalise, write 64 columns
+      lap(3);
       const uint32_t gl = tg + it.ntiles - 1;
       sm->xsum[half][0][r] = l;
       sm->xsum[half][1][r] = l_r;
@@ -404,6 +457,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constan
       tc_fence_before();
       mbar_arrive(&sm->o_free[qb]);
     }
+    lap(4);
+    if (warp == 2 && lane == 0) tflush(0);
   }
   tc_fence_before();
   __syncthreads();
@@ -435,7 +490,7 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
   p.n_kb = (int)n_kb; p.S = D.S; p.Nb = D.Nb; p.sb = D.sb; p.BH = D.BH;
   p.scale_log2 = D.scale * 1.4426950408889634f;
   p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
-  p.capacity = cap; p.status = status;
+  p.capacity = cap; p.status = status; p.prof = debug_wait_profile();
   VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)SMEM_BYTES));
   attn_fwd_tc_kernel<false><<<grid_items(cap / BM + n_kb), THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
@@ -459,7 +514,7 @@ int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, voi
   p.n_kb = 0; p.S = D.S; p.Nb = 1; p.sb = D.S; p.BH = D.BH;
   p.scale_log2 = D.scale * 1.4426950408889634f;
   p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = nullptr; p.part_lse = nullptr;
-  p.capacity = 0; p.status = status;
+  p.capacity = 0; p.status = status; p.prof = debug_wait_profile();
   VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)SMEM_BYTES));
   const long long items = (long long)D.BH * ((D.S + BM - 1) / BM);

@@ -831,6 +831,10 @@ int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, con
 
 // Registers (or clears, with null) a device buffer of 16 uint64 counters for the dK/dV kernel's
 // wait-time diagnostics.  Not part of the method; see the kernel for the counter layout.
+namespace vmoba {
+unsigned long long* debug_wait_profile() { return tcb::g_wait_profile; }
+}  // namespace vmoba
+
 extern "C" void vmoba_debug_wait_profile(void* dev_counters16) {
   vmoba::tcb::g_wait_profile = static_cast<unsigned long long*>(dev_counters16);
 }

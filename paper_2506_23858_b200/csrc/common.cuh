@@ -199,4 +199,7 @@ __device__ void block_exclusive_scan(In in, int* __restrict__ out, long long n, 
   __syncthreads();
 }
 
+// Device counters set through vmoba_debug_wait_profile (null when diagnostics are off).
+unsigned long long* debug_wait_profile();
+
 }  // namespace vmoba
