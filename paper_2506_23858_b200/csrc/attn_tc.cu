@@ -18,6 +18,7 @@
 // neighbouring items overlap; QK^T of tile t+1 is issued before P V of tile t.
 // TMEM: 2 x 128 columns of scores (P aliases them) + 2 x 128 columns of O.
 #include <algorithm>
+#include <cstdlib>
 
 #include "attn_simt.cuh"
 #include "sm100.cuh"
@@ -469,12 +470,29 @@ static int grid_items(long long items) { return (int)std::max<long long>(1, std:
 
 }  // namespace tc
 
+int tc_sparse_fwd_wide(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
+                       const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
+                       int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o,
+                       float* part_lse, cudaStream_t st);
+int tc_dense_fwd_wide(const Dims& D, const void* q, const void* k, const void* v, void* o, void* o_resid, float* lse,
+                      int32_t* status, cudaStream_t st);
+
+// Key ranges of at least this many keys go to the kernel with 256-row items: its per-item set-up is
+// longer, and it pays only when an item streams many key tiles.
+static int wide_min_keys() {
+  static int v = [] { const char* e = getenv("VMOBA_WIDE_MIN_KEYS"); return e ? atoi(e) : 1024; }();
+  return v;
+}
+
 // Forward over the work lists (bf16, head_dim 128).  Returns VMOBA_ERR_CUDA if the tensor maps or
 // the launch fail.
 int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                   const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
                   int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o, float* part_lse,
                   cudaStream_t st) {
+  if (D.sb >= wide_min_keys())
+    return tc_sparse_fwd_wide(D, q, k, v, kb_ptr, q_idx, q_ptr, q_pairs, cap, o, o_resid, lse, status, item_ptr, item_tab,
+                              max_items, part_o, part_lse, st);
   using namespace tc;
   CUtensorMap tmK, tmV;
   const uint64_t rows = (uint64_t)D.BH * D.S;
@@ -503,6 +521,7 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
 
 int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, void* o, void* o_resid, float* lse,
                  int32_t* status, cudaStream_t st) {
+  if (D.S >= wide_min_keys()) return tc_dense_fwd_wide(D, q, k, v, o, o_resid, lse, status, st);
   using namespace tc;
   CUtensorMap tmK, tmV;
   const uint64_t rows = (uint64_t)D.BH * D.S;
