@@ -20,8 +20,7 @@ int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, voi
 
 // attn_tc_bwd.cu: tensor-core backward kernels (bf16, head_dim 128)
 int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
-                  const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap,
-                  const int* item_ptr, const int* item_tab, float* dq_acc, void* dq, void* dk, void* dv,
+                  const float* Dv, const int* kb_ptr, const int* q_idx, long long cap, float* dq_acc, void* dk, void* dv,
                   int32_t* status, cudaStream_t st);
 int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* Dv, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st);
@@ -89,16 +88,14 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
   simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>((const T*)o, (const T*)o_resid,
                                                                         (const T*)d_o, nq, w.Dv);
   if (use_tensor_cores(D)) {
-    simt::zero_multi_rows_kernel<DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, q_ptr, nq);
-    count_launches(1);
-    simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, 128, cap, w.item_ptr);
-    simt::item_tab_kernel<<<(int)std::min<long long>((n_kb + 255) / 256, 148 * 4), 256, 0, st>>>(
-        w.item_ptr, n_kb, max_items_128(D, cap), w.item_tab);
-    count_launches(3);
-    int rc = tc_sparse_bwd(D, q, k, v, d_o, lse, w.Dv, kb_ptr, q_idx, q_ptr, cap, w.item_ptr, w.item_tab, w.dq_acc, dq,
-                           dk, dv, status, st);
+    // the backward kernel adds every dQ contribution into the fp32 accumulator: clear the rows of all
+    // selecting queries, convert them afterwards (rows of queries without a block become zero)
+    const int min_nb = 1;
+    simt::zero_multi_rows_kernel<DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, q_ptr, nq, min_nb);
+    count_launches(2);
+    int rc = tc_sparse_bwd(D, q, k, v, d_o, lse, w.Dv, kb_ptr, q_idx, cap, w.dq_acc, dk, dv, status, st);
     if (rc) return rc;
-    simt::cast_rows_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, q_ptr, nq, 1);
+    simt::cast_rows_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, q_ptr, nq, 1, min_nb);
     VMOBA_LAUNCH_OK(1);
     return VMOBA_OK;
   }

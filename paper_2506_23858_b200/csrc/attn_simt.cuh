@@ -456,29 +456,29 @@ attn_bwd_dq_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
 template <typename T, int DH>
 __global__ void __launch_bounds__(256)
 cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, const int* __restrict__ q_ptr, long long n_queries,
-                 int sparse_rows) {
+                 int sparse_rows, int min_nb) {
   constexpr int C = DH / 32;
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
   for (long long g = warp; g < n_queries; g += nwarps) {
     const int nb = sparse_rows ? q_ptr[g + 1] - q_ptr[g] : 2;
-    if (nb == 1) continue;
+    if (nb > 0 && nb < min_nb) continue;   // written directly by the attention kernel
 #pragma unroll
     for (int c = 0; c < C; ++c) dst[g * DH + lane * C + c] = from_f32<T>(nb == 0 ? 0.f : src[g * DH + lane * C + c]);
   }
 }
 
-// Zeroes the accumulator rows of the queries with two or more selected blocks (the only rows the
+// Zeroes the accumulator rows of the queries with at least min_nb selected blocks (the only rows the
 // attention kernel adds into), instead of clearing the whole [queries, head_dim] fp32 buffer.
 template <int DH>
 __global__ void __launch_bounds__(256)
-zero_multi_rows_kernel(float* __restrict__ acc, const int* __restrict__ q_ptr, long long n_queries) {
+zero_multi_rows_kernel(float* __restrict__ acc, const int* __restrict__ q_ptr, long long n_queries, int min_nb) {
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
   for (long long g = warp; g < n_queries; g += nwarps) {
-    if (q_ptr[g + 1] - q_ptr[g] < 2) continue;
+    if (q_ptr[g + 1] - q_ptr[g] < min_nb) continue;
     float4* row = reinterpret_cast<float4*>(acc + g * DH);
     for (int c = lane; c < DH / 4; c += 32) row[c] = make_float4(0.f, 0.f, 0.f, 0.f);
   }

@@ -1,21 +1,24 @@
 // Tensor-core attention backward for bf16, head_dim 128: the training backward of Step 3 of
-// VMoBA (mask constant) and of the dense path.  Two kernels, both persistent (one CTA per SM):
+// VMoBA (mask constant).  One persistent kernel (one CTA per SM), key-stationary:
 //
-//   dK/dV  key-stationary.  Item = 128 keys of one key block (or of the sequence).  K and V tiles
-//          stay in shared memory; the queries that selected the block stream through in gathered
-//          chunks of 64 (Q and dO rows, 3-deep ring).  Per chunk, with keys on the TMEM lanes:
-//            S^T = K Q^T,  dP^T = V dO^T            (two SS MMAs)
-//            P^T = exp2(c S^T - lse),  dS^T = P^T (dP^T - D)   (threads = key rows)
-//            dV += P^T dO,  dK += dS^T Q            (two TS MMAs, A = bf16 P^T / dS^T in TMEM;
-//                                                    B = the same dO / Q tiles read MN-major)
-//          Every key belongs to exactly one item: dK and dV are written once, no atomics.
-//   dQ     query-stationary over the forward's work items (128 gathered queries x one key block):
-//            S = Q K^T,  dP = dO V^T,  dS = P (dP - D),  dQ += dS K
-//          A query's blocks add their contributions into an fp32 accumulator (atomics); the dense
-//          path writes dQ directly.
+//   Item = 128 keys of one key block.  The K and V tiles stay in shared memory; the queries that
+//   selected the block stream through in gathered chunks of 64 (Q and dO rows, 3-deep ring).  Per
+//   chunk, with keys on the TMEM lanes:
+//     S^T = K Q^T,  dP^T = V dO^T                        (two SS MMAs, N = 64)
+//     P^T = exp2(c S^T - lse),  dS^T = P^T (dP^T - D)    (threads = key rows)
+//     dQ^T = K^T dS^T                                    (SS MMA: K tile read MN-major as A, dS^T from a
+//                                                         [keys][queries] bf16 tile in shared memory)
+//     dV += P^T dO,  dK += dS^T Q                        (two TS MMAs, A = bf16 P^T / dS^T in TMEM;
+//                                                         B = the same dO / Q tiles read MN-major)
+//   Every key belongs to exactly one item: dK and dV are written once, no atomics.  dQ^T of a chunk
+//   is read out of TMEM by four writer warps, transposed through shared memory and added into an
+//   fp32 accumulator with one bulk reduction per query row; the L2's fp32 reduction rate is what
+//   bounds this kernel on long key blocks.
 //
 // D = rowsum(dO * O) and lse come in per query; exp runs in the exp2 domain (c = scale * log2 e).
+// The dense path uses the kernels with 128-query units in the companion file.
 #include <algorithm>
+#include <cstdlib>
 
 #include "attn_simt.cuh"
 #include "sm100.cuh"
@@ -81,6 +84,17 @@ __device__ __forceinline__ void gather_store128(uint8_t* dst, int tid, const uin
 }
 
 // 16-byte vector reduction into global memory (fp32 add).
+// Bulk reduction: adds `bytes` (a multiple of 16) of fp32 from shared memory into global memory.
+__device__ __forceinline__ void bulk_reduce_add_f32(float* gdst, const float* ssrc, uint32_t bytes) {
+  asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(ssrc)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// named barrier of the four dQ writer warps
+__device__ __forceinline__ void writer_sync() { asm volatile("bar.sync 5, 128;" ::: "memory"); }
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
@@ -120,12 +134,20 @@ struct KvSmem {
   uint64_t acc_free;                         // epilogue has read dV / dK (128 compute arrivals)
   uint32_t tmem_base;
   int abort_flag;
+  uint64_t dq_full[2];                       // fused variant: dQ^T of a unit complete (commit)
+  uint64_t dq_free[2];                       // fused variant: dQ^T read out of TMEM (128 writer arrivals)
   alignas(16) float lse2[NQ][QC];
   alignas(16) float Dq[NQ][QC];
 };
+constexpr int DSTILE = 128 * 128;            // dS^T of a unit in shared memory: [128 keys][64 queries] bf16 (16 KB)
+// split kernels: K/V double buffered across items; fused kernel: one K/V pair, one dS^T tile, the dQ staging tile
 constexpr size_t KV_SMEM_BYTES = 1024 + 4 * TILE + NQ * 2 * CTILE + sizeof(KvSmem) + 32;
+constexpr int DQSTAGE = QC * DH * 4;         // dQ of a unit as [64 queries][128] fp32 rows for the bulk reductions (32 KB)
+constexpr size_t KVF_SMEM_BYTES = 1024 + 2 * TILE + NQ * 2 * CTILE + DSTILE + DQSTAGE + 8 * QC * 4 + sizeof(KvSmem) + 32;
 constexpr int KV_THREADS = 448;   // TMA, MMA, 8 compute warps, 4 loader warps
+constexpr int KVF_THREADS = 576;  // ... plus 4 dQ writer warps
 constexpr uint32_t IDESC_K64 = make_idesc_bf16(128, QC, false, false);   // S^T, dP^T: N = 64 queries
+constexpr uint32_t IDESC_DQT = make_idesc_bf16(128, QC, true, true);     // dQ^T = K^T dS^T: both operands MN-major
 
 struct KvParams {
   const __nv_bfloat16 *q, *d_o;
@@ -135,6 +157,7 @@ struct KvParams {
   float scale, scale_log2;
   long long capacity;
   __nv_bfloat16 *dk, *dv;
+  float* dq_acc;               // fused variant: fp32 [queries][head_dim], zeroed rows of all selecting queries
   int32_t* status;
   unsigned long long* prof;    // optional wait-time counters (diagnostics), or null
 };
@@ -194,15 +217,19 @@ __device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, i
   return it;
 }
 
-template <bool DENSE>
-__global__ void __launch_bounds__(KV_THREADS, 1)
+template <bool DENSE, bool FUSE>
+__global__ void __launch_bounds__(FUSE ? KVF_THREADS : KV_THREADS, 1)
 attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const KvParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sK = base;                  // [2][TILE]
-  uint8_t* sV = base + 2 * TILE;       // [2][TILE]
-  uint8_t* sC = base + 4 * TILE;       // [NQ][Q chunk | dO chunk]
-  KvSmem* sm = reinterpret_cast<KvSmem*>(sC + NQ * 2 * CTILE);
+  constexpr int KVB = FUSE ? 1 : 2;    // K/V buffers
+  uint8_t* sK = base;                  // [KVB][TILE]
+  uint8_t* sV = base + KVB * TILE;     // [KVB][TILE]
+  uint8_t* sC = base + 2 * KVB * TILE; // [NQ][Q chunk | dO chunk]
+  uint8_t* sDS = sC + NQ * 2 * CTILE;  // fused variant: dS^T of the current unit [DSTILE]
+  float* s_stage = reinterpret_cast<float*>(sDS + DSTILE);                         // fused variant: [QC][DH] fp32
+  int* s_qrow = reinterpret_cast<int*>(sDS + DSTILE + DQSTAGE);                    // fused variant: [unit % 8][query] accumulator row, -1 = padding
+  KvSmem* sm = reinterpret_cast<KvSmem*>(sDS + (FUSE ? DSTILE + DQSTAGE + 8 * QC * 4 : 0));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm->abort_flag;
   // diagnostics: cycles spent in each wait site by one representative thread per role
@@ -228,6 +255,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sm->kv_full[b], 1); mbar_init(&sm->kv_empty[b], 1);
       mbar_init(&sm->sdp_full[b], 1); mbar_init(&sm->pds_ready[b], 256);
+      mbar_init(&sm->dq_full[b], 1); mbar_init(&sm->dq_free[b], 128);
     }
     for (int b = 0; b < NQ; ++b) { mbar_init(&sm->chunk_full[b], 128); mbar_init(&sm->chunk_empty[b], 1); }
     mbar_init(&sm->acc_done, 1);
@@ -258,8 +286,12 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
         const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
         if (it.n_units == 0) continue;
-        const int b = n & 1;
-        if (n >= 2) twait(0, &sm->kv_empty[b], ((n >> 1) - 1) & 1);
+        const int b = FUSE ? 0 : (n & 1);
+        if (FUSE) {
+          if (n >= 1) twait(0, &sm->kv_empty[0], (n - 1) & 1);
+        } else if (n >= 2) {
+          twait(0, &sm->kv_empty[b], ((n >> 1) - 1) & 1);
+        }
         const int y = (int)it.head_off + it.key0;
         mbar_expect_tx(&sm->kv_full[b], 2 * TILE);
         tma_load_2d(sK + b * TILE, &tmK, &sm->kv_full[b], 0, y);
@@ -269,7 +301,8 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         ++n;
       }
       if (*abort_flag)
-        for (uint32_t f = n > 2 ? n - 2 : 0; f < n; ++f) mbar_wait(&sm->kv_full[f & 1], (f >> 1) & 1, abort_flag, p.status);
+        for (uint32_t f = n > 2 ? n - 2 : 0; f < n; ++f)
+          mbar_wait(&sm->kv_full[FUSE ? 0 : (f & 1)], (FUSE ? f : (f >> 1)) & 1, abort_flag, p.status);
       tflush(0, 1);      // [0] kv_empty, [1] total
     }
   } else if (warp == 1) {
@@ -279,13 +312,16 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
         const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
         if (it.n_units == 0) continue;
-        const int b = n & 1;
-        twait(0, &sm->kv_full[b], (n >> 1) & 1);
+        const int b = FUSE ? 0 : (n & 1);
+        twait(0, &sm->kv_full[b], (FUSE ? n : (n >> 1)) & 1);
         tc_fence_after();
         const uint64_t dK0 = desc_k(smem_u32(sK + b * TILE), 0), dV0 = desc_k(smem_u32(sV + b * TILE), 0);
+        const uint64_t mK0 = desc_mn(smem_u32(sK + b * TILE), 0);     // K^T as MN-major A operand (fused dQ^T)
         auto issue_sdp = [&](int i) {
           const uint32_t u = u0 + i;
           const int cb = u % NQ, tb = u & 1;
+          // fused: the dP^T buffer last held dQ^T of unit u - 2, which the writer warps must have read
+          if (FUSE && u >= 2) twait(3, &sm->dq_free[tb], ((u - 2) >> 1) & 1);
           twait(1, &sm->chunk_full[cb], (u / NQ) & 1);
           tc_fence_after();
           const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE);
@@ -300,8 +336,9 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           mma_commit(&sm->sdp_full[tb]);
         };
         issue_sdp(0);
+        if (FUSE && it.n_units > 1) issue_sdp(1);
         for (int i = 0; i < it.n_units; ++i) {
-          if (i + 1 < it.n_units) issue_sdp(i + 1);
+          if (!FUSE && i + 1 < it.n_units) issue_sdp(i + 1);
           const uint32_t u = u0 + i;
           const int cb = u % NQ, tb = u & 1;
           twait(2, &sm->pds_ready[tb], (u >> 1) & 1);
@@ -314,14 +351,27 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           const uint64_t mQ0 = cdesc_mn(sQ_addr, 0), mO0 = cdesc_mn(sQ_addr + CTILE, 0);
           const uint32_t pt = tmem + ST_COL + tb * QC, dst_ = tmem + DPT_COL + tb * QC;
           const uint32_t acc0 = i > 0 ? 1u : 0u;
-          // P^T / dS^T of queries 32h .. 32h+31 sit in columns 32h .. 32h+15 of their buffer
+          if (FUSE) {
+            // dQ^T [head dim x 64 queries] = K^T dS^T over the tile's keys, into the unit's dP^T columns
+            // (already read by the compute warps); issued first so that its read-out overlaps dV / dK
+            const uint64_t mS0 = make_smem_desc(smem_u32(sDS), DSTILE, 1024);
+            const int kk = (it.valid + 15) >> 4;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+              if (ks < kk) mma_ss(dst_, mK0 + mnoff(ks), mS0 + mnoff(ks), IDESC_DQT, ks > 0 ? 1u : 0u);
+            mma_commit(&sm->dq_full[tb]);
+          }
+          // P^T of queries 32h .. 32h+31 sits in columns 32h .. 32h+15 of the S^T buffer; dS^T in the same
+          // columns of the dP^T buffer (split kernels) or in columns 32h+16 .. 32h+31 of the S^T buffer (fused)
+          const uint32_t ds_t = FUSE ? pt + 16 : dst_;
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
             if (ks < ksteps) {
               mma_ts(tmem + DV_COL, pt + (ks >> 1) * 32 + (ks & 1) * 8, mO0 + mnoff(ks), IDESC_TN, ks > 0 ? 1u : acc0);
-              mma_ts(tmem + DK_COL, dst_ + (ks >> 1) * 32 + (ks & 1) * 8, mQ0 + mnoff(ks), IDESC_TN, ks > 0 ? 1u : acc0);
+              mma_ts(tmem + DK_COL, ds_t + (ks >> 1) * 32 + (ks & 1) * 8, mQ0 + mnoff(ks), IDESC_TN, ks > 0 ? 1u : acc0);
             }
           mma_commit(&sm->chunk_empty[cb]);
+          if (FUSE && i + 2 < it.n_units) issue_sdp(i + 2);
         }
         mma_commit(&sm->kv_empty[b]);
         mma_commit(&sm->acc_done);
@@ -330,7 +380,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       }
       tflush(2, 4);      // [2] kv_full, [3] chunk_full, [4] pds_ready, [5] acc_free, [6] total
     }
-  } else if (warp >= 10) {
+  } else if (warp >= 10 && warp < 14) {
     // ------------------------------------------------------------------ loaders: gather Q / dO chunks (run ahead)
     const int lt = threadIdx.x - 320;   // 0..127
     uint32_t u0 = 0;
@@ -346,22 +396,75 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         gather_chunk64(nullptr, p.q + it.head_off * DH, rows, lt, row_of, vq);
         gather_chunk64(nullptr, p.d_o + it.head_off * DH, rows, lt, row_of, vo);
         float l2 = INFINITY, dd = 0.f;     // padded queries: P = exp2(-inf) = 0
+        int qr = -1;
         if (lt < rows) {
           const long long G_ = it.head_off + row_of(lt);
           l2 = p.lse[G_] * LOG2E;
           dd = p.Dv[G_];
+          qr = (int)G_;
         }
         if (u >= NQ) twait(0, &sm->chunk_empty[cb], ((u / NQ) - 1) & 1);
         uint8_t* dst = sC + cb * 2 * CTILE;
         store_chunk64(dst, lt, vq);
         store_chunk64(dst + CTILE, lt, vo);
-        if (lt < QC) { sm->lse2[cb][lt] = l2; sm->Dq[cb][lt] = dd; }
+        if (lt < QC) { sm->lse2[cb][lt] = l2; sm->Dq[cb][lt] = dd; if (FUSE) s_qrow[(u & 7) * QC + lt] = qr; }
         fence_async_proxy();
         mbar_arrive(&sm->chunk_full[cb]);
       }
       u0 += it.n_units;
     }
     if (lt == 0) tflush(7, 1);     // [7] chunk_empty, [8] total
+  } else if (FUSE && warp >= 14) {
+    // ------------------------------------------------------------------ dQ writers: thread = head-dim index
+    // Read dQ^T of a unit out of TMEM, release the buffer, transpose it through shared memory into 64
+    // rows of 128 floats and add each row into the fp32 accumulator with one bulk reduction.
+    const int quad = warp & 3;
+    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const int d = quad * 32 + lane;
+    uint32_t u0 = 0;
+    for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+      const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+      for (int i = 0; i < it.n_units; ++i) {
+        const uint32_t u = u0 + i;
+        const int tb = u & 1;
+        long long tw0 = p.prof ? clock64() : 0;
+        mbar_wait(&sm->dq_full[tb], (u >> 1) & 1, abort_flag, p.status);
+        if (p.prof) { const long long t = clock64(); wp[0] += t - tw0; tw0 = t; }
+        tc_fence_after();
+        uint32_t a[32], c2[32];
+        tmem_ld32(tmem + lane_addr + DPT_COL + tb * QC, a);
+        tmem_ld32(tmem + lane_addr + DPT_COL + tb * QC + 32, c2);
+        tmem_ld_wait();
+        tc_fence_before();
+        mbar_arrive(&sm->dq_free[tb]);
+        // the staging tile is free once the previous unit's bulk reductions have read it
+        if (p.prof) { const long long t = clock64(); wp[1] += t - tw0; tw0 = t; }
+        if (warp == 14) bulk_wait_read0();
+        writer_sync();
+        if (p.prof) { const long long t = clock64(); wp[2] += t - tw0; tw0 = t; }
+#pragma unroll
+        for (int c = 0; c < 32; ++c) s_stage[c * DH + d] = __uint_as_float(a[c]) * p.scale;
+#pragma unroll
+        for (int c = 0; c < 32; ++c) s_stage[(32 + c) * DH + d] = __uint_as_float(c2[c]) * p.scale;
+        fence_async_proxy();
+        writer_sync();
+        if (warp == 14) {
+          const int* qr = s_qrow + (u & 7) * QC;
+#pragma unroll
+          for (int c = lane; c < QC; c += 32) {
+            const int row = qr[c];
+            if (row >= 0) bulk_reduce_add_f32(p.dq_acc + (long long)row * DH, s_stage + c * DH, DH * 4);
+          }
+          bulk_commit();
+        }
+        if (p.prof) { const long long t = clock64(); wp[3] += t - tw0; tw0 = t; }
+      }
+      u0 += it.n_units;
+    }
+    if (p.prof && warp == 14 && lane == 0) {
+      atomicAdd(p.prof + 9, wp[0]); atomicAdd(p.prof + 14, wp[1]); atomicAdd(p.prof + 15, wp[2]); atomicAdd(p.prof + 1, wp[3]);
+    }
+    if (warp == 14) bulk_wait0();    // shared memory must stay valid until the last reductions have read it
   } else {
     // ------------------------------------------------------------------ compute: thread = (key row, half of the unit's queries)
     const int quad = warp & 3;
@@ -413,7 +516,22 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           dk_[2 * e + 1] = pack_bf16(p2 * (__uint_as_float(dv_[4 * e + 2]) - d4.z), p3 * (__uint_as_float(dv_[4 * e + 3]) - d4.w));
         }
         tmem_st16(st_t, pk);       // P^T (bf16 pairs) over the first 16 of this thread's 32 S^T columns
-        tmem_st16(dp_t, dk_);      // dS^T likewise over its dP^T columns
+        if (FUSE) {
+          tmem_st16(st_t + 16, dk_);   // dS^T over the other 16: the dP^T columns are about to receive dQ^T
+          // and once more, as the row of this key in the [keys][queries] shared-memory tile that dQ^T reads;
+          // rows beyond the key range hold other blocks' keys and must not contribute
+          uint8_t* dsrow = sDS + r * 128;
+          const bool live = r < it.valid;
+          // one tile: the previous unit's dQ^T must have finished reading it
+          if (u >= 1) mbar_wait(&sm->dq_full[(u - 1) & 1], ((u - 1) >> 1) & 1, abort_flag, p.status);
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            *reinterpret_cast<uint4*>(dsrow + (((4 * half + j) ^ (r & 7)) << 4)) =
+                live ? make_uint4(dk_[4 * j], dk_[4 * j + 1], dk_[4 * j + 2], dk_[4 * j + 3]) : make_uint4(0u, 0u, 0u, 0u);
+          fence_async_proxy();
+        } else {
+          tmem_st16(dp_t, dk_);    // dS^T likewise over its dP^T columns
+        }
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(&sm->pds_ready[tb]);
@@ -451,287 +569,6 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-// ==========================================================================================
-// dQ
-// ==========================================================================================
-// Item = 128 gathered queries x one key block (the forward's work items).  Keys stream in units of
-// 64 through a 2-stage TMA ring; S and dP are double buffered in TMEM (64 columns each) and the dQ
-// accumulator is double buffered across items, so the epilogue of one item overlaps the MMAs of
-// the next.  Loader warps gather Q / dO rows (and lse, D, output row) of the NEXT item meanwhile.
-constexpr int KU = 64;                       // keys per unit
-// Two shared-memory splits: short key blocks (few units per item) double buffer the gathered
-// Q / dO tiles across items and keep a 2-deep K/V ring; long blocks keep one Q / dO tile and a
-// 4-deep K/V ring, because there the ring depth hides the TMA latency.
-constexpr int DQ_NS_MAX = 4;
-struct DqSmem {
-  uint64_t kv_full[DQ_NS_MAX], kv_empty[DQ_NS_MAX];  // K+V unit (TMA / commit)
-  uint64_t qdo_full[2], qdo_empty[2];        // gathered Q/dO of an item (128 loader arrivals / commit)
-  uint64_t sdp_full[2];                      // S and dP of a unit ready (commit)
-  uint64_t ds_ready[2];                      // dS written (128 compute arrivals)
-  uint64_t dq_done[2];                       // all MMAs of the item done (commit)
-  uint64_t dq_free[2];                       // epilogue has read the accumulator (128 compute arrivals)
-  uint32_t tmem_base;
-  int abort_flag;
-  float lse2[2][128];
-  float Dr[2][128];
-  long long G[2][128];                       // flat output row of each query, -1 for padding rows
-  int direct[2][128];                        // query has a single block: write bf16 directly
-};
-constexpr size_t dq_smem_bytes(int QB, int NS) { return 1024 + QB * 2 * TILE + NS * 2 * CTILE + sizeof(DqSmem) + 32; }
-constexpr int DQ_THREADS = 448;   // TMA, MMA, 8 compute warps, 4 loader warps
-
-struct DqParams {
-  const __nv_bfloat16 *q, *d_o;
-  const float *lse, *Dv;
-  const int *kb_ptr, *q_idx, *q_ptr, *item_ptr, *item_tab;
-  int n_kb, S, Nb, sb, BH;
-  float scale, scale_log2;
-  long long capacity;
-  float* dq_acc;            // sparse, queries with several blocks: fp32 accumulator [BH*S, 128]
-  __nv_bfloat16* dq;        // dense, and sparse queries with a single block: written directly
-  int32_t* status;
-};
-
-struct DqItem {
-  int bh, key_begin, n_keys, list_lo, n_rows, n_units;
-  long long head_off;
-};
-
-template <bool DENSE>
-__device__ __forceinline__ DqItem dq_decode(const DqParams& p, int item) {
-  DqItem it;
-  if (DENSE) {
-    const int tiles = (p.S + BM - 1) / BM;
-    it.bh = item / tiles;
-    const int t = item - it.bh * tiles;
-    it.key_begin = 0; it.n_keys = p.S; it.list_lo = t * BM; it.n_rows = min(BM, p.S - it.list_lo);
-  } else {
-    const int kbi = __ldg(p.item_tab + item);
-    const int chunk = item - __ldg(p.item_ptr + kbi);
-    it.bh = kbi / p.Nb;
-    const int j = kbi - it.bh * p.Nb;
-    it.key_begin = j * p.sb; it.n_keys = p.sb;
-    const long long end = min((long long)__ldg(p.kb_ptr + kbi + 1), p.capacity);
-    it.list_lo = __ldg(p.kb_ptr + kbi) + chunk * BM;
-    it.n_rows = (int)min((long long)BM, end - it.list_lo);
-  }
-  it.n_units = (it.n_keys + KU - 1) / KU;
-  it.head_off = (long long)it.bh * p.S;
-  return it;
-}
-
-template <bool DENSE, int QB, int DQ_NS>
-__global__ void __launch_bounds__(DQ_THREADS, 1)
-attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const DqParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQdO = base;                    // [QB][Q tile | dO tile]
-  uint8_t* sKV = base + QB * 2 * TILE;     // [DQ_NS][K unit | V unit]
-  DqSmem* sm = reinterpret_cast<DqSmem*>(sKV + DQ_NS * 2 * CTILE);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  volatile int* abort_flag = &sm->abort_flag;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < DQ_NS; ++s) { mbar_init(&sm->kv_full[s], 1); mbar_init(&sm->kv_empty[s], 1); }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(&sm->qdo_full[b], 128); mbar_init(&sm->qdo_empty[b], 1);
-      mbar_init(&sm->sdp_full[b], 1); mbar_init(&sm->ds_ready[b], 256);
-      mbar_init(&sm->dq_done[b], 1); mbar_init(&sm->dq_free[b], 256);
-    }
-    sm->abort_flag = 0;
-    fence_barrier_init();
-    prefetch_tmap(&tmK);
-    prefetch_tmap(&tmV);
-  }
-  if (warp == 1) {
-    tmem_alloc(&sm->tmem_base, TMEM_COLS);
-    tmem_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = sm->tmem_base;
-  constexpr uint32_t S_COL = 0, DP_COL = 128, DQ_COL = 256;   // S, dP: two 64-column buffers; dQ: two 128-column buffers
-  const int n_items = DENSE ? p.BH * ((p.S + BM - 1) / BM) : p.item_ptr[p.n_kb];
-
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer: K and V units
-    if (lane == 0) {
-      uint32_t f = 0;
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const DqItem it = dq_decode<DENSE>(p, item);
-        const int row0 = (int)it.head_off + it.key_begin;
-        for (int i = 0; i < it.n_units; ++i, ++f) {
-          const int s = f % DQ_NS;
-          if (f >= DQ_NS) mbar_wait(&sm->kv_empty[s], ((f / DQ_NS) - 1) & 1, abort_flag, p.status);
-          uint8_t* dst = sKV + s * 2 * CTILE;
-          const int y = row0 + i * KU;
-          mbar_expect_tx(&sm->kv_full[s], 2 * CTILE);
-          tma_load_2d(dst, &tmK, &sm->kv_full[s], 0, y);
-          tma_load_2d(dst + CPANEL, &tmK, &sm->kv_full[s], 64, y);
-          tma_load_2d(dst + CTILE, &tmV, &sm->kv_full[s], 0, y);
-          tma_load_2d(dst + CTILE + CPANEL, &tmV, &sm->kv_full[s], 64, y);
-        }
-      }
-      if (*abort_flag)
-        for (uint32_t g = f > DQ_NS ? f - DQ_NS : 0; g < f; ++g)
-          mbar_wait(&sm->kv_full[g % DQ_NS], (g / DQ_NS) & 1, abort_flag, p.status);
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      uint32_t n = 0, u0 = 0;
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
-        const DqItem it = dq_decode<DENSE>(p, item);
-        const int qb = n & 1;                 // accumulator / scalar slot
-        const int qs = n % QB;                // Q / dO tile slot
-        mbar_wait(&sm->qdo_full[qs], (n / QB) & 1, abort_flag, p.status);
-        tc_fence_after();
-        const uint32_t sQ_addr = smem_u32(sQdO + qs * 2 * TILE), sdO_addr = sQ_addr + TILE;
-        auto n_mma_of = [&](int i) { return (min(KU, it.n_keys - i * KU) + 15) & ~15; };
-        auto issue_sdp = [&](int i) {
-          const uint32_t u = u0 + i;
-          const int s = u % DQ_NS, tb = u & 1;
-          mbar_wait(&sm->kv_full[s], (u / DQ_NS) & 1, abort_flag, p.status);
-          tc_fence_after();
-          const uint32_t idesc = make_idesc_bf16(BM, n_mma_of(i), false, false);
-          const uint32_t sK_addr = smem_u32(sKV + s * 2 * CTILE), sV_addr = sK_addr + CTILE;
-#pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks)
-            mma_ss(tmem + S_COL + tb * KU, desc_k(sQ_addr, ks), cdesc_k(sK_addr, ks), idesc, ks > 0 ? 1u : 0u);
-#pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks)
-            mma_ss(tmem + DP_COL + tb * KU, desc_k(sdO_addr, ks), cdesc_k(sV_addr, ks), idesc, ks > 0 ? 1u : 0u);
-          mma_commit(&sm->sdp_full[tb]);
-        };
-        issue_sdp(0);
-        for (int i = 0; i < it.n_units; ++i) {
-          if (i + 1 < it.n_units) issue_sdp(i + 1);
-          const uint32_t u = u0 + i;
-          const int s = u % DQ_NS, tb = u & 1;
-          mbar_wait(&sm->ds_ready[tb], (u >> 1) & 1, abort_flag, p.status);
-          // this accumulator was last used two items ago: its epilogue must have read it
-          if (i == 0 && n >= 2) mbar_wait(&sm->dq_free[qb], ((n >> 1) - 1) & 1, abort_flag, p.status);
-          tc_fence_after();
-          const int ksteps = n_mma_of(i) >> 4;
-          const uint32_t sK_addr = smem_u32(sKV + s * 2 * CTILE);
-          // dS of keys 32h .. 32h+31 sits in columns 32h .. 32h+15 of the dP buffer
-          for (int ks = 0; ks < ksteps; ++ks)
-            mma_ts(tmem + DQ_COL + qb * 128, tmem + DP_COL + tb * KU + (ks >> 1) * 32 + (ks & 1) * 8, cdesc_mn(sK_addr, ks),
-                   IDESC_TN, (i > 0 || ks > 0) ? 1u : 0u);
-          mma_commit(&sm->kv_empty[s]);
-        }
-        mma_commit(&sm->qdo_empty[qs]);
-        mma_commit(&sm->dq_done[qb]);
-        u0 += it.n_units;
-      }
-    }
-  } else if (warp >= 10) {
-    // ------------------------------------------------------------------ loaders: Q / dO rows of the next items
-    const int lt = threadIdx.x - 320;   // 0..127
-    uint32_t n = 0;
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
-      const DqItem it = dq_decode<DENSE>(p, item);
-      const int qb = n & 1, qs = n % QB;
-      auto row_of = [&](int r) { return DENSE ? it.list_lo + r : __ldg(p.q_idx + it.list_lo + r); };
-      // this thread's own row (lt) for the per-row scalars; issue before the big gathers
-      long long G_ = -1;
-      float l2 = INFINITY, dd = 0.f;
-      int direct = DENSE ? 1 : 0;
-      if (lt < it.n_rows) {
-        G_ = it.head_off + row_of(lt);
-        l2 = p.lse[G_] * LOG2E;
-        dd = p.Dv[G_];
-        if (!DENSE) direct = (p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1;
-      }
-      uint4 vq[16];
-      gather_load128(p.q + it.head_off * DH, it.n_rows, lt, row_of, vq);
-      if (n >= QB) mbar_wait(&sm->qdo_empty[qs], ((n / QB) - 1) & 1, abort_flag, p.status);
-      // the scalar slots alternate by item; with a single Q / dO tile the compute warps may still be
-      // reading slot qb of item n-2 only if they lag two items behind, which qdo_empty(n-1) excludes
-      uint8_t* dst = sQdO + qs * 2 * TILE;
-      gather_store128(dst, lt, vq);
-      gather_load128(p.d_o + it.head_off * DH, it.n_rows, lt, row_of, vq);
-      gather_store128(dst + TILE, lt, vq);
-      sm->lse2[qb][lt] = l2; sm->Dr[qb][lt] = dd; sm->G[qb][lt] = G_; sm->direct[qb][lt] = direct;
-      fence_async_proxy();
-      mbar_arrive(&sm->qdo_full[qs]);
-    }
-  } else {
-    // ------------------------------------------------------------------ compute: thread = (query row, half of the unit's keys)
-    const int quad = warp & 3;
-    const int half = (warp - 2) >> 2;                 // warps 2-5: keys 0-31 of a unit, warps 6-9: keys 32-63
-    const int r = quad * 32 + lane;
-    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    uint32_t n = 0, u0 = 0;
-    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
-      const DqItem it = dq_decode<DENSE>(p, item);
-      const int qb = n & 1, qs = n % QB;
-      mbar_wait(&sm->qdo_full[qs], (n / QB) & 1, abort_flag, p.status);   // publishes the per-row scalars
-      const float lse2 = sm->lse2[qb][r], Dr = sm->Dr[qb][r];
-      const long long G_ = sm->G[qb][r];
-      const int direct = sm->direct[qb][r];
-      for (int i = 0; i < it.n_units; ++i) {
-        const uint32_t u = u0 + i;
-        const int tb = u & 1;
-        const int valid = min(KU, it.n_keys - i * KU) - 32 * half;     // valid keys among this thread's 32
-        mbar_wait(&sm->sdp_full[tb], (u >> 1) & 1, abort_flag, p.status);
-        tc_fence_after();
-        const uint32_t s_t = tmem + lane_addr + S_COL + tb * KU + 32 * half;
-        const uint32_t dp_t = tmem + lane_addr + DP_COL + tb * KU + 32 * half;
-        uint32_t sv[32], dv_[32];
-        tmem_ld32(s_t, sv);
-        tmem_ld32(dp_t, dv_);
-        tmem_ld_wait();
-        uint32_t ds[16];
-#pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const float p0 = ex2(fmaf(__uint_as_float(sv[2 * e]), p.scale_log2, -lse2));
-          const float p1 = ex2(fmaf(__uint_as_float(sv[2 * e + 1]), p.scale_log2, -lse2));
-          const float x0 = (2 * e < valid) ? p0 * (__uint_as_float(dv_[2 * e]) - Dr) : 0.f;
-          const float x1 = (2 * e + 1 < valid) ? p1 * (__uint_as_float(dv_[2 * e + 1]) - Dr) : 0.f;
-          ds[e] = pack_bf16(x0, x1);
-        }
-        tmem_st16(dp_t, ds);      // dS (bf16 pairs) over the first 16 of this thread's 32 dP columns
-        tmem_st_wait();
-        tc_fence_before();
-        mbar_arrive(&sm->ds_ready[tb]);
-      }
-      u0 += it.n_units;
-      // ---- epilogue: each half writes 64 of the 128 dQ columns of its row
-      mbar_wait(&sm->dq_done[qb], (n >> 1) & 1, abort_flag, p.status);
-      tc_fence_after();
-#pragma unroll 1
-      for (int cg2 = 0; cg2 < 2; ++cg2) {
-        const int cgrp = half * 2 + cg2;
-        uint32_t a[32];
-        tmem_ld32(tmem + lane_addr + DQ_COL + qb * 128 + cgrp * 32, a);
-        tmem_ld_wait();
-        if (G_ >= 0) {
-          if (direct) {
-            __nv_bfloat16* dst = p.dq + G_ * DH + cgrp * 32;
-#pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              store4(dst + i, make_float4(__uint_as_float(a[i]) * p.scale, __uint_as_float(a[i + 1]) * p.scale,
-                                          __uint_as_float(a[i + 2]) * p.scale, __uint_as_float(a[i + 3]) * p.scale));
-          } else {
-            float* dst = p.dq_acc + G_ * DH + cgrp * 32;
-#pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              red_add_v4(dst + i, __uint_as_float(a[i]) * p.scale, __uint_as_float(a[i + 1]) * p.scale,
-                         __uint_as_float(a[i + 2]) * p.scale, __uint_as_float(a[i + 3]) * p.scale);
-          }
-        }
-      }
-      tc_fence_before();
-      mbar_arrive(&sm->dq_free[qb]);
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
-}
-
 static int grid_items(long long items) { return (int)std::max<long long>(1, std::min<long long>(items, 148)); }
 
 }  // namespace tcb
@@ -743,24 +580,15 @@ int tc_long_dkdv(const Dims& D, bool dense, const void* q, const void* k, const 
 int tc_long_dq(const Dims& D, bool dense, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap, const int* item_ptr,
                const int* item_tab, float* dq_acc, void* dq, int32_t* status, cudaStream_t st);
-static bool use_long_kernels(const Dims& D) { (void)D; return false; }   // measured slower than the 64-column unit kernels on every sparse workload tried
-
 // Backward over the work lists (bf16, head_dim 128).  Dv holds rowsum(dO * O) per query; dq_acc is
-// a zeroed fp32 accumulator that the caller converts to bf16 afterwards.
+// an fp32 accumulator whose rows of selecting queries are zero; the caller converts it to bf16.
 int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
-                  const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap,
-                  const int* item_ptr, const int* item_tab, float* dq_acc, void* dq, void* dk, void* dv,
+                  const float* Dv, const int* kb_ptr, const int* q_idx, long long cap, float* dq_acc, void* dk, void* dv,
                   int32_t* status, cudaStream_t st) {
-  if (use_long_kernels(D)) {
-    int rc = tc_long_dkdv(D, false, q, k, v, d_o, lse, Dv, kb_ptr, q_idx, cap, dk, dv, status, tcb::g_wait_profile, st);
-    if (rc) return rc;
-    return tc_long_dq(D, false, q, k, v, d_o, lse, Dv, kb_ptr, q_idx, q_ptr, cap, item_ptr, item_tab, dq_acc, dq, status, st);
-  }
   using namespace tcb;
-  CUtensorMap tmK, tmV, tmK64, tmV64;
+  CUtensorMap tmK, tmV;
   const uint64_t rows = (uint64_t)D.BH * D.S;
-  if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN) ||
-      !sm100::make_tmap_bf16_rows(&tmK64, k, rows, DH, KU) || !sm100::make_tmap_bf16_rows(&tmV64, v, rows, DH, KU))
+  if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN))
     return VMOBA_ERR_CUDA;
   const long long n_kb = (long long)D.BH * D.Nb;
   KvParams kp;
@@ -768,63 +596,21 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
   kp.kb_ptr = kb_ptr; kp.q_idx = q_idx; kp.S = D.S; kp.Nb = D.Nb; kp.sb = D.sb; kp.BH = D.BH;
   kp.scale = D.scale; kp.scale_log2 = D.scale * LOG2E; kp.capacity = cap;
   kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status; kp.prof = tcb::g_wait_profile;
-  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)KV_SMEM_BYTES));
+  kp.dq_acc = dq_acc;
   const long long kv_items = n_kb * ((D.sb + BN - 1) / BN);
-  attn_bwd_dkdv_tc_kernel<false><<<grid_items(kv_items), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, kp);
-  DqParams qp;
-  qp.q = kp.q; qp.d_o = kp.d_o; qp.lse = lse; qp.Dv = Dv; qp.kb_ptr = kb_ptr; qp.q_idx = q_idx; qp.item_ptr = item_ptr;
-  qp.item_tab = item_tab;
-  qp.n_kb = (int)n_kb; qp.S = D.S; qp.Nb = D.Nb; qp.sb = D.sb; qp.BH = D.BH; qp.scale = D.scale;
-  qp.scale_log2 = D.scale * LOG2E; qp.capacity = cap; qp.dq_acc = dq_acc; qp.dq = (__nv_bfloat16*)dq; qp.status = status;
-  qp.q_ptr = q_ptr;
-  if (D.sb >= 1024) {
-    constexpr size_t SM = dq_smem_bytes(1, 4);
-    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<false, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM));
-    attn_bwd_dq_tc_kernel<false, 1, 4><<<grid_items(cap / BM + n_kb), DQ_THREADS, SM, st>>>(tmK64, tmV64, qp);
-  } else {
-    constexpr size_t SM = dq_smem_bytes(2, 2);
-    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<false, 2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM));
-    attn_bwd_dq_tc_kernel<false, 2, 2><<<grid_items(cap / BM + n_kb), DQ_THREADS, SM, st>>>(tmK64, tmV64, qp);
-  }
-  VMOBA_LAUNCH_OK(2);
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)KVF_SMEM_BYTES));
+  attn_bwd_dkdv_tc_kernel<false, true><<<grid_items(kv_items), KVF_THREADS, KVF_SMEM_BYTES, st>>>(tmK, tmV, kp);
+  VMOBA_LAUNCH_OK(1);
   return VMOBA_OK;
 }
 
+// Dense backward: the kernels with 128-query units (one key range spanning the sequence).
 int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* Dv, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st) {
-  {
-    int rc = tc_long_dkdv(D, true, q, k, v, d_o, lse, Dv, nullptr, nullptr, 0, dk, dv, status, tcb::g_wait_profile, st);
-    if (rc) return rc;
-    return tc_long_dq(D, true, q, k, v, d_o, lse, Dv, nullptr, nullptr, nullptr, 0, nullptr, nullptr, nullptr, dq, status, st);
-  }
-  using namespace tcb;
-  CUtensorMap tmK, tmV, tmK64, tmV64;
-  const uint64_t rows = (uint64_t)D.BH * D.S;
-  if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN) ||
-      !sm100::make_tmap_bf16_rows(&tmK64, k, rows, DH, KU) || !sm100::make_tmap_bf16_rows(&tmV64, v, rows, DH, KU))
-    return VMOBA_ERR_CUDA;
-  KvParams kp;
-  kp.q = (const __nv_bfloat16*)q; kp.d_o = (const __nv_bfloat16*)d_o; kp.lse = lse; kp.Dv = Dv;
-  kp.kb_ptr = nullptr; kp.q_idx = nullptr; kp.S = D.S; kp.Nb = 1; kp.sb = D.S; kp.BH = D.BH;
-  kp.scale = D.scale; kp.scale_log2 = D.scale * LOG2E; kp.capacity = 0;
-  kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status; kp.prof = tcb::g_wait_profile;
-  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)KV_SMEM_BYTES));
-  const long long tiles = (D.S + BN - 1) / BN;
-  attn_bwd_dkdv_tc_kernel<true><<<grid_items(D.BH * tiles), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, kp);
-  DqParams qp;
-  qp.q = kp.q; qp.d_o = kp.d_o; qp.lse = lse; qp.Dv = Dv; qp.kb_ptr = nullptr; qp.q_idx = nullptr; qp.item_ptr = nullptr;
-  qp.item_tab = nullptr;
-  qp.n_kb = 0; qp.S = D.S; qp.Nb = 1; qp.sb = D.S; qp.BH = D.BH; qp.scale = D.scale; qp.scale_log2 = D.scale * LOG2E;
-  qp.capacity = 0; qp.dq_acc = nullptr; qp.dq = (__nv_bfloat16*)dq; qp.status = status; qp.q_ptr = nullptr;
-  {
-    constexpr size_t SM = dq_smem_bytes(1, 4);
-    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dq_tc_kernel<true, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SM));
-    attn_bwd_dq_tc_kernel<true, 1, 4><<<grid_items(D.BH * tiles), DQ_THREADS, SM, st>>>(tmK64, tmV64, qp);
-  }
-  VMOBA_LAUNCH_OK(2);
-  return VMOBA_OK;
+  int rc = tc_long_dkdv(D, true, q, k, v, d_o, lse, Dv, nullptr, nullptr, 0, dk, dv, status, tcb::g_wait_profile, st);
+  if (rc) return rc;
+  return tc_long_dq(D, true, q, k, v, d_o, lse, Dv, nullptr, nullptr, nullptr, 0, nullptr, nullptr, nullptr, dq, status, st);
 }
 
 }  // namespace vmoba
