@@ -20,6 +20,7 @@
 namespace vmoba {
 
 constexpr int kBins = 2048;
+constexpr int kBins0 = 512;    // level 0 uses fewer bins, each replicated once per lane
 constexpr int kSegThreads = 512;
 
 struct HeadState {
@@ -27,7 +28,7 @@ struct HeadState {
   float anchor[3];             // lower edge of the interval refined at each level
   float inv[3];                // bins per unit score at each level
   int bin[3];                  // crossing bin found at each level
-  int level_ok;
+  int resolved;                // the level-1 crossing bin held a single distinct score: level 2 is skipped
   double Z;                    // sum of all weights
   double target;               // tau * Z
   double mass_above;           // weight of everything above the crossing bin so far
@@ -39,7 +40,7 @@ struct HeadState {
 // bin of a score at refinement level L given the state; monotone non-decreasing in s.
 __device__ __forceinline__ int bin_at(const HeadState& hs, int L, float s) {
   float t = (s - hs.anchor[L]) * hs.inv[L];
-  int b = t > 0.f ? (int)fminf(t, (float)(kBins - 1)) : 0;
+  int b = t > 0.f ? (int)fminf(t, (float)((L == 0 ? kBins0 : kBins) - 1)) : 0;
   return b;
 }
 
@@ -51,7 +52,15 @@ __device__ __forceinline__ void for_each_score(const float* __restrict__ base, l
   if ((reinterpret_cast<uintptr_t>(base) & 15u) == 0) {
     long long P4 = P >> 2;
     const float4* b4 = reinterpret_cast<const float4*>(base);
-    for (long long i = tid; i < P4; i += nth) {
+    long long i = tid;
+    for (; i + 3 * nth < P4; i += 4 * nth) {     // four independent 16-byte loads in flight
+      float4 x[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) x[j] = __ldg(b4 + i + j * nth);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { f(x[j].x); f(x[j].y); f(x[j].z); f(x[j].w); }
+    }
+    for (; i < P4; i += nth) {
       float4 x = __ldg(b4 + i);
       f(x.x); f(x.y); f(x.z); f(x.w);
     }
@@ -88,21 +97,26 @@ __global__ void init_state_kernel(HeadState* st, int BH) {
   st[i] = h;
 }
 
-// Level L histogram: pairs that fall in the crossing bins of all earlier levels add
-// (1, exp(sigma * (s - max))) to their level-L bin.  At the last level the smallest key of
-// each bin is tracked too, which turns the crossing bin into an exact fp32 cutoff.
+// Level L >= 1 histogram: pairs that fall in the crossing bins of all earlier levels add
+// (1, exp(sigma * (s - max))) to their level-L bin.  The smallest key of each bin is tracked too,
+// which turns the last crossing bin into an exact fp32 cutoff; at level 1 also the largest, so that
+// a crossing bin with a single distinct score ends the search there.
 template <int L>
 __global__ void __launch_bounds__(256)
 hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __restrict__ st, float sigma,
-            unsigned int* __restrict__ g_cnt, double* __restrict__ g_w, uint32_t* __restrict__ g_minkey) {
+            unsigned int* __restrict__ g_cnt, double* __restrict__ g_w, uint32_t* __restrict__ g_minkey,
+            uint32_t* __restrict__ g_maxkey) {
   __shared__ unsigned int s_cnt[kBins];
   __shared__ float s_w[kBins];
-  __shared__ uint32_t s_min[L == 2 ? kBins : 1];
+  __shared__ uint32_t s_min[kBins];
+  __shared__ uint32_t s_max[L == 1 ? kBins : 1];
   const int bh = blockIdx.y;
   const HeadState hs = st[bh];
+  if (L == 2 && hs.resolved) return;     // level 1 already pinned the cutoff: nothing to refine
   for (int i = threadIdx.x; i < kBins; i += blockDim.x) {
     s_cnt[i] = 0; s_w[i] = 0.f;
-    if (L == 2) s_min[i] = 0xffffffffu;
+    s_min[i] = 0xffffffffu;
+    if (L == 1) s_max[i] = 0u;
   }
   __syncthreads();
   const float smax = key_float(hs.max_key);
@@ -112,7 +126,8 @@ hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __re
     int b = bin_at(hs, L, s);
     atomicAdd(&s_cnt[b], 1u);
     atomicAdd(&s_w[b], expf(sigma * (s - smax)));
-    if (L == 2) atomicMin(&s_min[b], float_key(s));
+    atomicMin(&s_min[b], float_key(s));
+    if (L == 1) atomicMax(&s_max[b], float_key(s));
   });
   __syncthreads();
   for (int i = threadIdx.x; i < kBins; i += blockDim.x) {
@@ -120,8 +135,36 @@ hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __re
     if (c) {
       atomicAdd(&g_cnt[(long long)bh * kBins + i], c);
       atomicAdd(&g_w[(long long)bh * kBins + i], (double)s_w[i]);
-      if (L == 2) atomicMin(&g_minkey[(long long)bh * kBins + i], s_min[i]);
+      atomicMin(&g_minkey[(long long)bh * kBins + i], s_min[i]);
+      if (L == 1) atomicMax(&g_maxkey[(long long)bh * kBins + i], s_max[i]);
     }
+  }
+}
+
+// Level 0 sees every pair, and scores cluster: with one set of bins most lanes of a warp hit the
+// same few addresses and the shared-memory atomics serialise.  Here every bin has one copy per lane
+// in 32 consecutive words (a warp's updates always fall into 32 different banks), and only the
+// masses are kept: the scan needs no counts at this level.
+constexpr int kRep = 32;
+__global__ void __launch_bounds__(512)
+hist0_kernel(const float* __restrict__ scores, long long P, const HeadState* __restrict__ st, float sigma,
+             double* __restrict__ g_w) {
+  extern __shared__ float s_wr[];   // [kBins0][kRep]
+  const int bh = blockIdx.y;
+  const HeadState hs = st[bh];
+  for (int i = threadIdx.x; i < kBins0 * kRep; i += blockDim.x) s_wr[i] = 0.f;
+  __syncthreads();
+  const float smax = key_float(hs.max_key);
+  const int rep = threadIdx.x & (kRep - 1);
+  for_each_score(scores + (long long)bh * P, P, [&](float s) {
+    atomicAdd(&s_wr[bin_at(hs, 0, s) * kRep + rep], expf(sigma * (s - smax)));
+  });
+  __syncthreads();
+  for (int i = threadIdx.x; i < kBins0; i += blockDim.x) {
+    float w = 0.f;
+#pragma unroll
+    for (int r = 0; r < kRep; ++r) w += s_wr[i * kRep + ((r + i) & (kRep - 1))];
+    if (w > 0.f) atomicAdd(&g_w[(long long)bh * kBins + i], (double)w);
   }
 }
 
@@ -130,7 +173,8 @@ hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __re
 template <int L>
 __global__ void __launch_bounds__(1024)
 scan_kernel(HeadState* __restrict__ st, float tau, unsigned int* __restrict__ g_cnt, double* __restrict__ g_w,
-            uint32_t* __restrict__ g_minkey, int64_t* __restrict__ k_per_head, float* __restrict__ cutoff_per_head) {
+            uint32_t* __restrict__ g_minkey, uint32_t* __restrict__ g_maxkey, int64_t* __restrict__ k_per_head,
+            float* __restrict__ cutoff_per_head) {
   __shared__ double s_wsum[32];
   __shared__ unsigned long long s_csum[32];
   __shared__ int s_cross;
@@ -139,16 +183,20 @@ scan_kernel(HeadState* __restrict__ st, float tau, unsigned int* __restrict__ g_
   const int bh = blockIdx.x;
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   HeadState hs = st[bh];
+  if (L == 2 && hs.resolved) return;     // cutoff written at level 1; the histogram arrays are clear
   // element e = 0..2047 walks bins from the top: bin = 2047 - e; thread t owns e = 2t, 2t+1
   const long long hb = (long long)bh * kBins;
-  double w0 = g_w[hb + (kBins - 1 - 2 * t)], w1 = g_w[hb + (kBins - 2 - 2 * t)];
-  unsigned long long c0 = g_cnt[hb + (kBins - 1 - 2 * t)], c1 = g_cnt[hb + (kBins - 2 - 2 * t)];
-  uint32_t mk0 = 0xffffffffu, mk1 = 0xffffffffu;
-  if (L == 2) { mk0 = g_minkey[hb + (kBins - 1 - 2 * t)]; mk1 = g_minkey[hb + (kBins - 2 - 2 * t)]; }
+  const long long i0 = hb + (kBins - 1 - 2 * t), i1 = hb + (kBins - 2 - 2 * t);
+  double w0 = g_w[i0], w1 = g_w[i1];
+  // level 0 keeps masses only: a bin counts as occupied when its mass is positive
+  unsigned long long c0 = L == 0 ? (w0 > 0.0) : g_cnt[i0], c1 = L == 0 ? (w1 > 0.0) : g_cnt[i1];
+  uint32_t mk0 = 0xffffffffu, mk1 = 0xffffffffu, xk0 = 0u, xk1 = 0u;
+  if (L >= 1) { mk0 = g_minkey[i0]; mk1 = g_minkey[i1]; }
+  if (L == 1) { xk0 = g_maxkey[i0]; xk1 = g_maxkey[i1]; }
   // clear for the next level / next call
-  g_w[hb + (kBins - 1 - 2 * t)] = 0.0; g_w[hb + (kBins - 2 - 2 * t)] = 0.0;
-  g_cnt[hb + (kBins - 1 - 2 * t)] = 0u; g_cnt[hb + (kBins - 2 - 2 * t)] = 0u;
-  if (L == 2) { g_minkey[hb + (kBins - 1 - 2 * t)] = 0xffffffffu; g_minkey[hb + (kBins - 2 - 2 * t)] = 0xffffffffu; }
+  g_w[i0] = 0.0; g_w[i1] = 0.0;
+  if (L >= 1) { g_cnt[i0] = 0u; g_cnt[i1] = 0u; g_minkey[i0] = 0xffffffffu; g_minkey[i1] = 0xffffffffu; }
+  if (L == 1) { g_maxkey[i0] = 0u; g_maxkey[i1] = 0u; }
   double wl = w0 + w1;
   unsigned long long cl = c0 + c1;
   // inclusive warp scan
@@ -197,8 +245,9 @@ scan_kernel(HeadState* __restrict__ st, float tau, unsigned int* __restrict__ g_
   const int e_cross = kBins - 1 - cross_bin;
   __shared__ double s_above_w;
   __shared__ unsigned long long s_above_c;
-  if (2 * t == e_cross) { s_above_w = w_excl; s_above_c = c_excl; }
-  if (2 * t + 1 == e_cross) { s_above_w = w_excl + w0; s_above_c = c_excl + c0; }
+  __shared__ uint32_t s_cross_min, s_cross_max;
+  if (2 * t == e_cross) { s_above_w = w_excl; s_above_c = c_excl; s_cross_min = mk0; s_cross_max = xk0; }
+  if (2 * t + 1 == e_cross) { s_above_w = w_excl + w0; s_above_c = c_excl + c0; s_cross_min = mk1; s_cross_max = xk1; }
   if (L == 2) {
     // exact cutoff: smallest key among the bins at or above the crossing bin
     uint32_t mk = 0xffffffffu;
@@ -215,6 +264,13 @@ scan_kernel(HeadState* __restrict__ st, float tau, unsigned int* __restrict__ g_
     if (L < 2) {
       hs.anchor[L + 1] = hs.inv[L] > 0.f ? hs.anchor[L] + (float)cross_bin / hs.inv[L] : hs.anchor[L];
       hs.inv[L + 1] = fminf(hs.inv[L] * (float)kBins, 1e30f);
+      // one distinct score in the crossing bin: everything above it is below the target and the
+      // bin reaches it, so that score is the cutoff
+      if (L == 1 && tau < 1.0f && s_cross_min == s_cross_max && s_cross_min != 0xffffffffu) {
+        hs.resolved = 1;
+        hs.cutoff_key = s_cross_min;
+        cutoff_per_head[bh] = key_float(hs.cutoff_key);
+      }
     } else {
       hs.cutoff_key = s_minkey;
       if (tau >= 1.0f) hs.cutoff_key = hs.min_key;
@@ -231,7 +287,7 @@ __global__ void setup_level0_kernel(HeadState* st, int BH) {
   float lo = key_float(st[i].min_key), hi = key_float(st[i].max_key);
   float range = hi - lo;
   st[i].anchor[0] = lo;
-  st[i].inv[0] = range > 0.f ? (float)kBins / range : 0.f;
+  st[i].inv[0] = range > 0.f ? (float)kBins0 / range : 0.f;
 }
 
 // mark: a CTA takes a segment of QSEG consecutive queries of one head (a contiguous run of
@@ -239,10 +295,13 @@ __global__ void setup_level0_kernel(HeadState* st, int BH) {
 // then writes mask words, per-(segment, block) counts and the segment's pair total.
 __global__ void __launch_bounds__(kSegThreads)
 mark_kernel(const float* __restrict__ scores, const HeadState* __restrict__ st, int S, int Nb, int mw, int QSEG,
-            int nseg, uint32_t* __restrict__ mask_bits, int* __restrict__ seg_cnt, int* __restrict__ seg_total) {
+            int nseg, uint32_t* __restrict__ mask_bits, int* __restrict__ seg_cnt, int* __restrict__ seg_total,
+            uint32_t* __restrict__ tmask) {
   extern __shared__ uint32_t sm[];
+  const int TW = QSEG >> 5;                           // words of a block's column over the segment's queries
   uint32_t* s_mask = sm;                              // [QSEG][mw]
   int* s_cnt = reinterpret_cast<int*>(sm + QSEG * mw);  // [Nb]
+  uint32_t* s_tm = sm + QSEG * mw + Nb;               // [Nb][TW]: the same bits, one row per key block
   __shared__ int s_total;
   const int seg = blockIdx.x, bh = blockIdx.y;
   const int q0 = seg * QSEG;
@@ -250,6 +309,7 @@ mark_kernel(const float* __restrict__ scores, const HeadState* __restrict__ st, 
   const uint32_t cutoff = st[bh].cutoff_key;
   for (int i = threadIdx.x; i < QSEG * mw; i += blockDim.x) s_mask[i] = 0u;
   for (int i = threadIdx.x; i < Nb; i += blockDim.x) s_cnt[i] = 0;
+  for (int i = threadIdx.x; i < Nb * TW; i += blockDim.x) s_tm[i] = 0u;
   if (threadIdx.x == 0) s_total = 0;
   __syncthreads();
   const float* base = scores + ((long long)bh * S + q0) * Nb;
@@ -259,13 +319,26 @@ mark_kernel(const float* __restrict__ scores, const HeadState* __restrict__ st, 
       int ii = (int)i;
       int ql = ii / Nb, j = ii - ql * Nb;
       atomicOr(&s_mask[ql * mw + (j >> 5)], 1u << (j & 31));
+      atomicOr(&s_tm[j * TW + (ql >> 5)], 1u << (ql & 31));
       atomicAdd(&s_cnt[j], 1);
     }
   };
   if ((reinterpret_cast<uintptr_t>(base) & 15u) == 0) {
     const float4* b4 = reinterpret_cast<const float4*>(base);
     long long n4 = n >> 2;
-    for (long long i = threadIdx.x; i < n4; i += blockDim.x) {
+    // four independent 16-byte loads per thread in flight
+    long long i = threadIdx.x;
+    for (; i + 3 * (long long)blockDim.x < n4; i += 4 * (long long)blockDim.x) {
+      float4 x[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) x[j] = __ldg(b4 + i + j * (long long)blockDim.x);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const long long e = 4 * (i + j * (long long)blockDim.x);
+        mark(e, x[j].x); mark(e + 1, x[j].y); mark(e + 2, x[j].z); mark(e + 3, x[j].w);
+      }
+    }
+    for (; i < n4; i += blockDim.x) {
       float4 x = __ldg(b4 + i);
       mark(4 * i, x.x); mark(4 * i + 1, x.y); mark(4 * i + 2, x.z); mark(4 * i + 3, x.w);
     }
@@ -285,6 +358,8 @@ mark_kernel(const float* __restrict__ scores, const HeadState* __restrict__ st, 
   if ((threadIdx.x & 31) == 0 && local) atomicAdd(&s_total, local);
   int* sc = seg_cnt + ((long long)bh * nseg + seg) * Nb;
   for (int i = threadIdx.x; i < Nb; i += blockDim.x) sc[i] = s_cnt[i];
+  uint32_t* tm = tmask + ((long long)bh * nseg + seg) * Nb * TW;
+  for (int i = threadIdx.x; i < Nb * TW; i += blockDim.x) tm[i] = s_tm[i];
   __syncthreads();
   if (threadIdx.x == 0) seg_total[bh * nseg + seg] = s_total;
 }
@@ -325,12 +400,13 @@ offsets_kernel(const int* __restrict__ kb_total, int* __restrict__ kb_ptr, long 
   }
 }
 
-// fill: a CTA re-reads its segment's mask words, derives q_ptr for its queries and, one warp
-// per key block, ranks the selecting queries in ascending order to place them in q_idx; the
-// same position is recorded in the query-major list q_pairs.
+// fill: a CTA re-reads its segment's mask words and derives q_ptr for its queries; then, one warp
+// per key block, the block's column of the segment (a few words written by the mark kernel) gives
+// the selecting queries in ascending order without touching the unset bits: each is placed in
+// q_idx, and the same position is recorded in the query-major list q_pairs.
 __global__ void __launch_bounds__(kSegThreads)
-fill_kernel(const uint32_t* __restrict__ mask_bits, int S, int Nb, int mw, int QSEG, int nseg,
-            const int* __restrict__ kb_ptr, const int* __restrict__ seg_cnt, const int* __restrict__ seg_qoff,
+fill_kernel(const uint32_t* __restrict__ mask_bits, const uint32_t* __restrict__ tmask, int S, int Nb, int mw, int QSEG,
+            int nseg, const int* __restrict__ kb_ptr, const int* __restrict__ seg_cnt, const int* __restrict__ seg_qoff,
             int* __restrict__ q_idx, int* __restrict__ q_ptr, int* __restrict__ q_pairs, long long capacity) {
   extern __shared__ uint32_t sm[];
   uint32_t* s_mask = sm;                                   // [QSEG][mw]
@@ -339,6 +415,7 @@ fill_kernel(const uint32_t* __restrict__ mask_bits, int S, int Nb, int mw, int Q
   const int seg = blockIdx.x, bh = blockIdx.y;
   const int q0 = seg * QSEG;
   const int nq = min(QSEG, S - q0);
+  const int TW = QSEG >> 5;
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5, nwarps = blockDim.x >> 5;
   const uint32_t* gm = mask_bits + ((long long)bh * S + q0) * mw;
   for (int i = t; i < QSEG * mw; i += blockDim.x) s_mask[i] = i < nq * mw ? gm[i] : 0u;
@@ -374,27 +451,33 @@ fill_kernel(const uint32_t* __restrict__ mask_bits, int S, int Nb, int mw, int Q
   }
   __syncthreads();
   const int* sc = seg_cnt + ((long long)bh * nseg + seg) * Nb;
+  const uint32_t* tm = tmask + ((long long)bh * nseg + seg) * Nb * TW;
   for (int j = warp; j < Nb; j += nwarps) {
-    long long base = (long long)kb_ptr[(long long)bh * Nb + j] + sc[j];
+    // lane l holds the block's bits of queries 32 l .. 32 l + 31 of the segment (TW <= 16 words)
+    uint32_t word = lane < TW ? tm[j * TW + lane] : 0u;
+    int before = __popc(word);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int x = __shfl_up_sync(0xffffffffu, before, o);
+      if (lane >= o) before += x;
+    }
+    before -= __popc(word);                                 // selecting queries in the lower words
+    const long long base = (long long)kb_ptr[(long long)bh * Nb + j] + sc[j];
     const int wj = j >> 5;
     const uint32_t bit = 1u << (j & 31);
-    int run = 0;
-    for (int qs = 0; qs < nq; qs += 32) {
-      int ql = qs + lane;
-      uint32_t word = ql < nq ? s_mask[ql * mw + wj] : 0u;
-      bool sel = (word & bit) != 0;
-      unsigned ball = __ballot_sync(0xffffffffu, sel);
-      if (sel) {
-        long long pos = base + run + __popc(ball & ((1u << lane) - 1u));
-        if (pos < capacity) {
-          q_idx[pos] = q0 + ql;
-          int within = __popc(word & (bit - 1u));
-          for (int w = 0; w < wj; ++w) within += __popc(s_mask[ql * mw + w]);
-          long long qp = (long long)qbase + s_qoff[ql] + within;
-          if (qp < capacity) q_pairs[qp] = (int)pos;
-        }
+    while (word) {
+      const int b = __ffs(word) - 1;
+      word &= word - 1;
+      const int ql = 32 * lane + b;
+      const long long pos = base + before;
+      ++before;
+      if (pos < capacity) {
+        q_idx[pos] = q0 + ql;
+        int within = __popc(s_mask[ql * mw + wj] & (bit - 1u));
+        for (int w = 0; w < wj; ++w) within += __popc(s_mask[ql * mw + w]);
+        const long long qp = (long long)qbase + s_qoff[ql] + within;
+        if (qp < capacity) q_pairs[qp] = (int)pos;
       }
-      run += __popc(ball);
     }
   }
 }
@@ -412,6 +495,8 @@ struct SelectWs {
   unsigned int* g_cnt;
   double* g_w;
   uint32_t* g_minkey;
+  uint32_t* g_maxkey;
+  uint32_t* tmask;
   int* seg_cnt;
   int* seg_total;
   int* seg_qoff;
@@ -428,6 +513,8 @@ static SelectWs carve_select(const Dims& D, void* ws) {
   w.g_cnt = c.take<unsigned int>((size_t)D.BH * kBins);
   w.g_w = c.take<double>((size_t)D.BH * kBins);
   w.g_minkey = c.take<uint32_t>((size_t)D.BH * kBins);
+  w.g_maxkey = c.take<uint32_t>((size_t)D.BH * kBins);
+  w.tmask = c.take<uint32_t>((size_t)D.BH * nseg * D.Nb * (QSEG >> 5));
   w.seg_cnt = c.take<int>((size_t)D.BH * nseg * D.Nb);
   w.seg_total = c.take<int>((size_t)D.BH * nseg);
   w.seg_qoff = c.take<int>((size_t)D.BH * nseg + 1);
@@ -467,6 +554,7 @@ extern "C" int vmoba_select(const vmoba_shape* shape, const float* scores, float
   VMOBA_CUDA_OK(cudaMemsetAsync(w.g_cnt, 0, (size_t)D.BH * kBins * sizeof(unsigned int), st));
   VMOBA_CUDA_OK(cudaMemsetAsync(w.g_w, 0, (size_t)D.BH * kBins * sizeof(double), st));
   VMOBA_CUDA_OK(cudaMemsetAsync(w.g_minkey, 0xff, (size_t)D.BH * kBins * sizeof(uint32_t), st));
+  VMOBA_CUDA_OK(cudaMemsetAsync(w.g_maxkey, 0, (size_t)D.BH * kBins * sizeof(uint32_t), st));
 
   // enough CTAs per head to fill the machine, few enough that the per-CTA flush stays small
   long long per_head = (P / 4 + 255) / 256;
@@ -474,25 +562,31 @@ extern "C" int vmoba_select(const vmoba_shape* shape, const float* scores, float
   dim3 grid(gx, D.BH);
   minmax_kernel<<<grid, 256, 0, st>>>(scores, P, w.state);
   setup_level0_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH);
-  hist_kernel<0><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey);
-  scan_kernel<0><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, k_per_head, cutoff_per_head);
-  hist_kernel<1><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey);
-  scan_kernel<1><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, k_per_head, cutoff_per_head);
-  hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey);
-  scan_kernel<2><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, k_per_head, cutoff_per_head);
+  {
+    constexpr int smem0 = kBins0 * kRep * (int)sizeof(float);
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(hist0_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem0));
+    // three 512-thread CTAs per SM hold their replicated bins side by side
+    int gx0 = (int)std::min<long long>(std::max<long long>(per_head / 16, 1), std::max(1, 148 * 3 / D.BH));
+    hist0_kernel<<<dim3(gx0, D.BH), 512, smem0, st>>>(scores, P, w.state, D.scale, w.g_w);
+  }
+  scan_kernel<0><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head, cutoff_per_head);
+  hist_kernel<1><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
+  scan_kernel<1><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head, cutoff_per_head);
+  hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
+  scan_kernel<2><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head, cutoff_per_head);
   VMOBA_LAUNCH_OK(9);
 
-  size_t smem = (size_t)QSEG * D.mask_words * 4 + (size_t)std::max(D.Nb, QSEG) * 4;
+  size_t smem = (size_t)QSEG * D.mask_words * 4 + (size_t)std::max(D.Nb, QSEG) * 4 + (size_t)D.Nb * (QSEG >> 5) * 4;
   VMOBA_CUDA_OK(cudaFuncSetAttribute(mark_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   VMOBA_CUDA_OK(cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 sgrid(nseg, D.BH);
   mark_kernel<<<sgrid, kSegThreads, smem, st>>>(scores, w.state, D.S, D.Nb, D.mask_words, QSEG, nseg, mask_bits,
-                                                w.seg_cnt, w.seg_total);
+                                                w.seg_cnt, w.seg_total, w.tmask);
   long long nkb = (long long)D.BH * D.Nb;
   seg_prefix_kernel<<<(unsigned)((nkb + 255) / 256), 256, 0, st>>>(w.seg_cnt, w.kb_total, D.BH, D.Nb, nseg);
   offsets_kernel<<<1, 1024, 0, st>>>(w.kb_total, kb_ptr, nkb, w.seg_total, w.seg_qoff, (long long)D.BH * nseg,
                                      D.BH, D.Nb, k_per_head, capacity, q_ptr + (long long)D.BH * D.S, dev_status);
-  fill_kernel<<<sgrid, kSegThreads, smem, st>>>(mask_bits, D.S, D.Nb, D.mask_words, QSEG, nseg, kb_ptr, w.seg_cnt,
+  fill_kernel<<<sgrid, kSegThreads, smem, st>>>(mask_bits, w.tmask, D.S, D.Nb, D.mask_words, QSEG, nseg, kb_ptr, w.seg_cnt,
                                                 w.seg_qoff, q_idx, q_ptr, q_pairs, capacity);
   VMOBA_LAUNCH_OK(4);
   return VMOBA_OK;
