@@ -217,26 +217,58 @@ merge_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pairs, lon
     for (int c = 0; c < C; ++c) acc[c] = 0.f;
     float out_lse = -INFINITY;
     if (n > 0) {
+      // lane i of each group of 32 pairs fetches the position and lse of pair i once; the row
+      // weights then travel by shuffle.  A truncated list (capacity exceeded) may hold unwritten
+      // entries: keep every index in range.
       float mx = -INFINITY;
-      // a truncated list (capacity exceeded) may hold unwritten entries: keep every index in range
-      auto pair_pos = [&](long long i) { return (long long)min(max(q_pairs[i], 0), (int)(capacity - 1)); };
-      for (long long i = lo; i < hi; ++i) mx = fmaxf(mx, part_lse[pair_pos(i)]);
-      float tot = 0.f;
-      for (long long i = lo; i < hi; ++i) tot += expf(part_lse[pair_pos(i)] - mx);
-      const float inv = 1.0f / tot;
-      for (long long i = lo; i < hi; ++i) {
-        const long long pos = pair_pos(i);
-        const float wgt = expf(part_lse[pos] - mx) * inv;
-#pragma unroll
-        for (int c = 0; c < C; ++c) acc[c] = fmaf(wgt, to_f32<PT>(part_o[pos * DH + lane * C + c]), acc[c]);
+      for (long long i0 = lo; i0 < hi; i0 += 32) {
+        const long long i = i0 + lane;
+        const float l = i < hi ? part_lse[min(max(q_pairs[i], 0), (int)(capacity - 1))] : -INFINITY;
+        mx = fmaxf(mx, l);
       }
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+      float tot = 0.f;
+      for (long long i0 = lo; i0 < hi; i0 += 32) {
+        const long long i = i0 + lane;
+        int my_pos = 0;
+        float my_w = 0.f;
+        if (i < hi) {
+          my_pos = min(max(q_pairs[i], 0), (int)(capacity - 1));
+          my_w = expf(part_lse[my_pos] - mx);
+        }
+        tot += my_w;
+        const int m = (int)min((long long)32, hi - i0);
+        for (int k = 0; k < m; ++k) {
+          const long long pos = __shfl_sync(0xffffffffu, my_pos, k);
+          const float wgt = __shfl_sync(0xffffffffu, my_w, k);
+          if constexpr (C == 4 && sizeof(PT) == 4) {
+            const float4 v = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(part_o) + pos * DH + lane * 4);
+            acc[0] = fmaf(wgt, v.x, acc[0]); acc[1] = fmaf(wgt, v.y, acc[1]);
+            acc[2] = fmaf(wgt, v.z, acc[2]); acc[3] = fmaf(wgt, v.w, acc[3]);
+          } else {
+#pragma unroll
+            for (int c = 0; c < C; ++c) acc[c] = fmaf(wgt, to_f32<PT>(part_o[pos * DH + lane * C + c]), acc[c]);
+          }
+        }
+      }
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, s);
+      const float inv = 1.0f / tot;
+#pragma unroll
+      for (int c = 0; c < C; ++c) acc[c] *= inv;
       out_lse = mx + logf(tot);
     }
+    if constexpr (C == 4) {
+      store4_resid(o + g * DH + lane * 4, o_resid ? o_resid + g * DH + lane * 4 : nullptr,
+                   make_float4(acc[0], acc[1], acc[2], acc[3]));
+    } else {
 #pragma unroll
-    for (int c = 0; c < C; ++c) {
-      const T hi = from_f32<T>(acc[c]);
-      o[g * DH + lane * C + c] = hi;
-      if (o_resid) o_resid[g * DH + lane * C + c] = from_f32<T>(acc[c] - to_f32<T>(hi));
+      for (int c = 0; c < C; ++c) {
+        const T hi_ = from_f32<T>(acc[c]);
+        o[g * DH + lane * C + c] = hi_;
+        if (o_resid) o_resid[g * DH + lane * C + c] = from_f32<T>(acc[c] - to_f32<T>(hi_));
+      }
     }
     if (lane == 0) lse[g] = out_lse;
   }
@@ -464,8 +496,13 @@ cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, const int* 
   for (long long g = warp; g < n_queries; g += nwarps) {
     const int nb = sparse_rows ? q_ptr[g + 1] - q_ptr[g] : 2;
     if (nb > 0 && nb < min_nb) continue;   // written directly by the attention kernel
+    if constexpr (C == 4) {
+      const float4 v = nb == 0 ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(src + g * DH + lane * 4);
+      store4(dst + g * DH + lane * 4, v);
+    } else {
 #pragma unroll
-    for (int c = 0; c < C; ++c) dst[g * DH + lane * C + c] = from_f32<T>(nb == 0 ? 0.f : src[g * DH + lane * C + c]);
+      for (int c = 0; c < C; ++c) dst[g * DH + lane * C + c] = from_f32<T>(nb == 0 ? 0.f : src[g * DH + lane * C + c]);
+    }
   }
 }
 
