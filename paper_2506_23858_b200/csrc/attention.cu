@@ -10,7 +10,7 @@ namespace vmoba {
 size_t select_ws_bytes(const Dims& D);   // select.cu
 size_t scores_ws_bytes(const Dims& D);   // scores.cu
 
-// attn_tc.cu: tensor-core forward kernels (bf16, head_dim 128)
+// attn_tc_fwd.cu: tensor-core forward kernel (bf16, head_dim 128)
 int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                   const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
                   int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o, float* part_lse,

@@ -1,5 +1,8 @@
-// Tensor-core attention forward for long key ranges (bf16, head_dim 128): 256 query rows per item.
+// Tensor-core attention forward for bf16, head_dim 128 (Step 3 of VMoBA and its dense limit).
 //
+// One persistent CTA per SM walks the work items.  An item is up to 256 query rows (sparse: a chunk of
+// the queries that selected key block j, gathered by index; dense: 256 consecutive rows) against a
+// contiguous key range (the block, or the whole sequence), streamed in tiles of 128 keys.
 // With 128 query rows per CTA every 128-key tile of K and V (64 KB) feeds only 1024 tensor-pipe
 // cycles, and the L2-to-SM path, not the tensor pipe, sets the pace.  Here a CTA owns TWO 128-row
 // query tiles (A and B) that share each K/V tile, which halves the bytes per MMA, and the two
@@ -480,8 +483,9 @@ static int grid_items(long long items) { return (int)std::max<long long>(1, std:
 
 }  // namespace tcw
 
-// Forward over the work lists with 256-row items (bf16, head_dim 128).
-int tc_sparse_fwd_wide(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
+// Forward over the work lists (bf16, head_dim 128).  Returns VMOBA_ERR_CUDA if the tensor maps or
+// the launch fail.
+int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                        const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
                        int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o,
                        float* part_lse, cudaStream_t st) {
@@ -511,7 +515,7 @@ int tc_sparse_fwd_wide(const Dims& D, const void* q, const void* k, const void* 
   return VMOBA_OK;
 }
 
-int tc_dense_fwd_wide(const Dims& D, const void* q, const void* k, const void* v, void* o, void* o_resid, float* lse,
+int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, void* o, void* o_resid, float* lse,
                       int32_t* status, cudaStream_t st) {
   using namespace tcw;
   CUtensorMap tmK, tmV;
