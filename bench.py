@@ -413,10 +413,14 @@ def main():
             stages[s] = {"ms": ms, "bound": "tensor", "achieved": ach, "unit": "TFLOP/s",
                          "frac": ach / pk["tensor_sustained"]}
     dom = max(stage_names, key=lambda s: stage_ms[s])
+    # DRAM bytes per launch of the stage's main kernel, from the committed ncu capture of this workload
     traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        traffic = json.load(open(tpath)).get(args.workload, {}).get(dom)
+    tpath = os.path.join(ROOT, "profiles", f"traffic_bench_{args.workload}.txt")
+    if os.path.exists(tpath) and args.heads <= 0:
+        for line in open(tpath):
+            f = line.split()
+            if len(f) == 2 and f[0] == dom:
+                traffic = int(f[1])
     roofline = {"kernel": dom, "bound": stages[dom]["bound"], "achieved": stages[dom]["achieved"],
                 "peak": pk["hbm"] if stages[dom]["bound"] == "hbm" else pk["tensor_sustained"],
                 "unit": stages[dom]["unit"], "frac": stages[dom]["frac"], "traffic": traffic,
