@@ -160,6 +160,54 @@ def select_topk_per_query(scores, k):
     return mask
 
 
+def select_threshold_per_query(scores, tau, sigma):
+    """"threshold + local" of the block-choice ablation (Table 3b): the cumulative-similarity rule of
+    Eq. 4 applied to each query on its own instead of to the head-wide pool.
+
+    For query i: p_ij = softmax_j(sigma * S_hat_ij) over its N_b blocks (fp64), blocks ordered by
+    S_hat descending (ties: lower block index first), k_i = min{m : sum of the first m p >= tau}
+    (tau >= 1 or never reached -> N_b); the first k_i blocks are kept.  Every query keeps at least
+    one block.  Returns (mask [s, N_b] bool, k [s] int).
+    """
+    if not (tau > 0.0):
+        raise ValueError("tau must be in (0, 1]")
+    s, n_b = scores.shape
+    mask = np.zeros((s, n_b), dtype=bool)
+    ks = np.zeros(s, dtype=np.int64)
+    for i in range(s):
+        row = scores[i].astype(np.float64)
+        order = np.argsort(-row, kind="stable")
+        if tau >= 1.0:
+            k = n_b
+        else:
+            x = sigma * row
+            w = np.exp(x - x.max())
+            p = w / w.sum()
+            c = np.cumsum(p[order])
+            hit = np.nonzero(c >= tau)[0]
+            k = int(hit[0]) + 1 if hit.size else n_b
+        mask[i, order[:k]] = True
+        ks[i] = k
+    return mask, ks
+
+
+def select_topk_global(scores, k):
+    """"topk + global" of the block-choice ablation (Table 3b): the head-wide pool of Eq. 3 with a
+    fixed budget instead of the threshold of Eq. 4.  The budget is the one "topk + local" spends,
+    K = k * s pairs per head (capped at the pool size); the K best pairs of the head are kept
+    (ties: ascending flat index).  Returns (mask [s, N_b] bool, K, cutoff = fp32 score of the K-th pair).
+    """
+    if k < 1:
+        raise ValueError("k must be positive")
+    s, n_b = scores.shape
+    flat = scores.reshape(-1)
+    K = min(k * s, flat.size)
+    order = np.argsort(-flat.astype(np.float64), kind="stable")
+    mask = np.zeros(flat.size, dtype=bool)
+    mask[order[:K]] = True
+    return mask.reshape(s, n_b), K, np.float32(flat[order[K - 1]])
+
+
 # --------------------------------------------------------------------------------------
 # Step 3: attention over the selected blocks (Section 3.1, Step 3) and its gradient
 # --------------------------------------------------------------------------------------

@@ -280,6 +280,61 @@ def test_select_topk_per_query():
     assert orc.select_topk_per_query(sc, 9).all()
 
 
+def test_select_threshold_per_query_hand_case():
+    # one row, sigma = 1: weights e^0, e^-1, e^-2, e^-3 -> probabilities 0.6439, 0.2369, 0.0871, 0.0321
+    sc = np.array([[3.0, 2.0, 0.0, 1.0]], dtype=np.float32)
+    for tau, want in [(0.5, [1, 0, 0, 0]), (0.6439, [1, 0, 0, 0]), (0.65, [1, 1, 0, 0]), (0.88, [1, 1, 0, 0]),
+                      (0.89, [1, 1, 0, 1]), (0.97, [1, 1, 1, 1]), (1.0, [1, 1, 1, 1])]:
+        m, k = orc.select_threshold_per_query(sc, tau, 1.0)
+        assert m[0].astype(int).tolist() == want, tau
+        assert k[0] == sum(want)
+
+
+def test_select_threshold_per_query_is_the_global_rule_on_one_row():
+    # with a single query the head-wide pool IS the row: both rules must agree
+    rng = np.random.default_rng(5)
+    for _ in range(20):
+        sc = rng.normal(size=(1, 37)).astype(np.float32) * 3
+        tau = float(rng.uniform(0.05, 0.95))
+        m_row, k_row = orc.select_threshold_per_query(sc, tau, 0.7)
+        m_pool, k_pool, _ = orc.select(sc, tau, 0.7)
+        assert (m_row == m_pool).all() and k_row[0] == k_pool
+
+
+def test_select_threshold_per_query_rows_are_independent_and_never_empty():
+    rng = np.random.default_rng(6)
+    sc = rng.normal(size=(9, 12)).astype(np.float32)
+    m, k = orc.select_threshold_per_query(sc, 0.3, 2.0)
+    assert (m.sum(1) == k).all() and (k >= 1).all()
+    for i in range(9):
+        mi, _ = orc.select_threshold_per_query(sc[i:i + 1], 0.3, 2.0)
+        assert (mi[0] == m[i]).all()
+    # ties: equal scores are taken in block order
+    m, k = orc.select_threshold_per_query(np.zeros((1, 4), np.float32), 0.5, 1.0)
+    assert m[0].tolist() == [True, True, False, False]
+    with pytest.raises(ValueError):
+        orc.select_threshold_per_query(sc, 0.0, 1.0)
+
+
+def test_select_topk_global():
+    sc = np.array([[1, 5, 3, 3], [0, 0, 0, 0], [9, 8, 7, 6]], dtype=np.float32)
+    m, K, cut = orc.select_topk_global(sc, 2)          # budget 6 of 12: 9 8 7 6 5 and the first 3
+    assert K == 6 and cut == 3.0
+    assert m.astype(int).tolist() == [[0, 1, 1, 0], [0, 0, 0, 0], [1, 1, 1, 1]]
+    # one query: the pool is the row, so the rule is the per-query one
+    rng = np.random.default_rng(7)
+    row = rng.normal(size=(1, 23)).astype(np.float32)
+    assert (orc.select_topk_global(row, 5)[0] == orc.select_topk_per_query(row, 5)).all()
+    # the budget is capped by the pool
+    assert orc.select_topk_global(sc, 99)[0].all()
+    # brute force: exactly the K largest values
+    sc = rng.normal(size=(6, 7)).astype(np.float32)
+    m, K, cut = orc.select_topk_global(sc, 3)
+    assert m.sum() == K == 18 and sc[m].min() >= sc[~m].max() and cut == sc[m].min()
+    with pytest.raises(ValueError):
+        orc.select_topk_global(sc, 0)
+
+
 # ---------------------------------------------------------------- attention forward
 def _rand_head(s, d, seed):
     rng = np.random.default_rng(seed)
