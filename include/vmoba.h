@@ -130,6 +130,34 @@ int vmoba_select(const vmoba_shape* shape, const float* scores, float tau, uint3
                  int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The block-choice variants of Table 3b ("Block choice design ablation") and of the training-free
+ * setting of Table 4 / Appendix A ("Local + TopK"): the same outputs as vmoba_select, chosen by
+ *   VMOBA_SELECT_THRESHOLD_GLOBAL  the method's own rule; identical to vmoba_select(tau)
+ *   VMOBA_SELECT_TOPK_GLOBAL       head-wide pool of Eq. 3, fixed budget: the K = min(topk * S, S * N_b)
+ *                                  best pairs of the head (every pair tied with the K-th is kept)
+ *   VMOBA_SELECT_THRESHOLD_LOCAL   Eq. 4 applied to each query on its own: softmax of its N_b scores at
+ *                                  temperature softmax_scale, blocks in descending order until the
+ *                                  cumulative mass is >= tau; ties in block order; never an empty row
+ *   VMOBA_SELECT_TOPK_LOCAL        each query keeps its min(topk, N_b) best blocks (the MoBA rule);
+ *                                  ties in block order; exactly that many per query
+ * tau in (0, 1] is read by the threshold modes, topk >= 1 by the top-k modes.  The local modes need
+ * N_b <= 1024 (VMOBA_ERR_SHAPE otherwise).  cutoff_per_head receives the score of the last pair taken
+ * (global modes) or the smallest score selected in the head (local modes).  Workspace:
+ * vmoba_workspace_bytes(shape, VMOBA_STAGE_SELECT, 0), as for vmoba_select.
+ */
+typedef enum {
+  VMOBA_SELECT_THRESHOLD_GLOBAL = 0,
+  VMOBA_SELECT_TOPK_GLOBAL = 1,
+  VMOBA_SELECT_THRESHOLD_LOCAL = 2,
+  VMOBA_SELECT_TOPK_LOCAL = 3
+} vmoba_select_rule;
+
+int vmoba_select_rule_apply(const vmoba_shape* shape, const float* scores, int32_t rule, float tau, int32_t topk,
+                            uint32_t* mask_bits, int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr,
+                            int32_t* q_pairs, int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
+                            int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * vmoba_select for callers that cannot hand over scratch memory.  (The paper has no counterpart:
  * this is a packaging variant of the selection stage, not a step of the method.)
  *

@@ -95,6 +95,9 @@ def lib():
     L.vmoba_select.restype = ctypes.c_int
     L.vmoba_select.argtypes = [sp, vp, ctypes.c_float, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp]
     L.vmoba_select_static.restype = ctypes.c_int
+    L.vmoba_select_rule_apply.restype = ctypes.c_int
+    L.vmoba_select_rule_apply.argtypes = [sp, vp, ctypes.c_int32, ctypes.c_float, ctypes.c_int32, vp, vp, vp, vp, vp, i64, vp, vp, vp,
+                                          vp, sz, vp]
     L.vmoba_select_static.argtypes = [sp, vp, ctypes.c_float, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp]
     L.vmoba_select_static_scratch_bytes.restype = sz
     L.vmoba_select_static_scratch_bytes.argtypes = []
@@ -159,6 +162,19 @@ def vmoba_select(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, c
     _check(lib().vmoba_select(ctypes.byref(shape), _ptr(scores), float(tau), _ptr(mask_bits), _ptr(kb_ptr),
                               _ptr(q_idx), _ptr(q_ptr), _ptr(q_pairs), int(capacity), _ptr(k_per_head),
                               _ptr(cutoff_per_head), _ptr(dev_status), p, n, _stream(stream)), "vmoba_select")
+
+
+SELECT_THRESHOLD_GLOBAL, SELECT_TOPK_GLOBAL, SELECT_THRESHOLD_LOCAL, SELECT_TOPK_LOCAL = 0, 1, 2, 3
+
+
+def vmoba_select_rule_apply(shape, scores, rule, tau, topk, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity,
+                            k_per_head, cutoff_per_head, dev_status, ws, stream=None):
+    """vmoba_select with one of the four block-choice rules (threshold / top-k, head-wide / per query)."""
+    p, n = _ws_args(ws)
+    _check(lib().vmoba_select_rule_apply(ctypes.byref(shape), _ptr(scores), int(rule), float(tau), int(topk),
+                                         _ptr(mask_bits), _ptr(kb_ptr), _ptr(q_idx), _ptr(q_ptr), _ptr(q_pairs),
+                                         int(capacity), _ptr(k_per_head), _ptr(cutoff_per_head), _ptr(dev_status), p, n,
+                                         _stream(stream)), "vmoba_select_rule_apply")
 
 
 def vmoba_select_static(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity, k_per_head,

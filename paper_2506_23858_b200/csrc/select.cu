@@ -14,6 +14,7 @@
 //   offsets : CSR offsets by key block (kb_ptr) and by query (q_ptr)
 //   fill    : q_idx (queries of each key block, ascending) and q_pairs (pairs of each query)
 #include <algorithm>
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -94,6 +95,7 @@ __global__ void init_state_kernel(HeadState* st, int BH) {
   memset(&h, 0, sizeof(h));
   h.min_key = 0xffffffffu;
   h.max_key = 0u;
+  h.cutoff_key = 0xffffffffu;      // the per-query rules take the minimum of their row cutoffs into it
   st[i] = h;
 }
 
@@ -103,7 +105,7 @@ __global__ void init_state_kernel(HeadState* st, int BH) {
 // a crossing bin with a single distinct score ends the search there.
 template <int L>
 __global__ void __launch_bounds__(256)
-hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __restrict__ st, float sigma,
+hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __restrict__ st, float sigma, int unit_w,
             unsigned int* __restrict__ g_cnt, double* __restrict__ g_w, uint32_t* __restrict__ g_minkey,
             uint32_t* __restrict__ g_maxkey) {
   __shared__ unsigned int s_cnt[kBins];
@@ -125,7 +127,7 @@ hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __re
     if (L >= 2 && bin_at(hs, 1, s) != hs.bin[1]) return;
     int b = bin_at(hs, L, s);
     atomicAdd(&s_cnt[b], 1u);
-    atomicAdd(&s_w[b], expf(sigma * (s - smax)));
+    atomicAdd(&s_w[b], unit_w ? 1.0f : expf(sigma * (s - smax)));
     atomicMin(&s_min[b], float_key(s));
     if (L == 1) atomicMax(&s_max[b], float_key(s));
   });
@@ -147,7 +149,7 @@ hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __re
 // masses are kept: the scan needs no counts at this level.
 constexpr int kRep = 32;
 __global__ void __launch_bounds__(512)
-hist0_kernel(const float* __restrict__ scores, long long P, const HeadState* __restrict__ st, float sigma,
+hist0_kernel(const float* __restrict__ scores, long long P, const HeadState* __restrict__ st, float sigma, int unit_w,
              double* __restrict__ g_w) {
   extern __shared__ float s_wr[];   // [kBins0][kRep]
   const int bh = blockIdx.y;
@@ -157,7 +159,7 @@ hist0_kernel(const float* __restrict__ scores, long long P, const HeadState* __r
   const float smax = key_float(hs.max_key);
   const int rep = threadIdx.x & (kRep - 1);
   for_each_score(scores + (long long)bh * P, P, [&](float s) {
-    atomicAdd(&s_wr[bin_at(hs, 0, s) * kRep + rep], expf(sigma * (s - smax)));
+    atomicAdd(&s_wr[bin_at(hs, 0, s) * kRep + rep], unit_w ? 1.0f : expf(sigma * (s - smax)));
   });
   __syncthreads();
   for (int i = threadIdx.x; i < kBins0; i += blockDim.x) {
@@ -172,7 +174,8 @@ hist0_kernel(const float* __restrict__ scores, long long P, const HeadState* __r
 // which the cumulative mass first reaches the target, record it and clear the histogram.
 template <int L>
 __global__ void __launch_bounds__(1024)
-scan_kernel(HeadState* __restrict__ st, float tau, unsigned int* __restrict__ g_cnt, double* __restrict__ g_w,
+scan_kernel(HeadState* __restrict__ st, float tau, double count_target, unsigned int* __restrict__ g_cnt,
+            double* __restrict__ g_w,
             uint32_t* __restrict__ g_minkey, uint32_t* __restrict__ g_maxkey, int64_t* __restrict__ k_per_head,
             float* __restrict__ cutoff_per_head) {
   __shared__ double s_wsum[32];
@@ -228,7 +231,12 @@ scan_kernel(HeadState* __restrict__ st, float tau, unsigned int* __restrict__ g_
   __shared__ double s_total;
   if (t == 1023) s_total = w_excl + wl;
   __syncthreads();
-  if (L == 0) { hs.Z = s_total; hs.target = (double)tau * s_total; hs.mass_above = 0.0; hs.cnt_above = 0ull; }
+  // unit weights (count_target >= 0): the masses are pair counts and the target is the budget itself
+  if (L == 0) {
+    hs.Z = s_total;
+    hs.target = count_target >= 0.0 ? count_target : (double)tau * s_total;
+    hs.mass_above = 0.0; hs.cnt_above = 0ull;
+  }
   const double need = hs.target - hs.mass_above;    // mass still to be covered inside this level
   // crossing element: first e with inclusive mass >= need (and a non-empty bin)
   int my_cross = -1;
@@ -482,6 +490,197 @@ fill_kernel(const uint32_t* __restrict__ mask_bits, const uint32_t* __restrict__
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Per-query ("local") rules: one warp per query row, N_b <= 1024 so that lane l holds the blocks
+// j = l + 32 i as order-preserving keys.  The cutoff of a row is the largest key c with
+// measure{key >= c} >= target, found bit by bit from the top (measure = count for top-k, softmax
+// mass for the threshold rule); blocks above it are taken, blocks tied with it in block order until
+// the target is met.  Block j = l + 32 i is bit l of mask word i: a ballot IS the mask word.
+constexpr int kLocalMaxWords = 32;
+// MW: compile-time bound on the mask words of a row (the loops over a lane's blocks unroll to it)
+template <bool TOPK, int MW>
+__global__ void __launch_bounds__(256)
+select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, float sigma, float tau, int topk,
+                    uint32_t* __restrict__ mask_bits, HeadState* __restrict__ st, long long n_rows) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  for (long long row = warp; row < n_rows; row += nwarps) {
+    const float* sr = scores + row * Nb;
+    uint32_t key[MW];
+    uint32_t kmax = 0u;
+#pragma unroll
+    for (int i = 0; i < MW; ++i) {
+      const int j = lane + 32 * i;
+      key[i] = (i < mw && j < Nb) ? float_key(__ldg(sr + j)) : 0u;     // 0 is below every real score's key
+      kmax = max(kmax, key[i]);
+    }
+    kmax = __reduce_max_sync(0xffffffffu, kmax);
+    double w[TOPK ? 1 : MW];
+    double target;
+    if (TOPK) {
+      target = (double)min(topk, Nb);
+    } else {
+      const float smax = key_float(kmax);
+      double z = 0.0;
+#pragma unroll
+      for (int i = 0; i < MW; ++i) {
+        w[i] = key[i] ? (double)expf(sigma * (key_float(key[i]) - smax)) : 0.0;
+        z += w[i];
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+      target = (double)tau * z;
+    }
+    auto measure_ge = [&](uint32_t c) {
+      if (TOPK) {
+        int n = 0;
+#pragma unroll
+        for (int i = 0; i < MW; ++i) n += (i < mw && key[i] >= c) ? 1 : 0;
+        return (double)__reduce_add_sync(0xffffffffu, n);
+      } else {
+        double m = 0.0;
+#pragma unroll
+        for (int i = 0; i < MW; ++i) m += (i < mw && key[i] >= c) ? w[TOPK ? 0 : i] : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m += __shfl_xor_sync(0xffffffffu, m, o);
+        return m;
+      }
+    };
+    // Short selections (the usual case: a handful of blocks per query) are taken one block at a time,
+    // best first, lowest block index among equals, exactly the order the rule is stated in; the
+    // cumulative mass of the threshold rule is the running sum of the winners' weights.
+    {
+      constexpr int kRounds = 24;
+      const int rounds = TOPK ? ((int)target <= kRounds ? (int)target : 0) : (tau < 1.0f ? min(kRounds, Nb) : 0);
+      uint32_t taken = 0u;              // bit i: this lane's block lane + 32 i is selected
+      uint32_t c_last = 0u;
+      double acc = 0.0;
+      bool done = false;
+      for (int r = 0; r < rounds && !done; ++r) {
+        uint32_t m = 0u;
+#pragma unroll
+        for (int i = 0; i < MW; ++i) m = max(m, ((taken >> i) & 1u) ? 0u : key[i]);
+        m = __reduce_max_sync(0xffffffffu, m);
+        if (m == 0u) { done = true; break; }          // every block of the row is taken
+        int my_j = INT32_MAX;
+#pragma unroll
+        for (int i = MW - 1; i >= 0; --i)
+          if (key[i] == m && !((taken >> i) & 1u)) my_j = lane + 32 * i;
+        const int j_min = __reduce_min_sync(0xffffffffu, my_j);
+        if ((j_min & 31) == lane) taken |= 1u << (j_min >> 5);
+        c_last = m;
+        if (TOPK) {
+          done = r + 1 == rounds;
+        } else {
+          acc += (double)expf(sigma * (key_float(m) - key_float(kmax)));
+          done = acc >= target;
+        }
+      }
+      if (done) {
+        uint32_t my_word = 0u;
+#pragma unroll
+        for (int i = 0; i < MW; ++i) {
+          const uint32_t word = __ballot_sync(0xffffffffu, (taken >> i) & 1u);
+          if (lane == i) my_word = word;
+        }
+        if (lane < mw) mask_bits[row * mw + lane] = my_word;
+        if (lane == 0) atomicMin(&st[row / S].cutoff_key, c_last);
+        continue;
+      }
+    }
+    // General path: bitwise search for the cutoff key.
+    uint32_t c = 0u;
+    if (!TOPK && tau >= 1.0f) {
+      c = 1u;                                  // everything: every real key is >= 1
+    } else {
+      for (int b = 31; b >= 0; --b) {
+        const uint32_t cand = c | (1u << b);
+        if (cand <= kmax && measure_ge(cand) >= target) c = cand;
+      }
+      if (c == 0u) c = 1u;                     // rounding kept the mass below the target: take the row
+    }
+    // what the blocks strictly above the cutoff already cover, and how many of the tied ones are needed
+    const double above = c == 0xffffffffu ? 0.0 : measure_ge(c + 1u);
+    int n_ties = 0;
+    double w_tie = 0.0;
+#pragma unroll
+    for (int i = 0; i < MW; ++i)
+      if (i < mw && key[i] == c) { n_ties += 1; if (!TOPK) w_tie = w[TOPK ? 0 : i]; }
+    n_ties = __reduce_add_sync(0xffffffffu, n_ties);
+    int need;
+    if (TOPK) {
+      need = (int)(target - above);
+    } else {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) w_tie = fmax(w_tie, __shfl_xor_sync(0xffffffffu, w_tie, o));
+      need = (tau >= 1.0f || !(w_tie > 0.0)) ? n_ties : (int)ceil((target - above) / w_tie);
+    }
+    need = max(1, min(need, n_ties));
+    int run = 0;
+    uint32_t my_word = 0u;
+#pragma unroll
+    for (int i = 0; i < MW; ++i) {
+      if (i < mw) {
+        const bool eq = key[i] == c;
+        const uint32_t e = __ballot_sync(0xffffffffu, eq);
+        const bool sel = key[i] > c || (eq && run + __popc(e & lt_mask) < need);
+        const uint32_t word = __ballot_sync(0xffffffffu, sel);
+        if (lane == i) my_word = word;
+        run += __popc(e);
+      }
+    }
+    if (lane < mw) mask_bits[row * mw + lane] = my_word;
+    if (lane == 0) atomicMin(&st[row / S].cutoff_key, c);
+  }
+}
+
+__global__ void local_cutoff_kernel(const HeadState* __restrict__ st, float* __restrict__ cutoff_per_head, int BH) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < BH) cutoff_per_head[i] = key_float(st[i].cutoff_key);
+}
+
+// The mark pass of the local rules: the mask words exist already; a segment's CTA derives the
+// per-block columns, the per-(segment, block) counts and the segment's pair total from them.
+__global__ void __launch_bounds__(kSegThreads)
+mark_from_mask_kernel(const uint32_t* __restrict__ mask_bits, int S, int Nb, int mw, int QSEG, int nseg,
+                      int* __restrict__ seg_cnt, int* __restrict__ seg_total, uint32_t* __restrict__ tmask) {
+  extern __shared__ uint32_t sm[];
+  const int TW = QSEG >> 5;
+  int* s_cnt = reinterpret_cast<int*>(sm);            // [Nb]
+  uint32_t* s_tm = sm + Nb;                           // [Nb][TW]
+  __shared__ int s_total;
+  const int seg = blockIdx.x, bh = blockIdx.y;
+  const int q0 = seg * QSEG;
+  const int nq = min(QSEG, S - q0);
+  for (int i = threadIdx.x; i < Nb; i += blockDim.x) s_cnt[i] = 0;
+  for (int i = threadIdx.x; i < Nb * TW; i += blockDim.x) s_tm[i] = 0u;
+  if (threadIdx.x == 0) s_total = 0;
+  __syncthreads();
+  const uint32_t* gm = mask_bits + ((long long)bh * S + q0) * mw;
+  int local = 0;
+  for (int i = threadIdx.x; i < nq * mw; i += blockDim.x) {
+    uint32_t word = gm[i];
+    const int ql = i / mw, wj = i - ql * mw;
+    local += __popc(word);
+    while (word) {
+      const int j = 32 * wj + __ffs(word) - 1;
+      word &= word - 1;
+      atomicOr(&s_tm[j * TW + (ql >> 5)], 1u << (ql & 31));
+      atomicAdd(&s_cnt[j], 1);
+    }
+  }
+  local = __reduce_add_sync(0xffffffffu, local);
+  if ((threadIdx.x & 31) == 0 && local) atomicAdd(&s_total, local);
+  __syncthreads();
+  int* sc = seg_cnt + ((long long)bh * nseg + seg) * Nb;
+  for (int i = threadIdx.x; i < Nb; i += blockDim.x) sc[i] = s_cnt[i];
+  uint32_t* tm = tmask + ((long long)bh * nseg + seg) * Nb * TW;
+  for (int i = threadIdx.x; i < Nb * TW; i += blockDim.x) tm[i] = s_tm[i];
+  if (threadIdx.x == 0) seg_total[bh * nseg + seg] = s_total;
+}
+
 static int seg_queries(int mw) {
   int q = 4096 / mw;            // keep the shared mask tile <= 16 KB
   q = q / 32 * 32;
@@ -529,67 +728,119 @@ size_t select_ws_bytes(const Dims& D) { return carve_select(D, nullptr).bytes; }
 
 using namespace vmoba;
 
-extern "C" int vmoba_select(const vmoba_shape* shape, const float* scores, float tau, uint32_t* mask_bits,
-                            int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr, int32_t* q_pairs,
-                            int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
-                            int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+static int select_impl(const vmoba_shape* shape, const float* scores, int rule, float tau, int topk, uint32_t* mask_bits,
+                       int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr, int32_t* q_pairs, int64_t capacity,
+                       int64_t* k_per_head, float* cutoff_per_head, int32_t* dev_status, void* ws, size_t ws_bytes,
+                       void* stream) {
   Dims D;
   int rc = make_dims(shape, &D);
   if (rc) return rc;
-  if (!(tau > 0.0f) || tau > 1.0f) return VMOBA_ERR_ARG;
+  const bool by_topk = rule == VMOBA_SELECT_TOPK_GLOBAL || rule == VMOBA_SELECT_TOPK_LOCAL;
+  const bool local = rule == VMOBA_SELECT_THRESHOLD_LOCAL || rule == VMOBA_SELECT_TOPK_LOCAL;
+  if (rule < VMOBA_SELECT_THRESHOLD_GLOBAL || rule > VMOBA_SELECT_TOPK_LOCAL) return VMOBA_ERR_ARG;
+  if (by_topk ? topk < 1 : (!(tau > 0.0f) || tau > 1.0f)) return VMOBA_ERR_ARG;
   if (!scores || !mask_bits || !kb_ptr || !q_idx || !q_ptr || !q_pairs || !k_per_head || !cutoff_per_head ||
       !dev_status || !ws)
     return VMOBA_ERR_ARG;
   if (!aligned16(scores) || !aligned16(ws)) return VMOBA_ERR_ARG;
   if (capacity <= 0 || capacity > (int64_t)INT32_MAX) return VMOBA_ERR_ARG;
-  if (D.Nb > 8192) return VMOBA_ERR_SHAPE;
+  if (D.Nb > 8192 || (local && D.Nb > 32 * kLocalMaxWords)) return VMOBA_ERR_SHAPE;
   SelectWs w = carve_select(D, ws);
   if (ws_bytes < w.bytes) return VMOBA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const long long P = (long long)D.S * D.Nb;
   const int QSEG = seg_queries(D.mask_words);
   const int nseg = (D.S + QSEG - 1) / QSEG;
+  const size_t smem = (size_t)QSEG * D.mask_words * 4 + (size_t)std::max(D.Nb, QSEG) * 4 + (size_t)D.Nb * (QSEG >> 5) * 4;
+  const dim3 sgrid(nseg, D.BH);
 
   init_state_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH);
-  VMOBA_CUDA_OK(cudaMemsetAsync(w.g_cnt, 0, (size_t)D.BH * kBins * sizeof(unsigned int), st));
-  VMOBA_CUDA_OK(cudaMemsetAsync(w.g_w, 0, (size_t)D.BH * kBins * sizeof(double), st));
-  VMOBA_CUDA_OK(cudaMemsetAsync(w.g_minkey, 0xff, (size_t)D.BH * kBins * sizeof(uint32_t), st));
-  VMOBA_CUDA_OK(cudaMemsetAsync(w.g_maxkey, 0, (size_t)D.BH * kBins * sizeof(uint32_t), st));
+  if (local) {
+    // per-query rules: the mask comes straight from the rows; cutoff_key collects the smallest selected key
+    const long long n_rows = (long long)D.BH * D.S;
+    const int blocks = (int)std::min<long long>((n_rows + 7) / 8, 148 * 8);
+    auto launch_local = [&](auto topk_tag, auto mw_tag) {
+      select_local_kernel<decltype(topk_tag)::value, decltype(mw_tag)::value><<<blocks, 256, 0, st>>>(
+          scores, D.S, D.Nb, D.mask_words, D.scale, tau, topk, mask_bits, w.state, n_rows);
+    };
+    auto by_words = [&](auto topk_tag) {
+      if (D.mask_words <= 4) launch_local(topk_tag, std::integral_constant<int, 4>());
+      else if (D.mask_words <= 8) launch_local(topk_tag, std::integral_constant<int, 8>());
+      else if (D.mask_words <= 16) launch_local(topk_tag, std::integral_constant<int, 16>());
+      else launch_local(topk_tag, std::integral_constant<int, kLocalMaxWords>());
+    };
+    if (by_topk) by_words(std::true_type()); else by_words(std::false_type());
+    local_cutoff_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, cutoff_per_head, D.BH);
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(mark_from_mask_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    mark_from_mask_kernel<<<sgrid, kSegThreads, smem, st>>>(mask_bits, D.S, D.Nb, D.mask_words, QSEG, nseg, w.seg_cnt,
+                                                            w.seg_total, w.tmask);
+    VMOBA_LAUNCH_OK(4);
+  } else {
+    // head-wide rules: weighted quantile of the pool (unit weights and a pair budget for top-k)
+    double count_target = -1.0;
+    if (by_topk) {
+      count_target = (double)std::min<long long>((long long)topk * D.S, P);
+      tau = count_target >= (double)P ? 1.0f : 0.5f;      // tau only tells the scan whether everything is taken
+    }
+    const int unit_w = by_topk ? 1 : 0;
+    VMOBA_CUDA_OK(cudaMemsetAsync(w.g_cnt, 0, (size_t)D.BH * kBins * sizeof(unsigned int), st));
+    VMOBA_CUDA_OK(cudaMemsetAsync(w.g_w, 0, (size_t)D.BH * kBins * sizeof(double), st));
+    VMOBA_CUDA_OK(cudaMemsetAsync(w.g_minkey, 0xff, (size_t)D.BH * kBins * sizeof(uint32_t), st));
+    VMOBA_CUDA_OK(cudaMemsetAsync(w.g_maxkey, 0, (size_t)D.BH * kBins * sizeof(uint32_t), st));
 
-  // enough CTAs per head to fill the machine, few enough that the per-CTA flush stays small
-  long long per_head = (P / 4 + 255) / 256;
-  int gx = (int)std::min<long long>(std::max<long long>(per_head / 8, 1), std::max(1, 148 * 8 / D.BH));
-  dim3 grid(gx, D.BH);
-  minmax_kernel<<<grid, 256, 0, st>>>(scores, P, w.state);
-  setup_level0_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH);
-  {
-    constexpr int smem0 = kBins0 * kRep * (int)sizeof(float);
-    VMOBA_CUDA_OK(cudaFuncSetAttribute(hist0_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem0));
-    // three 512-thread CTAs per SM hold their replicated bins side by side
-    int gx0 = (int)std::min<long long>(std::max<long long>(per_head / 16, 1), std::max(1, 148 * 3 / D.BH));
-    hist0_kernel<<<dim3(gx0, D.BH), 512, smem0, st>>>(scores, P, w.state, D.scale, w.g_w);
+    // enough CTAs per head to fill the machine, few enough that the per-CTA flush stays small
+    long long per_head = (P / 4 + 255) / 256;
+    int gx = (int)std::min<long long>(std::max<long long>(per_head / 8, 1), std::max(1, 148 * 8 / D.BH));
+    dim3 grid(gx, D.BH);
+    minmax_kernel<<<grid, 256, 0, st>>>(scores, P, w.state);
+    setup_level0_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH);
+    {
+      constexpr int smem0 = kBins0 * kRep * (int)sizeof(float);
+      VMOBA_CUDA_OK(cudaFuncSetAttribute(hist0_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem0));
+      // three 512-thread CTAs per SM hold their replicated bins side by side
+      int gx0 = (int)std::min<long long>(std::max<long long>(per_head / 16, 1), std::max(1, 148 * 3 / D.BH));
+      hist0_kernel<<<dim3(gx0, D.BH), 512, smem0, st>>>(scores, P, w.state, D.scale, unit_w, w.g_w);
+    }
+    scan_kernel<0><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,
+                                         cutoff_per_head);
+    hist_kernel<1><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
+    scan_kernel<1><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,
+                                         cutoff_per_head);
+    hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
+    scan_kernel<2><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,
+                                         cutoff_per_head);
+    VMOBA_LAUNCH_OK(9);
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(mark_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    mark_kernel<<<sgrid, kSegThreads, smem, st>>>(scores, w.state, D.S, D.Nb, D.mask_words, QSEG, nseg, mask_bits,
+                                                  w.seg_cnt, w.seg_total, w.tmask);
+    VMOBA_LAUNCH_OK(1);
   }
-  scan_kernel<0><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head, cutoff_per_head);
-  hist_kernel<1><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
-  scan_kernel<1><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head, cutoff_per_head);
-  hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
-  scan_kernel<2><<<D.BH, 1024, 0, st>>>(w.state, tau, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head, cutoff_per_head);
-  VMOBA_LAUNCH_OK(9);
 
-  size_t smem = (size_t)QSEG * D.mask_words * 4 + (size_t)std::max(D.Nb, QSEG) * 4 + (size_t)D.Nb * (QSEG >> 5) * 4;
-  VMOBA_CUDA_OK(cudaFuncSetAttribute(mark_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   VMOBA_CUDA_OK(cudaFuncSetAttribute(fill_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  dim3 sgrid(nseg, D.BH);
-  mark_kernel<<<sgrid, kSegThreads, smem, st>>>(scores, w.state, D.S, D.Nb, D.mask_words, QSEG, nseg, mask_bits,
-                                                w.seg_cnt, w.seg_total, w.tmask);
   long long nkb = (long long)D.BH * D.Nb;
   seg_prefix_kernel<<<(unsigned)((nkb + 255) / 256), 256, 0, st>>>(w.seg_cnt, w.kb_total, D.BH, D.Nb, nseg);
   offsets_kernel<<<1, 1024, 0, st>>>(w.kb_total, kb_ptr, nkb, w.seg_total, w.seg_qoff, (long long)D.BH * nseg,
                                      D.BH, D.Nb, k_per_head, capacity, q_ptr + (long long)D.BH * D.S, dev_status);
   fill_kernel<<<sgrid, kSegThreads, smem, st>>>(mask_bits, w.tmask, D.S, D.Nb, D.mask_words, QSEG, nseg, kb_ptr, w.seg_cnt,
                                                 w.seg_qoff, q_idx, q_ptr, q_pairs, capacity);
-  VMOBA_LAUNCH_OK(4);
+  VMOBA_LAUNCH_OK(3);
   return VMOBA_OK;
+}
+
+extern "C" int vmoba_select(const vmoba_shape* shape, const float* scores, float tau, uint32_t* mask_bits,
+                            int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr, int32_t* q_pairs,
+                            int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
+                            int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  return select_impl(shape, scores, VMOBA_SELECT_THRESHOLD_GLOBAL, tau, 0, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity,
+                     k_per_head, cutoff_per_head, dev_status, ws, ws_bytes, stream);
+}
+
+extern "C" int vmoba_select_rule_apply(const vmoba_shape* shape, const float* scores, int32_t rule, float tau, int32_t topk,
+                                       uint32_t* mask_bits, int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr,
+                                       int32_t* q_pairs, int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
+                                       int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  return select_impl(shape, scores, rule, tau, topk, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity, k_per_head,
+                     cutoff_per_head, dev_status, ws, ws_bytes, stream);
 }
 
 // ------------------------------------------------------------------------------------------

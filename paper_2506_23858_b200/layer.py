@@ -77,6 +77,11 @@ class VmobaLayer:
                         self.q_idx, self.q_ptr, self.q_pairs, self.capacity, self.k_per_head, self.cutoff,
                         self.dev_status, self.ws)
 
+    def select_rule(self, rule, tau=0.25, topk=1, scores=None):
+        vb.vmoba_select_rule_apply(self.shape, self.scores if scores is None else scores, rule, tau, topk, self.mask_bits,
+                                   self.kb_ptr, self.q_idx, self.q_ptr, self.q_pairs, self.capacity, self.k_per_head,
+                                   self.cutoff, self.dev_status, self.ws)
+
     def attn_fwd(self):
         vb.vmoba_attn_fwd(self.shape, self.q_bm, self.k_bm, self.v_bm, self.kb_ptr, self.q_idx, self.q_ptr,
                           self.q_pairs, self.capacity, self.o_bm, self.o_resid, self.lse, self.dev_status, self.ws)
