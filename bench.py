@@ -46,6 +46,8 @@ def workloads(name):
         return [gen.C4], True
     if name == "c5":
         return [gen.C5.with_(name="c5_" + k, block=b) for k, b in gen.C5_BLOCKS.items()], True
+    if name == "t55k":   # the paper's 55K-token fine-tuning grid with its own block counts (Table 4), three layers
+        return [gen.T55.with_(name="t55k_" + k, block=b) for k, b in gen.T55_BLOCKS.items()], True
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -217,11 +219,15 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="vmoba", choices=["vmoba", "reference"])
-    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "t55k"])
     ap.add_argument("--cpu-rows", type=int, default=256, help="query rows per unit the CPU oracle baseline evaluates")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dense", action="store_true", help="also time the dense vmoba_full_attn path on the same inputs")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--rule", default="threshold_global",
+                    choices=["threshold_global", "topk_global", "threshold_local", "topk_local"],
+                    help="block-choice rule (Table 3b); the paper's training-free runs use topk_local")
+    ap.add_argument("--topk", default="", help="k of the top-k rules: one value, or one per layer (e.g. 2,6,18)")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small profiling runs)")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -264,13 +270,23 @@ def main():
     outs = {n: torch.empty_like(dev["q"]) for n in (["o"] + (["dq", "dk", "dv"] if with_bwd else []))}
     host_out = {n: torch.empty_like(host["q"]).pin_memory() for n in outs}
 
+    rule = {"threshold_global": vb.SELECT_THRESHOLD_GLOBAL, "topk_global": vb.SELECT_TOPK_GLOBAL,
+            "threshold_local": vb.SELECT_THRESHOLD_LOCAL, "topk_local": vb.SELECT_TOPK_LOCAL}[args.rule]
+    topks = [int(x) for x in args.topk.split(",")] if args.topk else [2]
+
+    def do_select(layer, w, i):
+        if rule == vb.SELECT_THRESHOLD_GLOBAL:
+            layer.select(w.tau)
+        else:
+            layer.select_rule(rule, tau=w.tau, topk=topks[min(i, len(topks) - 1)])
+
     # capacity of the work lists: measured selection size of this workload plus headroom
     L = []
     for w in layers:
         shape = vb.shape_of(w)
         probe = VmobaLayer(shape, capacity=1)          # scores + selection only, to size the lists
         probe.partition(dev["q"], probe.q_bm); probe.partition(dev["k"], probe.k_bm)
-        probe.block_scores(); probe.select(w.tau)
+        probe.block_scores(); do_select(probe, w, len(L))
         torch.cuda.synchronize()
         n_sel = probe.n_selected()
         del probe
@@ -293,7 +309,7 @@ def main():
             layer.partition(dev["v"], layer.v_bm)
             mark("partition")
             layer.block_scores(); mark("scores")
-            layer.select(layer_tau[id(layer)]); mark("select")
+            do_select(layer, layer_w[id(layer)], layer_pos[id(layer)]); mark("select")
             layer.attn_fwd(); mark("attn_fwd")
             layer.partition(outs["o"], layer.o_bm, inverse=True); mark("partition")
             if with_bwd:
@@ -306,6 +322,8 @@ def main():
         return evs
 
     layer_tau = {id(layer): w.tau for layer, w in zip(L, layers)}
+    layer_w = {id(layer): w for layer, w in zip(L, layers)}
+    layer_pos = {id(layer): i for i, layer in enumerate(L)}
 
     def barrier():
         if world > 1:
@@ -454,7 +472,8 @@ def main():
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w0.dtype, "data": "synthetic",
         "config": {"workload": args.workload, "passes": "fwd+bwd" if with_bwd else "fwd", "B": w0.B,
                    "heads": w0.heads, "head_dim": w0.head_dim, "grid": [w0.T, w0.H, w0.W],
-                   "blocks": [list(w.block) for w in layers], "tau": w0.tau, "inputs": w0.recipe,
+                   "blocks": [list(w.block) for w in layers], "tau": w0.tau, "rule": args.rule,
+                   **({"topk": topks} if "topk" in args.rule else {}), "inputs": w0.recipe,
                    "l2": l2_note},
         "clocks": clocks,
         "e2e": {"value": flops_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,

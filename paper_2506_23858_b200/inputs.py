@@ -72,6 +72,10 @@ C3_TAUS = (0.1, 0.25, 0.5, 1.0)
 C4 = Workload("c4_train_3d", 2, 12, 128, 21, 30, 52, (3, 6, 13), 0.25, "bf16", "smooth", 1)
 C5_BLOCKS = {"1d": (1, 45, 80), "2d": (21, 9, 10), "3d": (3, 9, 10)}
 C5 = Workload("c5_720p", 1, 40, 128, 21, 45, 80, (3, 9, 10), 0.25, "bf16", "smooth", 1)
+# The paper's own fine-tuning grid (Table 2 / Table 4: 93x576x1024 video, latent 24x36x64 = 55,296 tokens,
+# 8 / 48 / 72 key blocks for the 1D / 2D / 3D layers, tau = 0.25) on Wan-1.3B-sized heads.
+T55_BLOCKS = {"1d": (3, 36, 64), "2d": (24, 6, 8), "3d": (8, 12, 8)}
+T55 = Workload("t55k_train", 1, 12, 128, 24, 36, 64, (8, 12, 8), 0.25, "bf16", "smooth", 1)
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
