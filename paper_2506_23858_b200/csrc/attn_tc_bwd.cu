@@ -18,7 +18,6 @@
 // D = rowsum(dO * O) and lse come in per query; exp runs in the exp2 domain (c = scale * log2 e).
 // The dense path uses the kernels with 128-query units in the companion file.
 #include <algorithm>
-#include <cstdlib>
 
 #include "attn_simt.cuh"
 #include "sm100.cuh"

@@ -1,18 +1,19 @@
-// Backward kernels for long key blocks / long query lists (bf16, head_dim 128): the same math as
-// attn_tc_bwd.cu, organised for throughput rather than for short items.
+// Backward kernels of the dense path (bf16, head_dim 128): one key range spanning the sequence, so
+// each query meets every key tile and dQ is kept query-stationary instead of being reduced through
+// memory.  The same math as attn_tc_bwd.cu, in two kernels:
 //
 //   * every contraction runs as N = 128 MMAs (an N = 64 shared-memory MMA is bound by operand
 //     reads at about 60 % of the tensor rate; N = 128 runs at the full rate);
-//   * gathered Q / dO rows arrive by TMA row gathers (tile::gather4) issued by one warp, several
-//     tiles ahead, instead of by loader warps;
 //   * the element-wise step and the second pair of MMAs are pipelined at a granularity of 32
 //     columns: as soon as the compute warps have turned 32 columns of S / dP into bf16 P / dS in
 //     TMEM, the MMA warp issues the two k-steps that consume them.
 //
-// dK/dV: item = 128 keys x all queries that selected the block, in units of 128 queries.
-//        TMEM: S^T | dP^T | dV | dK, 128 columns each.  K/V tile single-buffered, Q/dO ring of 2.
-// dQ:    item = 128 gathered queries x one key block, in units of 128 keys.
+// dK/dV: item = 128 keys x all queries, in units of 128 queries (eight loader warps copy the Q / dO
+//        rows).  TMEM: S^T | dP^T | dV | dK, 128 columns each.  K/V tile single-buffered, Q/dO ring of 2.
+// dQ:    item = 128 queries x the key range, in units of 128 keys.
 //        TMEM: S | dP | dQ (x2, alternating by item).  Q/dO tile single-buffered, K/V ring of 2.
+// The kernels also carry index-list (gathered) variants of their loads from the time they served the
+// sparse path; those template branches are not instantiated any more.
 #include <algorithm>
 
 #include "attn_simt.cuh"
@@ -644,15 +645,11 @@ int tc_long_dkdv(const Dims& D, bool dense, const void* q, const void* k, const 
   kp.Nb = dense ? 1 : D.Nb; kp.sb = dense ? D.S : D.sb;
   kp.scale = D.scale; kp.scale_log2 = D.scale * 1.4426950408889634f; kp.capacity = cap;
   kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status; kp.prof = prof;
-  if (dense) {
-    VMOBA_CUDA_OK(cudaFuncSetAttribute(dkdv_long_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KV_SMEM_BYTES));
-    const long long items = (long long)D.BH * ((D.S + BN - 1) / BN);
-    dkdv_long_kernel<true><<<grid_items(items), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, tmQ, tmO, kp);
-  } else {
-    VMOBA_CUDA_OK(cudaFuncSetAttribute(dkdv_long_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KV_SMEM_BYTES));
-    const long long items = (long long)D.BH * D.Nb * ((D.sb + BN - 1) / BN);
-    dkdv_long_kernel<false><<<grid_items(items), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, tmQ, tmO, kp);
-  }
+  // Only the dense instantiation is dispatched: the sparse lists go through the fused kernel.
+  if (!dense) return VMOBA_ERR_ARG;
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(dkdv_long_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KV_SMEM_BYTES));
+  const long long items = (long long)D.BH * ((D.S + BN - 1) / BN);
+  dkdv_long_kernel<true><<<grid_items(items), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, tmQ, tmO, kp);
   VMOBA_LAUNCH_OK(1);
   return VMOBA_OK;
 }
@@ -675,14 +672,10 @@ int tc_long_dq(const Dims& D, bool dense, const void* q, const void* k, const vo
   qp.n_kb = dense ? 0 : D.BH * D.Nb; qp.S = D.S; qp.BH = D.BH; qp.Nb = dense ? 1 : D.Nb; qp.sb = dense ? D.S : D.sb;
   qp.scale = D.scale; qp.scale_log2 = D.scale * 1.4426950408889634f; qp.capacity = cap;
   qp.dq_acc = dq_acc; qp.dq = (__nv_bfloat16*)dq; qp.status = status;
-  if (dense) {
-    VMOBA_CUDA_OK(cudaFuncSetAttribute(dq_long_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DQ_SMEM_BYTES));
-    const long long items = (long long)D.BH * ((D.S + BM - 1) / BM);
-    dq_long_kernel<true><<<grid_items(items), THREADS, DQ_SMEM_BYTES, st>>>(tmK, tmV, tmQ, tmO, qp);
-  } else {
-    VMOBA_CUDA_OK(cudaFuncSetAttribute(dq_long_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DQ_SMEM_BYTES));
-    dq_long_kernel<false><<<grid_items(cap / BM + (long long)D.BH * D.Nb), THREADS, DQ_SMEM_BYTES, st>>>(tmK, tmV, tmQ, tmO, qp);
-  }
+  if (!dense) return VMOBA_ERR_ARG;     // see tc_long_dkdv
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(dq_long_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DQ_SMEM_BYTES));
+  const long long items = (long long)D.BH * ((D.S + BM - 1) / BM);
+  dq_long_kernel<true><<<grid_items(items), THREADS, DQ_SMEM_BYTES, st>>>(tmK, tmV, tmQ, tmO, qp);
   VMOBA_LAUNCH_OK(1);
   return VMOBA_OK;
 }
