@@ -149,7 +149,11 @@ typedef enum {
   VMOBA_SELECT_THRESHOLD_GLOBAL = 0,
   VMOBA_SELECT_TOPK_GLOBAL = 1,
   VMOBA_SELECT_THRESHOLD_LOCAL = 2,
-  VMOBA_SELECT_TOPK_LOCAL = 3
+  VMOBA_SELECT_TOPK_LOCAL = 3,
+  /* may be OR-ed into any rule: every query also keeps the key block it lies in (the convention of
+   * MoBA, which always attends the current block), so that the head-wide rules leave no query
+   * without a block.  The paper's own rule does not do this; it is an option, off by default. */
+  VMOBA_SELECT_KEEP_OWN_BLOCK = 0x100
 } vmoba_select_rule;
 
 int vmoba_select_rule_apply(const vmoba_shape* shape, const float* scores, int32_t rule, float tau, int32_t topk,

@@ -165,6 +165,7 @@ def vmoba_select(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, c
 
 
 SELECT_THRESHOLD_GLOBAL, SELECT_TOPK_GLOBAL, SELECT_THRESHOLD_LOCAL, SELECT_TOPK_LOCAL = 0, 1, 2, 3
+SELECT_KEEP_OWN_BLOCK = 0x100      # OR into a rule: every query also keeps the key block it lies in
 
 
 def vmoba_select_rule_apply(shape, scores, rule, tau, topk, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity,

@@ -303,8 +303,8 @@ __global__ void setup_level0_kernel(HeadState* st, int BH) {
 // then writes mask words, per-(segment, block) counts and the segment's pair total.
 __global__ void __launch_bounds__(kSegThreads)
 mark_kernel(const float* __restrict__ scores, const HeadState* __restrict__ st, int S, int Nb, int mw, int QSEG,
-            int nseg, uint32_t* __restrict__ mask_bits, int* __restrict__ seg_cnt, int* __restrict__ seg_total,
-            uint32_t* __restrict__ tmask) {
+            int nseg, int own_sb, uint32_t* __restrict__ mask_bits, int* __restrict__ seg_cnt,
+            int* __restrict__ seg_total, uint32_t* __restrict__ tmask) {
   extern __shared__ uint32_t sm[];
   const int TW = QSEG >> 5;                           // words of a block's column over the segment's queries
   uint32_t* s_mask = sm;                              // [QSEG][mw]
@@ -323,9 +323,10 @@ mark_kernel(const float* __restrict__ scores, const HeadState* __restrict__ st, 
   const float* base = scores + ((long long)bh * S + q0) * Nb;
   const long long n = (long long)nq * Nb;
   auto mark = [&](long long i, float s) {
-    if (float_key(s) >= cutoff) {
-      int ii = (int)i;
-      int ql = ii / Nb, j = ii - ql * Nb;
+    int ii = (int)i;
+    int ql = ii / Nb, j = ii - ql * Nb;
+    // own_sb > 0: a query also keeps the block it lies in (block-major position / tokens per block)
+    if (float_key(s) >= cutoff || (own_sb > 0 && (q0 + ql) / own_sb == j)) {
       atomicOr(&s_mask[ql * mw + (j >> 5)], 1u << (j & 31));
       atomicOr(&s_tm[j * TW + (ql >> 5)], 1u << (ql & 31));
       atomicAdd(&s_cnt[j], 1);
@@ -500,7 +501,7 @@ constexpr int kLocalMaxWords = 32;
 // MW: compile-time bound on the mask words of a row (the loops over a lane's blocks unroll to it)
 template <bool TOPK, int MW>
 __global__ void __launch_bounds__(256)
-select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, float sigma, float tau, int topk,
+select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, float sigma, float tau, int topk, int own_sb,
                     uint32_t* __restrict__ mask_bits, HeadState* __restrict__ st, long long n_rows) {
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -508,6 +509,8 @@ select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, flo
   const uint32_t lt_mask = (1u << lane) - 1u;
   for (long long row = warp; row < n_rows; row += nwarps) {
     const float* sr = scores + row * Nb;
+    const int own = own_sb > 0 ? (int)(row % S) / own_sb : -1;      // the query's own block, if it is to be kept
+    const uint32_t own_bit = (own >= 0 && (own >> 5) == lane) ? 1u << (own & 31) : 0u;
     uint32_t key[MW];
     uint32_t kmax = 0u;
 #pragma unroll
@@ -585,7 +588,7 @@ select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, flo
           const uint32_t word = __ballot_sync(0xffffffffu, (taken >> i) & 1u);
           if (lane == i) my_word = word;
         }
-        if (lane < mw) mask_bits[row * mw + lane] = my_word;
+        if (lane < mw) mask_bits[row * mw + lane] = my_word | own_bit;
         if (lane == 0) atomicMin(&st[row / S].cutoff_key, c_last);
         continue;
       }
@@ -631,7 +634,7 @@ select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, flo
         run += __popc(e);
       }
     }
-    if (lane < mw) mask_bits[row * mw + lane] = my_word;
+    if (lane < mw) mask_bits[row * mw + lane] = my_word | own_bit;
     if (lane == 0) atomicMin(&st[row / S].cutoff_key, c);
   }
 }
@@ -735,6 +738,9 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
   Dims D;
   int rc = make_dims(shape, &D);
   if (rc) return rc;
+  // D is known here: a query at block-major position p lies in key block p / s_b
+  const int own_sb = (rule & VMOBA_SELECT_KEEP_OWN_BLOCK) ? D.sb : 0;
+  rule &= ~VMOBA_SELECT_KEEP_OWN_BLOCK;
   const bool by_topk = rule == VMOBA_SELECT_TOPK_GLOBAL || rule == VMOBA_SELECT_TOPK_LOCAL;
   const bool local = rule == VMOBA_SELECT_THRESHOLD_LOCAL || rule == VMOBA_SELECT_TOPK_LOCAL;
   if (rule < VMOBA_SELECT_THRESHOLD_GLOBAL || rule > VMOBA_SELECT_TOPK_LOCAL) return VMOBA_ERR_ARG;
@@ -761,7 +767,7 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
     const int blocks = (int)std::min<long long>((n_rows + 7) / 8, 148 * 8);
     auto launch_local = [&](auto topk_tag, auto mw_tag) {
       select_local_kernel<decltype(topk_tag)::value, decltype(mw_tag)::value><<<blocks, 256, 0, st>>>(
-          scores, D.S, D.Nb, D.mask_words, D.scale, tau, topk, mask_bits, w.state, n_rows);
+          scores, D.S, D.Nb, D.mask_words, D.scale, tau, topk, own_sb, mask_bits, w.state, n_rows);
     };
     auto by_words = [&](auto topk_tag) {
       if (D.mask_words <= 4) launch_local(topk_tag, std::integral_constant<int, 4>());
@@ -811,7 +817,7 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
                                          cutoff_per_head);
     VMOBA_LAUNCH_OK(9);
     VMOBA_CUDA_OK(cudaFuncSetAttribute(mark_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    mark_kernel<<<sgrid, kSegThreads, smem, st>>>(scores, w.state, D.S, D.Nb, D.mask_words, QSEG, nseg, mask_bits,
+    mark_kernel<<<sgrid, kSegThreads, smem, st>>>(scores, w.state, D.S, D.Nb, D.mask_words, QSEG, nseg, own_sb, mask_bits,
                                                   w.seg_cnt, w.seg_total, w.tmask);
     VMOBA_LAUNCH_OK(1);
   }

@@ -188,3 +188,29 @@ def test_local_rules_at_full_size_on_sampled_rows():
         ref, k_ref = orc.select_threshold_per_query(sc, 0.5, w.head_dim ** -0.5)
         differ = (got != ref).any(axis=1)
         assert differ.sum() <= 4 and (np.abs(got.sum(axis=1) - k_ref) <= 1).all(), (name, int(differ.sum()))
+
+
+def test_keep_own_block_option():
+    """VMOBA_SELECT_KEEP_OWN_BLOCK: the mask is the rule's mask OR the block each query lies in."""
+    w = MID
+    data, ora = _prep(w)
+    L = _layer_with_scores(w, ora)
+    own = np.zeros((w.S, w.n_blocks), dtype=bool)
+    own[np.arange(w.S), np.arange(w.S) // w.block_tokens] = True
+    for rule, kw, ref_of in (
+            (vb.SELECT_THRESHOLD_GLOBAL, dict(tau=0.25), lambda sc: orc.select(sc, 0.25, ora["scale"])[0]),
+            (vb.SELECT_TOPK_LOCAL, dict(topk=2), lambda sc: orc.select_topk_per_query(sc, 2)),
+            (vb.SELECT_THRESHOLD_LOCAL, dict(tau=0.25), lambda sc: orc.select_threshold_per_query(sc, 0.25, ora["scale"])[0])):
+        base = _run(L, w, rule, **kw).copy()
+        got = _run(L, w, rule | vb.SELECT_KEEP_OWN_BLOCK, **kw)
+        for i, hd in enumerate(ora["heads"]):
+            assert np.array_equal(got[i], base[i] | own), (rule, i)
+        assert (got.sum(axis=2) >= 1).all()
+        _check_lists(L, w, got)
+    # end to end: no query is left without keys, so no output row is zero and every lse is finite
+    for name, buf in (("q", L.q_bm), ("k", L.k_bm), ("v", L.v_bm)):
+        buf.copy_(U.bm_to_device(w, U.block_major(w, data, name, ora["perm"])))
+    L.select_rule(vb.SELECT_THRESHOLD_GLOBAL | vb.SELECT_KEEP_OWN_BLOCK, tau=0.25)
+    L.attn_fwd()
+    L.check_status()
+    assert torch.isfinite(L.lse).all()
