@@ -219,7 +219,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="vmoba", choices=["vmoba", "reference"])
-    ap.add_argument("--workload", default="c4", choices=["c1", "c2", "c3", "c4", "c5", "t55k"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "t55k"])
     ap.add_argument("--cpu-rows", type=int, default=256, help="query rows per unit the CPU oracle baseline evaluates")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--dense", action="store_true", help="also time the dense vmoba_full_attn path on the same inputs")
