@@ -164,28 +164,37 @@ def run_reference(args):
     cores = torch.get_num_threads()
     times, flops_tot = [], 0.0
     detail = None
-    warmup, steps = min(args.warmup, 1), args.steps
+    # One untimed step first (also when W = 0): it tells how long a step takes.  If W + K such steps would
+    # not end within a few minutes, later steps sample fewer of the workload's layers (the value is work /
+    # time of whatever was sampled), and only if one layer is still too slow, fewer steps.
+    warmup, steps = 1, args.steps
+    n_used = len(layers)
     it = 0
     while it < warmup + steps:
         wall = time.perf_counter()
         t, f = 0.0, 0.0
-        for w in layers:
+        for w in layers[:n_used]:
             tt, ff, detail = oracle_sample(w, with_bwd, args.cpu_rows, seed=it)
             t += tt; f += ff
         wall = time.perf_counter() - wall
         if it >= warmup:
             times.append(t); flops_tot = f
-        elif wall * (warmup + steps) > 240.0:
-            steps = max(1, int(240.0 / wall) - warmup)     # keep the whole run within a few minutes
+        else:
+            budget = 240.0 / (warmup + steps)
+            if wall > budget:
+                n_used = max(1, int(len(layers) * budget / wall))
+                per_step = wall * n_used / len(layers)
+                if per_step > budget:
+                    steps = max(1, int(240.0 / per_step) - warmup)
         it += 1
     sec = statistics.mean(times)
     units = layers[0].B * layers[0].heads
     value = flops_tot / sec / 1e12
-    sample = (f"1 of {units} (batch, head) units per layer; partition, centroids, scores, selection in full; "
-              f"attention on {args.cpu_rows} sampled query rows, time scaled to the unit's selected pairs")
+    sample = (f"1 of {units} (batch, head) units of {n_used} of the {len(layers)} layers; partition, centroids, scores, "
+              f"selection in full; attention on {args.cpu_rows} sampled query rows, time scaled to the unit's selected pairs")
     line = {
         "impl": "reference", "metric": "vmoba_layer_selected_pair_tflops", "value": value, "unit": "TFLOP/s",
-        "n_gpus": args.gpus, "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3 * units,
+        "n_gpus": args.gpus, "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3 * units * len(layers) / n_used,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": args.workload, "passes": "fwd+bwd" if with_bwd else "fwd"},
         "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
