@@ -191,6 +191,36 @@ def select_threshold_per_query(scores, tau, sigma):
     return mask, ks
 
 
+def select_rownorm(scores, tau, sigma):
+    """Eq. 3 + Eq. 4 under the other reading of "normalized similarity scores": each query's scores
+    are normalised on their own, p_ij = softmax_j(sigma * S_hat_ij) / s (fp64; the head's pool then
+    sums to one), the pool is ordered by p descending (ties: ascending flat index) and pairs are
+    taken until the cumulative p reaches tau (tau >= 1 or never reached: all).  Unlike the pool-wide
+    softmax this is not a single raw-score cutoff per head: a query with a flat row needs a higher
+    raw score than a query with a peaked one.
+    Returns (mask [s, N_b] bool, k, cutoff) with cutoff = ln(s * p) of the last pair taken, i.e.
+    sigma * S_hat minus the row's log-sum-exp.
+    """
+    if not (tau > 0.0):
+        raise ValueError("tau must be in (0, 1]")
+    s, n_b = scores.shape
+    x = sigma * scores.astype(np.float64)
+    m = x.max(axis=1, keepdims=True)
+    lse = m + np.log(np.exp(x - m).sum(axis=1, keepdims=True))
+    logp = (x - lse).reshape(-1)                      # ln(s * p)
+    P = logp.size
+    order = np.argsort(-logp, kind="stable")
+    if tau >= 1.0:
+        k = P
+    else:
+        c = np.cumsum(np.exp(logp[order]) / s)
+        hit = np.nonzero(c >= tau)[0]
+        k = int(hit[0]) + 1 if hit.size else P
+    mask = np.zeros(P, dtype=bool)
+    mask[order[:k]] = True
+    return mask.reshape(s, n_b), k, float(logp[order[k - 1]])
+
+
 def select_topk_global(scores, k):
     """"topk + global" of the block-choice ablation (Table 3b): the head-wide pool of Eq. 3 with a
     fixed budget instead of the threshold of Eq. 4.  The budget is the one "topk + local" spends,

@@ -316,6 +316,36 @@ def test_select_threshold_per_query_rows_are_independent_and_never_empty():
         orc.select_threshold_per_query(sc, 0.0, 1.0)
 
 
+def test_select_rownorm():
+    # two queries, sigma = 1.  Row 0 is peaked: softmax (0.9526, 0.0474); row 1 is flat: (0.5, 0.5).
+    # Pool probabilities (divided by s = 2): 0.4763, 0.0237, 0.25, 0.25 -> order (0,0), (1,0), (1,1), (0,1)
+    sc = np.array([[3.0, 0.0], [7.0, 7.0]], dtype=np.float32)
+    for tau, want, k_want in [(0.4, [[1, 0], [0, 0]], 1), (0.5, [[1, 0], [1, 0]], 2), (0.73, [[1, 0], [1, 1]], 3),
+                              (0.98, [[1, 1], [1, 1]], 4), (1.0, [[1, 1], [1, 1]], 4)]:
+        m, k, cut = orc.select_rownorm(sc, tau, 1.0)
+        assert m.astype(int).tolist() == want and k == k_want, tau
+    # the raw scores of row 1 (7.0) exceed every score of row 0, yet row 0's peak is taken first:
+    # the pool-wide softmax of Eq. 4's other reading would take both 7.0s first
+    assert orc.select(sc, 0.4, 1.0)[0].astype(int).tolist() == [[0, 0], [1, 0]]
+    # one query: both readings coincide (the row is the pool)
+    rng = np.random.default_rng(8)
+    row = rng.normal(size=(1, 31)).astype(np.float32) * 2
+    for tau in (0.1, 0.5, 0.9):
+        assert (orc.select_rownorm(row, tau, 0.6)[0] == orc.select(row, tau, 0.6)[0]).all()
+    # rows shifted by constants are normalised away: the mask does not change
+    sc = rng.normal(size=(12, 9)).astype(np.float32)
+    shift = rng.normal(size=(12, 1)).astype(np.float32) * 8
+    a, ka, _ = orc.select_rownorm(sc.astype(np.float64), 0.3, 1.0)
+    b, kb, _ = orc.select_rownorm(sc.astype(np.float64) + shift.astype(np.float64), 0.3, 1.0)
+    assert (a == b).all() and ka == kb
+    # brute force: the kept set is exactly the top-k of p and its mass is the first to reach tau
+    x = sc.astype(np.float64)
+    p = np.exp(x) / np.exp(x).sum(axis=1, keepdims=True) / 12
+    assert p[a].min() >= p[~a].max() and p[a].sum() >= 0.3 and p[a].sum() - p[a].min() < 0.3
+    with pytest.raises(ValueError):
+        orc.select_rownorm(sc, 0.0, 1.0)
+
+
 def test_select_topk_global():
     sc = np.array([[1, 5, 3, 3], [0, 0, 0, 0], [9, 8, 7, 6]], dtype=np.float32)
     m, K, cut = orc.select_topk_global(sc, 2)          # budget 6 of 12: 9 8 7 6 5 and the first 3
