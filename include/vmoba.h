@@ -62,7 +62,8 @@ typedef enum {
   VMOBA_STAGE_ATTN_FWD = 2,
   VMOBA_STAGE_ATTN_BWD = 3,
   VMOBA_STAGE_FULL_FWD = 4,
-  VMOBA_STAGE_FULL_BWD = 5
+  VMOBA_STAGE_FULL_BWD = 5,
+  VMOBA_STAGE_SELECT_ROWNORM = 6   /* vmoba_select_rule_apply with VMOBA_SELECT_THRESHOLD_GLOBAL_ROWNORM */
 } vmoba_stage;
 
 typedef struct {
@@ -150,6 +151,12 @@ typedef enum {
   VMOBA_SELECT_TOPK_GLOBAL = 1,
   VMOBA_SELECT_THRESHOLD_LOCAL = 2,
   VMOBA_SELECT_TOPK_LOCAL = 3,
+  /* the method's own rule under the other reading of "normalized similarity scores" (Eq. 4): each
+   * query's scores are normalised by a softmax over its own N_b blocks, then pooled over the head
+   * (divided by S) and taken in descending order of that probability until the sum reaches tau.
+   * cutoff_per_head receives softmax_scale * score - logsumexp(row) of the last pair taken.  Needs
+   * the larger workspace vmoba_workspace_bytes(shape, VMOBA_STAGE_SELECT_ROWNORM, 0). */
+  VMOBA_SELECT_THRESHOLD_GLOBAL_ROWNORM = 4,
   /* may be OR-ed into any rule: every query also keeps the key block it lies in (the convention of
    * MoBA, which always attends the current block), so that the head-wide rules leave no query
    * without a block.  The paper's own rule does not do this; it is an option, off by default. */

@@ -13,7 +13,7 @@ from . import build as _build
 
 OK, ERR_ARG, ERR_SHAPE, ERR_WORKSPACE, ERR_CAPACITY, ERR_TIMEOUT, ERR_CUDA, ERR_NOT_IMPLEMENTED = range(8)
 F32, BF16 = 0, 1
-STAGE_SCORES, STAGE_SELECT, STAGE_ATTN_FWD, STAGE_ATTN_BWD, STAGE_FULL_FWD, STAGE_FULL_BWD = range(6)
+STAGE_SCORES, STAGE_SELECT, STAGE_ATTN_FWD, STAGE_ATTN_BWD, STAGE_FULL_FWD, STAGE_FULL_BWD, STAGE_SELECT_ROWNORM = range(7)
 
 EXPORTS = (
     "vmoba_status_string", "vmoba_kernel_launches", "vmoba_workspace_bytes", "vmoba_partition", "vmoba_block_scores",
@@ -165,6 +165,7 @@ def vmoba_select(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, c
 
 
 SELECT_THRESHOLD_GLOBAL, SELECT_TOPK_GLOBAL, SELECT_THRESHOLD_LOCAL, SELECT_TOPK_LOCAL = 0, 1, 2, 3
+SELECT_THRESHOLD_GLOBAL_ROWNORM = 4  # Eq. 4 with per-query softmax normalisation; needs STAGE_SELECT_ROWNORM scratch
 SELECT_KEEP_OWN_BLOCK = 0x100      # OR into a rule: every query also keeps the key block it lies in
 
 

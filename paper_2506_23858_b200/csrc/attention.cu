@@ -8,6 +8,7 @@
 namespace vmoba {
 
 size_t select_ws_bytes(const Dims& D);   // select.cu
+size_t select_rownorm_ws_bytes(const Dims& D);
 size_t scores_ws_bytes(const Dims& D);   // scores.cu
 
 // attn_tc_fwd.cu: tensor-core forward kernel (bf16, head_dim 128)
@@ -183,6 +184,7 @@ extern "C" size_t vmoba_workspace_bytes(const vmoba_shape* shape, int stage, int
   switch (stage) {
     case VMOBA_STAGE_SCORES: return scores_ws_bytes(D);
     case VMOBA_STAGE_SELECT: return select_ws_bytes(D);
+    case VMOBA_STAGE_SELECT_ROWNORM: return select_rownorm_ws_bytes(D);
     case VMOBA_STAGE_ATTN_FWD: return carve_fwd(D, capacity, nullptr).bytes;
     case VMOBA_STAGE_ATTN_BWD: return carve_bwd(D, false, nullptr, capacity).bytes;
     case VMOBA_STAGE_FULL_FWD: return 256;

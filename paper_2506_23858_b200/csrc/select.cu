@@ -684,6 +684,30 @@ mark_from_mask_kernel(const uint32_t* __restrict__ mask_bits, int S, int Nb, int
   if (threadIdx.x == 0) seg_total[bh * nseg + seg] = s_total;
 }
 
+// Row normalisation for the second reading of Eq. 4: out[i][j] = sigma * s[i][j] - logsumexp_j(sigma * s[i][:]),
+// the logarithm of S times the pair's probability when every query is normalised on its own.  One
+// warp per query row; the head-wide quantile search then runs on `out` with unit temperature.
+__global__ void __launch_bounds__(256)
+rownorm_kernel(const float* __restrict__ scores, float* __restrict__ out, int Nb, float sigma, long long n_rows) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
+  for (long long row = warp; row < n_rows; row += nwarps) {
+    const float* sr = scores + row * Nb;
+    float mx = -INFINITY;
+    for (int j = lane; j < Nb; j += 32) mx = fmaxf(mx, sigma * __ldg(sr + j));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float z = 0.f;
+    for (int j = lane; j < Nb; j += 32) z += expf(sigma * __ldg(sr + j) - mx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    const float lse = mx + logf(z);
+    float* orow = out + row * Nb;
+    for (int j = lane; j < Nb; j += 32) orow[j] = sigma * __ldg(sr + j) - lse;
+  }
+}
+
 static int seg_queries(int mw) {
   int q = 4096 / mw;            // keep the shared mask tile <= 16 KB
   q = q / 32 * 32;
@@ -726,6 +750,10 @@ static SelectWs carve_select(const Dims& D, void* ws) {
 }
 
 size_t select_ws_bytes(const Dims& D) { return carve_select(D, nullptr).bytes; }
+// the row-normalised rule also keeps a transformed copy of the score matrix behind the common scratch
+size_t select_rownorm_ws_bytes(const Dims& D) {
+  return ((carve_select(D, nullptr).bytes + 255) / 256) * 256 + (size_t)D.BH * D.S * D.Nb * sizeof(float);
+}
 
 }  // namespace vmoba
 
@@ -741,6 +769,8 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
   // D is known here: a query at block-major position p lies in key block p / s_b
   const int own_sb = (rule & VMOBA_SELECT_KEEP_OWN_BLOCK) ? D.sb : 0;
   rule &= ~VMOBA_SELECT_KEEP_OWN_BLOCK;
+  const bool rownorm = rule == VMOBA_SELECT_THRESHOLD_GLOBAL_ROWNORM;
+  if (rownorm) rule = VMOBA_SELECT_THRESHOLD_GLOBAL;
   const bool by_topk = rule == VMOBA_SELECT_TOPK_GLOBAL || rule == VMOBA_SELECT_TOPK_LOCAL;
   const bool local = rule == VMOBA_SELECT_THRESHOLD_LOCAL || rule == VMOBA_SELECT_TOPK_LOCAL;
   if (rule < VMOBA_SELECT_THRESHOLD_GLOBAL || rule > VMOBA_SELECT_TOPK_LOCAL) return VMOBA_ERR_ARG;
@@ -752,9 +782,19 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
   if (capacity <= 0 || capacity > (int64_t)INT32_MAX) return VMOBA_ERR_ARG;
   if (D.Nb > 8192 || (local && D.Nb > 32 * kLocalMaxWords)) return VMOBA_ERR_SHAPE;
   SelectWs w = carve_select(D, ws);
-  if (ws_bytes < w.bytes) return VMOBA_ERR_WORKSPACE;
+  if (ws_bytes < (rownorm ? select_rownorm_ws_bytes(D) : w.bytes)) return VMOBA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const long long P = (long long)D.S * D.Nb;
+  float sigma = D.scale;
+  if (rownorm) {
+    // search on the row-normalised log-probabilities with unit temperature
+    float* lp = reinterpret_cast<float*>(static_cast<char*>(ws) + ((w.bytes + 255) / 256) * 256);
+    const long long n_rows = (long long)D.BH * D.S;
+    rownorm_kernel<<<(int)std::min<long long>((n_rows + 7) / 8, 148 * 8), 256, 0, st>>>(scores, lp, D.Nb, D.scale, n_rows);
+    VMOBA_LAUNCH_OK(1);
+    scores = lp;
+    sigma = 1.0f;
+  }
   const int QSEG = seg_queries(D.mask_words);
   const int nseg = (D.S + QSEG - 1) / QSEG;
   const size_t smem = (size_t)QSEG * D.mask_words * 4 + (size_t)std::max(D.Nb, QSEG) * 4 + (size_t)D.Nb * (QSEG >> 5) * 4;
@@ -805,14 +845,14 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
       VMOBA_CUDA_OK(cudaFuncSetAttribute(hist0_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem0));
       // three 512-thread CTAs per SM hold their replicated bins side by side
       int gx0 = (int)std::min<long long>(std::max<long long>(per_head / 16, 1), std::max(1, 148 * 3 / D.BH));
-      hist0_kernel<<<dim3(gx0, D.BH), 512, smem0, st>>>(scores, P, w.state, D.scale, unit_w, w.g_w);
+      hist0_kernel<<<dim3(gx0, D.BH), 512, smem0, st>>>(scores, P, w.state, sigma, unit_w, w.g_w);
     }
     scan_kernel<0><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,
                                          cutoff_per_head);
-    hist_kernel<1><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
+    hist_kernel<1><<<grid, 256, 0, st>>>(scores, P, w.state, sigma, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
     scan_kernel<1><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,
                                          cutoff_per_head);
-    hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, D.scale, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
+    hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, sigma, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
     scan_kernel<2><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,
                                          cutoff_per_head);
     VMOBA_LAUNCH_OK(9);

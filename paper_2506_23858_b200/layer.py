@@ -78,9 +78,16 @@ class VmobaLayer:
                         self.dev_status, self.ws)
 
     def select_rule(self, rule, tau=0.25, topk=1, scores=None):
+        ws = self.ws
+        if (rule & 0xff) == vb.SELECT_THRESHOLD_GLOBAL_ROWNORM:
+            # this rule keeps a transformed copy of the score matrix in its scratch: allocated on first use
+            need = vb.workspace_bytes(self.shape, vb.STAGE_SELECT_ROWNORM, self.capacity)
+            if getattr(self, "ws_rownorm", None) is None or self.ws_rownorm.numel() < need:
+                self.ws_rownorm = torch.empty(need, dtype=torch.uint8, device=self.ws.device)
+            ws = self.ws_rownorm
         vb.vmoba_select_rule_apply(self.shape, self.scores if scores is None else scores, rule, tau, topk, self.mask_bits,
                                    self.kb_ptr, self.q_idx, self.q_ptr, self.q_pairs, self.capacity, self.k_per_head,
-                                   self.cutoff, self.dev_status, self.ws)
+                                   self.cutoff, self.dev_status, ws)
 
     def attn_fwd(self):
         vb.vmoba_attn_fwd(self.shape, self.q_bm, self.k_bm, self.v_bm, self.kb_ptr, self.q_idx, self.q_ptr,

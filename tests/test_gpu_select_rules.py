@@ -214,3 +214,32 @@ def test_keep_own_block_option():
     L.attn_fwd()
     L.check_status()
     assert torch.isfinite(L.lse).all()
+
+
+@pytest.mark.parametrize("w", CASES, ids=IDS)
+def test_rownorm_threshold_matches_oracle(w):
+    """Eq. 4 with per-query softmax normalisation: equal to the oracle on every pair whose row-normalised
+    log-probability is farther than the score band from the oracle's cutoff."""
+    data, ora = _prep(w)
+    L = _layer_with_scores(w, ora)
+    for tau in (0.25, 0.6, 1.0):
+        got = _run(L, w, vb.SELECT_THRESHOLD_GLOBAL_ROWNORM, tau=tau)
+        kph = L.k_per_head.cpu().numpy(); cut = L.cutoff.cpu().numpy()
+        for i, hd in enumerate(ora["heads"]):
+            m_ref, k_ref, c_ref = orc.select_rownorm(hd["scores"], tau, ora["scale"])
+            x = ora["scale"] * hd["scores"].astype(np.float64)
+            mx = x.max(axis=1, keepdims=True)
+            logp = x - (mx + np.log(np.exp(x - mx).sum(axis=1, keepdims=True)))
+            decided = np.abs(logp - c_ref) > U.SCORE_BAND
+            assert np.array_equal(got[i][decided], m_ref[decided]), (tau, i)
+            assert kph[i] == got[i].sum()
+            if tau < 1.0:
+                assert abs(float(cut[i]) - c_ref) <= U.SCORE_BAND
+            assert abs(int(kph[i]) - k_ref) <= max(8, int(2e-3 * k_ref)), (tau, i, kph[i], k_ref)
+        _check_lists(L, w, got)
+    assert got.all()
+    # too small a workspace is refused on the host
+    with pytest.raises(vb.VmobaError):
+        vb.vmoba_select_rule_apply(L.shape, L.scores, vb.SELECT_THRESHOLD_GLOBAL_ROWNORM, 0.25, 1, L.mask_bits, L.kb_ptr,
+                                   L.q_idx, L.q_ptr, L.q_pairs, L.capacity, L.k_per_head, L.cutoff, L.dev_status,
+                                   L.ws[:vb.workspace_bytes(L.shape, vb.STAGE_SELECT, 0)])
