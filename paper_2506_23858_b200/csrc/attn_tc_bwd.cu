@@ -216,6 +216,9 @@ __device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, i
   return it;
 }
 
+// Only <DENSE = false, FUSE = true> is instantiated.  FUSE = false is the same kernel without the
+// dQ^T MMA, the dS^T tile and the writer warps (dS^T then goes to the dP^T columns, K/V are double
+// buffered across items); DENSE = true walks all queries of the sequence instead of an index list.
 template <bool DENSE, bool FUSE>
 __global__ void __launch_bounds__(FUSE ? KVF_THREADS : KV_THREADS, 1)
 attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const KvParams p) {
