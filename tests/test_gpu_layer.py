@@ -188,3 +188,10 @@ def test_config5_720p_shape_forward_backward(name):
     shape = vb.shape_of(w)
     cap = int(0.3 * default_capacity(shape, w.tau)) if name == "3d" else None
     _full_size(w, True, [(0, 2)], n_rows=48, n_blocks=1, capacity=cap)
+
+
+def test_config5_all_40_heads_one_layer():
+    """Config 5 exactly as bench.py times it (B=1, 40 heads, 75,600 tokens), the 2D layer, forward and
+    backward; sampled rows and key blocks of the first and the last head against the oracle."""
+    w = gen.C5.with_(name="c5_full_2d", block=gen.C5_BLOCKS["2d"])
+    _full_size(w, True, [(0, 0), (0, 39)], n_rows=32, n_blocks=1)
