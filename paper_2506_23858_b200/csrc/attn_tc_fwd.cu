@@ -141,6 +141,19 @@ __device__ __forceinline__ void exp_pack64(const uint32_t (&sv)[64], float scale
   }
 }
 
+// Eight consecutive outputs as bf16 (one 16-byte store) and, if asked for, their rounding residuals
+// bf16(v - bf16(v)), computed in registers.
+__device__ __forceinline__ void store8_resid(__nv_bfloat16* dst, __nv_bfloat16* rdst, const float (&v)[8]) {
+  uint32_t h[4], r[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    h[k] = pack_bf16(v[2 * k], v[2 * k + 1]);
+    r[k] = pack_bf16(v[2 * k] - __uint_as_float(h[k] << 16), v[2 * k + 1] - __uint_as_float(h[k] & 0xffff0000u));
+  }
+  *reinterpret_cast<uint4*>(dst) = make_uint4(h[0], h[1], h[2], h[3]);
+  if (rdst) *reinterpret_cast<uint4*>(rdst) = make_uint4(r[0], r[1], r[2], r[3]);
+}
+
 template <bool DENSE>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
@@ -451,10 +464,12 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             __nv_bfloat16* dst = p.o + G_ * DH + col;
             __nv_bfloat16* rdst = p.o_resid ? p.o_resid + G_ * DH + col : nullptr;
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              store4_resid(dst + i, rdst ? rdst + i : nullptr,
-                           make_float4(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
-                                       __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv));
+            for (int i = 0; i < 32; i += 8) {
+              float v8[8];
+#pragma unroll
+              for (int k = 0; k < 8; ++k) v8[k] = __uint_as_float(ov[i + k]) * inv;
+              store8_resid(dst + i, rdst ? rdst + i : nullptr, v8);
+            }
           } else {
             float* dst = p.part_o + pos * DH + col;
 #pragma unroll
