@@ -550,12 +550,18 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         tmem_ld_wait();
         if (r < it.valid) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 4) {
-            store4(dv_row + cgrp * 32 + i, make_float4(__uint_as_float(a[i]), __uint_as_float(a[i + 1]),
-                                                       __uint_as_float(a[i + 2]), __uint_as_float(a[i + 3])));
-            store4(dk_row + cgrp * 32 + i,
-                   make_float4(__uint_as_float(bb[i]) * p.scale, __uint_as_float(bb[i + 1]) * p.scale,
-                               __uint_as_float(bb[i + 2]) * p.scale, __uint_as_float(bb[i + 3]) * p.scale));
+          for (int i = 0; i < 32; i += 8) {       // eight bf16 = one 16-byte store
+            uint4 hv, hk;
+            hv.x = pack_bf16(__uint_as_float(a[i]), __uint_as_float(a[i + 1]));
+            hv.y = pack_bf16(__uint_as_float(a[i + 2]), __uint_as_float(a[i + 3]));
+            hv.z = pack_bf16(__uint_as_float(a[i + 4]), __uint_as_float(a[i + 5]));
+            hv.w = pack_bf16(__uint_as_float(a[i + 6]), __uint_as_float(a[i + 7]));
+            hk.x = pack_bf16(__uint_as_float(bb[i]) * p.scale, __uint_as_float(bb[i + 1]) * p.scale);
+            hk.y = pack_bf16(__uint_as_float(bb[i + 2]) * p.scale, __uint_as_float(bb[i + 3]) * p.scale);
+            hk.z = pack_bf16(__uint_as_float(bb[i + 4]) * p.scale, __uint_as_float(bb[i + 5]) * p.scale);
+            hk.w = pack_bf16(__uint_as_float(bb[i + 6]) * p.scale, __uint_as_float(bb[i + 7]) * p.scale);
+            *reinterpret_cast<uint4*>(dv_row + cgrp * 32 + i) = hv;
+            *reinterpret_cast<uint4*>(dk_row + cgrp * 32 + i) = hk;
           }
         }
       }
