@@ -242,17 +242,21 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer: the whole warp walks the loop, one
+    // elected lane issues (warp-uniform control flow; see elect_one)
+    {
+      const bool leader = elect_one();
+      const int n_items_u = __reduce_max_sync(0xffffffffu, n_items);
       uint32_t fills = 0;              // key tiles consumed so far (ring position of K and of V)
       uint32_t n = 0;                  // items done so far
       uint32_t tcnt[2] = {0, 0};       // key tiles done per query tile (phase of s_full / p_ready / o_done)
       uint32_t ecnt[2] = {0, 0};       // items done per query tile (phase of o_free)
       const uint64_t dQ[2] = {make_smem_desc(smem_u32(sQ), 16, 1024), make_smem_desc(smem_u32(sQ + TILE), 16, 1024)};
-      for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
-        const FwdItem it = decode_item<DENSE>(p, item);
+      for (int item = blockIdx.x; item < n_items_u; item += gridDim.x, ++n) {
+        FwdItem it = decode_item<DENSE>(p, item);
+        it.nx = __reduce_max_sync(0xffffffffu, it.nx);
         lap(5);
-        mbar_wait(&sm->q_full, n & 1, abort_flag, p.status);
+        mbar_wait_warp(&sm->q_full, n & 1, abort_flag, p.status);
         lap(0);
         tc_fence_after();
         auto qk = [&](int x, int t, int s) {
@@ -261,61 +265,61 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
           const uint64_t dK0 = make_smem_desc(smem_u32(sK + s * TILE), 16, 1024);
 #pragma unroll
           for (int ks = 0; ks < DH / 16; ++ks)
-            mma_ss(tmem + x * 128, dQ[x] + koff(ks), dK0 + koff(ks), idesc, ks > 0 ? 1u : 0u);
-          mma_commit(&sm->s_full[x]);
+            if (leader) mma_ss(tmem + x * 128, dQ[x] + koff(ks), dK0 + koff(ks), idesc, ks > 0 ? 1u : 0u);
+          if (leader) mma_commit(&sm->s_full[x]);
         };
         auto pv = [&](int x, int t, uint32_t f) {
           const int s = f % STAGES;
           lap(5);
-          mbar_wait(&sm->p_ready[x], tcnt[x] & 1, abort_flag, p.status);
+          mbar_wait_warp(&sm->p_ready[x], tcnt[x] & 1, abort_flag, p.status);
           lap(2);
-          mbar_wait(&sm->v_full[s], (f / STAGES) & 1, abort_flag, p.status);
+          mbar_wait_warp(&sm->v_full[s], (f / STAGES) & 1, abort_flag, p.status);
           lap(3);
           // the accumulator was last used by the previous item on this query tile: its epilogue must have read it
-          if (t == 0 && ecnt[x] >= 1) mbar_wait(&sm->o_free[x], (ecnt[x] - 1) & 1, abort_flag, p.status);
+          if (t == 0 && ecnt[x] >= 1) mbar_wait_warp(&sm->o_free[x], (ecnt[x] - 1) & 1, abort_flag, p.status);
           lap(4);
           tc_fence_after();
           const int ksteps = (min(BN, it.n_keys - t * BN) + 15) >> 4;
           const uint64_t mV0 = make_smem_desc(smem_u32(sV + s * TILE), PANEL, 1024);
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
-            if (ks < ksteps)   // P of keys 16 ks .. 16 ks + 15 sits in columns 64 + 8 ks .. of the tile's score buffer
+            if (leader && ks < ksteps)   // P of keys 16 ks .. 16 ks + 15 sits in columns 64 + 8 ks .. of the tile's score buffer
               mma_ts(tmem + O_COL + x * 128, tmem + x * 128 + 64 + ks * 8, mV0 + mnoff(ks), IDESC_PV,
                      (t > 0 || ks > 0) ? 1u : 0u);
-          mma_commit(&sm->o_done[x]);
+          if (leader) mma_commit(&sm->o_done[x]);
           tcnt[x] += 1;
         };
         for (int t = 0; t < it.ntiles; ++t) {
           const uint32_t f = fills + t;
           const int s = f % STAGES;
           lap(5);
-          mbar_wait(&sm->k_full[s], (f / STAGES) & 1, abort_flag, p.status);
+          mbar_wait_warp(&sm->k_full[s], (f / STAGES) & 1, abort_flag, p.status);
           lap(1);
           tc_fence_after();
           qk(0, t, s);
           if (it.nx == 2) {
             if (t > 0) {
               pv(1, t - 1, f - 1);
-              mma_commit(&sm->v_empty[(f - 1) % STAGES]);
+              if (leader) mma_commit(&sm->v_empty[(f - 1) % STAGES]);
             }
             qk(1, t, s);
           }
-          mma_commit(&sm->k_empty[s]);
-          if (t == it.ntiles - 1) mma_commit(&sm->q_empty);
+          if (leader) mma_commit(&sm->k_empty[s]);
+          if (leader && t == it.ntiles - 1) mma_commit(&sm->q_empty);
           pv(0, t, f);
-          if (it.nx == 1) mma_commit(&sm->v_empty[s]);
+          if (leader && it.nx == 1) mma_commit(&sm->v_empty[s]);
         }
         if (it.nx == 2) {
           const uint32_t f = fills + it.ntiles - 1;
           pv(1, it.ntiles - 1, f);
-          mma_commit(&sm->v_empty[f % STAGES]);
+          if (leader) mma_commit(&sm->v_empty[f % STAGES]);
         }
         fills += it.ntiles;
         ecnt[0] += 1;
         if (it.nx == 2) ecnt[1] += 1;
       }
       lap(5);
-      tflush(8);
+      if (leader) tflush(8);
     }
   } else if (warp < 4 || warp >= 12) {
     // ------------------------------------------------------------------ loaders: Q rows of the next item
