@@ -172,40 +172,43 @@ dkdv_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       if (*abort_flag && n > 0) mbar_wait(&sm->kv_full, (n - 1) & 1, abort_flag, p.status);
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer: the whole warp walks the loop, one
+    // elected lane issues (warp-uniform control flow; see elect_one)
+    {
+      const bool leader = elect_one();
+      auto wwait = [&](int site, uint64_t* bar, uint32_t parity) { twait(site, bar, parity); __syncwarp(); };
       uint32_t n = 0, u0 = 0;
       const uint64_t dK0 = desc_k0(smem_u32(sK)), dV0 = desc_k0(smem_u32(sV));
       for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
         const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
         if (it.n_units == 0) continue;
-        twait(0, &sm->kv_full, n & 1);
+        wwait(0, &sm->kv_full, n & 1);
         for (int i = 0; i < it.n_units; ++i) {
           const uint32_t u = u0 + i;
           const int cb = u & 1;
-          twait(1, &sm->chunk_full[cb], (u >> 1) & 1);
+          wwait(1, &sm->chunk_full[cb], (u >> 1) & 1);
           tc_fence_after();
           const uint32_t sQ_addr = smem_u32(sC + cb * 2 * TILE);
           const uint64_t dQ0 = desc_k0(sQ_addr), dO0 = desc_k0(sQ_addr + TILE);
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) mma_ss(tmem + ST_COL, dK0 + koff(ks), dQ0 + koff(ks), IDESC_KK, ks > 0 ? 1u : 0u);
+          for (int ks = 0; ks < 8; ++ks) if (leader) mma_ss(tmem + ST_COL, dK0 + koff(ks), dQ0 + koff(ks), IDESC_KK, ks > 0 ? 1u : 0u);
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) mma_ss(tmem + DPT_COL, dV0 + koff(ks), dO0 + koff(ks), IDESC_KK, ks > 0 ? 1u : 0u);
-          mma_commit(&sm->sdp_full);
+          for (int ks = 0; ks < 8; ++ks) if (leader) mma_ss(tmem + DPT_COL, dV0 + koff(ks), dO0 + koff(ks), IDESC_KK, ks > 0 ? 1u : 0u);
+          if (leader) mma_commit(&sm->sdp_full);
           // dV / dK still hold the previous item until its epilogue has read them
-          if (i == 0 && n > 0) twait(3, &sm->acc_free, (n - 1) & 1);
+          if (i == 0 && n > 0) wwait(3, &sm->acc_free, (n - 1) & 1);
           const int rows = (int)min((long long)BM, it.list_hi - it.list_lo - (long long)i * BM);
           const int ksteps = (rows + 15) >> 4;
           const uint64_t mQ0 = desc_mn0(sQ_addr), mO0 = desc_mn0(sQ_addr + TILE);
 #pragma unroll
           for (int gi = 0; gi < 4; ++gi) {
             const int g = group_order(gi);
-            twait(2, &sm->grp_ready[g], u & 1);
+            wwait(2, &sm->grp_ready[g], u & 1);
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < 2; ++kk) {
               const int ks = 2 * g + kk;
-              if (ks < ksteps) {
+              if (leader && ks < ksteps) {
                 const uint32_t first = (i == 0 && gi == 0 && kk == 0) ? 0u : 1u;
                 // P^T / dS^T of queries 32g .. 32g+31 sit in columns 32g .. 32g+15 of their buffer
                 mma_ts(tmem + DV_COL, tmem + ST_COL + 32 * g + 8 * kk, mO0 + mnoff(ks), IDESC_TN, first);
@@ -213,14 +216,14 @@ dkdv_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
               }
             }
           }
-          mma_commit(&sm->chunk_empty[cb]);
+          if (leader) mma_commit(&sm->chunk_empty[cb]);
         }
-        mma_commit(&sm->kv_empty);
-        mma_commit(&sm->acc_done);
+        if (leader) mma_commit(&sm->kv_empty);
+        if (leader) mma_commit(&sm->acc_done);
         u0 += it.n_units;
         ++n;
       }
-      tflush(2, 4);      // [2] kv_full, [3] chunk_full, [4] grp_ready, [5] acc_free, [6] total
+      if (leader) tflush(2, 4);      // [2] kv_full, [3] chunk_full, [4] grp_ready, [5] acc_free, [6] total
     }
   } else if (warp >= 10) {
     // ------------------------------------------------------------------ loaders (8 warps): gather Q / dO units, one ahead
@@ -507,47 +510,49 @@ dq_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       for (uint32_t g = f > 2 ? f - 2 : 0; g < f; ++g) mbar_wait(&sm->kv_full[g & 1], (g >> 1) & 1, abort_flag, p.status);
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer: the whole warp walks the loop, one
+    // elected lane issues (warp-uniform control flow; see elect_one)
+    {
+      const bool leader = elect_one();
       uint32_t n = 0, f = 0;
       const uint64_t dQ0 = desc_k0(smem_u32(sQ)), dO0 = desc_k0(smem_u32(sdO));
       for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
         const DqItem it = dq_decode<DENSE>(p, item);
         const int acc = n & 1;
-        mbar_wait(&sm->qdo_full, n & 1, abort_flag, p.status);
+        mbar_wait_warp(&sm->qdo_full, n & 1, abort_flag, p.status);
         for (int t = 0; t < it.n_units; ++t, ++f) {
           const int s = f & 1;
-          mbar_wait(&sm->kv_full[s], (f >> 1) & 1, abort_flag, p.status);
+          mbar_wait_warp(&sm->kv_full[s], (f >> 1) & 1, abort_flag, p.status);
           tc_fence_after();
           const int n_mma = (min(BN, it.n_keys - t * BN) + 15) & ~15;
           const uint32_t idesc = make_idesc_bf16(BM, n_mma, false, false);
           const uint32_t sK_addr = smem_u32(sKV + s * 2 * TILE);
           const uint64_t dK0 = desc_k0(sK_addr), dV0 = desc_k0(sK_addr + TILE), mK0 = desc_mn0(sK_addr);
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) mma_ss(tmem + S_COL, dQ0 + koff(ks), dK0 + koff(ks), idesc, ks > 0 ? 1u : 0u);
+          for (int ks = 0; ks < 8; ++ks) if (leader) mma_ss(tmem + S_COL, dQ0 + koff(ks), dK0 + koff(ks), idesc, ks > 0 ? 1u : 0u);
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) mma_ss(tmem + DP_COL, dO0 + koff(ks), dV0 + koff(ks), idesc, ks > 0 ? 1u : 0u);
-          mma_commit(&sm->sdp_full);
+          for (int ks = 0; ks < 8; ++ks) if (leader) mma_ss(tmem + DP_COL, dO0 + koff(ks), dV0 + koff(ks), idesc, ks > 0 ? 1u : 0u);
+          if (leader) mma_commit(&sm->sdp_full);
           // this accumulator was last used two items ago: its epilogue must have read it
-          if (t == 0 && n >= 2) mbar_wait(&sm->dq_free[acc], ((n >> 1) - 1) & 1, abort_flag, p.status);
+          if (t == 0 && n >= 2) mbar_wait_warp(&sm->dq_free[acc], ((n >> 1) - 1) & 1, abort_flag, p.status);
           const int ksteps = n_mma >> 4;
 #pragma unroll
           for (int gi = 0; gi < 4; ++gi) {
             const int g = group_order(gi);
-            mbar_wait(&sm->grp_ready[g], f & 1, abort_flag, p.status);
+            mbar_wait_warp(&sm->grp_ready[g], f & 1, abort_flag, p.status);
             tc_fence_after();
 #pragma unroll
             for (int kk = 0; kk < 2; ++kk) {
               const int ks = 2 * g + kk;
-              if (ks < ksteps)
+              if (leader && ks < ksteps)
                 mma_ts(tmem + DQ_COL + acc * 128, tmem + DP_COL + 32 * g + 8 * kk, mK0 + mnoff(ks), IDESC_TN,
                        (t == 0 && gi == 0 && kk == 0) ? 0u : 1u);
             }
           }
-          mma_commit(&sm->kv_empty[s]);
+          if (leader) mma_commit(&sm->kv_empty[s]);
         }
-        mma_commit(&sm->qdo_empty);
-        mma_commit(&sm->dq_done[acc]);
+        if (leader) mma_commit(&sm->qdo_empty);
+        if (leader) mma_commit(&sm->dq_done[acc]);
       }
     }
   } else {

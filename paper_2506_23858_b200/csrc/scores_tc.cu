@@ -144,8 +144,10 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer: the whole warp walks the loop, one
+    // elected lane issues (warp-uniform control flow; see elect_one)
+    {
+      const bool leader = elect_one();
       uint32_t qn = 0, bn = 0;
       long long cur_group = -1;
       const uint32_t idesc = make_idesc_bf16(BM, p.rows_pass, false, false);
@@ -153,14 +155,14 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         const long long group = it / tiles;
         if (group != cur_group) {
           // all MMAs on the previous range were issued before this point: release it to the producer
-          if (cur_group >= 0) mma_commit(&sm->b_empty);
-          mbar_wait(&sm->b_full, bn & 1, abort_flag, p.status);
+          if (leader && cur_group >= 0) mma_commit(&sm->b_empty);
+          mbar_wait_warp(&sm->b_full, bn & 1, abort_flag, p.status);
           cur_group = group;
           ++bn;
         }
         const int s = qn & 1;
-        mbar_wait(&sm->q_full[s], (qn >> 1) & 1, abort_flag, p.status);
-        if (qn >= 2) mbar_wait(&sm->acc_empty[s], ((qn >> 1) - 1) & 1, abort_flag, p.status);
+        mbar_wait_warp(&sm->q_full[s], (qn >> 1) & 1, abort_flag, p.status);
+        if (qn >= 2) mbar_wait_warp(&sm->acc_empty[s], ((qn >> 1) - 1) & 1, abort_flag, p.status);
         tc_fence_after();
         const uint32_t d_tmem = tmem + (s ? 256u : 0u);
         const uint32_t sQ_addr = smem_u32(sQ + s * TILE);
@@ -171,11 +173,11 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           for (int ks = 0; ks < DH / 16; ++ks) {
             const uint64_t a = make_smem_desc(sQ_addr + (ks >> 2) * PANEL + (ks & 3) * 32, 16, 1024);
             const uint64_t b = make_smem_desc(sB_addr + (ks >> 2) * BPANEL + (ks & 3) * 32, 16, 1024);
-            mma_ss(d_tmem, a, b, idesc, (part > 0 || ks > 0) ? 1u : 0u);
+            if (leader) mma_ss(d_tmem, a, b, idesc, (part > 0 || ks > 0) ? 1u : 0u);
           }
         }
-        mma_commit(&sm->q_empty[s]);
-        mma_commit(&sm->acc_full[s]);
+        if (leader) mma_commit(&sm->q_empty[s]);
+        if (leader) mma_commit(&sm->acc_full[s]);
       }
     }
   } else {
