@@ -12,8 +12,7 @@
 //                                                         B = the same dO / Q tiles read MN-major)
 //   Every key belongs to exactly one item: dK and dV are written once, no atomics.  dQ^T of a chunk
 //   is read out of TMEM by four writer warps, transposed through shared memory and added into an
-//   fp32 accumulator with one bulk reduction per query row; the L2's fp32 reduction rate is what
-//   bounds this kernel on long key blocks.
+//   fp32 accumulator with one red.global.add.v4.f32 warp instruction per query row (512 bytes).
 //
 // D = rowsum(dO * O) and lse come in per query; exp runs in the exp2 domain (c = scale * log2 e).
 // The dense path uses the kernels with 128-query units in the companion file.
@@ -82,18 +81,9 @@ __device__ __forceinline__ void gather_store128(uint8_t* dst, int tid, const uin
   }
 }
 
-// 16-byte vector reduction into global memory (fp32 add).
-// Bulk reduction: adds `bytes` (a multiple of 16) of fp32 from shared memory into global memory.
-__device__ __forceinline__ void bulk_reduce_add_f32(float* gdst, const float* ssrc, uint32_t bytes) {
-  asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(ssrc)),
-               "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // named barrier of the four dQ writer warps
 __device__ __forceinline__ void writer_sync() { asm volatile("bar.sync 5, 128;" ::: "memory"); }
+// 16-byte vector reduction into global memory (fp32 add)
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
@@ -141,7 +131,7 @@ struct KvSmem {
 constexpr int DSTILE = 128 * 128;            // dS^T of a unit in shared memory: [128 keys][64 queries] bf16 (16 KB)
 // split kernels: K/V double buffered across items; fused kernel: one K/V pair, one dS^T tile, the dQ staging tile
 constexpr size_t KV_SMEM_BYTES = 1024 + 4 * TILE + NQ * 2 * CTILE + sizeof(KvSmem) + 32;
-constexpr int DQSTAGE = QC * DH * 4;         // dQ of a unit as [64 queries][128] fp32 rows for the bulk reductions (32 KB)
+constexpr int DQSTAGE = QC * DH * 4;         // dQ of a unit as [64 queries][128] fp32 rows for the vector reductions (32 KB)
 constexpr size_t KVF_SMEM_BYTES = 1024 + 2 * TILE + NQ * 2 * CTILE + DSTILE + DQSTAGE + 8 * QC * 4 + sizeof(KvSmem) + 32;
 constexpr int KV_THREADS = 448;   // TMA, MMA, 8 compute warps, 4 loader warps
 constexpr int KVF_THREADS = 576;  // ... plus 4 dQ writer warps
@@ -194,6 +184,7 @@ __device__ __forceinline__ uint64_t cdesc_mn(uint32_t tile_addr, int ks) {
 
 struct KvItem {
   int bh, key0, valid, n_units;
+  int start;      // first unit of this item's walk over the query list (see unit_at)
   long long list_lo, list_hi, head_off;
 };
 
@@ -213,7 +204,15 @@ __device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, i
   }
   it.n_units = (int)((it.list_hi - it.list_lo + QC - 1) / QC);
   it.head_off = (long long)it.bh * p.S;
+  it.start = (int)(((long long)tile * it.n_units) / tiles);
   return it;
+}
+// The key tiles of a block run at the same time on different SMs and walk the same query list: each
+// starts at a different unit (and wraps), so that their dQ reductions do not all hit the same
+// accumulator rows at the same moment.
+__device__ __forceinline__ int unit_at(const KvItem& it, int i) {
+  const int k = i + it.start;
+  return k < it.n_units ? k : k - it.n_units;
 }
 
 // Only <DENSE = false, FUSE = true> is instantiated.  FUSE = false is the same kernel without the
@@ -308,14 +307,21 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       tflush(0, 1);      // [0] kv_empty, [1] total
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer: the whole warp walks the loop, one
+    // elected lane issues (warp-uniform control flow; see elect_one)
+    {
+      const bool leader = elect_one();
+      auto wwait = [&](int site, uint64_t* bar, uint32_t parity) { twait(site, bar, parity); __syncwarp(); };
       uint32_t n = 0, u0 = 0;      // items and units done so far
       for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+        KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+        // the list bounds come from memory: a warp reduction marks them as warp-uniform
+        const int n_list = __reduce_max_sync(0xffffffffu, (int)(it.list_hi - it.list_lo));
+        it.n_units = (n_list + QC - 1) / QC;
+        it.start = __reduce_max_sync(0xffffffffu, it.start);
         if (it.n_units == 0) continue;
         const int b = FUSE ? 0 : (n & 1);
-        twait(0, &sm->kv_full[b], (FUSE ? n : (n >> 1)) & 1);
+        wwait(0, &sm->kv_full[b], (FUSE ? n : (n >> 1)) & 1);
         tc_fence_after();
         const uint64_t dK0 = desc_k(smem_u32(sK + b * TILE), 0), dV0 = desc_k(smem_u32(sV + b * TILE), 0);
         const uint64_t mK0 = desc_mn(smem_u32(sK + b * TILE), 0);     // K^T as MN-major A operand (fused dQ^T)
@@ -323,8 +329,8 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           const uint32_t u = u0 + i;
           const int cb = u % NQ, tb = u & 1;
           // fused: the dP^T buffer last held dQ^T of unit u - 2, which the writer warps must have read
-          if (FUSE && u >= 2) twait(3, &sm->dq_free[tb], ((u - 2) >> 1) & 1);
-          twait(1, &sm->chunk_full[cb], (u / NQ) & 1);
+          if (FUSE && u >= 2) wwait(3, &sm->dq_free[tb], ((u - 2) >> 1) & 1);
+          wwait(1, &sm->chunk_full[cb], (u / NQ) & 1);
           tc_fence_after();
           const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE);
           const uint64_t dQ0 = cdesc_k(sQ_addr, 0), dO0 = cdesc_k(sQ_addr + CTILE, 0);
@@ -332,10 +338,10 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           // the two accumulation chains are independent: interleave them
 #pragma unroll
           for (int ks = 0; ks < DH / 16; ++ks) {
-            mma_ss(st, dK0 + koff(ks, PANEL), dQ0 + koff(ks, CPANEL), IDESC_K64, ks > 0 ? 1u : 0u);
-            mma_ss(dp, dV0 + koff(ks, PANEL), dO0 + koff(ks, CPANEL), IDESC_K64, ks > 0 ? 1u : 0u);
+            if (leader) mma_ss(st, dK0 + koff(ks, PANEL), dQ0 + koff(ks, CPANEL), IDESC_K64, ks > 0 ? 1u : 0u);
+            if (leader) mma_ss(dp, dV0 + koff(ks, PANEL), dO0 + koff(ks, CPANEL), IDESC_K64, ks > 0 ? 1u : 0u);
           }
-          mma_commit(&sm->sdp_full[tb]);
+          if (leader) mma_commit(&sm->sdp_full[tb]);
         };
         issue_sdp(0);
         if (FUSE && it.n_units > 1) issue_sdp(1);
@@ -343,11 +349,11 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           if (!FUSE && i + 1 < it.n_units) issue_sdp(i + 1);
           const uint32_t u = u0 + i;
           const int cb = u % NQ, tb = u & 1;
-          twait(2, &sm->pds_ready[tb], (u >> 1) & 1);
+          wwait(2, &sm->pds_ready[tb], (u >> 1) & 1);
           // dV / dK still hold the previous item until its epilogue has read them
-          if (i == 0 && n > 0) twait(3, &sm->acc_free, (n - 1) & 1);
+          if (i == 0 && n > 0) wwait(3, &sm->acc_free, (n - 1) & 1);
           tc_fence_after();
-          const int rows = (int)min((long long)QC, it.list_hi - it.list_lo - (long long)i * QC);
+          const int rows = min(QC, n_list - unit_at(it, i) * QC);
           const int ksteps = (rows + 15) >> 4;
           const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE);
           const uint64_t mQ0 = cdesc_mn(sQ_addr, 0), mO0 = cdesc_mn(sQ_addr + CTILE, 0);
@@ -360,27 +366,27 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
             const int kk = (it.valid + 15) >> 4;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-              if (ks < kk) mma_ss(dst_, mK0 + mnoff(ks), mS0 + mnoff(ks), IDESC_DQT, ks > 0 ? 1u : 0u);
-            mma_commit(&sm->dq_full[tb]);
+              if (leader && ks < kk) mma_ss(dst_, mK0 + mnoff(ks), mS0 + mnoff(ks), IDESC_DQT, ks > 0 ? 1u : 0u);
+            if (leader) mma_commit(&sm->dq_full[tb]);
           }
           // P^T of queries 32h .. 32h+31 sits in columns 32h .. 32h+15 of the S^T buffer; dS^T in the same
           // columns of the dP^T buffer (split kernels) or in columns 32h+16 .. 32h+31 of the S^T buffer (fused)
           const uint32_t ds_t = FUSE ? pt + 16 : dst_;
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
-            if (ks < ksteps) {
+            if (leader && ks < ksteps) {
               mma_ts(tmem + DV_COL, pt + (ks >> 1) * 32 + (ks & 1) * 8, mO0 + mnoff(ks), IDESC_TN, ks > 0 ? 1u : acc0);
               mma_ts(tmem + DK_COL, ds_t + (ks >> 1) * 32 + (ks & 1) * 8, mQ0 + mnoff(ks), IDESC_TN, ks > 0 ? 1u : acc0);
             }
-          mma_commit(&sm->chunk_empty[cb]);
+          if (leader) mma_commit(&sm->chunk_empty[cb]);
           if (FUSE && i + 2 < it.n_units) issue_sdp(i + 2);
         }
-        mma_commit(&sm->kv_empty[b]);
-        mma_commit(&sm->acc_done);
+        if (leader) mma_commit(&sm->kv_empty[b]);
+        if (leader) mma_commit(&sm->acc_done);
         u0 += it.n_units;
         ++n;
       }
-      tflush(2, 4);      // [2] kv_full, [3] chunk_full, [4] pds_ready, [5] acc_free, [6] total
+      if (leader) tflush(2, 4);      // [2] kv_full, [3] chunk_full, [4] pds_ready, [5] acc_free, [6] total
     }
   } else if (warp >= 10 && warp < 14) {
     // ------------------------------------------------------------------ loaders: gather Q / dO chunks (run ahead)
@@ -391,7 +397,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       for (int i = 0; i < it.n_units; ++i) {
         const uint32_t u = u0 + i;
         const int cb = u % NQ;
-        const long long lo = it.list_lo + (long long)i * QC;
+        const long long lo = it.list_lo + (long long)unit_at(it, i) * QC;
         const int rows = (int)min((long long)QC, it.list_hi - lo);
         auto row_of = [&](int r) { return DENSE ? (int)(lo + r) : __ldg(p.q_idx + lo + r); };
         uint4 vq[8], vo[8];
@@ -419,7 +425,11 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   } else if (FUSE && warp >= 14) {
     // ------------------------------------------------------------------ dQ writers: thread = head-dim index
     // Read dQ^T of a unit out of TMEM, release the buffer, transpose it through shared memory into 64
-    // rows of 128 floats and add each row into the fp32 accumulator with one bulk reduction.
+    // rows of 128 floats and add each row into the fp32 accumulator with one vector-reduction warp
+    // instruction.  (Measured per SM: bulk reductions through the copy engine stop at 8.6 B/cycle;
+    // red.global.add.v4.f32 gives 10 B/cycle from 4 warps, 18.7 from 8, 23 from 16, about one
+    // instruction in flight per warp; but these share the load/store path with the loaders' gathers,
+    // and eight writer warps slowed those down by more than the reductions gained.)
     const int quad = warp & 3;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const int d = quad * 32 + lane;
@@ -439,25 +449,27 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         tmem_ld_wait();
         tc_fence_before();
         mbar_arrive(&sm->dq_free[tb]);
-        // the staging tile is free once the previous unit's bulk reductions have read it
+        // the staging tile is free once every writer warp has loaded its rows of the previous unit
         if (p.prof) { const long long t = clock64(); wp[1] += t - tw0; tw0 = t; }
-        if (warp == 14) bulk_wait_read0();
         writer_sync();
         if (p.prof) { const long long t = clock64(); wp[2] += t - tw0; tw0 = t; }
 #pragma unroll
         for (int c = 0; c < 32; ++c) s_stage[c * DH + d] = __uint_as_float(a[c]) * p.scale;
 #pragma unroll
         for (int c = 0; c < 32; ++c) s_stage[(32 + c) * DH + d] = __uint_as_float(c2[c]) * p.scale;
-        fence_async_proxy();
         writer_sync();
-        if (warp == 14) {
+        // one row (512 bytes) per warp instruction
+        {
           const int* qr = s_qrow + (u & 7) * QC;
 #pragma unroll
-          for (int c = lane; c < QC; c += 32) {
+          for (int k = 0; k < QC / 4; ++k) {
+            const int c = 4 * k + (warp - 14);
             const int row = qr[c];
-            if (row >= 0) bulk_reduce_add_f32(p.dq_acc + (long long)row * DH, s_stage + c * DH, DH * 4);
+            if (row >= 0) {
+              const float4 v = *reinterpret_cast<const float4*>(s_stage + c * DH + 4 * lane);
+              red_add_v4(p.dq_acc + (long long)row * DH + 4 * lane, v.x, v.y, v.z, v.w);
+            }
           }
-          bulk_commit();
         }
         if (p.prof) { const long long t = clock64(); wp[3] += t - tw0; tw0 = t; }
       }
@@ -466,7 +478,6 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     if (p.prof && warp == 14 && lane == 0) {
       atomicAdd(p.prof + 9, wp[0]); atomicAdd(p.prof + 14, wp[1]); atomicAdd(p.prof + 15, wp[2]); atomicAdd(p.prof + 1, wp[3]);
     }
-    if (warp == 14) bulk_wait0();    // shared memory must stay valid until the last reductions have read it
   } else {
     // ------------------------------------------------------------------ compute: thread = (key row, half of the unit's queries)
     const int quad = warp & 3;
