@@ -12,7 +12,8 @@
 //                                                         B = the same dO / Q tiles read MN-major)
 //   Every key belongs to exactly one item: dK and dV are written once, no atomics.  dQ^T of a chunk
 //   is read out of TMEM by four writer warps, transposed through shared memory and added into an
-//   fp32 accumulator with one red.global.add.v4.f32 warp instruction per query row (512 bytes).
+//   fp32 accumulator with one red.global.add.v4.f32 warp instruction per query row (512 bytes), the
+//   rows shared between the writer warps and two helper warps.
 //
 // D = rowsum(dO * O) and lse come in per query; exp runs in the exp2 domain (c = scale * log2 e).
 // The dense path uses the kernels with 128-query units in the companion file.
@@ -81,8 +82,10 @@ __device__ __forceinline__ void gather_store128(uint8_t* dst, int tid, const uin
   }
 }
 
-// named barrier of the four dQ writer warps
-__device__ __forceinline__ void writer_sync() { asm volatile("bar.sync 5, 128;" ::: "memory"); }
+// named barrier of the dQ writer and helper warps
+constexpr int RED_HELPERS = 2;               // warps that only send out staged dQ rows, next to the four writer warps
+constexpr int RED_WARPS = 4 + RED_HELPERS;
+__device__ __forceinline__ void writer_sync() { asm volatile("bar.sync 5, %0;" ::"n"(32 * RED_WARPS) : "memory"); }
 // 16-byte vector reduction into global memory (fp32 add)
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
@@ -134,7 +137,7 @@ constexpr size_t KV_SMEM_BYTES = 1024 + 4 * TILE + NQ * 2 * CTILE + sizeof(KvSme
 constexpr int DQSTAGE = QC * DH * 4;         // dQ of a unit as [64 queries][128] fp32 rows for the vector reductions (32 KB)
 constexpr size_t KVF_SMEM_BYTES = 1024 + 2 * TILE + NQ * 2 * CTILE + DSTILE + DQSTAGE + 8 * QC * 4 + sizeof(KvSmem) + 32;
 constexpr int KV_THREADS = 448;   // TMA, MMA, 8 compute warps, 4 loader warps
-constexpr int KVF_THREADS = 576;  // ... plus 4 dQ writer warps
+constexpr int KVF_THREADS = 576 + 32 * RED_HELPERS;  // ... plus 4 dQ writer warps and the reduction helper warps
 constexpr uint32_t IDESC_K64 = make_idesc_bf16(128, QC, false, false);   // S^T, dP^T: N = 64 queries
 constexpr uint32_t IDESC_DQT = make_idesc_bf16(128, QC, true, true);     // dQ^T = K^T dS^T: both operands MN-major
 
@@ -428,12 +431,37 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     // rows of 128 floats and add each row into the fp32 accumulator with one vector-reduction warp
     // instruction.  (Measured per SM: bulk reductions through the copy engine stop at 8.6 B/cycle;
     // red.global.add.v4.f32 gives 10 B/cycle from 4 warps, 18.7 from 8, 23 from 16, about one
-    // instruction in flight per warp; but these share the load/store path with the loaders' gathers,
-    // and eight writer warps slowed those down by more than the reductions gained.)
+    // instruction in flight per warp; but these share the load/store path with the loaders' gathers:
+    // two helper warps that only send rows pay off, a third or a second set of four writer warps slows
+    // the gathers down by more than the reductions gain.)
     const int quad = warp & 3;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const int d = quad * 32 + lane;
+    const int wi = warp - 14;                      // 0..3 writers, 4.. helpers
+    auto send_rows = [&](uint32_t u) {             // one row (512 bytes) per warp instruction, rows dealt round-robin
+      const int* qr = s_qrow + (u & 7) * QC;
+#pragma unroll
+      for (int c = wi; c < QC; c += RED_WARPS) {
+        const int row = qr[c];
+        if (row >= 0) {
+          const float4 v = *reinterpret_cast<const float4*>(s_stage + c * DH + 4 * lane);
+          red_add_v4(p.dq_acc + (long long)row * DH + 4 * lane, v.x, v.y, v.z, v.w);
+        }
+      }
+    };
     uint32_t u0 = 0;
+    if (wi >= 4) {
+      // helper warps: follow the writers' two barriers per unit and send their share of the staged rows
+      for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+        for (int i = 0; i < it.n_units; ++i) {
+          writer_sync();
+          writer_sync();
+          send_rows(u0 + i);
+        }
+        u0 += it.n_units;
+      }
+    } else {
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
       const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
       for (int i = 0; i < it.n_units; ++i) {
@@ -458,22 +486,11 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
 #pragma unroll
         for (int c = 0; c < 32; ++c) s_stage[(32 + c) * DH + d] = __uint_as_float(c2[c]) * p.scale;
         writer_sync();
-        // one row (512 bytes) per warp instruction
-        {
-          const int* qr = s_qrow + (u & 7) * QC;
-#pragma unroll
-          for (int k = 0; k < QC / 4; ++k) {
-            const int c = 4 * k + (warp - 14);
-            const int row = qr[c];
-            if (row >= 0) {
-              const float4 v = *reinterpret_cast<const float4*>(s_stage + c * DH + 4 * lane);
-              red_add_v4(p.dq_acc + (long long)row * DH + 4 * lane, v.x, v.y, v.z, v.w);
-            }
-          }
-        }
+        send_rows(u);
         if (p.prof) { const long long t = clock64(); wp[3] += t - tw0; tw0 = t; }
       }
       u0 += it.n_units;
+    }
     }
     if (p.prof && warp == 14 && lane == 0) {
       atomicAdd(p.prof + 9, wp[0]); atomicAdd(p.prof + 14, wp[1]); atomicAdd(p.prof + 15, wp[2]); atomicAdd(p.prof + 1, wp[3]);
