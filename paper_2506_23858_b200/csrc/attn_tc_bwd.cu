@@ -86,6 +86,13 @@ __device__ __forceinline__ void gather_store128(uint8_t* dst, int tid, const uin
 constexpr int RED_HELPERS = 2;               // warps that only send out staged dQ rows, next to the four writer warps
 constexpr int RED_WARPS = 4 + RED_HELPERS;
 __device__ __forceinline__ void writer_sync() { asm volatile("bar.sync 5, %0;" ::"n"(32 * RED_WARPS) : "memory"); }
+// Asynchronous 16-byte copy global -> shared (bypassing L1); `bytes` = 16, or 0 to write zeros.
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc, uint32_t bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 // 16-byte vector reduction into global memory (fp32 add)
 __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
@@ -393,19 +400,31 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     }
   } else if (warp >= 10 && warp < 14) {
     // ------------------------------------------------------------------ loaders: gather Q / dO chunks (run ahead)
+    // The rows go from global to shared memory as asynchronous 16-byte copies (no registers, no
+    // st.shared); a unit is published in the next iteration, once its copies have landed.
     const int lt = threadIdx.x - 320;   // 0..127
+    const int chunk = lt & 15, panel = chunk >> 3, cc = chunk & 7;
+    auto publish = [&](uint32_t u) {
+      fence_async_proxy();
+      mbar_arrive(&sm->chunk_full[u % NQ]);
+    };
     uint32_t u0 = 0;
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
       const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+      const __nv_bfloat16* qh = p.q + it.head_off * DH + chunk * 8;
+      const __nv_bfloat16* oh = p.d_o + it.head_off * DH + chunk * 8;
       for (int i = 0; i < it.n_units; ++i) {
         const uint32_t u = u0 + i;
         const int cb = u % NQ;
         const long long lo = it.list_lo + (long long)unit_at(it, i) * QC;
         const int rows = (int)min((long long)QC, it.list_hi - lo);
         auto row_of = [&](int r) { return DENSE ? (int)(lo + r) : __ldg(p.q_idx + lo + r); };
-        uint4 vq[8], vo[8];
-        gather_chunk64(nullptr, p.q + it.head_off * DH, rows, lt, row_of, vq);
-        gather_chunk64(nullptr, p.d_o + it.head_off * DH, rows, lt, row_of, vo);
+        int idx[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int row = (lt >> 4) + 8 * k;
+          idx[k] = row < rows ? row_of(row) : -1;       // -1: padding row, zero-filled
+        }
         float l2 = INFINITY, dd = 0.f;     // padded queries: P = exp2(-inf) = 0
         int qr = -1;
         if (lt < rows) {
@@ -414,16 +433,30 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           dd = p.Dv[G_];
           qr = (int)G_;
         }
+        // the previous unit is published as soon as its copies have landed (this unit's row indices and
+        // scalars are already on their way), not behind this unit's wait for a free ring slot
+        if (u >= 1) {
+          cp_async_wait<0>();
+          publish(u - 1);
+        }
         if (u >= NQ) twait(0, &sm->chunk_empty[cb], ((u / NQ) - 1) & 1);
-        uint8_t* dst = sC + cb * 2 * CTILE;
-        store_chunk64(dst, lt, vq);
-        store_chunk64(dst + CTILE, lt, vo);
+        const uint32_t dst = smem_u32(sC + cb * 2 * CTILE);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int row = (lt >> 4) + 8 * k;
+          const uint32_t off = panel * CPANEL + row * 128 + ((cc ^ (row & 7)) << 4);
+          const long long src = (long long)(idx[k] < 0 ? 0 : idx[k]) * DH;
+          const uint32_t bytes = idx[k] < 0 ? 0u : 16u;
+          cp_async16(dst + off, qh + src, bytes);
+          cp_async16(dst + CTILE + off, oh + src, bytes);
+        }
         if (lt < QC) { sm->lse2[cb][lt] = l2; sm->Dq[cb][lt] = dd; if (FUSE) s_qrow[(u & 7) * QC + lt] = qr; }
-        fence_async_proxy();
-        mbar_arrive(&sm->chunk_full[cb]);
+        cp_async_commit();
       }
       u0 += it.n_units;
     }
+    cp_async_wait<0>();
+    if (u0 >= 1) publish(u0 - 1);
     if (lt == 0) tflush(7, 1);     // [7] chunk_empty, [8] total
   } else if (FUSE && warp >= 14) {
     // ------------------------------------------------------------------ dQ writers: thread = head-dim index
