@@ -557,8 +557,9 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         twait(0, &sm->chunk_full[cb], (u / NQ) & 1);   // publishes lse2 / Dq of this unit
         twait(1, &sm->sdp_full[tb], (u >> 1) & 1);
         tc_fence_after();
-        const float4* lse2 = reinterpret_cast<const float4*>(sm->lse2[cb] + 32 * half);
-        const float4* Dq = reinterpret_cast<const float4*>(sm->Dq[cb] + 32 * half);
+        // lane l holds the log-sum-exp and D of query 32 half + l: one 128-byte load each per warp, handed
+        // round by shuffles (broadcast 16-byte loads from shared memory cost four wavefronts each)
+        const float my_lse2 = sm->lse2[cb][32 * half + lane], my_D = sm->Dq[cb][32 * half + lane];
         const uint32_t st_t = tmem + lane_addr + ST_COL + tb * QC + 32 * half;
         const uint32_t dp_t = tmem + lane_addr + DPT_COL + tb * QC + 32 * half;
         uint32_t sv[32], dv_[32];
@@ -568,7 +569,11 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         uint32_t pk[16], dk_[16];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          const float4 l4 = lse2[e], d4 = Dq[e];
+          float4 l4, d4;
+          l4.x = __shfl_sync(0xffffffffu, my_lse2, 4 * e);     l4.y = __shfl_sync(0xffffffffu, my_lse2, 4 * e + 1);
+          l4.z = __shfl_sync(0xffffffffu, my_lse2, 4 * e + 2); l4.w = __shfl_sync(0xffffffffu, my_lse2, 4 * e + 3);
+          d4.x = __shfl_sync(0xffffffffu, my_D, 4 * e);        d4.y = __shfl_sync(0xffffffffu, my_D, 4 * e + 1);
+          d4.z = __shfl_sync(0xffffffffu, my_D, 4 * e + 2);    d4.w = __shfl_sync(0xffffffffu, my_D, 4 * e + 3);
           const float p0 = ex2(fmaf(__uint_as_float(sv[4 * e]), p.scale_log2, -l4.x));
           const float p1 = ex2(fmaf(__uint_as_float(sv[4 * e + 1]), p.scale_log2, -l4.y));
           const float p2 = ex2(fmaf(__uint_as_float(sv[4 * e + 2]), p.scale_log2, -l4.z));
