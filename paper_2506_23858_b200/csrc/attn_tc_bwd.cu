@@ -338,19 +338,24 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         auto issue_sdp = [&](int i) {
           const uint32_t u = u0 + i;
           const int cb = u % NQ, tb = u & 1;
-          // fused: the dP^T buffer last held dQ^T of unit u - 2, which the writer warps must have read
-          if (FUSE && u >= 2) wwait(3, &sm->dq_free[tb], ((u - 2) >> 1) & 1);
           wwait(1, &sm->chunk_full[cb], (u / NQ) & 1);
           tc_fence_after();
           const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE);
           const uint64_t dQ0 = cdesc_k(sQ_addr, 0), dO0 = cdesc_k(sQ_addr + CTILE, 0);
           const uint32_t st = tmem + ST_COL + tb * QC, dp = tmem + DPT_COL + tb * QC;
-          // the two accumulation chains are independent: interleave them
+          // S^T first: its buffer is free (the MMAs that read P^T / dS^T of unit u - 2 were issued before),
+          // while the dP^T buffer last held dQ^T of unit u - 2, which the writer warps must have read;
+          // that hand-off completes behind the eight S^T MMAs instead of stalling the issue
 #pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks) {
+          for (int ks = 0; ks < DH / 16; ++ks)
             if (leader) mma_ss(st, dK0 + koff(ks, PANEL), dQ0 + koff(ks, CPANEL), IDESC_K64, ks > 0 ? 1u : 0u);
-            if (leader) mma_ss(dp, dV0 + koff(ks, PANEL), dO0 + koff(ks, CPANEL), IDESC_K64, ks > 0 ? 1u : 0u);
+          if (FUSE && u >= 2) {
+            wwait(3, &sm->dq_free[tb], ((u - 2) >> 1) & 1);
+            tc_fence_after();
           }
+#pragma unroll
+          for (int ks = 0; ks < DH / 16; ++ks)
+            if (leader) mma_ss(dp, dV0 + koff(ks, PANEL), dO0 + koff(ks, CPANEL), IDESC_K64, ks > 0 ? 1u : 0u);
           if (leader) mma_commit(&sm->sdp_full[tb]);
         };
         issue_sdp(0);
