@@ -2,7 +2,7 @@
 // VMoBA (mask constant).  One persistent kernel (one CTA per SM), key-stationary:
 //
 //   Item = 128 keys of one key block.  The K and V tiles stay in shared memory; the queries that
-//   selected the block stream through in gathered chunks of 64 (Q and dO rows, 3-deep ring).  Per
+//   selected the block stream through in gathered chunks of 64 (Q and dO rows, 4-deep ring).  Per
 //   chunk, with keys on the TMEM lanes:
 //     S^T = K Q^T,  dP^T = V dO^T                        (two SS MMAs, N = 64)
 //     P^T = exp2(c S^T - lse),  dS^T = P^T (dP^T - D)    (threads = key rows)
@@ -11,9 +11,9 @@
 //     dV += P^T dO,  dK += dS^T Q                        (two TS MMAs, A = bf16 P^T / dS^T in TMEM;
 //                                                         B = the same dO / Q tiles read MN-major)
 //   Every key belongs to exactly one item: dK and dV are written once, no atomics.  dQ^T of a chunk
-//   is read out of TMEM by four writer warps, transposed through shared memory and added into an
-//   fp32 accumulator with one red.global.add.v4.f32 warp instruction per query row (512 bytes), the
-//   rows shared between the writer warps and two helper warps.
+//   is read out of TMEM by four writer warps, transposed through shared memory (32 queries at a
+//   time) and added into an fp32 accumulator with one red.global.add.v4.f32 warp instruction per query
+//   row (512 bytes), the rows shared between the writer warps and two helper warps.
 //
 // D = rowsum(dO * O) and lse come in per query; exp runs in the exp2 domain (c = scale * log2 e).
 // The dense path uses the kernels with 128-query units in the companion file.
@@ -116,14 +116,14 @@ __device__ __forceinline__ uint64_t desc_mn(uint32_t tile_addr, int ks) {
 // ==========================================================================================
 // dK / dV
 // ==========================================================================================
-// Units of 64 queries flow through a 3-deep ring of gathered (Q, dO) chunks; S^T / dP^T are double
+// Units of 64 queries flow through a ring of gathered (Q, dO) chunks; S^T / dP^T are double
 // buffered in TMEM (64 columns each), so the tensor pipe computes unit u+1 while the compute warps
 // turn unit u into P^T / dS^T.  K and V tiles are double buffered across items, and the loader and
 // TMA warps run ahead of the MMA warp across item boundaries.
 constexpr int QC = 64;                       // queries per unit
 constexpr int CPANEL = QC * 128;             // bytes of one 64-column panel of a 64-row chunk (8 KB)
 constexpr int CTILE = 2 * CPANEL;            // [64 x 128] bf16 (16 KB)
-constexpr int NQ = 3;                        // chunk ring depth
+constexpr int NQ = 4;                        // chunk ring depth
 struct KvSmem {
   uint64_t kv_full[2], kv_empty[2];          // K+V tiles of an item (TMA / commit)
   uint64_t chunk_full[NQ], chunk_empty[NQ];  // gathered Q/dO chunk (128 loader arrivals / commit)
@@ -141,8 +141,10 @@ struct KvSmem {
 constexpr int DSTILE = 128 * 128;            // dS^T of a unit in shared memory: [128 keys][64 queries] bf16 (16 KB)
 // split kernels: K/V double buffered across items; fused kernel: one K/V pair, one dS^T tile, the dQ staging tile
 constexpr size_t KV_SMEM_BYTES = 1024 + 4 * TILE + NQ * 2 * CTILE + sizeof(KvSmem) + 32;
-constexpr int DQSTAGE = QC * DH * 4;         // dQ of a unit as [64 queries][128] fp32 rows for the vector reductions (32 KB)
-constexpr size_t KVF_SMEM_BYTES = 1024 + 2 * TILE + NQ * 2 * CTILE + DSTILE + DQSTAGE + 8 * QC * 4 + sizeof(KvSmem) + 32;
+constexpr int DQSTAGE = (QC / 2) * DH * 4;   // dQ of half a unit as [32 queries][128] fp32 rows for the vector reductions (16 KB)
+// no alignment slack: the kernel checks that its dynamic shared memory starts on a 1024-byte boundary
+constexpr size_t KVF_SMEM_BYTES = 2 * TILE + NQ * 2 * CTILE + DSTILE + DQSTAGE + sizeof(KvSmem) + 32;
+static_assert(KVF_SMEM_BYTES <= 232448, "fused backward: shared memory");
 constexpr int KV_THREADS = 448;   // TMA, MMA, 8 compute warps, 4 loader warps
 constexpr int KVF_THREADS = 576 + 32 * RED_HELPERS;  // ... plus 4 dQ writer warps and the reduction helper warps
 constexpr uint32_t IDESC_K64 = make_idesc_bf16(128, QC, false, false);   // S^T, dP^T: N = 64 queries
@@ -232,15 +234,19 @@ template <bool DENSE, bool FUSE>
 __global__ void __launch_bounds__(FUSE ? KVF_THREADS : KV_THREADS, 1)
 attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const KvParams p) {
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // the swizzled tiles need 1024-byte alignment; the fused variant has no room for alignment slack
+  if (FUSE && (smem_u32(smem_raw) & 1023u) != 0) {
+    if (threadIdx.x == 0) set_status(p.status, VMOBA_ERR_CUDA);
+    return;
+  }
+  uint8_t* base = FUSE ? smem_raw : reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int KVB = FUSE ? 1 : 2;    // K/V buffers
   uint8_t* sK = base;                  // [KVB][TILE]
   uint8_t* sV = base + KVB * TILE;     // [KVB][TILE]
   uint8_t* sC = base + 2 * KVB * TILE; // [NQ][Q chunk | dO chunk]
   uint8_t* sDS = sC + NQ * 2 * CTILE;  // fused variant: dS^T of the current unit [DSTILE]
-  float* s_stage = reinterpret_cast<float*>(sDS + DSTILE);                         // fused variant: [QC][DH] fp32
-  int* s_qrow = reinterpret_cast<int*>(sDS + DSTILE + DQSTAGE);                    // fused variant: [unit % 8][query] accumulator row, -1 = padding
-  KvSmem* sm = reinterpret_cast<KvSmem*>(sDS + (FUSE ? DSTILE + DQSTAGE + 8 * QC * 4 : 0));
+  float* s_stage = reinterpret_cast<float*>(sDS + DSTILE);                         // fused variant: [QC / 2][DH] fp32
+  KvSmem* sm = reinterpret_cast<KvSmem*>(sDS + (FUSE ? DSTILE + DQSTAGE : 0));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm->abort_flag;
   // diagnostics: cycles spent in each wait site by one representative thread per role
@@ -431,12 +437,10 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           idx[k] = row < rows ? row_of(row) : -1;       // -1: padding row, zero-filled
         }
         float l2 = INFINITY, dd = 0.f;     // padded queries: P = exp2(-inf) = 0
-        int qr = -1;
         if (lt < rows) {
           const long long G_ = it.head_off + row_of(lt);
           l2 = p.lse[G_] * LOG2E;
           dd = p.Dv[G_];
-          qr = (int)G_;
         }
         // the previous unit is published as soon as its copies have landed (this unit's row indices and
         // scalars are already on their way), not behind this unit's wait for a free ring slot
@@ -455,7 +459,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           cp_async16(dst + off, qh + src, bytes);
           cp_async16(dst + CTILE + off, oh + src, bytes);
         }
-        if (lt < QC) { sm->lse2[cb][lt] = l2; sm->Dq[cb][lt] = dd; if (FUSE) s_qrow[(u & 7) * QC + lt] = qr; }
+        if (lt < QC) { sm->lse2[cb][lt] = l2; sm->Dq[cb][lt] = dd; }
         cp_async_commit();
       }
       u0 += it.n_units;
@@ -476,26 +480,43 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     const int d = quad * 32 + lane;
     const int wi = warp - 14;                      // 0..3 writers, 4.. helpers
-    auto send_rows = [&](uint32_t u) {             // one row (512 bytes) per warp instruction, rows dealt round-robin
-      const int* qr = s_qrow + (u & 7) * QC;
+    constexpr int HR = QC / 2;                     // rows staged at a time
+    constexpr int RPW = (HR + RED_WARPS - 1) / RED_WARPS;   // rows of a half per warp, at most
+    // accumulator rows of this warp's share of a unit (row c = 32 h + wi + RED_WARPS k of the unit), -1 beyond the list
+    auto my_rows = [&](const KvItem& it, int i, int (&rowi)[2][RPW]) {
+      const long long lo = it.list_lo + (long long)unit_at(it, i) * QC;
+      const int rows = (int)min((long long)QC, it.list_hi - lo);
 #pragma unroll
-      for (int c = wi; c < QC; c += RED_WARPS) {
-        const int row = qr[c];
-        if (row >= 0) {
-          const float4 v = *reinterpret_cast<const float4*>(s_stage + c * DH + 4 * lane);
-          red_add_v4(p.dq_acc + (long long)row * DH + 4 * lane, v.x, v.y, v.z, v.w);
+      for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int k = 0; k < RPW; ++k) {
+          const int c = HR * h + wi + RED_WARPS * k;
+          rowi[h][k] = (wi + RED_WARPS * k < HR && c < rows) ? (int)it.head_off + (DENSE ? (int)(lo + c) : __ldg(p.q_idx + lo + c)) : -1;
+        }
+    };
+    auto send_rows = [&](int h, const int (&rowi)[2][RPW]) {     // one row (512 bytes) per warp instruction
+#pragma unroll
+      for (int k = 0; k < RPW; ++k) {
+        if (rowi[h][k] >= 0) {
+          const float4 v = *reinterpret_cast<const float4*>(s_stage + (wi + RED_WARPS * k) * DH + 4 * lane);
+          red_add_v4(p.dq_acc + (long long)rowi[h][k] * DH + 4 * lane, v.x, v.y, v.z, v.w);
         }
       }
     };
     uint32_t u0 = 0;
     if (wi >= 4) {
-      // helper warps: follow the writers' two barriers per unit and send their share of the staged rows
+      // helper warps: follow the writers' barriers (two per half unit) and send their share of the staged rows
       for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
         const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
         for (int i = 0; i < it.n_units; ++i) {
-          writer_sync();
-          writer_sync();
-          send_rows(u0 + i);
+          int rowi[2][RPW];
+          my_rows(it, i, rowi);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            writer_sync();
+            writer_sync();
+            send_rows(h, rowi);
+          }
         }
         u0 += it.n_units;
       }
@@ -505,6 +526,8 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       for (int i = 0; i < it.n_units; ++i) {
         const uint32_t u = u0 + i;
         const int tb = u & 1;
+        int rowi[2][RPW];
+        my_rows(it, i, rowi);
         long long tw0 = p.prof ? clock64() : 0;
         mbar_wait(&sm->dq_full[tb], (u >> 1) & 1, abort_flag, p.status);
         if (p.prof) { const long long t = clock64(); wp[0] += t - tw0; tw0 = t; }
@@ -515,16 +538,20 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         tmem_ld_wait();
         tc_fence_before();
         mbar_arrive(&sm->dq_free[tb]);
-        // the staging tile is free once every writer warp has loaded its rows of the previous unit
         if (p.prof) { const long long t = clock64(); wp[1] += t - tw0; tw0 = t; }
+        // first half of the unit's queries; the staging tile is free once every warp has loaded its rows of the previous half
         writer_sync();
         if (p.prof) { const long long t = clock64(); wp[2] += t - tw0; tw0 = t; }
 #pragma unroll
         for (int c = 0; c < 32; ++c) s_stage[c * DH + d] = __uint_as_float(a[c]) * p.scale;
-#pragma unroll
-        for (int c = 0; c < 32; ++c) s_stage[(32 + c) * DH + d] = __uint_as_float(c2[c]) * p.scale;
         writer_sync();
-        send_rows(u);
+        send_rows(0, rowi);
+        // second half
+        writer_sync();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) s_stage[c * DH + d] = __uint_as_float(c2[c]) * p.scale;
+        writer_sync();
+        send_rows(1, rowi);
         if (p.prof) { const long long t = clock64(); wp[3] += t - tw0; tw0 = t; }
       }
       u0 += it.n_units;
