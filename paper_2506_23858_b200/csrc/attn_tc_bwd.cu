@@ -196,7 +196,6 @@ __device__ __forceinline__ uint64_t cdesc_mn(uint32_t tile_addr, int ks) {
 
 struct KvItem {
   int bh, key0, valid, n_units;
-  int start;      // first unit of this item's walk over the query list (see unit_at)
   long long list_lo, list_hi, head_off;
 };
 
@@ -216,15 +215,7 @@ __device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, i
   }
   it.n_units = (int)((it.list_hi - it.list_lo + QC - 1) / QC);
   it.head_off = (long long)it.bh * p.S;
-  it.start = (int)(((long long)tile * it.n_units) / tiles);
   return it;
-}
-// The key tiles of a block run at the same time on different SMs and walk the same query list: each
-// starts at a different unit (and wraps), so that their dQ reductions do not all hit the same
-// accumulator rows at the same moment.
-__device__ __forceinline__ int unit_at(const KvItem& it, int i) {
-  const int k = i + it.start;
-  return k < it.n_units ? k : k - it.n_units;
 }
 
 // Only <DENSE = false, FUSE = true> is instantiated.  FUSE = false is the same kernel without the
@@ -334,7 +325,6 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         // the list bounds come from memory: a warp reduction marks them as warp-uniform
         const int n_list = __reduce_max_sync(0xffffffffu, (int)(it.list_hi - it.list_lo));
         it.n_units = (n_list + QC - 1) / QC;
-        it.start = __reduce_max_sync(0xffffffffu, it.start);
         if (it.n_units == 0) continue;
         const int b = FUSE ? 0 : (n & 1);
         wwait(0, &sm->kv_full[b], (FUSE ? n : (n >> 1)) & 1);
@@ -374,7 +364,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           // dV / dK still hold the previous item until its epilogue has read them
           if (i == 0 && n > 0) wwait(3, &sm->acc_free, (n - 1) & 1);
           tc_fence_after();
-          const int rows = min(QC, n_list - unit_at(it, i) * QC);
+          const int rows = min(QC, n_list - i * QC);
           const int ksteps = (rows + 15) >> 4;
           const uint32_t sQ_addr = smem_u32(sC + cb * 2 * CTILE);
           const uint64_t mQ0 = cdesc_mn(sQ_addr, 0), mO0 = cdesc_mn(sQ_addr + CTILE, 0);
@@ -427,7 +417,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       for (int i = 0; i < it.n_units; ++i) {
         const uint32_t u = u0 + i;
         const int cb = u % NQ;
-        const long long lo = it.list_lo + (long long)unit_at(it, i) * QC;
+        const long long lo = it.list_lo + (long long)i * QC;
         const int rows = (int)min((long long)QC, it.list_hi - lo);
         auto row_of = [&](int r) { return DENSE ? (int)(lo + r) : __ldg(p.q_idx + lo + r); };
         int idx[8];
@@ -484,7 +474,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     constexpr int RPW = (HR + RED_WARPS - 1) / RED_WARPS;   // rows of a half per warp, at most
     // accumulator rows of this warp's share of a unit (row c = 32 h + wi + RED_WARPS k of the unit), -1 beyond the list
     auto my_rows = [&](const KvItem& it, int i, int (&rowi)[2][RPW]) {
-      const long long lo = it.list_lo + (long long)unit_at(it, i) * QC;
+      const long long lo = it.list_lo + (long long)i * QC;
       const int rows = (int)min((long long)QC, it.list_hi - lo);
 #pragma unroll
       for (int h = 0; h < 2; ++h)
