@@ -239,6 +239,7 @@ merge_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pairs, lon
         }
         tot += my_w;
         const int m = (int)min((long long)32, hi - i0);
+#pragma unroll 4
         for (int k = 0; k < m; ++k) {
           const long long pos = __shfl_sync(0xffffffffu, my_pos, k);
           const float wgt = __shfl_sync(0xffffffffu, my_w, k);
