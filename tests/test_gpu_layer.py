@@ -124,6 +124,18 @@ def test_mid_size_layer_forward_backward(block):
             _check_head(w, data, res, b, h, rng, n_rows=400, n_blocks=3, with_bwd=True)
 
 
+@pytest.mark.parametrize("grid,block", [((6, 9, 20), (3, 9, 10)), ((4, 43, 3), (1, 43, 3)), ((2, 16, 32), (1, 16, 16))],
+                         ids=["270keys_tail14", "129keys_tail1", "256keys_no_tail"])
+def test_key_block_tails_forward_backward(grid, block):
+    """Key blocks whose last 128-key tile holds 14 keys (the 720p 3D blocks), one key, or is full."""
+    w = gen.Workload("tails", 1, 2, 128, grid[0], grid[1], grid[2], block, 0.25, "bf16", "smooth", 11)
+    data = gen.make_inputs(w)
+    res = _run_layer(w, data, with_bwd=True)
+    rng = np.random.default_rng(2)
+    for h in range(w.heads):
+        _check_head(w, data, res, 0, h, rng, n_rows=min(400, w.S), n_blocks=min(3, w.n_blocks), with_bwd=True)
+
+
 def test_mid_size_threshold_one_equals_dense_path():
     """tau = 1.0 through the sparse pipeline must equal the library's dense path and the oracle's dense attention."""
     w = MID.with_(tau=1.0, B=1, heads=2)
