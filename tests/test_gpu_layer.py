@@ -136,6 +136,21 @@ def test_key_block_tails_forward_backward(grid, block):
         _check_head(w, data, res, 0, h, rng, n_rows=min(400, w.S), n_blocks=min(3, w.n_blocks), with_bwd=True)
 
 
+@pytest.mark.parametrize("block", [(1, 12, 26), (3, 6, 13)], ids=["1d", "3d"])
+def test_wide_logit_range_forward_backward(block):
+    """Queries four times larger (exact in bf16): logits spread over tens of units, so the running maximum
+    of a row moves by more than the lazy-rescale threshold between key tiles and the accumulator is rescaled."""
+    w = MID.with_(block=block, B=1, heads=2)
+    data = gen.make_inputs(w)
+    data["q"] = data["q"] * 4.0
+    data["q_bits"] = gen.f32_to_bf16_bits(data["q"])
+    assert np.array_equal(gen.bf16_bits_to_f32(data["q_bits"]), data["q"])
+    res = _run_layer(w, data, with_bwd=True)
+    rng = np.random.default_rng(3)
+    for h in range(w.heads):
+        _check_head(w, data, res, 0, h, rng, n_rows=400, n_blocks=3, with_bwd=True)
+
+
 def test_mid_size_threshold_one_equals_dense_path():
     """tau = 1.0 through the sparse pipeline must equal the library's dense path and the oracle's dense attention."""
     w = MID.with_(tau=1.0, B=1, heads=2)
