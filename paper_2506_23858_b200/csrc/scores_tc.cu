@@ -8,8 +8,11 @@
 //
 // Persistent CTAs walk (head, block range, 128-query tile) items: the three centroid parts of
 // the block range stay in shared memory, query tiles stream through a 2-stage TMA ring, the
-// accumulator is double buffered in TMEM so that the epilogue (thread = query row, coalesced in
-// time fp32 stores of the [S, N_b] matrix -- the HBM-bound part) overlaps the next tile's MMAs.
+// accumulator is double buffered in TMEM so that the epilogue (the fp32 stores of the [S, N_b]
+// matrix -- the HBM-bound part) overlaps the next tile's MMAs.  The epilogue threads (thread = query
+// row) put 32 columns at a time into a swizzled shared-memory slab and one TMA store writes the slab
+// as full 128-byte row segments; when rows are not 16-byte multiples (N_b % 4 != 0) each thread
+// stores its own row instead.
 #include <algorithm>
 
 #include "sm100.cuh"
@@ -36,12 +39,14 @@ struct Smem {
 // B parts: 3 x (two 64-column panels of NT_MAX rows x 128 bytes)
 constexpr int BPANEL = NT_MAX * 128;
 constexpr int BPART = 2 * BPANEL;
-constexpr size_t SMEM_BYTES = 1024 + 2 * TILE + 3 * BPART + sizeof(Smem) + 64;
+constexpr int SLAB = BM * 128;            // 128 rows x 32 fp32 columns (16 KB), two of them
+constexpr size_t SMEM_BYTES = 1024 + 2 * TILE + 3 * BPART + 2 * SLAB + sizeof(Smem) + 64;
 
 struct Params {
   float* scores;
   int S, Nb, Nb_pad, BH;
   int n_pass, rows_pass;    // block ranges per head, rows per range (multiple of 16, <= NT_MAX)
+  int tma_store;            // rows are multiples of 16 bytes: the epilogue writes through tmS
   int32_t* status;
 };
 
@@ -68,12 +73,14 @@ split_centroids_kernel(const float* __restrict__ cent, __nv_bfloat16* __restrict
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
-scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmB, const Params p) {
+scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmB,
+                 const __grid_constant__ CUtensorMap tmS, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = base;                    // [2][TILE]
   uint8_t* sB = base + 2 * TILE;         // [3][BPART]
-  Smem* sm = reinterpret_cast<Smem*>(sB + 3 * BPART);
+  uint8_t* sOut = sB + 3 * BPART;        // [2][SLAB]; BPART is a multiple of 1024
+  Smem* sm = reinterpret_cast<Smem*>(sOut + 2 * SLAB);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm->abort_flag;
 
@@ -185,7 +192,7 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int quad = warp & 3;
     const int r = quad * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    uint32_t qn = 0;
+    uint32_t qn = 0, slabs = 0;
     for (long long it = it0; it < it1; ++it, ++qn) {
       const int tile = (int)(it % tiles);
       const long long group = it / tiles;
@@ -199,29 +206,45 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const int ncols = min(p.rows_pass, p.Nb - j0);       // real blocks in this range
       float* out = p.scores + ((long long)bh * p.S + row) * p.Nb + j0;
       const uint32_t a_tmem = tmem + lane_addr + (s ? 256u : 0u);
+      if (p.tma_store) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < p.rows_pass; c0 += 32) {
+          if (j0 + c0 >= p.Nb) break;                         // the remaining slabs are padding (uniform)
+          uint32_t v[32];
+          tmem_ld32(a_tmem + c0, v);
+          tmem_ld_wait();
+          uint8_t* slab = sOut + (slabs & 1) * SLAB;
+          // the slab's previous store (two slabs ago) must have read it
+          if (threadIdx.x == 64) bulk_wait_group_read<1>();
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            *reinterpret_cast<uint4*>(slab + r * 128 + ((i ^ (r & 7)) << 4)) = make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          fence_async_proxy();
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (threadIdx.x == 64) {
+            tma_store_3d(&tmS, slab, j0 + c0, tile * BM, (int)bh);   // rows beyond S and columns beyond N_b are clipped
+            bulk_commit_group();
+          }
+          ++slabs;
+        }
+      } else {
 #pragma unroll 1
       for (int c0 = 0; c0 < p.rows_pass; c0 += 32) {
         uint32_t v[32];
         tmem_ld32(a_tmem + c0, v);
         tmem_ld_wait();
         if (row < p.S) {
-          if ((p.Nb & 3) == 0) {
-            // rows start 16-byte aligned: 4 scores per store
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              if (c0 + i < ncols)     // ncols is a multiple of 4 here
-                *reinterpret_cast<float4*>(out + c0 + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
-                                                                       __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (c0 + i < ncols) out[c0 + i] = __uint_as_float(v[i]);
-          }
+          for (int i = 0; i < 32; ++i)
+            if (c0 + i < ncols) out[c0 + i] = __uint_as_float(v[i]);
         }
+      }
       }
       tc_fence_before();
       mbar_arrive(&sm->acc_empty[s]);
     }
+    if (threadIdx.x == 64) bulk_wait_group<0>();      // shared memory must outlive the last stores' reads
   }
   tc_fence_before();
   __syncthreads();
@@ -231,7 +254,7 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 }  // namespace sct
 
 size_t scores_tc_ws_bytes(const Dims& D) {
-  const size_t Nb_pad = (size_t)(D.Nb + 15) / 16 * 16;
+  const size_t Nb_pad = (size_t)(D.Nb + 31) / 32 * 32;
   return 3 * (size_t)D.BH * Nb_pad * sct::DH * sizeof(__nv_bfloat16) + 1024;
 }
 
@@ -239,22 +262,30 @@ size_t scores_tc_ws_bytes(const Dims& D) {
 int scores_tc(const Dims& D, const void* q_bm, const float* cent, float* scores, void* ws, int32_t* status,
               cudaStream_t st) {
   using namespace sct;
-  const int Nb_pad = (D.Nb + 15) / 16 * 16;
+  // ranges of whole 32-column slabs (the epilogue's store unit)
+  const int Nb_pad = (D.Nb + 31) / 32 * 32;
   const int n_pass = (Nb_pad + NT_MAX - 1) / NT_MAX;
-  int rows_pass = ((Nb_pad + n_pass - 1) / n_pass + 15) / 16 * 16;
+  const int rows_pass = ((Nb_pad + n_pass - 1) / n_pass + 31) / 32 * 32;
   __nv_bfloat16* parts = reinterpret_cast<__nv_bfloat16*>((reinterpret_cast<uintptr_t>(ws) + 1023) & ~uintptr_t(1023));
   const long long n = (long long)D.BH * Nb_pad * DH;
   split_centroids_kernel<<<(int)std::min<long long>((n + 255) / 256, 148 * 8), 256, 0, st>>>(cent, parts, D.Nb, Nb_pad, D.BH);
-  CUtensorMap tmQ, tmB;
+  CUtensorMap tmQ, tmB, tmS;
+  const int tma_store = (D.Nb % 4 == 0) && (reinterpret_cast<uintptr_t>(scores) % 16 == 0);
+  if (tma_store) {
+    if (!sm100::make_tmap_f32_planes(&tmS, scores, (uint64_t)D.BH, (uint64_t)D.S, (uint64_t)D.Nb, BM)) return VMOBA_ERR_CUDA;
+  } else {
+    tmS = CUtensorMap{};
+  }
   if (!sm100::make_tmap_bf16_rows(&tmQ, q_bm, (uint64_t)D.BH * D.S, DH, BM) ||
       !sm100::make_tmap_bf16_rows(&tmB, parts, (uint64_t)3 * D.BH * Nb_pad, DH, rows_pass))
     return VMOBA_ERR_CUDA;
   Params p;
   p.scores = scores; p.S = D.S; p.Nb = D.Nb; p.Nb_pad = Nb_pad; p.BH = D.BH; p.n_pass = n_pass; p.rows_pass = rows_pass;
+  p.tma_store = tma_store;
   p.status = status;
   VMOBA_CUDA_OK(cudaFuncSetAttribute(scores_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
   const long long items = (long long)D.BH * n_pass * ((D.S + BM - 1) / BM);
-  scores_tc_kernel<<<(int)std::max<long long>(1, std::min<long long>(items, 148)), THREADS, SMEM_BYTES, st>>>(tmQ, tmB, p);
+  scores_tc_kernel<<<(int)std::max<long long>(1, std::min<long long>(items, 148)), THREADS, SMEM_BYTES, st>>>(tmQ, tmB, tmS, p);
   VMOBA_LAUNCH_OK(2);
   return VMOBA_OK;
 }
