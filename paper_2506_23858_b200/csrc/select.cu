@@ -322,11 +322,17 @@ mark_kernel(const float* __restrict__ scores, const HeadState* __restrict__ st, 
   __syncthreads();
   const float* base = scores + ((long long)bh * S + q0) * Nb;
   const long long n = (long long)nq * Nb;
+  // (query, block) of element i of the segment by reciprocal: i < QSEG * Nb < 2^23, and (i + 0.5) / Nb is at
+  // least 0.5 / Nb away from an integer, the rounding error far less (a fix-up step covers the rest)
+  const float inv_nb = 1.0f / (float)Nb;
   auto mark = [&](long long i, float s) {
-    int ii = (int)i;
-    int ql = ii / Nb, j = ii - ql * Nb;
+    const bool sel = float_key(s) >= cutoff;
+    if (!sel && own_sb <= 0) return;          // the common case: no index arithmetic at all
+    const int ii = (int)i;
+    int ql = (int)(((float)ii + 0.5f) * inv_nb), j = ii - ql * Nb;
+    if (j < 0) { --ql; j += Nb; } else if (j >= Nb) { ++ql; j -= Nb; }     // belt and braces for huge Nb
     // own_sb > 0: a query also keeps the block it lies in (block-major position / tokens per block)
-    if (float_key(s) >= cutoff || (own_sb > 0 && (q0 + ql) / own_sb == j)) {
+    if (sel || (q0 + ql) / own_sb == j) {
       atomicOr(&s_mask[ql * mw + (j >> 5)], 1u << (j & 31));
       atomicOr(&s_tm[j * TW + (ql >> 5)], 1u << (ql & 31));
       atomicAdd(&s_cnt[j], 1);
