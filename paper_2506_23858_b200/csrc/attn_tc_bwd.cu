@@ -158,6 +158,7 @@ struct KvParams {
   float scale, scale_log2;
   long long capacity;
   __nv_bfloat16 *dk, *dv;
+  int dkv_32;                  // dk and dv are 32-byte aligned: rows go out with 32-byte stores
   float* dq_acc;               // fused variant: fp32 [queries][head_dim], zeroed rows of all selecting queries
   int32_t* status;
   unsigned long long* prof;    // optional wait-time counters (diagnostics), or null
@@ -638,18 +639,22 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         tmem_ld_wait();
         if (r < it.valid) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 8) {       // eight bf16 = one 16-byte store
-            uint4 hv, hk;
-            hv.x = pack_bf16(__uint_as_float(a[i]), __uint_as_float(a[i + 1]));
-            hv.y = pack_bf16(__uint_as_float(a[i + 2]), __uint_as_float(a[i + 3]));
-            hv.z = pack_bf16(__uint_as_float(a[i + 4]), __uint_as_float(a[i + 5]));
-            hv.w = pack_bf16(__uint_as_float(a[i + 6]), __uint_as_float(a[i + 7]));
-            hk.x = pack_bf16(__uint_as_float(bb[i]) * p.scale, __uint_as_float(bb[i + 1]) * p.scale);
-            hk.y = pack_bf16(__uint_as_float(bb[i + 2]) * p.scale, __uint_as_float(bb[i + 3]) * p.scale);
-            hk.z = pack_bf16(__uint_as_float(bb[i + 4]) * p.scale, __uint_as_float(bb[i + 5]) * p.scale);
-            hk.w = pack_bf16(__uint_as_float(bb[i + 6]) * p.scale, __uint_as_float(bb[i + 7]) * p.scale);
-            *reinterpret_cast<uint4*>(dv_row + cgrp * 32 + i) = hv;
-            *reinterpret_cast<uint4*>(dk_row + cgrp * 32 + i) = hk;
+          for (int i = 0; i < 32; i += 16) {      // sixteen bf16 = one 32-byte store (two 16-byte stores if unaligned)
+            uint32_t hv[8], hk[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              hv[k] = pack_bf16(__uint_as_float(a[i + 2 * k]), __uint_as_float(a[i + 2 * k + 1]));
+              hk[k] = pack_bf16(__uint_as_float(bb[i + 2 * k]) * p.scale, __uint_as_float(bb[i + 2 * k + 1]) * p.scale);
+            }
+            if (p.dkv_32) {
+              st_global_v8(dv_row + cgrp * 32 + i, hv[0], hv[1], hv[2], hv[3], hv[4], hv[5], hv[6], hv[7]);
+              st_global_v8(dk_row + cgrp * 32 + i, hk[0], hk[1], hk[2], hk[3], hk[4], hk[5], hk[6], hk[7]);
+            } else {
+              *reinterpret_cast<uint4*>(dv_row + cgrp * 32 + i) = make_uint4(hv[0], hv[1], hv[2], hv[3]);
+              *reinterpret_cast<uint4*>(dv_row + cgrp * 32 + i + 8) = make_uint4(hv[4], hv[5], hv[6], hv[7]);
+              *reinterpret_cast<uint4*>(dk_row + cgrp * 32 + i) = make_uint4(hk[0], hk[1], hk[2], hk[3]);
+              *reinterpret_cast<uint4*>(dk_row + cgrp * 32 + i + 8) = make_uint4(hk[4], hk[5], hk[6], hk[7]);
+            }
           }
         }
       }
@@ -693,6 +698,7 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
   kp.scale = D.scale; kp.scale_log2 = D.scale * LOG2E; kp.capacity = cap;
   kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status; kp.prof = tcb::g_wait_profile;
   kp.dq_acc = dq_acc;
+  kp.dkv_32 = (reinterpret_cast<uintptr_t>(dk) % 32) == 0 && (reinterpret_cast<uintptr_t>(dv) % 32) == 0;
   const long long kv_items = n_kb * ((D.sb + BN - 1) / BN);
   VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)KVF_SMEM_BYTES));

@@ -69,6 +69,7 @@ struct Params {
   float* part_o;
   float* part_lse;
   long long capacity;
+  int part_o_32;         // part_o is 32-byte aligned: rows go out with 32-byte stores
   int32_t* status;
   unsigned long long* prof;   // optional per-section cycle counters (diagnostics), or null
 };
@@ -141,17 +142,23 @@ __device__ __forceinline__ void exp_pack64(const uint32_t (&sv)[64], float scale
   }
 }
 
-// Eight consecutive outputs as bf16 (one 16-byte store) and, if asked for, their rounding residuals
-// bf16(v - bf16(v)), computed in registers.
-__device__ __forceinline__ void store8_resid(__nv_bfloat16* dst, __nv_bfloat16* rdst, const float (&v)[8]) {
-  uint32_t h[4], r[4];
+// N (8 or 16) consecutive outputs as bf16 (one 16- or 32-byte store) and, if asked for, their rounding
+// residuals bf16(v - bf16(v)), computed in registers.
+template <int N>
+__device__ __forceinline__ void store_resid(__nv_bfloat16* dst, __nv_bfloat16* rdst, const float (&v)[N]) {
+  uint32_t h[N / 2], r[N / 2];
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
+  for (int k = 0; k < N / 2; ++k) {
     h[k] = pack_bf16(v[2 * k], v[2 * k + 1]);
     r[k] = pack_bf16(v[2 * k] - __uint_as_float(h[k] << 16), v[2 * k + 1] - __uint_as_float(h[k] & 0xffff0000u));
   }
-  *reinterpret_cast<uint4*>(dst) = make_uint4(h[0], h[1], h[2], h[3]);
-  if (rdst) *reinterpret_cast<uint4*>(rdst) = make_uint4(r[0], r[1], r[2], r[3]);
+  if constexpr (N == 16) {
+    st_global_v8(dst, h[0], h[1], h[2], h[3], h[4], h[5], h[6], h[7]);
+    if (rdst) st_global_v8(rdst, r[0], r[1], r[2], r[3], r[4], r[5], r[6], r[7]);
+  } else {
+    *reinterpret_cast<uint4*>(dst) = make_uint4(h[0], h[1], h[2], h[3]);
+    if (rdst) *reinterpret_cast<uint4*>(rdst) = make_uint4(r[0], r[1], r[2], r[3]);
+  }
 }
 
 template <bool DENSE>
@@ -468,19 +475,27 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
             __nv_bfloat16* dst = p.o + G_ * DH + col;
             __nv_bfloat16* rdst = p.o_resid ? p.o_resid + G_ * DH + col : nullptr;
 #pragma unroll
-            for (int i = 0; i < 32; i += 8) {
+            for (int i = 0; i < 32; i += 8) {     // 16-byte stores (32-byte ones were slower here: more values live at once)
               float v8[8];
 #pragma unroll
               for (int k = 0; k < 8; ++k) v8[k] = __uint_as_float(ov[i + k]) * inv;
-              store8_resid(dst + i, rdst ? rdst + i : nullptr, v8);
+              store_resid<8>(dst + i, rdst ? rdst + i : nullptr, v8);
             }
           } else {
             float* dst = p.part_o + pos * DH + col;
+            if (!p.part_o_32) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              *reinterpret_cast<float4*>(dst + i) =
-                  make_float4(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
-                              __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv);
+              for (int i = 0; i < 32; i += 4)
+                *reinterpret_cast<float4*>(dst + i) =
+                    make_float4(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
+                                __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv);
+            } else
+#pragma unroll
+            for (int i = 0; i < 32; i += 8)       // 32-byte stores: a thread's row is 512 contiguous bytes
+              st_global_v8(dst + i, __uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
+                           __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv,
+                           __uint_as_float(ov[i + 4]) * inv, __uint_as_float(ov[i + 5]) * inv,
+                           __uint_as_float(ov[i + 6]) * inv, __uint_as_float(ov[i + 7]) * inv);
           }
         }
       }
@@ -524,6 +539,7 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
   p.scale_log2 = D.scale * 1.4426950408889634f;
   p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
   p.capacity = cap; p.status = status; p.prof = debug_wait_profile();
+  p.part_o_32 = (reinterpret_cast<uintptr_t>(part_o) % 32) == 0;
   VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_wide_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)SMEM_BYTES));
   attn_fwd_wide_kernel<false><<<grid_items(cap / IM + n_kb), THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
@@ -547,7 +563,8 @@ int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, voi
   p.n_kb = 0; p.S = D.S; p.Nb = 1; p.sb = D.S; p.BH = D.BH;
   p.scale_log2 = D.scale * 1.4426950408889634f;
   p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = nullptr; p.part_lse = nullptr;
-  p.capacity = 0; p.status = status; p.prof = debug_wait_profile();
+  p.capacity = 0; p.part_o_32 = 0;
+  p.status = status; p.prof = debug_wait_profile();
   VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_wide_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)SMEM_BYTES));
   const long long items = (long long)D.BH * ((D.S + IM - 1) / IM);
