@@ -27,7 +27,7 @@ namespace tcb {
 
 using namespace sm100;
 
-constexpr int BM = 128, BN = 128, DH = 128;
+constexpr int BN = 128, DH = 128;
 constexpr int PANEL = 128 * 128;
 constexpr int TILE = 2 * PANEL;
 constexpr uint32_t TMEM_COLS = 512;
@@ -35,7 +35,6 @@ constexpr float LOG2E = 1.4426950408889634f;
 // Diagnostics: when a device buffer of 16 counters is registered, the dK/dV kernels add the cycles
 // their roles spend in each wait (one representative thread per role and CTA).
 static unsigned long long* g_wait_profile = nullptr;
-constexpr uint32_t IDESC_KK = make_idesc_bf16(128, 128, false, false);   // A, B both K-major in shared memory
 constexpr uint32_t IDESC_TN = make_idesc_bf16(128, 128, false, true);    // A from TMEM, B MN-major
 
 // 16 threads per row: copy `n_rows` gathered 256-byte rows into a swizzled K-major tile (two
@@ -114,18 +113,18 @@ __device__ __forceinline__ uint64_t desc_mn(uint32_t tile_addr, int ks) {
 }
 
 // ==========================================================================================
-// dK / dV
+// dK / dV / dQ
 // ==========================================================================================
 // Units of 64 queries flow through a ring of gathered (Q, dO) chunks; S^T / dP^T are double
 // buffered in TMEM (64 columns each), so the tensor pipe computes unit u+1 while the compute warps
-// turn unit u into P^T / dS^T.  K and V tiles are double buffered across items, and the loader and
-// TMA warps run ahead of the MMA warp across item boundaries.
+// turn unit u into P^T / dS^T.  One K / V pair is resident per item; the loader warps run ahead of
+// the MMA warp across item boundaries.
 constexpr int QC = 64;                       // queries per unit
 constexpr int CPANEL = QC * 128;             // bytes of one 64-column panel of a 64-row chunk (8 KB)
 constexpr int CTILE = 2 * CPANEL;            // [64 x 128] bf16 (16 KB)
 constexpr int NQ = 4;                        // chunk ring depth
 struct KvSmem {
-  uint64_t kv_full[2], kv_empty[2];          // K+V tiles of an item (TMA / commit)
+  uint64_t kv_full[2], kv_empty[2];          // K+V tiles of an item (TMA / commit); index 0 is in use
   uint64_t chunk_full[NQ], chunk_empty[NQ];  // gathered Q/dO chunk (128 loader arrivals / commit)
   uint64_t sdp_full[2];                      // S^T and dP^T of a unit ready (commit)
   uint64_t pds_ready[2];                     // P^T and dS^T written (128 compute arrivals)
@@ -133,19 +132,17 @@ struct KvSmem {
   uint64_t acc_free;                         // epilogue has read dV / dK (128 compute arrivals)
   uint32_t tmem_base;
   int abort_flag;
-  uint64_t dq_full[2];                       // fused variant: dQ^T of a unit complete (commit)
-  uint64_t dq_free[2];                       // fused variant: dQ^T read out of TMEM (128 writer arrivals)
+  uint64_t dq_full[2];                       // dQ^T of a unit complete (commit)
+  uint64_t dq_free[2];                       // dQ^T read out of TMEM (128 writer arrivals)
   alignas(16) float lse2[NQ][QC];
   alignas(16) float Dq[NQ][QC];
 };
 constexpr int DSTILE = 128 * 128;            // dS^T of a unit in shared memory: [128 keys][64 queries] bf16 (16 KB)
-// split kernels: K/V double buffered across items; fused kernel: one K/V pair, one dS^T tile, the dQ staging tile
-constexpr size_t KV_SMEM_BYTES = 1024 + 4 * TILE + NQ * 2 * CTILE + sizeof(KvSmem) + 32;
+// one K/V pair, the chunk ring, one dS^T tile, the dQ staging tile
 constexpr int DQSTAGE = (QC / 2) * DH * 4;   // dQ of half a unit as [32 queries][128] fp32 rows for the vector reductions (16 KB)
 // no alignment slack: the kernel checks that its dynamic shared memory starts on a 1024-byte boundary
 constexpr size_t KVF_SMEM_BYTES = 2 * TILE + NQ * 2 * CTILE + DSTILE + DQSTAGE + sizeof(KvSmem) + 32;
 static_assert(KVF_SMEM_BYTES <= 232448, "fused backward: shared memory");
-constexpr int KV_THREADS = 448;   // TMA, MMA, 8 compute warps, 4 loader warps
 constexpr int KVF_THREADS = 576 + 32 * RED_HELPERS;  // ... plus 4 dQ writer warps and the reduction helper warps
 constexpr uint32_t IDESC_K64 = make_idesc_bf16(128, QC, false, false);   // S^T, dP^T: N = 64 queries
 constexpr uint32_t IDESC_DQT = make_idesc_bf16(128, QC, true, true);     // dQ^T = K^T dS^T: both operands MN-major
@@ -159,7 +156,7 @@ struct KvParams {
   long long capacity;
   __nv_bfloat16 *dk, *dv;
   int dkv_32;                  // dk and dv are 32-byte aligned: rows go out with 32-byte stores
-  float* dq_acc;               // fused variant: fp32 [queries][head_dim], zeroed rows of all selecting queries
+  float* dq_acc;               // fp32 [queries][head_dim], zeroed rows of all selecting queries
   int32_t* status;
   unsigned long long* prof;    // optional wait-time counters (diagnostics), or null
 };
@@ -219,26 +216,23 @@ __device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, i
   return it;
 }
 
-// Only <DENSE = false, FUSE = true> is instantiated.  FUSE = false is the same kernel without the
-// dQ^T MMA, the dS^T tile and the writer warps (dS^T then goes to the dP^T columns, K/V are double
-// buffered across items); DENSE = true walks all queries of the sequence instead of an index list.
-template <bool DENSE, bool FUSE>
-__global__ void __launch_bounds__(FUSE ? KVF_THREADS : KV_THREADS, 1)
+// Only DENSE = false is instantiated (DENSE = true walks all queries of the sequence instead of an index list).
+template <bool DENSE>
+__global__ void __launch_bounds__(KVF_THREADS, 1)
 attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const KvParams p) {
   extern __shared__ uint8_t smem_raw[];
-  // the swizzled tiles need 1024-byte alignment; the fused variant has no room for alignment slack
-  if (FUSE && (smem_u32(smem_raw) & 1023u) != 0) {
+  // the swizzled tiles need 1024-byte alignment and there is no room for alignment slack
+  if ((smem_u32(smem_raw) & 1023u) != 0) {
     if (threadIdx.x == 0) set_status(p.status, VMOBA_ERR_CUDA);
     return;
   }
-  uint8_t* base = FUSE ? smem_raw : reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  constexpr int KVB = FUSE ? 1 : 2;    // K/V buffers
-  uint8_t* sK = base;                  // [KVB][TILE]
-  uint8_t* sV = base + KVB * TILE;     // [KVB][TILE]
-  uint8_t* sC = base + 2 * KVB * TILE; // [NQ][Q chunk | dO chunk]
-  uint8_t* sDS = sC + NQ * 2 * CTILE;  // fused variant: dS^T of the current unit [DSTILE]
-  float* s_stage = reinterpret_cast<float*>(sDS + DSTILE);                         // fused variant: [QC / 2][DH] fp32
-  KvSmem* sm = reinterpret_cast<KvSmem*>(sDS + (FUSE ? DSTILE + DQSTAGE : 0));
+  uint8_t* base = smem_raw;
+  uint8_t* sK = base;                  // [TILE]
+  uint8_t* sV = base + TILE;           // [TILE]
+  uint8_t* sC = base + 2 * TILE;       // [NQ][Q chunk | dO chunk]
+  uint8_t* sDS = sC + NQ * 2 * CTILE;  // dS^T of the current unit [DSTILE]
+  float* s_stage = reinterpret_cast<float*>(sDS + DSTILE);                         // [QC / 2][DH] fp32
+  KvSmem* sm = reinterpret_cast<KvSmem*>(sDS + DSTILE + DQSTAGE);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm->abort_flag;
   // diagnostics: cycles spent in each wait site by one representative thread per role
@@ -295,23 +289,18 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
         const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
         if (it.n_units == 0) continue;
-        const int b = FUSE ? 0 : (n & 1);
-        if (FUSE) {
-          if (n >= 1) twait(0, &sm->kv_empty[0], (n - 1) & 1);
-        } else if (n >= 2) {
-          twait(0, &sm->kv_empty[b], ((n >> 1) - 1) & 1);
-        }
+        // one K / V pair: the next item's tiles wait for the current item's last MMA
+        if (n >= 1) twait(0, &sm->kv_empty[0], (n - 1) & 1);
         const int y = (int)it.head_off + it.key0;
-        mbar_expect_tx(&sm->kv_full[b], 2 * TILE);
-        tma_load_2d(sK + b * TILE, &tmK, &sm->kv_full[b], 0, y);
-        tma_load_2d(sK + b * TILE + PANEL, &tmK, &sm->kv_full[b], 64, y);
-        tma_load_2d(sV + b * TILE, &tmV, &sm->kv_full[b], 0, y);
-        tma_load_2d(sV + b * TILE + PANEL, &tmV, &sm->kv_full[b], 64, y);
+        mbar_expect_tx(&sm->kv_full[0], 2 * TILE);
+        tma_load_2d(sK, &tmK, &sm->kv_full[0], 0, y);
+        tma_load_2d(sK + PANEL, &tmK, &sm->kv_full[0], 64, y);
+        tma_load_2d(sV, &tmV, &sm->kv_full[0], 0, y);
+        tma_load_2d(sV + PANEL, &tmV, &sm->kv_full[0], 64, y);
         ++n;
       }
       if (*abort_flag)
-        for (uint32_t f = n > 2 ? n - 2 : 0; f < n; ++f)
-          mbar_wait(&sm->kv_full[FUSE ? 0 : (f & 1)], (FUSE ? f : (f >> 1)) & 1, abort_flag, p.status);
+        for (uint32_t f = n > 2 ? n - 2 : 0; f < n; ++f) mbar_wait(&sm->kv_full[0], f & 1, abort_flag, p.status);
       tflush(0, 1);      // [0] kv_empty, [1] total
     }
   } else if (warp == 1) {
@@ -327,11 +316,10 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         const int n_list = __reduce_max_sync(0xffffffffu, (int)(it.list_hi - it.list_lo));
         it.n_units = (n_list + QC - 1) / QC;
         if (it.n_units == 0) continue;
-        const int b = FUSE ? 0 : (n & 1);
-        wwait(0, &sm->kv_full[b], (FUSE ? n : (n >> 1)) & 1);
+        wwait(0, &sm->kv_full[0], n & 1);
         tc_fence_after();
-        const uint64_t dK0 = desc_k(smem_u32(sK + b * TILE), 0), dV0 = desc_k(smem_u32(sV + b * TILE), 0);
-        const uint64_t mK0 = desc_mn(smem_u32(sK + b * TILE), 0);     // K^T as MN-major A operand (fused dQ^T)
+        const uint64_t dK0 = desc_k(smem_u32(sK), 0), dV0 = desc_k(smem_u32(sV), 0);
+        const uint64_t mK0 = desc_mn(smem_u32(sK), 0);     // K^T as MN-major A operand (fused dQ^T)
         auto issue_sdp = [&](int i) {
           const uint32_t u = u0 + i;
           const int cb = u % NQ, tb = u & 1;
@@ -346,7 +334,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
 #pragma unroll
           for (int ks = 0; ks < DH / 16; ++ks)
             if (leader) mma_ss(st, dK0 + koff(ks, PANEL), dQ0 + koff(ks, CPANEL), IDESC_K64, ks > 0 ? 1u : 0u);
-          if (FUSE && u >= 2) {
+          if (u >= 2) {
             wwait(3, &sm->dq_free[tb], ((u - 2) >> 1) & 1);
             tc_fence_after();
           }
@@ -356,9 +344,8 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           if (leader) mma_commit(&sm->sdp_full[tb]);
         };
         issue_sdp(0);
-        if (FUSE && it.n_units > 1) issue_sdp(1);
+        if (it.n_units > 1) issue_sdp(1);
         for (int i = 0; i < it.n_units; ++i) {
-          if (!FUSE && i + 1 < it.n_units) issue_sdp(i + 1);
           const uint32_t u = u0 + i;
           const int cb = u % NQ, tb = u & 1;
           wwait(2, &sm->pds_ready[tb], (u >> 1) & 1);
@@ -371,7 +358,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           const uint64_t mQ0 = cdesc_mn(sQ_addr, 0), mO0 = cdesc_mn(sQ_addr + CTILE, 0);
           const uint32_t pt = tmem + ST_COL + tb * QC, dst_ = tmem + DPT_COL + tb * QC;
           const uint32_t acc0 = i > 0 ? 1u : 0u;
-          if (FUSE) {
+          {
             // dQ^T [head dim x 64 queries] = K^T dS^T over the tile's keys, into the unit's dP^T columns
             // (already read by the compute warps); issued first so that its read-out overlaps dV / dK
             const uint64_t mS0 = make_smem_desc(smem_u32(sDS), DSTILE, 1024);
@@ -381,9 +368,9 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
               if (leader && ks < kk) mma_ss(dst_, mK0 + mnoff(ks), mS0 + mnoff(ks), IDESC_DQT, ks > 0 ? 1u : 0u);
             if (leader) mma_commit(&sm->dq_full[tb]);
           }
-          // P^T of queries 32h .. 32h+31 sits in columns 32h .. 32h+15 of the S^T buffer; dS^T in the same
-          // columns of the dP^T buffer (split kernels) or in columns 32h+16 .. 32h+31 of the S^T buffer (fused)
-          const uint32_t ds_t = FUSE ? pt + 16 : dst_;
+          // P^T of queries 32h .. 32h+31 sits in columns 32h .. 32h+15 of the S^T buffer, dS^T in columns
+          // 32h+16 .. 32h+31 (the dP^T columns are receiving dQ^T)
+          const uint32_t ds_t = pt + 16;
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
             if (leader && ks < ksteps) {
@@ -391,9 +378,9 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
               mma_ts(tmem + DK_COL, ds_t + (ks >> 1) * 32 + (ks & 1) * 8, mQ0 + mnoff(ks), IDESC_TN, ks > 0 ? 1u : acc0);
             }
           if (leader) mma_commit(&sm->chunk_empty[cb]);
-          if (FUSE && i + 2 < it.n_units) issue_sdp(i + 2);
+          if (i + 2 < it.n_units) issue_sdp(i + 2);
         }
-        if (leader) mma_commit(&sm->kv_empty[b]);
+        if (leader) mma_commit(&sm->kv_empty[0]);
         if (leader) mma_commit(&sm->acc_done);
         u0 += it.n_units;
         ++n;
@@ -458,7 +445,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     cp_async_wait<0>();
     if (u0 >= 1) publish(u0 - 1);
     if (lt == 0) tflush(7, 1);     // [7] chunk_empty, [8] total
-  } else if (FUSE && warp >= 14) {
+  } else if (warp >= 14) {
     // ------------------------------------------------------------------ dQ writers: thread = head-dim index
     // Read dQ^T of a unit out of TMEM, release the buffer, transpose it through shared memory into 64
     // rows of 128 floats and add each row into the fp32 accumulator with one vector-reduction warp
@@ -607,7 +594,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
           dk_[2 * e + 1] = pack_bf16(p2 * (__uint_as_float(dv_[4 * e + 2]) - d4.z), p3 * (__uint_as_float(dv_[4 * e + 3]) - d4.w));
         }
         tmem_st16(st_t, pk);       // P^T (bf16 pairs) over the first 16 of this thread's 32 S^T columns
-        if (FUSE) {
+        {
           tmem_st16(st_t + 16, dk_);   // dS^T over the other 16: the dP^T columns are about to receive dQ^T
           // and once more, as the row of this key in the [keys][queries] shared-memory tile that dQ^T reads;
           // rows beyond the key range hold other blocks' keys and must not contribute
@@ -620,8 +607,6 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
             *reinterpret_cast<uint4*>(dsrow + (((4 * half + j) ^ (r & 7)) << 4)) =
                 live ? make_uint4(dk_[4 * j], dk_[4 * j + 1], dk_[4 * j + 2], dk_[4 * j + 3]) : make_uint4(0u, 0u, 0u, 0u);
           fence_async_proxy();
-        } else {
-          tmem_st16(dp_t, dk_);    // dS^T likewise over its dP^T columns
         }
         tmem_st_wait();
         tc_fence_before();
@@ -700,9 +685,9 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
   kp.dq_acc = dq_acc;
   kp.dkv_32 = (reinterpret_cast<uintptr_t>(dk) % 32) == 0 && (reinterpret_cast<uintptr_t>(dv) % 32) == 0;
   const long long kv_items = n_kb * ((D.sb + BN - 1) / BN);
-  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)KVF_SMEM_BYTES));
-  attn_bwd_dkdv_tc_kernel<false, true><<<grid_items(kv_items), KVF_THREADS, KVF_SMEM_BYTES, st>>>(tmK, tmV, kp);
+  attn_bwd_dkdv_tc_kernel<false><<<grid_items(kv_items), KVF_THREADS, KVF_SMEM_BYTES, st>>>(tmK, tmV, kp);
   VMOBA_LAUNCH_OK(1);
   return VMOBA_OK;
 }
