@@ -37,50 +37,6 @@ constexpr float LOG2E = 1.4426950408889634f;
 static unsigned long long* g_wait_profile = nullptr;
 constexpr uint32_t IDESC_TN = make_idesc_bf16(128, 128, false, true);    // A from TMEM, B MN-major
 
-// 16 threads per row: copy `n_rows` gathered 256-byte rows into a swizzled K-major tile (two
-// 64-column panels of 128-byte rows); rows beyond n_rows are zero-filled.
-template <int NTHREADS, typename RowOf>
-__device__ __forceinline__ void gather_tile(uint8_t* dst, const __nv_bfloat16* head_base, int n_rows, int tid, RowOf row_of) {
-  constexpr int PASSES = 128 / (NTHREADS / 16);
-  const int chunk = tid & 15;
-  const int panel = chunk >> 3, cc = chunk & 7;
-  // issue every load of this thread before the first store: the gather is latency-bound otherwise
-  uint4 v[PASSES];
-#pragma unroll
-  for (int i = 0; i < PASSES; ++i) {
-    const int row = (tid >> 4) + i * (NTHREADS / 16);
-    v[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (row < n_rows) v[i] = __ldg(reinterpret_cast<const uint4*>(head_base + (long long)row_of(row) * DH) + chunk);
-  }
-#pragma unroll
-  for (int i = 0; i < PASSES; ++i) {
-    const int row = (tid >> 4) + i * (NTHREADS / 16);
-    *reinterpret_cast<uint4*>(dst + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v[i];
-  }
-}
-
-// The same gather split in two, so that a wait can sit between the loads and the stores
-// (128 threads, 16 rows per thread).
-template <typename RowOf>
-__device__ __forceinline__ void gather_load128(const __nv_bfloat16* head_base, int n_rows, int tid, RowOf row_of, uint4 (&v)[16]) {
-  const int chunk = tid & 15;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const int row = (tid >> 4) + i * 8;
-    v[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (row < n_rows) v[i] = __ldg(reinterpret_cast<const uint4*>(head_base + (long long)row_of(row) * DH) + chunk);
-  }
-}
-__device__ __forceinline__ void gather_store128(uint8_t* dst, int tid, const uint4 (&v)[16]) {
-  const int chunk = tid & 15;
-  const int panel = chunk >> 3, cc = chunk & 7;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const int row = (tid >> 4) + i * 8;
-    *reinterpret_cast<uint4*>(dst + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v[i];
-  }
-}
-
 // named barrier of the dQ writer and helper warps
 constexpr int RED_HELPERS = 2;               // warps that only send out staged dQ rows, next to the four writer warps
 constexpr int RED_WARPS = 4 + RED_HELPERS;
@@ -161,28 +117,6 @@ struct KvParams {
   unsigned long long* prof;    // optional wait-time counters (diagnostics), or null
 };
 
-// 16 threads per row: gather `n_rows` (<= 64) 256-byte rows into a swizzled [64 x 128] chunk tile.
-template <typename RowOf>
-__device__ __forceinline__ void gather_chunk64(uint8_t* dst, const __nv_bfloat16* head_base, int n_rows, int tid, RowOf row_of,
-                                               uint4 (&v)[8]) {
-  const int chunk = tid & 15;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int row = (tid >> 4) + i * 8;
-    v[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (row < n_rows) v[i] = __ldg(reinterpret_cast<const uint4*>(head_base + (long long)row_of(row) * DH) + chunk);
-  }
-  (void)dst;
-}
-__device__ __forceinline__ void store_chunk64(uint8_t* dst, int tid, const uint4 (&v)[8]) {
-  const int chunk = tid & 15;
-  const int panel = chunk >> 3, cc = chunk & 7;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int row = (tid >> 4) + i * 8;
-    *reinterpret_cast<uint4*>(dst + panel * CPANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v[i];
-  }
-}
 // chunk tile as K-major B operand (N = 64 queries, K = head dim), k-step ks of 8
 __device__ __forceinline__ uint64_t cdesc_k(uint32_t tile_addr, int ks) {
   return make_smem_desc(tile_addr + (ks >> 2) * CPANEL + (ks & 3) * 32, 16, 1024);
