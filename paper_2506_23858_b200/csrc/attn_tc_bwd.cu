@@ -99,7 +99,8 @@ constexpr int DQSTAGE = (QC / 2) * DH * 4;   // dQ of half a unit as [32 queries
 // no alignment slack: the kernel checks that its dynamic shared memory starts on a 1024-byte boundary
 constexpr size_t KVF_SMEM_BYTES = 2 * TILE + NQ * 2 * CTILE + DSTILE + DQSTAGE + sizeof(KvSmem) + 32;
 static_assert(KVF_SMEM_BYTES <= 232448, "fused backward: shared memory");
-constexpr int KVF_THREADS = 576 + 32 * RED_HELPERS;  // ... plus 4 dQ writer warps and the reduction helper warps
+// warps: TMA, MMA, 8 compute, 4 loaders, 4 dQ writers, then the reduction helpers
+constexpr int KVF_THREADS = 576 + 32 * RED_HELPERS;
 constexpr uint32_t IDESC_K64 = make_idesc_bf16(128, QC, false, false);   // S^T, dP^T: N = 64 queries
 constexpr uint32_t IDESC_DQT = make_idesc_bf16(128, QC, true, true);     // dQ^T = K^T dS^T: both operands MN-major
 
