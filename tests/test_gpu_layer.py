@@ -151,6 +151,20 @@ def test_wide_logit_range_forward_backward(block):
         _check_head(w, data, res, 0, h, rng, n_rows=400, n_blocks=3, with_bwd=True)
 
 
+def test_repeated_runs_reproduce():
+    """Everything but dQ is written once, by one owner: repeated runs must agree bit for bit (a race between the
+    roles of a kernel shows up here first).  dQ is an fp32 sum of per-key-tile parts whose order is not fixed."""
+    w = MID.with_(block=(1, 12, 26))
+    data = gen.make_inputs(w)
+    runs = [_run_layer(w, data, with_bwd=True) for _ in range(3)]
+    for r in runs[1:]:
+        for name in ("o", "dk", "dv"):
+            assert torch.equal(r[name], runs[0][name]), name
+        assert torch.equal(r["L"].lse, runs[0]["L"].lse)
+        diff = (r["dq"].float() - runs[0]["dq"].float()).abs().max().item()
+        assert diff <= 2.0 ** -6 * max(1.0, runs[0]["dq"].float().abs().max().item())
+
+
 def test_mid_size_threshold_one_equals_dense_path():
     """tau = 1.0 through the sparse pipeline must equal the library's dense path and the oracle's dense attention."""
     w = MID.with_(tau=1.0, B=1, heads=2)
