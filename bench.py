@@ -165,16 +165,18 @@ def run_reference(args):
     times, flops_tot = [], 0.0
     detail = None
     # One untimed step first (also when W = 0): it tells how long a step takes.  If W + K such steps would
-    # not end within a few minutes, later steps sample fewer of the workload's layers (the value is work /
-    # time of whatever was sampled), and only if one layer is still too slow, fewer steps.
+    # not end within a few minutes, the later steps take a smaller sample: first fewer query rows for the
+    # attention, then fewer of the workload's layers (the value is work / time of whatever was sampled), and
+    # only if that is still too slow, fewer steps.
     warmup, steps = 1, args.steps
     n_used = len(layers)
+    rows = args.cpu_rows
     it = 0
     while it < warmup + steps:
         wall = time.perf_counter()
         t, f = 0.0, 0.0
         for w in layers[:n_used]:
-            tt, ff, detail = oracle_sample(w, with_bwd, args.cpu_rows, seed=it)
+            tt, ff, detail = oracle_sample(w, with_bwd, rows, seed=it)
             t += tt; f += ff
         wall = time.perf_counter() - wall
         if it >= warmup:
@@ -182,16 +184,19 @@ def run_reference(args):
         else:
             budget = 240.0 / (warmup + steps)
             if wall > budget:
-                n_used = max(1, int(len(layers) * budget / wall))
-                per_step = wall * n_used / len(layers)
-                if per_step > budget:
-                    steps = max(1, int(240.0 / per_step) - warmup)
+                rows = max(32, int(rows * budget / wall) // 32 * 32)
+                est = wall * (0.25 + 0.75 * rows / args.cpu_rows)      # part of a step does not depend on the rows
+                if est > budget:
+                    n_used = max(1, int(len(layers) * budget / est))
+                    est = est * n_used / len(layers)
+                    if est > 2.0 * budget:
+                        steps = max(1, int(240.0 / est) - warmup)
         it += 1
     sec = statistics.mean(times)
     units = layers[0].B * layers[0].heads
     value = flops_tot / sec / 1e12
     sample = (f"1 of {units} (batch, head) units of {n_used} of the {len(layers)} layers; partition, centroids, scores, "
-              f"selection in full; attention on {args.cpu_rows} sampled query rows, time scaled to the unit's selected pairs")
+              f"selection in full; attention on {rows} sampled query rows, time scaled to the unit's selected pairs")
     line = {
         "impl": "reference", "metric": "vmoba_layer_selected_pair_tflops", "value": value, "unit": "TFLOP/s",
         "n_gpus": args.gpus, "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3 * units * len(layers) / n_used,
