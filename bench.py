@@ -4,10 +4,11 @@
 A step is one pass of the whole layer over one batch of synthetic video-DiT-shaped input:
 partition(q, k, v) -> centroids + scores -> global threshold selection -> sparse attention
 forward -> inverse partition(o), and for training workloads the backward:
-partition(dO) -> sparse attention backward -> inverse partition(dq, dk, dv).  Workloads with
+partition(dO) -> sparse attention backward writing dq, dk, dv in raster order (bf16, head_dim 128;
+otherwise the backward followed by their inverse partitions).  Workloads with
 several partitions (c3, c5) run the layer once per partition (1D, 2D, 3D) per step.
 
-    python bench.py --gpus 1 --steps 20 --warmup 3                # default workload: c4
+    python bench.py --gpus 1 --steps 20 --warmup 3                # default workload: c5
     python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
     python bench.py --impl reference                               # the CPU oracle, timed
 
@@ -242,6 +243,8 @@ def main():
                     choices=["threshold_global", "topk_global", "threshold_local", "topk_local"],
                     help="block-choice rule (Table 3b); the paper's training-free runs use topk_local")
     ap.add_argument("--topk", default="", help="k of the top-k rules: one value, or one per layer (e.g. 2,6,18)")
+    ap.add_argument("--no-fold", action="store_true",
+                    help="write dq, dk, dv block-major and run their inverse partitions (instead of the backward writing raster order)")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small profiling runs)")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -310,6 +313,8 @@ def main():
     stage_names = ["partition", "scores", "select", "attn_fwd"] + (["attn_bwd"] if with_bwd else [])
     stage_ms = {s: 0.0 for s in stage_names}
 
+    fold = with_bwd and not args.no_fold and L[0].can_fold_inverse(outs["dq"], outs["dk"], outs["dv"])
+
     def step(record, dev=dev, outs=outs):
         evs = []
 
@@ -319,7 +324,7 @@ def main():
 
         for layer in L:
             mark("start")
-            layer.partition(dev["q"], layer.q_bm); layer.partition(dev["k"], layer.k_bm)
+            layer.partition(dev["q"], layer.q_bm, perm=layer.perm); layer.partition(dev["k"], layer.k_bm)
             layer.partition(dev["v"], layer.v_bm)
             mark("partition")
             layer.block_scores(); mark("scores")
@@ -328,11 +333,15 @@ def main():
             layer.partition(outs["o"], layer.o_bm, inverse=True); mark("partition")
             if with_bwd:
                 layer.partition(dev["do"], layer.do_bm); mark("partition")
-                layer.attn_bwd(); mark("attn_bwd")
-                layer.partition(outs["dq"], layer.dq_bm, inverse=True)
-                layer.partition(outs["dk"], layer.dk_bm, inverse=True)
-                layer.partition(outs["dv"], layer.dv_bm, inverse=True)
-                mark("partition")
+                if fold:
+                    # the backward kernels write dq, dk, dv in raster order themselves (inverse of Eq. 1 folded in)
+                    layer.attn_bwd_raster_out(outs["dq"], outs["dk"], outs["dv"]); mark("attn_bwd")
+                else:
+                    layer.attn_bwd(); mark("attn_bwd")
+                    layer.partition(outs["dq"], layer.dq_bm, inverse=True)
+                    layer.partition(outs["dk"], layer.dk_bm, inverse=True)
+                    layer.partition(outs["dv"], layer.dv_bm, inverse=True)
+                    mark("partition")
         return evs
 
     layer_tau = {id(layer): w.tau for layer, w in zip(L, layers)}
@@ -453,7 +462,7 @@ def main():
 
     es = 2 if w0.dtype == "bf16" else 4
     tensor_bytes = w0.B * w0.S * w0.heads * w0.head_dim * es
-    n_part = len(layers) * (8 if with_bwd else 4)
+    n_part = len(layers) * ((5 if fold else 8) if with_bwd else 4)     # partition passes of a step
     alg = {
         "partition": ("hbm", 2.0 * tensor_bytes * n_part),
         "scores": ("hbm", sum(2.0 * tensor_bytes + 4.0 * w.B * w.heads * (w.S * w.n_blocks + w.n_blocks * w.head_dim)

@@ -489,7 +489,7 @@ attn_bwd_dq_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
 template <typename T, int DH>
 __global__ void __launch_bounds__(256)
 cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, const int* __restrict__ q_ptr, long long n_queries,
-                 int sparse_rows, int min_nb) {
+                 int sparse_rows, int min_nb, const RowMap map = RowMap()) {
   constexpr int C = DH / 32;
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -497,12 +497,13 @@ cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, const int* 
   for (long long g = warp; g < n_queries; g += nwarps) {
     const int nb = sparse_rows ? q_ptr[g + 1] - q_ptr[g] : 2;
     if (nb > 0 && nb < min_nb) continue;   // written directly by the attention kernel
+    T* out = dst + map.off(g, DH);
     if constexpr (C == 4) {
       const float4 v = nb == 0 ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(src + g * DH + lane * 4);
-      store4(dst + g * DH + lane * 4, v);
+      store4(out + lane * 4, v);
     } else {
 #pragma unroll
-      for (int c = 0; c < C; ++c) dst[g * DH + lane * C + c] = from_f32<T>(nb == 0 ? 0.f : src[g * DH + lane * C + c]);
+      for (int c = 0; c < C; ++c) out[lane * C + c] = from_f32<T>(nb == 0 ? 0.f : src[g * DH + lane * C + c]);
     }
   }
 }

@@ -113,6 +113,7 @@ struct KvParams {
   long long capacity;
   __nv_bfloat16 *dk, *dv;
   int dkv_32;                  // dk and dv are 32-byte aligned: rows go out with 32-byte stores
+  RowMap out_map;              // where the dK / dV rows go (block-major, or raster order through perm)
   float* dq_acc;               // fp32 [queries][head_dim], zeroed rows of all selecting queries
   int32_t* status;
   unsigned long long* prof;    // optional wait-time counters (diagnostics), or null
@@ -482,8 +483,9 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     uint32_t n = 0, u0 = 0;
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
       const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
-      __nv_bfloat16* dv_row = p.dv + (it.head_off + it.key0 + r) * DH;
-      __nv_bfloat16* dk_row = p.dk + (it.head_off + it.key0 + r) * DH;
+      const long long row_off = r < it.valid ? p.out_map.off(it.head_off + it.key0 + r, DH) : 0;
+      __nv_bfloat16* dv_row = p.dv + row_off;
+      __nv_bfloat16* dk_row = p.dk + row_off;
       if (it.n_units == 0) {
         // no query selected this block: its keys get zero gradients
         if (r < it.valid) {
@@ -605,7 +607,7 @@ int tc_long_dq(const Dims& D, bool dense, const void* q, const void* k, const vo
 // an fp32 accumulator whose rows of selecting queries are zero; the caller converts it to bf16.
 int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                   const float* Dv, const int* kb_ptr, const int* q_idx, long long cap, float* dq_acc, void* dk, void* dv,
-                  int32_t* status, cudaStream_t st) {
+                  int32_t* status, cudaStream_t st, const RowMap& out_map) {
   using namespace tcb;
   CUtensorMap tmK, tmV;
   const uint64_t rows = (uint64_t)D.BH * D.S;
@@ -618,7 +620,9 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
   kp.scale = D.scale; kp.scale_log2 = D.scale * LOG2E; kp.capacity = cap;
   kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status; kp.prof = tcb::g_wait_profile;
   kp.dq_acc = dq_acc;
-  kp.dkv_32 = (reinterpret_cast<uintptr_t>(dk) % 32) == 0 && (reinterpret_cast<uintptr_t>(dv) % 32) == 0;
+  kp.out_map = out_map;
+  kp.dkv_32 = (reinterpret_cast<uintptr_t>(dk) % 32) == 0 && (reinterpret_cast<uintptr_t>(dv) % 32) == 0 &&
+              (!out_map.perm || (out_map.sb % 16 == 0 && out_map.st % 16 == 0 && out_map.sh % 16 == 0));
   const long long kv_items = n_kb * ((D.sb + BN - 1) / BN);
   VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)KVF_SMEM_BYTES));

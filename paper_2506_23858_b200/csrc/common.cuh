@@ -26,6 +26,25 @@ struct Dims {
   float scale;
 };
 
+// Where row (batch, head, block-major position p) of an output tensor lives.  perm == nullptr: block-major,
+// row G = (batch * heads + head) * S + p at G * head_dim.  Otherwise raster order [B, S, heads, head_dim]
+// through element strides: batch * sb + perm[p] * st + head * sh (the inverse of Eq. 1 folded into the
+// kernel that writes the rows).
+struct RowMap {
+  const int* perm = nullptr;
+  long long sb = 0, st = 0, sh = 0;
+  int heads = 1, S = 1;
+#ifdef __CUDACC__
+  __device__ __forceinline__ long long off(long long G, int dh) const {
+    if (!perm) return G * dh;
+    const long long bh = G / S;
+    const int p = (int)(G - bh * S);
+    const long long b = bh / heads, hd = bh - b * heads;
+    return b * sb + (long long)__ldg(perm + p) * st + hd * sh;
+  }
+#endif
+};
+
 // Validates a shape and fills the derived sizes (Eq. 1 needs the grid divisible by the block).
 inline int make_dims(const vmoba_shape* s, Dims* o) {
   if (!s) return VMOBA_ERR_ARG;

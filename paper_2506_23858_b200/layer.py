@@ -47,6 +47,7 @@ class VmobaLayer:
         self.k_per_head = torch.empty(BH, dtype=torch.int64, device=dev)
         self.cutoff = torch.empty(BH, dtype=torch.float32, device=dev)
         self.lse = torch.empty(BH * S, dtype=torch.float32, device=dev)
+        self.perm = torch.empty(S, dtype=torch.int32, device=dev)     # raster token of block-major position p (Eq. 1)
         self.dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
         stages = [vb.STAGE_SCORES, vb.STAGE_SELECT, vb.STAGE_ATTN_FWD]
         if with_backward:
@@ -98,10 +99,22 @@ class VmobaLayer:
                           self.kb_ptr, self.q_idx, self.q_ptr, self.capacity, self.dq_bm, self.dk_bm, self.dv_bm,
                           self.dev_status, self.ws)
 
+    def can_fold_inverse(self, dq_out, dk_out, dv_out) -> bool:
+        """Whether the backward kernels can write these raster-order gradients themselves."""
+        strides = self.raster_strides(dq_out)
+        return (self.shape.dtype == vb.BF16 and self.d == 128 and self.raster_strides(dk_out) == strides
+                and self.raster_strides(dv_out) == strides)
+
+    def attn_bwd_raster_out(self, dq_out, dk_out, dv_out):
+        """Backward writing dq, dk, dv in raster order (needs self.perm from the forward's partition of q)."""
+        vb.vmoba_attn_bwd_raster_out(self.shape, self.q_bm, self.k_bm, self.v_bm, self.o_bm, self.o_resid, self.lse,
+                                     self.do_bm, self.kb_ptr, self.q_idx, self.q_ptr, self.capacity, dq_out, dk_out,
+                                     dv_out, self.raster_strides(dq_out), self.perm, self.dev_status, self.ws)
+
     # ---- whole layer --------------------------------------------------------------------
     def forward(self, q, k, v, tau, o_out):
         """q, k, v, o_out: [B, S, heads, d] raster-order tensors on the device."""
-        self.partition(q, self.q_bm)
+        self.partition(q, self.q_bm, perm=self.perm)
         self.partition(k, self.k_bm)
         self.partition(v, self.v_bm)
         self.block_scores()
@@ -109,9 +122,17 @@ class VmobaLayer:
         self.attn_fwd()
         self.partition(o_out, self.o_bm, inverse=True)
 
-    def backward(self, do, dq_out, dk_out, dv_out):
-        """Gradients of the last forward(); do and the outputs are raster-order [B, S, heads, d]."""
+    def backward(self, do, dq_out, dk_out, dv_out, fold_inverse=None):
+        """Gradients of the last forward(); do and the outputs are raster-order [B, S, heads, d].
+
+        fold_inverse: let the backward kernels write dq, dk, dv in raster order themselves (bf16, head_dim 128,
+        outputs with equal strides) instead of three inverse partition passes; default: whenever possible."""
         self.partition(do, self.do_bm)
+        if fold_inverse is None:
+            fold_inverse = self.can_fold_inverse(dq_out, dk_out, dv_out)
+        if fold_inverse:
+            self.attn_bwd_raster_out(dq_out, dk_out, dv_out)
+            return
         self.attn_bwd()
         self.partition(dq_out, self.dq_bm, inverse=True)
         self.partition(dk_out, self.dk_bm, inverse=True)

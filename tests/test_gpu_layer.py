@@ -151,6 +151,35 @@ def test_wide_logit_range_forward_backward(block):
         _check_head(w, data, res, 0, h, rng, n_rows=400, n_blocks=3, with_bwd=True)
 
 
+@pytest.mark.parametrize("block", [(1, 12, 26), (3, 6, 13)], ids=["1d", "3d"])
+def test_backward_writing_raster_order_equals_inverse_partition(block):
+    """vmoba_attn_bwd_raster_out folds the inverse of Eq. 1 into the gradient writes: dK and dV must equal
+    vmoba_attn_bwd followed by the inverse partition bit for bit, dQ up to the order of its fp32 sum."""
+    w = MID.with_(block=block)
+    data = gen.make_inputs(w)
+    shape = vb.shape_of(w)
+    L = VmobaLayer(shape, capacity=default_capacity(shape, w.tau), with_backward=True)
+    q, k, v, do = (U.to_device(w, data, n) for n in ("q", "k", "v", "do"))
+    o = torch.empty_like(q)
+    L.forward(q, k, v, w.tau, o)
+    got = [torch.full_like(q, float("nan")) for _ in range(3)]
+    ref = [torch.empty_like(q) for _ in range(3)]
+    L.backward(do, *got, fold_inverse=True)
+    L.backward(do, *ref, fold_inverse=False)
+    torch.cuda.synchronize()
+    L.check_status()
+    assert torch.equal(got[1], ref[1]) and torch.equal(got[2], ref[2])
+    assert not torch.isnan(got[0].float()).any()
+    diff = (got[0].float() - ref[0].float()).abs().max().item()
+    assert diff <= 2.0 ** -6 * max(1.0, ref[0].float().abs().max().item())
+    # a strided destination: the gradients of a fused [B, S, heads, 3, d] buffer
+    fused = torch.full((w.B, w.S, w.heads, 3, w.head_dim), float("nan"), dtype=q.dtype, device=q.device)
+    L.backward(do, fused[:, :, :, 0], fused[:, :, :, 1], fused[:, :, :, 2], fold_inverse=True)
+    torch.cuda.synchronize()
+    L.check_status()
+    assert torch.equal(fused[:, :, :, 1], ref[1]) and torch.equal(fused[:, :, :, 2], ref[2])
+
+
 def test_repeated_runs_reproduce():
     """Everything but dQ is written once, by one owner: repeated runs must agree bit for bit (a race between the
     roles of a kernel shows up here first).  dQ is an fp32 sum of per-key-tile parts whose order is not fixed."""
