@@ -5,7 +5,7 @@ A step is one pass of the whole layer over one batch of synthetic video-DiT-shap
 partition(q, k, v) -> centroids + scores -> global threshold selection -> sparse attention
 forward -> inverse partition(o), and for training workloads the backward:
 partition(dO) -> sparse attention backward writing dq, dk, dv in raster order (bf16, head_dim 128;
-otherwise the backward followed by their inverse partitions).  Workloads with
+otherwise the backward followed by the inverse partitions of the gradients).  Workloads with
 several partitions (c3, c5) run the layer once per partition (1D, 2D, 3D) per step.
 
     python bench.py --gpus 1 --steps 20 --warmup 3                # default workload: c5
@@ -244,7 +244,9 @@ def main():
                     help="block-choice rule (Table 3b); the paper's training-free runs use topk_local")
     ap.add_argument("--topk", default="", help="k of the top-k rules: one value, or one per layer (e.g. 2,6,18)")
     ap.add_argument("--no-fold", action="store_true",
-                    help="write dq, dk, dv block-major and run their inverse partitions (instead of the backward writing raster order)")
+                    help="partition dO and inverse-partition dq, dk, dv in passes of their own (instead of the backward reading / writing raster order)")
+    ap.add_argument("--fold-do", action="store_true",
+                    help="also let the backward read dO in raster order (pays with few heads: c4 yes, c5 no)")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small profiling runs)")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -332,11 +334,14 @@ def main():
             layer.attn_fwd(); mark("attn_fwd")
             layer.partition(outs["o"], layer.o_bm, inverse=True); mark("partition")
             if with_bwd:
-                layer.partition(dev["do"], layer.do_bm); mark("partition")
-                if fold:
-                    # the backward kernels write dq, dk, dv in raster order themselves (inverse of Eq. 1 folded in)
-                    layer.attn_bwd_raster_out(outs["dq"], outs["dk"], outs["dv"]); mark("attn_bwd")
+                if fold and args.fold_do:
+                    # the backward kernels read dO and write dq, dk, dv in raster order themselves (Eq. 1 folded in)
+                    layer.attn_bwd_raster(dev["do"], outs["dq"], outs["dk"], outs["dv"]); mark("attn_bwd")
+                elif fold:
+                    layer.partition(dev["do"], layer.do_bm); mark("partition")
+                    layer.attn_bwd_raster(None, outs["dq"], outs["dk"], outs["dv"]); mark("attn_bwd")
                 else:
+                    layer.partition(dev["do"], layer.do_bm); mark("partition")
                     layer.attn_bwd(); mark("attn_bwd")
                     layer.partition(outs["dq"], layer.dq_bm, inverse=True)
                     layer.partition(outs["dk"], layer.dk_bm, inverse=True)
@@ -462,7 +467,7 @@ def main():
 
     es = 2 if w0.dtype == "bf16" else 4
     tensor_bytes = w0.B * w0.S * w0.heads * w0.head_dim * es
-    n_part = len(layers) * ((5 if fold else 8) if with_bwd else 4)     # partition passes of a step
+    n_part = len(layers) * (((4 if args.fold_do else 5) if fold else 8) if with_bwd else 4)     # partition passes of a step
     alg = {
         "partition": ("hbm", 2.0 * tensor_bytes * n_part),
         "scores": ("hbm", sum(2.0 * tensor_bytes + 4.0 * w.B * w.heads * (w.S * w.n_blocks + w.n_blocks * w.head_dim)

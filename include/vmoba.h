@@ -223,18 +223,22 @@ int vmoba_attn_bwd(const vmoba_shape* shape, const void* q_bm, const void* k_bm,
                    void* dv_bm, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
 
 /*
- * The same backward with the inverse of Eq. 1 folded into the kernels that write the gradients: dq, dk and
- * dv are written in RASTER order, [B, S, heads, head_dim] addressed by element strides raster_strides_bsh =
- * {batch, token, head} (head_dim contiguous, every stride a multiple of 16 bytes), the row of block-major
- * position p going to token perm[p] (perm: device int32 [S], as produced by vmoba_partition).  Saves the
- * three inverse vmoba_partition passes of a training step.  Inputs, workspace and errors as vmoba_attn_bwd;
- * bf16 with head_dim 128 only (VMOBA_ERR_NOT_IMPLEMENTED otherwise).
+ * The same backward with Eq. 1 and its inverse folded into the kernels that read dO and write the gradients:
+ * d_o is read and dq, dk, dv are written in RASTER order, [B, S, heads, head_dim] addressed by element strides
+ * {batch, token, head} (do_strides_bsh for d_o, grad_strides_bsh for the three gradients; head_dim contiguous,
+ * every stride a multiple of 16 bytes), the row of block-major position p being token perm[p] (perm: device
+ * int32 [S], as produced by vmoba_partition).  do_strides_bsh may be NULL: d_o is then block-major like the
+ * other inputs.  Saves the three inverse partition passes of a training step and, with a raster d_o, the
+ * partition pass of dO (its gathered reads from raster order cost more than that pass when the head count is
+ * large: see the design notes).  The other inputs, the workspace and the errors are those of vmoba_attn_bwd; bf16
+ * with head_dim 128 only (VMOBA_ERR_NOT_IMPLEMENTED otherwise).
  */
-int vmoba_attn_bwd_raster_out(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
-                              const void* o_bm, const void* o_resid_or_null, const float* lse, const void* do_bm,
-                              const int32_t* kb_ptr, const int32_t* q_idx, const int32_t* q_ptr, int64_t capacity,
-                              void* dq, void* dk, void* dv, const int64_t raster_strides_bsh[3],
-                              const int32_t* perm, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+int vmoba_attn_bwd_raster(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
+                          const void* o_bm, const void* o_resid_or_null, const float* lse, const void* d_o,
+                          const int64_t do_strides_bsh[3], const int32_t* kb_ptr, const int32_t* q_idx,
+                          const int32_t* q_ptr, int64_t capacity, void* dq, void* dk, void* dv,
+                          const int64_t grad_strides_bsh[3], const int32_t* perm, int32_t* dev_status, void* ws,
+                          size_t ws_bytes, void* stream);
 
 /*
  * Dense softmax attention over all S keys: the tau = 1 limit of the layer and the speed-up

@@ -22,7 +22,7 @@ int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, voi
 // attn_tc_bwd.cu: tensor-core backward kernels (bf16, head_dim 128)
 int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                   const float* Dv, const int* kb_ptr, const int* q_idx, long long cap, float* dq_acc, void* dk, void* dv,
-                  int32_t* status, cudaStream_t st, const RowMap& out_map);
+                  int32_t* status, cudaStream_t st, const RowMap& out_map, const RowMap& do_map);
 int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* Dv, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st);
 
@@ -82,21 +82,21 @@ template <typename T, int DH>
 static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* o,
                            const void* o_resid, const float* lse, const void* d_o, const int* kb_ptr, const int* q_idx,
                            const int* q_ptr, long long cap, void* dq, void* dk, void* dv, int32_t* status, void* ws,
-                           cudaStream_t st, const RowMap& out_map) {
-  // gradients in raster order (out_map.perm set) are written by the tensor-core kernels only
-  if (out_map.perm && !use_tensor_cores(D)) return VMOBA_ERR_NOT_IMPLEMENTED;
+                           cudaStream_t st, const RowMap& out_map, const RowMap& do_map) {
+  // raster-order dO / gradients (perm set) are handled by the tensor-core kernels only
+  if ((out_map.perm || do_map.perm) && !use_tensor_cores(D)) return VMOBA_ERR_NOT_IMPLEMENTED;
   BwdWs w = carve_bwd(D, false, ws, cap);
   const long long n_kb = (long long)D.BH * D.Nb;
   const long long nq = (long long)D.BH * D.S;
   simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>((const T*)o, (const T*)o_resid,
-                                                                        (const T*)d_o, nq, w.Dv);
+                                                                        (const T*)d_o, nq, w.Dv, do_map);
   if (use_tensor_cores(D)) {
     // the backward kernel adds every dQ contribution into the fp32 accumulator: clear the rows of all
     // selecting queries, convert them afterwards (rows of queries without a block become zero)
     const int min_nb = 1;
     simt::zero_multi_rows_kernel<DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, q_ptr, nq, min_nb);
     count_launches(2);
-    int rc = tc_sparse_bwd(D, q, k, v, d_o, lse, w.Dv, kb_ptr, q_idx, cap, w.dq_acc, dk, dv, status, st, out_map);
+    int rc = tc_sparse_bwd(D, q, k, v, d_o, lse, w.Dv, kb_ptr, q_idx, cap, w.dq_acc, dk, dv, status, st, out_map, do_map);
     if (rc) return rc;
     simt::cast_rows_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, q_ptr, nq, 1, min_nb, out_map);
     VMOBA_LAUNCH_OK(1);
@@ -240,38 +240,46 @@ extern "C" int vmoba_attn_bwd(const vmoba_shape* shape, const void* q_bm, const 
   if (D.dtype != VMOBA_BF16) o_resid_or_null = nullptr;
   if (!aligned16(o_resid_or_null)) return VMOBA_ERR_ARG;
   VMOBA_DISPATCH(simt_sparse_bwd, D, q_bm, k_bm, v_bm, o_bm, o_resid_or_null, lse, do_bm, kb_ptr, q_idx, q_ptr,
-                 capacity, dq_bm, dk_bm, dv_bm, dev_status, ws, st, RowMap());
+                 capacity, dq_bm, dk_bm, dv_bm, dev_status, ws, st, RowMap(), RowMap());
 }
 
-extern "C" int vmoba_attn_bwd_raster_out(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
-                                         const void* o_bm, const void* o_resid_or_null, const float* lse,
-                                         const void* do_bm, const int32_t* kb_ptr, const int32_t* q_idx,
-                                         const int32_t* q_ptr, int64_t capacity, void* dq, void* dk, void* dv,
-                                         const int64_t raster_strides_bsh[3], const int32_t* perm,
-                                         int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+extern "C" int vmoba_attn_bwd_raster(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
+                                     const void* o_bm, const void* o_resid_or_null, const float* lse,
+                                     const void* d_o, const int64_t do_strides_bsh[3], const int32_t* kb_ptr,
+                                     const int32_t* q_idx, const int32_t* q_ptr, int64_t capacity, void* dq, void* dk,
+                                     void* dv, const int64_t grad_strides_bsh[3], const int32_t* perm,
+                                     int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
   Dims D;
   int rc = make_dims(shape, &D);
   if (rc) return rc;
-  if (!q_bm || !k_bm || !v_bm || !o_bm || !lse || !do_bm || !kb_ptr || !q_idx || !q_ptr || !dq || !dk || !dv ||
-      !raster_strides_bsh || !perm || !dev_status || !ws)
+  if (!q_bm || !k_bm || !v_bm || !o_bm || !lse || !d_o || !kb_ptr || !q_idx || !q_ptr || !dq || !dk || !dv ||
+      !grad_strides_bsh || !perm || !dev_status || !ws)
     return VMOBA_ERR_ARG;
-  if (!aligned16(q_bm) || !aligned16(k_bm) || !aligned16(v_bm) || !aligned16(o_bm) || !aligned16(do_bm) ||
+  if (!aligned16(q_bm) || !aligned16(k_bm) || !aligned16(v_bm) || !aligned16(o_bm) || !aligned16(d_o) ||
       !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(ws))
     return VMOBA_ERR_ARG;
   // rows must stay 16-byte aligned
   const int per16 = 16 / D.es;
-  for (int i = 0; i < 3; ++i)
-    if (raster_strides_bsh[i] < 0 || raster_strides_bsh[i] % per16) return VMOBA_ERR_ARG;
+  for (int i = 0; i < 3; ++i) {
+    if (grad_strides_bsh[i] < 0 || grad_strides_bsh[i] % per16) return VMOBA_ERR_ARG;
+    if (do_strides_bsh && (do_strides_bsh[i] < 0 || do_strides_bsh[i] % per16)) return VMOBA_ERR_ARG;
+  }
   if (capacity <= 0 || capacity > (int64_t)INT32_MAX) return VMOBA_ERR_ARG;
   if (ws_bytes < carve_bwd(D, false, nullptr, capacity).bytes) return VMOBA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (D.dtype != VMOBA_BF16) o_resid_or_null = nullptr;
   if (!aligned16(o_resid_or_null)) return VMOBA_ERR_ARG;
-  RowMap map;
-  map.perm = perm; map.sb = raster_strides_bsh[0]; map.st = raster_strides_bsh[1]; map.sh = raster_strides_bsh[2];
-  map.heads = D.heads; map.S = D.S;
-  VMOBA_DISPATCH(simt_sparse_bwd, D, q_bm, k_bm, v_bm, o_bm, o_resid_or_null, lse, do_bm, kb_ptr, q_idx, q_ptr,
-                 capacity, dq, dk, dv, dev_status, ws, st, map);
+  RowMap out_map, do_map;
+  out_map.perm = perm;
+  out_map.heads = do_map.heads = D.heads;
+  out_map.S = do_map.S = D.S;
+  out_map.sb = grad_strides_bsh[0]; out_map.st = grad_strides_bsh[1]; out_map.sh = grad_strides_bsh[2];
+  if (do_strides_bsh) {     // else d_o is block-major
+    do_map.perm = perm;
+    do_map.sb = do_strides_bsh[0]; do_map.st = do_strides_bsh[1]; do_map.sh = do_strides_bsh[2];
+  }
+  VMOBA_DISPATCH(simt_sparse_bwd, D, q_bm, k_bm, v_bm, o_bm, o_resid_or_null, lse, d_o, kb_ptr, q_idx, q_ptr,
+                 capacity, dq, dk, dv, dev_status, ws, st, out_map, do_map);
 }
 
 extern "C" int vmoba_full_attn(const vmoba_shape* shape, const void* q, const void* k, const void* v, void* o,

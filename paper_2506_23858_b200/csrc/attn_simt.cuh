@@ -280,18 +280,19 @@ merge_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pairs, lon
 template <typename T, int DH>
 __global__ void __launch_bounds__(256)
 rowdot_kernel(const T* __restrict__ o, const T* __restrict__ o_resid, const T* __restrict__ d_o, long long n_queries,
-              float* __restrict__ Dv) {
+              float* __restrict__ Dv, const RowMap do_map = RowMap()) {
   constexpr int C = DH / 32;
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
   for (long long g = warp; g < n_queries; g += nwarps) {
     float a = 0.f;
+    const T* do_row = d_o + do_map.off(g, DH);
 #pragma unroll
     for (int c = 0; c < C; ++c) {
       float ov = to_f32<T>(o[g * DH + lane * C + c]);
       if (o_resid) ov += to_f32<T>(o_resid[g * DH + lane * C + c]);
-      a = fmaf(ov, to_f32<T>(d_o[g * DH + lane * C + c]), a);
+      a = fmaf(ov, to_f32<T>(do_row[lane * C + c]), a);
     }
 #pragma unroll
     for (int s = 16; s > 0; s >>= 1) a += __shfl_xor_sync(0xffffffffu, a, s);

@@ -114,6 +114,7 @@ struct KvParams {
   __nv_bfloat16 *dk, *dv;
   int dkv_32;                  // dk and dv are 32-byte aligned: rows go out with 32-byte stores
   RowMap out_map;              // where the dK / dV rows go (block-major, or raster order through perm)
+  RowMap do_map;               // where the dO rows come from (likewise)
   float* dq_acc;               // fp32 [queries][head_dim], zeroed rows of all selecting queries
   int32_t* status;
   unsigned long long* prof;    // optional wait-time counters (diagnostics), or null
@@ -337,7 +338,10 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
       const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
       const __nv_bfloat16* qh = p.q + it.head_off * DH + chunk * 8;
-      const __nv_bfloat16* oh = p.d_o + it.head_off * DH + chunk * 8;
+      // dO rows: block-major, or in raster order through perm (the batch / head part of the address once per item)
+      const bool do_raster = p.do_map.perm != nullptr;
+      const int b_ = it.bh / p.do_map.heads, hd_ = it.bh - b_ * p.do_map.heads;
+      const __nv_bfloat16* oh = p.d_o + (do_raster ? b_ * p.do_map.sb + hd_ * p.do_map.sh : it.head_off * DH) + chunk * 8;
       for (int i = 0; i < it.n_units; ++i) {
         const uint32_t u = u0 + i;
         const int cb = u % NQ;
@@ -368,10 +372,12 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         for (int k = 0; k < 8; ++k) {
           const int row = (lt >> 4) + 8 * k;
           const uint32_t off = panel * CPANEL + row * 128 + ((cc ^ (row & 7)) << 4);
-          const long long src = (long long)(idx[k] < 0 ? 0 : idx[k]) * DH;
+          const int ik = idx[k] < 0 ? 0 : idx[k];
+          const long long src = (long long)ik * DH;
+          const long long osrc = do_raster ? (long long)__ldg(p.do_map.perm + ik) * p.do_map.st : src;
           const uint32_t bytes = idx[k] < 0 ? 0u : 16u;
           cp_async16(dst + off, qh + src, bytes);
-          cp_async16(dst + CTILE + off, oh + src, bytes);
+          cp_async16(dst + CTILE + off, oh + osrc, bytes);
         }
         if (lt < QC) { sm->lse2[cb][lt] = l2; sm->Dq[cb][lt] = dd; }
         cp_async_commit();
@@ -607,7 +613,7 @@ int tc_long_dq(const Dims& D, bool dense, const void* q, const void* k, const vo
 // an fp32 accumulator whose rows of selecting queries are zero; the caller converts it to bf16.
 int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                   const float* Dv, const int* kb_ptr, const int* q_idx, long long cap, float* dq_acc, void* dk, void* dv,
-                  int32_t* status, cudaStream_t st, const RowMap& out_map) {
+                  int32_t* status, cudaStream_t st, const RowMap& out_map, const RowMap& do_map) {
   using namespace tcb;
   CUtensorMap tmK, tmV;
   const uint64_t rows = (uint64_t)D.BH * D.S;
@@ -621,6 +627,7 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
   kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status; kp.prof = tcb::g_wait_profile;
   kp.dq_acc = dq_acc;
   kp.out_map = out_map;
+  kp.do_map = do_map;
   kp.dkv_32 = (reinterpret_cast<uintptr_t>(dk) % 32) == 0 && (reinterpret_cast<uintptr_t>(dv) % 32) == 0 &&
               (!out_map.perm || (out_map.sb % 16 == 0 && out_map.st % 16 == 0 && out_map.sh % 16 == 0));
   const long long kv_items = n_kb * ((D.sb + BN - 1) / BN);

@@ -105,11 +105,14 @@ class VmobaLayer:
         return (self.shape.dtype == vb.BF16 and self.d == 128 and self.raster_strides(dk_out) == strides
                 and self.raster_strides(dv_out) == strides)
 
-    def attn_bwd_raster_out(self, dq_out, dk_out, dv_out):
-        """Backward writing dq, dk, dv in raster order (needs self.perm from the forward's partition of q)."""
-        vb.vmoba_attn_bwd_raster_out(self.shape, self.q_bm, self.k_bm, self.v_bm, self.o_bm, self.o_resid, self.lse,
-                                     self.do_bm, self.kb_ptr, self.q_idx, self.q_ptr, self.capacity, dq_out, dk_out,
-                                     dv_out, self.raster_strides(dq_out), self.perm, self.dev_status, self.ws)
+    def attn_bwd_raster(self, do_raster_or_none, dq_out, dk_out, dv_out):
+        """Backward writing dq, dk, dv in raster order (needs self.perm from the forward's partition of q); dO is
+        read in raster order too if given, else from self.do_bm."""
+        do = self.do_bm if do_raster_or_none is None else do_raster_or_none
+        dos = None if do_raster_or_none is None else self.raster_strides(do)
+        vb.vmoba_attn_bwd_raster(self.shape, self.q_bm, self.k_bm, self.v_bm, self.o_bm, self.o_resid, self.lse, do,
+                                 dos, self.kb_ptr, self.q_idx, self.q_ptr, self.capacity, dq_out,
+                                 dk_out, dv_out, self.raster_strides(dq_out), self.perm, self.dev_status, self.ws)
 
     # ---- whole layer --------------------------------------------------------------------
     def forward(self, q, k, v, tau, o_out):
@@ -122,16 +125,20 @@ class VmobaLayer:
         self.attn_fwd()
         self.partition(o_out, self.o_bm, inverse=True)
 
-    def backward(self, do, dq_out, dk_out, dv_out, fold_inverse=None):
+    def backward(self, do, dq_out, dk_out, dv_out, fold_inverse=None, fold_do=False):
         """Gradients of the last forward(); do and the outputs are raster-order [B, S, heads, d].
 
         fold_inverse: let the backward kernels write dq, dk, dv in raster order themselves (bf16, head_dim 128,
-        outputs with equal strides) instead of three inverse partition passes; default: whenever possible."""
-        self.partition(do, self.do_bm)
+        outputs with equal strides) instead of three inverse partition passes; default: whenever possible.
+        fold_do: also let them read dO in raster order instead of partitioning it first (pays with few heads)."""
         if fold_inverse is None:
             fold_inverse = self.can_fold_inverse(dq_out, dk_out, dv_out)
+        if fold_inverse and fold_do:
+            self.attn_bwd_raster(do, dq_out, dk_out, dv_out)
+            return
+        self.partition(do, self.do_bm)
         if fold_inverse:
-            self.attn_bwd_raster_out(dq_out, dk_out, dv_out)
+            self.attn_bwd_raster(None, dq_out, dk_out, dv_out)
             return
         self.attn_bwd()
         self.partition(dq_out, self.dq_bm, inverse=True)

@@ -153,8 +153,8 @@ def test_wide_logit_range_forward_backward(block):
 
 @pytest.mark.parametrize("block", [(1, 12, 26), (3, 6, 13)], ids=["1d", "3d"])
 def test_backward_writing_raster_order_equals_inverse_partition(block):
-    """vmoba_attn_bwd_raster_out folds the inverse of Eq. 1 into the gradient writes: dK and dV must equal
-    vmoba_attn_bwd followed by the inverse partition bit for bit, dQ up to the order of its fp32 sum."""
+    """vmoba_attn_bwd_raster folds Eq. 1 into the reads of dO and its inverse into the gradient writes: dK and dV
+    must equal partition + vmoba_attn_bwd + inverse partition bit for bit, dQ up to the order of its fp32 sum."""
     w = MID.with_(block=block)
     data = gen.make_inputs(w)
     shape = vb.shape_of(w)
@@ -164,7 +164,7 @@ def test_backward_writing_raster_order_equals_inverse_partition(block):
     L.forward(q, k, v, w.tau, o)
     got = [torch.full_like(q, float("nan")) for _ in range(3)]
     ref = [torch.empty_like(q) for _ in range(3)]
-    L.backward(do, *got, fold_inverse=True)
+    L.backward(do, *got, fold_inverse=True, fold_do=True)
     L.backward(do, *ref, fold_inverse=False)
     torch.cuda.synchronize()
     L.check_status()
@@ -174,7 +174,7 @@ def test_backward_writing_raster_order_equals_inverse_partition(block):
     assert diff <= 2.0 ** -6 * max(1.0, ref[0].float().abs().max().item())
     # a strided destination: the gradients of a fused [B, S, heads, 3, d] buffer
     fused = torch.full((w.B, w.S, w.heads, 3, w.head_dim), float("nan"), dtype=q.dtype, device=q.device)
-    L.backward(do, fused[:, :, :, 0], fused[:, :, :, 1], fused[:, :, :, 2], fold_inverse=True)
+    L.backward(do, fused[:, :, :, 0], fused[:, :, :, 1], fused[:, :, :, 2], fold_inverse=True)     # dO block-major
     torch.cuda.synchronize()
     L.check_status()
     assert torch.equal(fused[:, :, :, 1], ref[1]) and torch.equal(fused[:, :, :, 2], ref[2])
