@@ -495,14 +495,34 @@ cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, const int* 
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
-  for (long long g = warp; g < n_queries; g += nwarps) {
-    const int nb = sparse_rows ? q_ptr[g + 1] - q_ptr[g] : 2;
-    if (nb > 0 && nb < min_nb) continue;   // written directly by the attention kernel
-    T* out = dst + map.off(g, DH);
-    if constexpr (C == 4) {
-      const float4 v = nb == 0 ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(src + g * DH + lane * 4);
-      store4(out + lane * 4, v);
-    } else {
+  if constexpr (C == 4) {
+    // Four rows per warp and trip, in phases (list bounds, row offsets, loads, stores), so that the
+    // loads of the four rows are in flight together.
+    constexpr int R = 4;
+    for (long long g0 = warp * R; g0 < n_queries; g0 += nwarps * R) {
+      int nb[R];
+      long long off[R];
+      float4 v[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const long long g = g0 + r;
+        nb[r] = g >= n_queries ? 1 : (sparse_rows ? __ldg(q_ptr + g + 1) - __ldg(q_ptr + g) : 2);
+        if (g >= n_queries || (nb[r] > 0 && nb[r] < min_nb)) nb[r] = -1;   // no row, or written by the attention kernel
+      }
+#pragma unroll
+      for (int r = 0; r < R; ++r) off[r] = nb[r] >= 0 ? map.off(g0 + r, DH) : 0;
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+        v[r] = nb[r] > 0 ? *reinterpret_cast<const float4*>(src + (g0 + r) * DH + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+        if (nb[r] >= 0) store4(dst + off[r] + lane * 4, v[r]);
+    }
+  } else {
+    for (long long g = warp; g < n_queries; g += nwarps) {
+      const int nb = sparse_rows ? q_ptr[g + 1] - q_ptr[g] : 2;
+      if (nb > 0 && nb < min_nb) continue;   // written directly by the attention kernel
+      T* out = dst + map.off(g, DH);
 #pragma unroll
       for (int c = 0; c < C; ++c) out[lane * C + c] = from_f32<T>(nb == 0 ? 0.f : src[g * DH + lane * C + c]);
     }

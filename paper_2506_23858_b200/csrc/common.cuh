@@ -37,9 +37,19 @@ struct RowMap {
 #ifdef __CUDACC__
   __device__ __forceinline__ long long off(long long G, int dh) const {
     if (!perm) return G * dh;
-    const long long bh = G / S;
-    const int p = (int)(G - bh * S);
-    const long long b = bh / heads, hd = bh - b * heads;
+    long long b, hd;
+    int p;
+    if ((unsigned long long)G <= 0x7fffffffull) {   // the usual case: 32-bit quotients
+      const unsigned g = (unsigned)G, bh = g / (unsigned)S, b32 = bh / (unsigned)heads;
+      p = (int)(g - bh * (unsigned)S);
+      b = b32;
+      hd = bh - b32 * (unsigned)heads;
+    } else {
+      const long long bh = G / S;
+      p = (int)(G - bh * S);
+      b = bh / heads;
+      hd = bh - b * heads;
+    }
     return b * sb + (long long)__ldg(perm + p) * st + hd * sh;
   }
 #endif
