@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the Blackwell (sm_100a) features the attention kernels use:
-// mbarrier, TMA tiled loads (no multicast), tcgen05 MMA / TMEM load-store-alloc, proxy fences.
+// mbarrier, TMA tiled loads into this CTA only, tcgen05 MMA / TMEM load-store-alloc, proxy fences.
 // Every wait is bounded: after the limit it records VMOBA_ERR_TIMEOUT in the device status word
 // and lets the caller carry on, so a kernel always terminates and frees its TMEM.
 #pragma once
