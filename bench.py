@@ -155,6 +155,18 @@ def oracle_sample(w, with_bwd, n_rows, seed=0):
                                          pairs_unit=int(k_sel))
 
 
+def workload_config(args, layers, with_bwd):
+    """The `config` object of the JSON line (both arms print the same one; the product arm adds its L2 note)."""
+    w0 = layers[0]
+    cfg = {"workload": args.workload, "passes": "fwd+bwd" if with_bwd else "fwd", "B": w0.B, "heads": w0.heads,
+           "head_dim": w0.head_dim, "grid": [w0.T, w0.H, w0.W], "blocks": [list(w.block) for w in layers],
+           "tau": w0.tau, "rule": args.rule}
+    if "topk" in args.rule:
+        cfg["topk"] = [int(x) for x in args.topk.split(",")] if args.topk else [2]
+    cfg["inputs"] = w0.recipe
+    return cfg
+
+
 def run_reference(args):
     """--impl reference: the oracle as it stands, on the host cores, bounded sample per step."""
     rank = int(os.environ.get("RANK", "0"))
@@ -202,7 +214,7 @@ def run_reference(args):
         "impl": "reference", "metric": "vmoba_layer_selected_pair_tflops", "value": value, "unit": "TFLOP/s",
         "n_gpus": args.gpus, "steps": steps, "warmup": warmup, "ms_per_step": sec * 1e3 * units * len(layers) / n_used,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "passes": "fwd+bwd" if with_bwd else "fwd"},
+        "config": workload_config(args, layers, with_bwd),
         "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
@@ -529,11 +541,7 @@ def main():
         "metric": "vmoba_layer_selected_pair_tflops", "value": flops_all / (ms_per_step * 1e-3) / 1e12,
         "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w0.dtype, "data": "synthetic",
-        "config": {"workload": args.workload, "passes": "fwd+bwd" if with_bwd else "fwd", "B": w0.B,
-                   "heads": w0.heads, "head_dim": w0.head_dim, "grid": [w0.T, w0.H, w0.W],
-                   "blocks": [list(w.block) for w in layers], "tau": w0.tau, "rule": args.rule,
-                   **({"topk": topks} if "topk" in args.rule else {}), "inputs": w0.recipe,
-                   "l2": l2_note},
+        "config": {**workload_config(args, layers, with_bwd), "l2": l2_note},
         "clocks": clocks,
         "e2e": {"value": flops_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": len(names) * tensor_bytes, "d2h_bytes_per_step": len(outs) * tensor_bytes},
