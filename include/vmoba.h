@@ -249,6 +249,25 @@ int vmoba_full_attn(const vmoba_shape* shape, const void* q, const void* k, cons
                     float* lse, const void* do_or_null, void* dq, void* dk, void* dv,
                     int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * Diagnostics; not part of the method.  Registers a device buffer of 16 uint64 counters (NULL: clears the
+ * registration) into which the tensor-core attention kernels launched afterwards ADD, per CTA, the clock
+ * cycles that one representative thread of each warp role spent in each section of its loop; divide by the
+ * grid size (one CTA per SM) for cycles per CTA.  The caller zeroes the buffer before a launch, reads it after
+ * synchronising, and keeps it alive until it is cleared here.  Process-wide, not thread-safe; kernels run a
+ * little slower while a buffer is registered, and their results do not change.
+ *   forward kernel:  [0] softmax thread waiting for scores, [1] score read + row maximum, [2] accumulator
+ *     rescale, [3] exponentials + P written, [4] epilogue (wait for the last P V, normalise, write), [6] its
+ *     total; MMA warp: [8] wait for Q, [9] for K, [10] for P, [11] for V, [12] for a free accumulator,
+ *     [13] issuing, [14] its total.
+ *   backward kernel: [0] TMA warp waiting for free K / V buffers; [1] the TMA warp's total plus the writer
+ *     warp's staging and reductions (one slot); MMA warp: [2] wait for K / V, [3] for a gathered chunk, [4] for
+ *     P^T / dS^T, [5] for free accumulators or the dQ^T buffer, [6] its total; loaders: [7] wait for a free
+ *     chunk, [8] total; compute warps: [10] wait for a chunk, [11] for S^T / dP^T, [12] for the dK / dV hand-off,
+ *     [13] total; writer warp: [9] wait for dQ^T, [14] reading it from TMEM, [15] waiting at the staging barrier.
+ */
+void vmoba_debug_wait_profile(void* dev_counters16);
+
 #ifdef __cplusplus
 }
 #endif

@@ -18,6 +18,7 @@ STAGE_SCORES, STAGE_SELECT, STAGE_ATTN_FWD, STAGE_ATTN_BWD, STAGE_FULL_FWD, STAG
 EXPORTS = (
     "vmoba_status_string", "vmoba_kernel_launches", "vmoba_workspace_bytes", "vmoba_partition", "vmoba_block_scores",
     "vmoba_select", "vmoba_select_static", "vmoba_select_static_scratch_bytes", "vmoba_attn_fwd", "vmoba_attn_bwd", "vmoba_attn_bwd_raster", "vmoba_full_attn",
+    "vmoba_debug_wait_profile",
 )
 
 
@@ -108,6 +109,8 @@ def lib():
     L.vmoba_attn_bwd_raster.restype = ctypes.c_int
     L.vmoba_attn_bwd_raster.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(ctypes.c_int64), vp, vp, vp, i64,
                                         vp, vp, vp, ctypes.POINTER(ctypes.c_int64), vp, vp, vp, sz, vp]
+    L.vmoba_debug_wait_profile.restype = None
+    L.vmoba_debug_wait_profile.argtypes = [vp]
     L.vmoba_full_attn.restype = ctypes.c_int
     L.vmoba_full_attn.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     _lib = L
@@ -229,3 +232,10 @@ def vmoba_full_attn(shape, q, k, v, o, lse, do=None, dq=None, dk=None, dv=None, 
     _check(lib().vmoba_full_attn(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(do),
                                  _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dev_status), p, n, _stream(stream)),
            "vmoba_full_attn")
+
+
+def vmoba_debug_wait_profile(counters=None):
+    """Registers a zeroed device tensor of 16 int64 counters for the attention kernels' section timers (None: clears)."""
+    if counters is not None and (counters.numel() < 16 or counters.element_size() != 8 or not counters.is_cuda):
+        raise ValueError("vmoba_debug_wait_profile: need a CUDA tensor of at least 16 64-bit counters")
+    lib().vmoba_debug_wait_profile(_ptr(counters))

@@ -194,6 +194,32 @@ def test_repeated_runs_reproduce():
         assert diff <= 2.0 ** -6 * max(1.0, runs[0]["dq"].float().abs().max().item())
 
 
+def test_section_timers_leave_results_unchanged():
+    """The diagnostic counters (cycles per warp role and loop section) fill in when a buffer is registered and the
+    outputs stay bit-identical (dQ up to its summation order)."""
+    w = MID.with_(block=(1, 12, 26))
+    data = gen.make_inputs(w)
+    plain = _run_layer(w, data, with_bwd=True)
+    counters = torch.zeros(16, dtype=torch.int64, device="cuda")
+    vb.vmoba_debug_wait_profile(counters)
+    try:
+        timed = _run_layer(w, data, with_bwd=True)
+        torch.cuda.synchronize()
+    finally:
+        vb.vmoba_debug_wait_profile(None)
+    c = counters.cpu().numpy()
+    assert c[6] > 0 and c[13] > 0 and c[8] > 0      # totals of three roles
+    assert np.all(c >= 0)
+    for name in ("o", "dk", "dv"):
+        assert torch.equal(timed[name], plain[name]), name
+    diff = (timed["dq"].float() - plain["dq"].float()).abs().max().item()
+    assert diff <= 2.0 ** -6 * max(1.0, plain["dq"].float().abs().max().item())
+    after = _run_layer(w, data, with_bwd=True)        # cleared: the buffer is no longer written
+    torch.cuda.synchronize()
+    assert np.array_equal(counters.cpu().numpy(), c)
+    assert torch.equal(after["o"], plain["o"])
+
+
 def test_mid_size_threshold_one_equals_dense_path():
     """tau = 1.0 through the sparse pipeline must equal the library's dense path and the oracle's dense attention."""
     w = MID.with_(tau=1.0, B=1, heads=2)
