@@ -39,6 +39,12 @@ struct HeadState {
 };
 
 // bin of a score at refinement level L given the state; monotone non-decreasing in s.
+// Unnormalised softmax weight of a pair relative to the head's largest score (Eq. 4 accumulates these
+// in descending score order).  One definition for every histogram level and for the final exact
+// steps, so that the masses they hand to each other are sums of the same numbers; the fast
+// exponential (one multiply, one ex2) is within a few ulp of expf over the range that carries mass.
+__device__ __forceinline__ float pair_weight(float sigma, float s, float smax) { return __expf(sigma * (s - smax)); }
+
 __device__ __forceinline__ int bin_at(const HeadState& hs, int L, float s) {
   float t = (s - hs.anchor[L]) * hs.inv[L];
   int b = t > 0.f ? (int)fminf(t, (float)((L == 0 ? kBins0 : kBins) - 1)) : 0;
@@ -127,7 +133,7 @@ hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __re
     if (L >= 2 && bin_at(hs, 1, s) != hs.bin[1]) return;
     int b = bin_at(hs, L, s);
     atomicAdd(&s_cnt[b], 1u);
-    atomicAdd(&s_w[b], unit_w ? 1.0f : expf(sigma * (s - smax)));
+    atomicAdd(&s_w[b], unit_w ? 1.0f : pair_weight(sigma, s, smax));
     atomicMin(&s_min[b], float_key(s));
     if (L == 1) atomicMax(&s_max[b], float_key(s));
   });
@@ -159,7 +165,7 @@ hist0_kernel(const float* __restrict__ scores, long long P, const HeadState* __r
   const float smax = key_float(hs.max_key);
   const int rep = threadIdx.x & (kRep - 1);
   for_each_score(scores + (long long)bh * P, P, [&](float s) {
-    atomicAdd(&s_wr[bin_at(hs, 0, s) * kRep + rep], unit_w ? 1.0f : expf(sigma * (s - smax)));
+    atomicAdd(&s_wr[bin_at(hs, 0, s) * kRep + rep], unit_w ? 1.0f : pair_weight(sigma, s, smax));
   });
   __syncthreads();
   for (int i = threadIdx.x; i < kBins0; i += blockDim.x) {
@@ -535,7 +541,7 @@ select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, flo
       double z = 0.0;
 #pragma unroll
       for (int i = 0; i < MW; ++i) {
-        w[i] = key[i] ? (double)expf(sigma * (key_float(key[i]) - smax)) : 0.0;
+        w[i] = key[i] ? (double)pair_weight(sigma, key_float(key[i]), smax) : 0.0;
         z += w[i];
       }
 #pragma unroll
@@ -583,7 +589,7 @@ select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, flo
         if (TOPK) {
           done = r + 1 == rounds;
         } else {
-          acc += (double)expf(sigma * (key_float(m) - key_float(kmax)));
+          acc += (double)pair_weight(sigma, key_float(m), key_float(kmax));
           done = acc >= target;
         }
       }
