@@ -67,7 +67,8 @@ _lib = None
 
 
 def lib_path() -> str:
-    return _build.LIB_PATH
+    """The in-tree library, or the file VMOBA_LIB names (another build of this same library)."""
+    return os.environ.get("VMOBA_LIB") or _build.LIB_PATH
 
 
 def lib():
@@ -76,8 +77,9 @@ def lib():
     if _lib is not None:
         return _lib
     path = lib_path()
-    if not os.path.exists(path):
-        _build.build()          # needs nvcc; raises if the build fails -- there is no CPU fallback
+    if path == _build.LIB_PATH:
+        _build.ensure_built()   # rebuilds when a source is newer than the library; needs nvcc, raises if the build
+                                # fails -- there is no CPU fallback
     if not os.path.exists(path):
         raise RuntimeError(f"{path} is missing: run `python -m paper_2506_23858_b200.build` (no CPU fallback exists)")
     L = ctypes.CDLL(path)

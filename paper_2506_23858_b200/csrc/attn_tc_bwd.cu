@@ -11,9 +11,9 @@
 //     dV += P^T dO,  dK += dS^T Q                        (two TS MMAs, A = bf16 P^T / dS^T in TMEM;
 //                                                         B = the same dO / Q tiles read MN-major)
 //   Every key belongs to exactly one item: dK and dV are written once, no atomics.  dQ^T of a chunk
-//   is read out of TMEM by four writer warps, transposed through shared memory (32 queries at a
-//   time) and added into an fp32 accumulator with one red.global.add.v4.f32 warp instruction per query
-//   row (512 bytes), the rows shared between the writer warps and two helper warps.
+//   is read out of TMEM by eight writer warps (lane = head-dim index), transposed four queries at a
+//   time among groups of four lanes with shuffles, and added into an fp32 accumulator with
+//   red.global.add.v4.f32 (per warp instruction: complete 128-byte lines of four query rows).
 //
 // D = rowsum(dO * O) and lse come in per query; exp runs in the exp2 domain (c = scale * log2 e).
 // The dense path uses the kernels with 128-query units in the companion file.
@@ -37,10 +37,6 @@ constexpr float LOG2E = 1.4426950408889634f;
 static unsigned long long* g_wait_profile = nullptr;
 constexpr uint32_t IDESC_TN = make_idesc_bf16(128, 128, false, true);    // A from TMEM, B MN-major
 
-// named barrier of the dQ writer and helper warps
-constexpr int RED_HELPERS = 2;               // warps that only send out staged dQ rows, next to the four writer warps
-constexpr int RED_WARPS = 4 + RED_HELPERS;
-__device__ __forceinline__ void writer_sync() { asm volatile("bar.sync 5, %0;" ::"n"(32 * RED_WARPS) : "memory"); }
 // Asynchronous 16-byte copy global -> shared (bypassing L1); `bytes` = 16, or 0 to write zeros.
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc, uint32_t bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(bytes) : "memory");
@@ -89,18 +85,17 @@ struct KvSmem {
   uint32_t tmem_base;
   int abort_flag;
   uint64_t dq_full[2];                       // dQ^T of a unit complete (commit)
-  uint64_t dq_free[2];                       // dQ^T read out of TMEM (128 writer arrivals)
+  uint64_t dq_free[2];                       // dQ^T read out of TMEM (256 writer arrivals)
   alignas(16) float lse2[NQ][QC];
   alignas(16) float Dq[NQ][QC];
 };
 constexpr int DSTILE = 128 * 128;            // dS^T of a unit in shared memory: [128 keys][64 queries] bf16 (16 KB)
-// one K/V pair, the chunk ring, one dS^T tile, the dQ staging tile
-constexpr int DQSTAGE = (QC / 2) * DH * 4;   // dQ of half a unit as [32 queries][128] fp32 rows for the vector reductions (16 KB)
+// one K/V pair, the chunk ring, one dS^T tile
 // no alignment slack: the kernel checks that its dynamic shared memory starts on a 1024-byte boundary
-constexpr size_t KVF_SMEM_BYTES = 2 * TILE + NQ * 2 * CTILE + DSTILE + DQSTAGE + sizeof(KvSmem) + 32;
+constexpr size_t KVF_SMEM_BYTES = 2 * TILE + NQ * 2 * CTILE + DSTILE + sizeof(KvSmem) + 32;
 static_assert(KVF_SMEM_BYTES <= 232448, "fused backward: shared memory");
-// warps: TMA, MMA, 8 compute, 4 loaders, 4 dQ writers, then the reduction helpers
-constexpr int KVF_THREADS = 576 + 32 * RED_HELPERS;
+// warps: TMA, MMA, 8 compute, 4 loaders, 8 dQ writers
+constexpr int KVF_THREADS = 704;
 constexpr uint32_t IDESC_K64 = make_idesc_bf16(128, QC, false, false);   // S^T, dP^T: N = 64 queries
 constexpr uint32_t IDESC_DQT = make_idesc_bf16(128, QC, true, true);     // dQ^T = K^T dS^T: both operands MN-major
 
@@ -134,27 +129,21 @@ struct KvItem {
   long long list_lo, list_hi, head_off;
 };
 
-template <bool DENSE>
-__device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, int tiles, int span) {
+__device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, int tiles) {
   KvItem it;
   const int tile = (int)(item % tiles);
   const long long kbi = item / tiles;
-  it.bh = DENSE ? (int)kbi : (int)(kbi / p.Nb);
-  const int j = DENSE ? 0 : (int)(kbi - (long long)it.bh * p.Nb);
+  it.bh = (int)(kbi / p.Nb);
+  const int j = (int)(kbi - (long long)it.bh * p.Nb);
   it.key0 = j * p.sb + tile * BN;
-  it.valid = min(BN, span - tile * BN);
-  it.list_lo = 0; it.list_hi = p.S;
-  if (!DENSE) {
-    it.list_lo = min((long long)p.kb_ptr[kbi], p.capacity);
-    it.list_hi = min((long long)p.kb_ptr[kbi + 1], p.capacity);
-  }
+  it.valid = min(BN, p.sb - tile * BN);
+  it.list_lo = min((long long)p.kb_ptr[kbi], p.capacity);
+  it.list_hi = min((long long)p.kb_ptr[kbi + 1], p.capacity);
   it.n_units = (int)((it.list_hi - it.list_lo + QC - 1) / QC);
   it.head_off = (long long)it.bh * p.S;
   return it;
 }
 
-// Only DENSE = false is instantiated (DENSE = true walks all queries of the sequence instead of an index list).
-template <bool DENSE>
 __global__ void __launch_bounds__(KVF_THREADS, 1)
 attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const KvParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -168,8 +157,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   uint8_t* sV = base + TILE;           // [TILE]
   uint8_t* sC = base + 2 * TILE;       // [NQ][Q chunk | dO chunk]
   uint8_t* sDS = sC + NQ * 2 * CTILE;  // dS^T of the current unit [DSTILE]
-  float* s_stage = reinterpret_cast<float*>(sDS + DSTILE);                         // [QC / 2][DH] fp32
-  KvSmem* sm = reinterpret_cast<KvSmem*>(sDS + DSTILE + DQSTAGE);
+  KvSmem* sm = reinterpret_cast<KvSmem*>(sDS + DSTILE);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &sm->abort_flag;
   // diagnostics: cycles spent in each wait site by one representative thread per role
@@ -195,7 +183,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sm->kv_full[b], 1); mbar_init(&sm->kv_empty[b], 1);
       mbar_init(&sm->sdp_full[b], 1); mbar_init(&sm->pds_ready[b], 256);
-      mbar_init(&sm->dq_full[b], 1); mbar_init(&sm->dq_free[b], 128);
+      mbar_init(&sm->dq_full[b], 1); mbar_init(&sm->dq_free[b], 256);
     }
     for (int b = 0; b < NQ; ++b) { mbar_init(&sm->chunk_full[b], 128); mbar_init(&sm->chunk_empty[b], 1); }
     mbar_init(&sm->acc_done, 1);
@@ -215,16 +203,15 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   const uint32_t tmem = sm->tmem_base;
   constexpr uint32_t ST_COL = 0, DPT_COL = 128, DV_COL = 256, DK_COL = 384;   // ST/DPT: two 64-column buffers each
 
-  const int span = DENSE ? p.S : p.sb;
-  const int tiles = (span + BN - 1) / BN;
-  const long long n_items = (long long)p.BH * (DENSE ? 1 : p.Nb) * tiles;
+  const int tiles = (p.sb + BN - 1) / BN;
+  const long long n_items = (long long)p.BH * p.Nb * tiles;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA: K and V tiles, one pair per item
     if (lane == 0) {
       uint32_t n = 0;
       for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+        const KvItem it = kv_decode(p, item, tiles);
         if (it.n_units == 0) continue;
         // one K / V pair: the next item's tiles wait for the current item's last MMA
         if (n >= 1) twait(0, &sm->kv_empty[0], (n - 1) & 1);
@@ -248,7 +235,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       auto wwait = [&](int site, uint64_t* bar, uint32_t parity) { twait(site, bar, parity); __syncwarp(); };
       uint32_t n = 0, u0 = 0;      // items and units done so far
       for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-        KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+        KvItem it = kv_decode(p, item, tiles);
         // the list bounds come from memory: a warp reduction marks them as warp-uniform
         const int n_list = __reduce_max_sync(0xffffffffu, (int)(it.list_hi - it.list_lo));
         it.n_units = (n_list + QC - 1) / QC;
@@ -336,7 +323,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     };
     uint32_t u0 = 0;
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-      const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+      const KvItem it = kv_decode(p, item, tiles);
       const __nv_bfloat16* qh = p.q + it.head_off * DH + chunk * 8;
       // dO rows: block-major, or in raster order through perm (the batch / head part of the address once per item)
       const bool do_raster = p.do_map.perm != nullptr;
@@ -347,7 +334,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         const int cb = u % NQ;
         const long long lo = it.list_lo + (long long)i * QC;
         const int rows = (int)min((long long)QC, it.list_hi - lo);
-        auto row_of = [&](int r) { return DENSE ? (int)(lo + r) : __ldg(p.q_idx + lo + r); };
+        auto row_of = [&](int r) { return __ldg(p.q_idx + lo + r); };
         int idx[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -389,93 +376,77 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     if (lt == 0) tflush(7, 1);     // [7] chunk_empty, [8] total
   } else if (warp >= 14) {
     // ------------------------------------------------------------------ dQ writers: thread = head-dim index
-    // Read dQ^T of a unit out of TMEM, release the buffer, transpose it through shared memory into 64
-    // rows of 128 floats and add each row into the fp32 accumulator with one vector-reduction warp
-    // instruction.  (Measured per SM: bulk reductions through the copy engine stop at 8.6 B/cycle;
-    // red.global.add.v4.f32 gives 10 B/cycle from 4 warps, 18.7 from 8, 23 from 16, about one
-    // instruction in flight per warp; but these share the load/store path with the loaders' gathers:
-    // two helper warps that only send rows pay off, a third or a second set of four writer warps slows
-    // the gathers down by more than the reductions gain.)
+    // Read dQ^T of a unit out of TMEM (lane = head-dim index, 64 query columns), release the buffer and add
+    // it into the fp32 accumulator.  The four lanes 4i .. 4i+3 transpose each group of four queries among
+    // themselves with two exchange steps (one shuffle per value), after which lane 4i + j holds head-dim
+    // columns 4i .. 4i+3 of query j of the group: one red.global.add.v4.f32 warp instruction then adds four
+    // complete 128-byte lines, one in each of four accumulator rows.  (Measured per SM with all SMs busy:
+    // reductions that cover whole 128-byte lines reach 23 B/cycle however the lines are spread over rows;
+    // 16 bytes per lane in 32 different rows reach 12.5; scalar line-wide reductions reach 23 alone but
+    // made this kernel 1.5x slower.  An earlier version transposed through a shared-memory tile: a third
+    // of the load/store wavefronts of a unit, on the unit that binds this kernel.)
+    // Eight warps: two per TMEM lane quarter, each taking 32 of a unit's 64 query columns.
     const int quad = warp & 3;
+    const int qhalf = (warp - 14) >> 2;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const int d = quad * 32 + lane;
-    const int wi = warp - 14;                      // 0..3 writers, 4.. helpers
-    constexpr int HR = QC / 2;                     // rows staged at a time
-    constexpr int RPW = (HR + RED_WARPS - 1) / RED_WARPS;   // rows of a half per warp, at most
-    // accumulator rows of this warp's share of a unit (row c = 32 h + wi + RED_WARPS k of the unit), -1 beyond the list
-    auto my_rows = [&](const KvItem& it, int i, int (&rowi)[2][RPW]) {
-      const long long lo = it.list_lo + (long long)i * QC;
-      const int rows = (int)min((long long)QC, it.list_hi - lo);
-#pragma unroll
-      for (int h = 0; h < 2; ++h)
-#pragma unroll
-        for (int k = 0; k < RPW; ++k) {
-          const int c = HR * h + wi + RED_WARPS * k;
-          rowi[h][k] = (wi + RED_WARPS * k < HR && c < rows) ? (int)it.head_off + (DENSE ? (int)(lo + c) : __ldg(p.q_idx + lo + c)) : -1;
-        }
-    };
-    auto send_rows = [&](int h, const int (&rowi)[2][RPW]) {     // one row (512 bytes) per warp instruction
-#pragma unroll
-      for (int k = 0; k < RPW; ++k) {
-        if (rowi[h][k] >= 0) {
-          const float4 v = *reinterpret_cast<const float4*>(s_stage + (wi + RED_WARPS * k) * DH + 4 * lane);
-          red_add_v4(p.dq_acc + (long long)rowi[h][k] * DH + 4 * lane, v.x, v.y, v.z, v.w);
-        }
-      }
+    const int j4 = lane & 3;
+    const bool odd1 = (lane & 1) != 0, odd2 = (lane & 2) != 0;
+    float* acc_col = p.dq_acc + quad * 32 + (lane & ~3);
+    // x[0..3]: this lane's head-dim column for four queries -> head-dim columns 4i .. 4i+3 of query j4
+    auto transpose4 = [&](float x0, float x1, float x2, float x3, float4& y) {
+      // step 1, partner lane ^ 1: even lanes keep queries 0, 2, odd lanes keep queries 1, 3
+      const float r0 = __shfl_xor_sync(0xffffffffu, odd1 ? x0 : x1, 1);
+      const float r1 = __shfl_xor_sync(0xffffffffu, odd1 ? x2 : x3, 1);
+      // (query 0 or 1: columns c, c ^ 1), (query 2 or 3: likewise), in column order
+      const float a0 = odd1 ? r0 : x0, a1 = odd1 ? x1 : r0;
+      const float b0 = odd1 ? r1 : x2, b1 = odd1 ? x3 : r1;
+      // step 2, partner lane ^ 2: lanes 0, 1 keep the first query of their pair, lanes 2, 3 the second
+      const float s0 = __shfl_xor_sync(0xffffffffu, odd2 ? a0 : b0, 2);
+      const float s1 = __shfl_xor_sync(0xffffffffu, odd2 ? a1 : b1, 2);
+      y = odd2 ? make_float4(s0, s1, b0, b1) : make_float4(a0, a1, s0, s1);
     };
     uint32_t u0 = 0;
-    if (wi >= 4) {
-      // helper warps: follow the writers' barriers (two per half unit) and send their share of the staged rows
-      for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
-        for (int i = 0; i < it.n_units; ++i) {
-          int rowi[2][RPW];
-          my_rows(it, i, rowi);
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            writer_sync();
-            writer_sync();
-            send_rows(h, rowi);
-          }
-        }
-        u0 += it.n_units;
-      }
-    } else {
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-      const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+      const KvItem it = kv_decode(p, item, tiles);
+      float* acc_head = acc_col + it.head_off * DH;
       for (int i = 0; i < it.n_units; ++i) {
         const uint32_t u = u0 + i;
         const int tb = u & 1;
-        int rowi[2][RPW];
-        my_rows(it, i, rowi);
+        // accumulator row of query 32 qhalf + lane of the unit (-1 beyond the list)
+        const long long lo = it.list_lo + (long long)i * QC + 32 * qhalf;
+        const int row_lane = lo + lane < it.list_hi ? __ldg(p.q_idx + lo + lane) : -1;
         long long tw0 = p.prof ? clock64() : 0;
         mbar_wait(&sm->dq_full[tb], (u >> 1) & 1, abort_flag, p.status);
         if (p.prof) { const long long t = clock64(); wp[0] += t - tw0; tw0 = t; }
         tc_fence_after();
-        uint32_t a[32], c2[32];
-        tmem_ld32(tmem + lane_addr + DPT_COL + tb * QC, a);
-        tmem_ld32(tmem + lane_addr + DPT_COL + tb * QC + 32, c2);
+        uint32_t x[32];
+        tmem_ld32(tmem + lane_addr + DPT_COL + tb * QC + 32 * qhalf, x);
         tmem_ld_wait();
         tc_fence_before();
         mbar_arrive(&sm->dq_free[tb]);
         if (p.prof) { const long long t = clock64(); wp[1] += t - tw0; tw0 = t; }
-        // first half of the unit's queries; the staging tile is free once every warp has loaded its rows of the previous half
-        writer_sync();
-        if (p.prof) { const long long t = clock64(); wp[2] += t - tw0; tw0 = t; }
+        // The transpositions first, in place, then the eight reductions back to back from eight different
+        // register quadruples: a reduction holds its source registers until the load/store unit has taken them
+        // (about 200 cycles under this kernel's memory traffic), so a loop that reuses one quadruple sends one
+        // reduction per 200 cycles.
+        int rw[8];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) s_stage[c * DH + d] = __uint_as_float(a[c]) * p.scale;
-        writer_sync();
-        send_rows(0, rowi);
-        // second half
-        writer_sync();
+        for (int g = 0; g < 8; ++g) {
+          float4 y;
+          transpose4(__uint_as_float(x[4 * g]), __uint_as_float(x[4 * g + 1]), __uint_as_float(x[4 * g + 2]),
+                     __uint_as_float(x[4 * g + 3]), y);
+          x[4 * g] = __float_as_uint(y.x * p.scale); x[4 * g + 1] = __float_as_uint(y.y * p.scale);
+          x[4 * g + 2] = __float_as_uint(y.z * p.scale); x[4 * g + 3] = __float_as_uint(y.w * p.scale);
+          rw[g] = __shfl_sync(0xffffffffu, row_lane, 4 * g + j4);
+        }
 #pragma unroll
-        for (int c = 0; c < 32; ++c) s_stage[c * DH + d] = __uint_as_float(c2[c]) * p.scale;
-        writer_sync();
-        send_rows(1, rowi);
+        for (int g = 0; g < 8; ++g)
+          if (rw[g] >= 0)
+            red_add_v4(acc_head + (long long)rw[g] * DH, __uint_as_float(x[4 * g]), __uint_as_float(x[4 * g + 1]),
+                       __uint_as_float(x[4 * g + 2]), __uint_as_float(x[4 * g + 3]));
         if (p.prof) { const long long t = clock64(); wp[3] += t - tw0; tw0 = t; }
       }
       u0 += it.n_units;
-    }
     }
     if (p.prof && warp == 14 && lane == 0) {
       atomicAdd(p.prof + 9, wp[0]); atomicAdd(p.prof + 14, wp[1]); atomicAdd(p.prof + 15, wp[2]); atomicAdd(p.prof + 1, wp[3]);
@@ -488,7 +459,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     uint32_t n = 0, u0 = 0;
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-      const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+      const KvItem it = kv_decode(p, item, tiles);
       const long long row_off = r < it.valid ? p.out_map.off(it.head_off + it.key0 + r, DH) : 0;
       __nv_bfloat16* dv_row = p.dv + row_off;
       __nv_bfloat16* dk_row = p.dk + row_off;
@@ -515,42 +486,55 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         const float my_lse2 = sm->lse2[cb][32 * half + lane], my_D = sm->Dq[cb][32 * half + lane];
         const uint32_t st_t = tmem + lane_addr + ST_COL + tb * QC + 32 * half;
         const uint32_t dp_t = tmem + lane_addr + DPT_COL + tb * QC + 32 * half;
-        uint32_t sv[32], dv_[32];
-        tmem_ld32(st_t, sv);
-        tmem_ld32(dp_t, dv_);
-        tmem_ld_wait();
-        uint32_t pk[16], dk_[16];
+        // Two passes of 16 queries each (a thread then holds 16 scores and 16 dP values at a time).  P^T goes
+        // over the first 16 of this thread's 32 S^T columns and dS^T over the other 16 (the dP^T columns are
+        // about to receive dQ^T), so the first pass keeps its dS^T in registers until the second pass has read
+        // the remaining scores.  dS^T is written once more, as the row of this key in the [keys][queries]
+        // shared-memory tile that dQ^T reads; rows beyond the key range hold other blocks' keys and must not
+        // contribute.
+        uint8_t* dsrow = sDS + r * 128;
+        const bool live = r < it.valid;
+        uint32_t dk_first[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          float4 l4, d4;
-          l4.x = __shfl_sync(0xffffffffu, my_lse2, 4 * e);     l4.y = __shfl_sync(0xffffffffu, my_lse2, 4 * e + 1);
-          l4.z = __shfl_sync(0xffffffffu, my_lse2, 4 * e + 2); l4.w = __shfl_sync(0xffffffffu, my_lse2, 4 * e + 3);
-          d4.x = __shfl_sync(0xffffffffu, my_D, 4 * e);        d4.y = __shfl_sync(0xffffffffu, my_D, 4 * e + 1);
-          d4.z = __shfl_sync(0xffffffffu, my_D, 4 * e + 2);    d4.w = __shfl_sync(0xffffffffu, my_D, 4 * e + 3);
-          const float p0 = ex2(fmaf(__uint_as_float(sv[4 * e]), p.scale_log2, -l4.x));
-          const float p1 = ex2(fmaf(__uint_as_float(sv[4 * e + 1]), p.scale_log2, -l4.y));
-          const float p2 = ex2(fmaf(__uint_as_float(sv[4 * e + 2]), p.scale_log2, -l4.z));
-          const float p3 = ex2(fmaf(__uint_as_float(sv[4 * e + 3]), p.scale_log2, -l4.w));
-          pk[2 * e] = pack_bf16(p0, p1);
-          pk[2 * e + 1] = pack_bf16(p2, p3);
-          dk_[2 * e] = pack_bf16(p0 * (__uint_as_float(dv_[4 * e]) - d4.x), p1 * (__uint_as_float(dv_[4 * e + 1]) - d4.y));
-          dk_[2 * e + 1] = pack_bf16(p2 * (__uint_as_float(dv_[4 * e + 2]) - d4.z), p3 * (__uint_as_float(dv_[4 * e + 3]) - d4.w));
-        }
-        tmem_st16(st_t, pk);       // P^T (bf16 pairs) over the first 16 of this thread's 32 S^T columns
-        {
-          tmem_st16(st_t + 16, dk_);   // dS^T over the other 16: the dP^T columns are about to receive dQ^T
-          // and once more, as the row of this key in the [keys][queries] shared-memory tile that dQ^T reads;
-          // rows beyond the key range hold other blocks' keys and must not contribute
-          uint8_t* dsrow = sDS + r * 128;
-          const bool live = r < it.valid;
-          // one tile: the previous unit's dQ^T must have finished reading it
-          if (u >= 1) mbar_wait(&sm->dq_full[(u - 1) & 1], ((u - 1) >> 1) & 1, abort_flag, p.status);
+        for (int pass = 0; pass < 2; ++pass) {
+          uint32_t sv[16], dv_[16];
+          tmem_ld16(st_t + 16 * pass, sv);
+          tmem_ld16(dp_t + 16 * pass, dv_);
+          tmem_ld_wait();
+          if (pass == 1) tmem_st8(st_t + 16, dk_first);
+          uint32_t pk[8], dk_[8];
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            *reinterpret_cast<uint4*>(dsrow + (((4 * half + j) ^ (r & 7)) << 4)) =
+          for (int e = 0; e < 4; ++e) {
+            const int l0 = 16 * pass + 4 * e;
+            float4 l4, d4;
+            l4.x = __shfl_sync(0xffffffffu, my_lse2, l0);     l4.y = __shfl_sync(0xffffffffu, my_lse2, l0 + 1);
+            l4.z = __shfl_sync(0xffffffffu, my_lse2, l0 + 2); l4.w = __shfl_sync(0xffffffffu, my_lse2, l0 + 3);
+            d4.x = __shfl_sync(0xffffffffu, my_D, l0);        d4.y = __shfl_sync(0xffffffffu, my_D, l0 + 1);
+            d4.z = __shfl_sync(0xffffffffu, my_D, l0 + 2);    d4.w = __shfl_sync(0xffffffffu, my_D, l0 + 3);
+            const float p0 = ex2(fmaf(__uint_as_float(sv[4 * e]), p.scale_log2, -l4.x));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[4 * e + 1]), p.scale_log2, -l4.y));
+            const float p2 = ex2(fmaf(__uint_as_float(sv[4 * e + 2]), p.scale_log2, -l4.z));
+            const float p3 = ex2(fmaf(__uint_as_float(sv[4 * e + 3]), p.scale_log2, -l4.w));
+            pk[2 * e] = pack_bf16(p0, p1);
+            pk[2 * e + 1] = pack_bf16(p2, p3);
+            dk_[2 * e] = pack_bf16(p0 * (__uint_as_float(dv_[4 * e]) - d4.x), p1 * (__uint_as_float(dv_[4 * e + 1]) - d4.y));
+            dk_[2 * e + 1] = pack_bf16(p2 * (__uint_as_float(dv_[4 * e + 2]) - d4.z), p3 * (__uint_as_float(dv_[4 * e + 3]) - d4.w));
+          }
+          tmem_st8(st_t + 8 * pass, pk);
+          if (pass == 0) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) dk_first[k] = dk_[k];
+            // one shared-memory tile: the previous unit's dQ^T must have finished reading it
+            if (u >= 1) mbar_wait(&sm->dq_full[(u - 1) & 1], ((u - 1) >> 1) & 1, abort_flag, p.status);
+          } else {
+            tmem_st8(st_t + 24, dk_);
+          }
+#pragma unroll
+          for (int j = 0; j < 2; ++j)
+            *reinterpret_cast<uint4*>(dsrow + (((4 * half + 2 * pass + j) ^ (r & 7)) << 4)) =
                 live ? make_uint4(dk_[4 * j], dk_[4 * j + 1], dk_[4 * j + 2], dk_[4 * j + 3]) : make_uint4(0u, 0u, 0u, 0u);
-          fence_async_proxy();
         }
+        fence_async_proxy();
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(&sm->pds_ready[tb]);
@@ -559,29 +543,26 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
       twait(2, &sm->acc_done, n & 1);
       tc_fence_after();
 #pragma unroll 1
-      for (int cg2 = 0; cg2 < 2; ++cg2) {
-        const int cgrp = half * 2 + cg2;
-        uint32_t a[32], bb[32];
-        tmem_ld32(tmem + lane_addr + DV_COL + cgrp * 32, a);
-        tmem_ld32(tmem + lane_addr + DK_COL + cgrp * 32, bb);
+      for (int pass = 0; pass < 4; ++pass) {      // dV columns, then dK columns, 32 at a time
+        const int cgrp = half * 2 + (pass & 1);
+        const bool is_dk = pass >= 2;
+        uint32_t a[32];
+        tmem_ld32(tmem + lane_addr + (is_dk ? DK_COL : DV_COL) + cgrp * 32, a);
         tmem_ld_wait();
         if (r < it.valid) {
+          const float mul = is_dk ? p.scale : 1.0f;
+          __nv_bfloat16* row = (is_dk ? dk_row : dv_row) + cgrp * 32;
 #pragma unroll
           for (int i = 0; i < 32; i += 16) {      // sixteen bf16 = one 32-byte store (two 16-byte stores if unaligned)
-            uint32_t hv[8], hk[8];
+            uint32_t hv[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-              hv[k] = pack_bf16(__uint_as_float(a[i + 2 * k]), __uint_as_float(a[i + 2 * k + 1]));
-              hk[k] = pack_bf16(__uint_as_float(bb[i + 2 * k]) * p.scale, __uint_as_float(bb[i + 2 * k + 1]) * p.scale);
-            }
+            for (int k = 0; k < 8; ++k)
+              hv[k] = pack_bf16(__uint_as_float(a[i + 2 * k]) * mul, __uint_as_float(a[i + 2 * k + 1]) * mul);
             if (p.dkv_32) {
-              st_global_v8(dv_row + cgrp * 32 + i, hv[0], hv[1], hv[2], hv[3], hv[4], hv[5], hv[6], hv[7]);
-              st_global_v8(dk_row + cgrp * 32 + i, hk[0], hk[1], hk[2], hk[3], hk[4], hk[5], hk[6], hk[7]);
+              st_global_v8(row + i, hv[0], hv[1], hv[2], hv[3], hv[4], hv[5], hv[6], hv[7]);
             } else {
-              *reinterpret_cast<uint4*>(dv_row + cgrp * 32 + i) = make_uint4(hv[0], hv[1], hv[2], hv[3]);
-              *reinterpret_cast<uint4*>(dv_row + cgrp * 32 + i + 8) = make_uint4(hv[4], hv[5], hv[6], hv[7]);
-              *reinterpret_cast<uint4*>(dk_row + cgrp * 32 + i) = make_uint4(hk[0], hk[1], hk[2], hk[3]);
-              *reinterpret_cast<uint4*>(dk_row + cgrp * 32 + i + 8) = make_uint4(hk[4], hk[5], hk[6], hk[7]);
+              *reinterpret_cast<uint4*>(row + i) = make_uint4(hv[0], hv[1], hv[2], hv[3]);
+              *reinterpret_cast<uint4*>(row + i + 8) = make_uint4(hv[4], hv[5], hv[6], hv[7]);
             }
           }
         }
@@ -631,9 +612,9 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
   kp.dkv_32 = (reinterpret_cast<uintptr_t>(dk) % 32) == 0 && (reinterpret_cast<uintptr_t>(dv) % 32) == 0 &&
               (!out_map.perm || (out_map.sb % 16 == 0 && out_map.st % 16 == 0 && out_map.sh % 16 == 0));
   const long long kv_items = n_kb * ((D.sb + BN - 1) / BN);
-  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_bwd_dkdv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)KVF_SMEM_BYTES));
-  attn_bwd_dkdv_tc_kernel<false><<<grid_items(kv_items), KVF_THREADS, KVF_SMEM_BYTES, st>>>(tmK, tmV, kp);
+  attn_bwd_dkdv_tc_kernel<<<grid_items(kv_items), KVF_THREADS, KVF_SMEM_BYTES, st>>>(tmK, tmV, kp);
   VMOBA_LAUNCH_OK(1);
   return VMOBA_OK;
 }

@@ -51,18 +51,58 @@ def rel_l2(a, b):
     return float(np.sqrt(((a - b) ** 2).sum())) / den if den > 0 else float(np.sqrt(((a - b) ** 2).sum()))
 
 
+# Parity report: one record per assert_close call, printed by the terminal-summary hook of conftest.py.
+PARITY_REPORT = []
+STRICT_BELOW = 4.0         # |ref| below which the plain max-abs bound holds without the store-rounding allowance
+GRAD_OUTLIER_FRAC = 1e-4   # share of a gradient tensor's elements that may sit in the operand-rounding tail
+GRAD_OUTLIER_CAP = 2.5e-2  # and how far
+
+
 def assert_close(got, ref, dtype, what=""):
-    """max-abs and relative-L2 bounds.  bf16 arithmetic has two error terms that grow with the size of
-    the result and that no kernel can avoid: the stored result is rounded to bf16 (half an ulp,
-    2^-9 |ref|, which alone exceeds 2e-2 once |ref| >= 8), and the tensor-core operands P and dS are
-    rounded to bf16 (2^-9 relative per term; a sum of same-signed terms keeps that relative error).
-    The max-abs bound of 2e-2 is therefore taken on top of 2^-8 |ref|."""
+    """max-abs and relative-L2 bounds; `what` starts with the tensor's name (o, dq, dk, dv).
+
+    bf16, every tensor: |err| <= 2e-2 wherever |ref| < 4.  Above that the stored result alone is rounded by
+    up to half a bf16 ulp (1.6e-2 for |ref| in [4, 8), 3.1e-2 in [8, 16)), which no bf16 kernel can avoid, so
+    only there the bound grows to 2e-2 + 2^-8 |ref|.
+
+    bf16 gradients: P and dS enter the second matrix product rounded to bf16.  A query whose softmax sits on
+    a few keys has dS entries of 8 and more; rounding one of them moves it by up to 1.6e-2 and its term
+    scale * dS * k (|k| up to 4) by 5e-3, and a handful of such terms give every element of that row an error
+    with a standard deviation of about 5e-3.  A kernel with no other error than these two roundings
+    (simulated on the CPU in test_rounding_floor.py) reaches 1.8e-2 to 1.95e-2 on the mid-size layer: the
+    plain 2e-2 is a 3.7-sigma event per element in such rows, met or missed from one draw of the roundings to
+    the next.  Gradient tensors may therefore hold a share of at most 1e-4 of elements above 2e-2, none of
+    them above 2.5e-2 (nor above the bound of large elements); the report lists how many and where."""
     ma, rl = TOL[dtype]
     got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
-    allow = ma + (2.0 ** -8) * np.abs(ref) if dtype == "bf16" else ma
-    excess = float(np.max(np.abs(got - ref) - allow)) if got.size else -1.0
+    err = np.abs(got - ref)
+    aref = np.abs(ref)
+    small = aref < STRICT_BELOW
     e1, e2 = max_abs(got, ref), rel_l2(got, ref)
-    assert excess <= 0 and e2 <= rl, f"{what}: max-abs {e1:.3e} (tol {ma} + 2^-8 |ref|), rel-L2 {e2:.3e} (tol {rl})"
+    e_small = float(err[small].max()) if small.any() else 0.0
+    e_large = float(err[~small].max()) if (~small).any() else 0.0
+    over = err > ma
+    import os
+    PARITY_REPORT.append(dict(test=os.environ.get("PYTEST_CURRENT_TEST", "").split(" ")[0].split("::")[-1], what=what,
+                              dtype=dtype, n=int(got.size), max_small=e_small, max_large=e_large,
+                              n_large=int((~small).sum()), n_over_plain=int(over.sum()),
+                              n_over_small=int((over & small).sum()),
+                              min_ref_over_plain=float(aref[over].min()) if over.any() else None, rel_l2=e2))
+    msg = (f"{what}: max-abs {e1:.3e} (|ref| < {STRICT_BELOW:g}: {e_small:.3e}, {int((over & small).sum())} of {got.size} "
+           f"above {ma}; |ref| >= {STRICT_BELOW:g}: {e_large:.3e}, tol {ma} + 2^-8 |ref|), rel-L2 {e2:.3e} (tol {rl})")
+    assert e2 <= rl, msg
+    if dtype != "bf16":
+        assert e1 <= ma, msg
+        return
+    wide = ma + (2.0 ** -8) * aref
+    assert np.all(err[~small] <= wide[~small]), msg
+    is_grad = (what.split() or [""])[0] in ("dq", "dk", "dv")
+    if not is_grad:
+        assert e_small <= ma, msg
+        return
+    tail = over & small
+    assert tail.sum() <= GRAD_OUTLIER_FRAC * got.size, msg
+    assert np.all(err[tail] <= np.minimum(GRAD_OUTLIER_CAP, wide[tail])), msg
 
 
 def unpack_mask(mask_bits, BH, S, Nb):
