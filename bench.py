@@ -49,6 +49,8 @@ def workloads(name):
         return [gen.C5.with_(name="c5_" + k, block=b) for k, b in gen.C5_BLOCKS.items()], True
     if name == "t55k":   # the paper's 55K-token fine-tuning grid with its own block counts (Table 4), three layers
         return [gen.T55.with_(name="t55k_" + k, block=b) for k, b in gen.T55_BLOCKS.items()], True
+    if name == "t56k":   # the paper's second training grid (Table 4: 141 x 480 x 832 video, latent 36 x 30 x 52)
+        return [gen.T56.with_(name="t56k_" + k, block=b) for k, b in gen.T56_BLOCKS.items()], True
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -246,10 +248,15 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="vmoba", choices=["vmoba", "reference"])
-    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "t55k"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "t55k", "t56k"])
+    ap.add_argument("--inputs", default="", choices=["", "smooth", "white", "sine"],
+                    help="override the workload's input recipe; 'white' = no locality component (selection pattern "
+                         "essentially random: the worst case for gathered work lists)")
     ap.add_argument("--cpu-rows", type=int, default=256, help="query rows per unit the CPU oracle baseline evaluates")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--dense", action="store_true", help="also time the dense vmoba_full_attn path on the same inputs")
+    ap.add_argument("--dense", action="store_true",
+                    help="also time the dense vmoba_full_attn path on the same inputs (always done for c5)")
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense comparison of c5")
     ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--rule", default="threshold_global",
                     choices=["threshold_global", "topk_global", "threshold_local", "topk_local"],
@@ -286,6 +293,8 @@ def main():
     layers, with_bwd = workloads(args.workload)
     if args.heads > 0:
         layers = [w.with_(heads=args.heads) for w in layers]
+    if args.inputs:
+        layers = [w.with_(recipe=args.inputs) for w in layers]
     layers = rank_workloads(layers, rank)
     w0 = layers[0]
     data = gen.make_inputs(w0, with_do=with_bwd)
@@ -447,9 +456,12 @@ def main():
     barrier()
     e2e_ms = e0.elapsed_time(e1) / args.e2e_steps
 
-    # ---- optional dense path on the same inputs
+    # ---- the dense path on the same inputs (config 5's speed-up denominator; Section 4.1's "Full Attention"):
+    # one dense layer, forward (+ backward), one warm-up call and two timed ones
     dense_ms = None
-    if args.dense:
+    if (args.dense or args.workload == "c5") and not args.no_dense:
+        del dev_b, outs_b, sets
+        torch.cuda.empty_cache()
         shape = vb.shape_of(w0)
         qd, kd, vd = (dev[n].permute(0, 2, 1, 3).contiguous() for n in "qkv")
         od = torch.empty_like(qd)
@@ -464,9 +476,13 @@ def main():
         torch.cuda.synchronize()
         d0 = torch.cuda.Event(enable_timing=True); d1 = torch.cuda.Event(enable_timing=True)
         d0.record()
-        vb.vmoba_full_attn(shape, qd, kd, vd, od, lse, dev_status=st, **extra)
+        for _ in range(2):
+            vb.vmoba_full_attn(shape, qd, kd, vd, od, lse, dev_status=st, **extra)
         d1.record(); torch.cuda.synchronize()
-        dense_ms = d0.elapsed_time(d1)
+        dense_ms = d0.elapsed_time(d1) / 2
+        if int(st.item()) != 0:
+            raise vb.VmobaError(int(st.item()), "dense path")
+        del qd, kd, vd, od, extra
 
     # ---- aggregate over ranks (max time, summed work)
     mult = 14.0 if with_bwd else 4.0
@@ -555,6 +571,13 @@ def main():
                        / ((stage_ms["attn_fwd"] + stage_ms.get("attn_bwd", 0.0)) * 1e-3) / 1e12,
         "dense_ms": dense_ms,
     }
+    if dense_ms is not None:
+        # one dense layer against one sparse layer (the step's time over its layers, every stage included)
+        dense_flops = (14.0 if with_bwd else 4.0) * w0.B * w0.heads * float(w0.S) ** 2 * w0.head_dim
+        line["dense"] = {"ms_per_layer": dense_ms, "tflops": dense_flops / (dense_ms * 1e-3) / 1e12,
+                         "frac": dense_flops / (dense_ms * 1e-3) / 1e12 / pk["tensor_sustained"],
+                         "sparse_ms_per_layer": ms_per_step / len(layers),
+                         "speedup_sparse_vs_dense": dense_ms / (ms_per_step / len(layers))}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -56,7 +56,7 @@ static BwdWs carve_bwd(const Dims& D, bool dense, void* ws, long long cap = 0) {
 }
 
 static int grid_for(long long items, int per_sm) {
-  long long g = std::min<long long>(items, 148ll * per_sm);
+  long long g = std::min<long long>(items, (long long)sm_count() * per_sm);
   return (int)std::max<long long>(g, 1);
 }
 

@@ -579,7 +579,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-static int grid_items(long long items) { return (int)std::max<long long>(1, std::min<long long>(items, 148)); }
+static int grid_items(long long items) { return (int)std::max<long long>(1, std::min<long long>(items, sm_count())); }
 
 }  // namespace tcb
 

@@ -631,7 +631,7 @@ dq_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-static int grid_items(long long items) { return (int)std::max<long long>(1, std::min<long long>(items, 148)); }
+static int grid_items(long long items) { return (int)std::max<long long>(1, std::min<long long>(items, sm_count())); }
 
 }  // namespace tcl
 

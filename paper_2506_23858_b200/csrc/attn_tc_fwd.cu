@@ -513,7 +513,7 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
   if (warp == 1) tmem_dealloc(tmem, TMEM_COLS);
 }
 
-static int grid_items(long long items) { return (int)std::max<long long>(1, std::min<long long>(items, 148)); }
+static int grid_items(long long items) { return (int)std::max<long long>(1, std::min<long long>(items, sm_count())); }
 
 }  // namespace tcw
 
@@ -530,7 +530,7 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
     return VMOBA_ERR_CUDA;
   const long long n_kb = (long long)D.BH * D.Nb;
   simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, IM, cap, item_ptr);
-  simt::item_tab_kernel<<<(int)std::min<long long>((n_kb + 255) / 256, 148 * 4), 256, 0, st>>>(item_ptr, n_kb, max_items,
+  simt::item_tab_kernel<<<(int)std::min<long long>((n_kb + 255) / 256, sm_count() * 4), 256, 0, st>>>(item_ptr, n_kb, max_items,
                                                                                                item_tab);
   Params p;
   p.q = (const __nv_bfloat16*)q; p.kb_ptr = kb_ptr; p.q_idx = q_idx; p.q_ptr = q_ptr; p.item_ptr = item_ptr;
@@ -544,7 +544,7 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
                                      (int)SMEM_BYTES));
   attn_fwd_wide_kernel<false><<<grid_items(cap / IM + n_kb), THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
   const long long nq = (long long)D.BH * D.S;
-  simt::merge_kernel<__nv_bfloat16, 128, float><<<(int)std::min<long long>((nq + 7) / 8, 148 * 16), 256, 0, st>>>(
+  simt::merge_kernel<__nv_bfloat16, 128, float><<<(int)std::min<long long>((nq + 7) / 8, sm_count() * 16), 256, 0, st>>>(
       q_ptr, q_pairs, nq, part_o, part_lse, cap, (__nv_bfloat16*)o, (__nv_bfloat16*)o_resid, lse);
   VMOBA_LAUNCH_OK(4);
   return VMOBA_OK;

@@ -83,6 +83,20 @@ inline int make_dims(const vmoba_shape* s, Dims* o) {
   return VMOBA_OK;
 }
 
+// Number of SMs of the current device, read once per device and thread (grids of the persistent kernels are
+// one CTA per SM; the streaming kernels size theirs as a multiple of it).
+inline int sm_count() {
+  thread_local int cached_dev = -1, cached_n = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+  if (dev != cached_dev) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 1;
+    cached_dev = dev; cached_n = n;
+  }
+  return cached_n;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -82,7 +82,7 @@ static int launch_partition(const Dims& D, const PermGeom& g, int inverse, const
   long long n_rows = (long long)D.BH * D.S;
   long long warps = (n_rows + 31) / 32;
   long long blocks = (warps + 7) / 8;
-  long long cap = 148ll * 8 * 4;
+  long long cap = (long long)sm_count() * 8 * 4;
   if (blocks > cap) blocks = cap;
   long long per_vec = 16 / D.es;
   partition_kernel<V><<<(unsigned)blocks, 256, 0, st>>>(

@@ -268,7 +268,7 @@ int scores_tc(const Dims& D, const void* q_bm, const float* cent, float* scores,
   const int rows_pass = ((Nb_pad + n_pass - 1) / n_pass + 31) / 32 * 32;
   __nv_bfloat16* parts = reinterpret_cast<__nv_bfloat16*>((reinterpret_cast<uintptr_t>(ws) + 1023) & ~uintptr_t(1023));
   const long long n = (long long)D.BH * Nb_pad * DH;
-  split_centroids_kernel<<<(int)std::min<long long>((n + 255) / 256, 148 * 8), 256, 0, st>>>(cent, parts, D.Nb, Nb_pad, D.BH);
+  split_centroids_kernel<<<(int)std::min<long long>((n + 255) / 256, sm_count() * 8), 256, 0, st>>>(cent, parts, D.Nb, Nb_pad, D.BH);
   CUtensorMap tmQ, tmB, tmS;
   const int tma_store = (D.Nb % 4 == 0) && (reinterpret_cast<uintptr_t>(scores) % 16 == 0);
   if (tma_store) {
@@ -285,7 +285,7 @@ int scores_tc(const Dims& D, const void* q_bm, const float* cent, float* scores,
   p.status = status;
   VMOBA_CUDA_OK(cudaFuncSetAttribute(scores_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
   const long long items = (long long)D.BH * n_pass * ((D.S + BM - 1) / BM);
-  scores_tc_kernel<<<(int)std::max<long long>(1, std::min<long long>(items, 148)), THREADS, SMEM_BYTES, st>>>(tmQ, tmB, tmS, p);
+  scores_tc_kernel<<<(int)std::max<long long>(1, std::min<long long>(items, sm_count())), THREADS, SMEM_BYTES, st>>>(tmQ, tmB, tmS, p);
   VMOBA_LAUNCH_OK(2);
   return VMOBA_OK;
 }

@@ -802,7 +802,7 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
     // search on the row-normalised log-probabilities with unit temperature
     float* lp = reinterpret_cast<float*>(static_cast<char*>(ws) + ((w.bytes + 255) / 256) * 256);
     const long long n_rows = (long long)D.BH * D.S;
-    rownorm_kernel<<<(int)std::min<long long>((n_rows + 7) / 8, 148 * 8), 256, 0, st>>>(scores, lp, D.Nb, D.scale, n_rows);
+    rownorm_kernel<<<(int)std::min<long long>((n_rows + 7) / 8, sm_count() * 8), 256, 0, st>>>(scores, lp, D.Nb, D.scale, n_rows);
     VMOBA_LAUNCH_OK(1);
     scores = lp;
     sigma = 1.0f;
@@ -816,7 +816,7 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
   if (local) {
     // per-query rules: the mask comes straight from the rows; cutoff_key collects the smallest selected key
     const long long n_rows = (long long)D.BH * D.S;
-    const int blocks = (int)std::min<long long>((n_rows + 7) / 8, 148 * 8);
+    const int blocks = (int)std::min<long long>((n_rows + 7) / 8, sm_count() * 8);
     auto launch_local = [&](auto topk_tag, auto mw_tag) {
       select_local_kernel<decltype(topk_tag)::value, decltype(mw_tag)::value><<<blocks, 256, 0, st>>>(
           scores, D.S, D.Nb, D.mask_words, D.scale, tau, topk, own_sb, mask_bits, w.state, n_rows);
@@ -848,7 +848,7 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
 
     // enough CTAs per head to fill the machine, few enough that the per-CTA flush stays small
     long long per_head = (P / 4 + 255) / 256;
-    int gx = (int)std::min<long long>(std::max<long long>(per_head / 8, 1), std::max(1, 148 * 8 / D.BH));
+    int gx = (int)std::min<long long>(std::max<long long>(per_head / 8, 1), std::max(1, sm_count() * 8 / D.BH));
     dim3 grid(gx, D.BH);
     minmax_kernel<<<grid, 256, 0, st>>>(scores, P, w.state);
     setup_level0_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH);
@@ -856,7 +856,7 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
       constexpr int smem0 = kBins0 * kRep * (int)sizeof(float);
       VMOBA_CUDA_OK(cudaFuncSetAttribute(hist0_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem0));
       // three 512-thread CTAs per SM hold their replicated bins side by side
-      int gx0 = (int)std::min<long long>(std::max<long long>(per_head / 16, 1), std::max(1, 148 * 3 / D.BH));
+      int gx0 = (int)std::min<long long>(std::max<long long>(per_head / 16, 1), std::max(1, sm_count() * 3 / D.BH));
       hist0_kernel<<<dim3(gx0, D.BH), 512, smem0, st>>>(scores, P, w.state, sigma, unit_w, w.g_w);
     }
     scan_kernel<0><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,

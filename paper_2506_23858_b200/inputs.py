@@ -7,11 +7,13 @@ T x H x W tokens, several heads, head_dim channels) and rounds them to the
 storage type.  Token order is raster (t, h, w) with w fastest; tensors are
 laid out [B, S, heads, head_dim] (what a DiT's q/k/v projections produce).
 
-Two recipes:
+Three recipes:
 
 * ``sine``  : x(t,h,w,head,c) = 0.5*sin(2*pi*(t/T + h/H + w/W) + phi_head) + N(0,1),
               phi_head = 2*pi*head/heads; the sine term is shared by q, k and v and by
               all channels; the noise is i.i.d. per element and independent for q, k, v.
+* ``white`` : x = N(0,1) only: no locality component at all (the unstructured variant: selection is
+              essentially random, the worst case for gathered work lists).
 * ``smooth``: x = N(0,1) + f, where f is, per (batch, head), one white N(0,1)
               field of shape [T,H,W,head_dim] blurred along T, H and W (not along
               channels) with a separable Gaussian (sigma = 2 tokens, radius 8,
@@ -76,6 +78,12 @@ C5 = Workload("c5_720p", 1, 40, 128, 21, 45, 80, (3, 9, 10), 0.25, "bf16", "smoo
 # 8 / 48 / 72 key blocks for the 1D / 2D / 3D layers, tau = 0.25) on Wan-1.3B-sized heads.
 T55_BLOCKS = {"1d": (3, 36, 64), "2d": (24, 6, 8), "3d": (8, 12, 8)}
 T55 = Workload("t55k_train", 1, 12, 128, 24, 36, 64, (8, 12, 8), 0.25, "bf16", "smooth", 1)
+# The paper's second training grid (Table 4: 141x480x832 video, latent 36x30x52 = 56,160 tokens; spatial blocks
+# of 5 x 13 tokens -> 24 blocks of 2340 keys, spatio-temporal blocks of 12 x 10 x 13 tokens -> 36 blocks of
+# 1560 keys).  The table's temporal entry for this grid is inconsistent (block size 3 but 7 blocks, where
+# 36 / 3 = 12); the 1D layer here takes the block size: 12 temporal blocks of 3 frames (4680 keys).
+T56_BLOCKS = {"1d": (3, 30, 52), "2d": (36, 5, 13), "3d": (12, 10, 13)}
+T56 = Workload("t56k_train", 1, 12, 128, 36, 30, 52, (12, 10, 13), 0.25, "bf16", "smooth", 1)
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:

@@ -154,6 +154,41 @@ class VmobaLayer:
         return int(self.k_per_head.sum().item())
 
 
+def dense_step_schedule(n_steps: int, dense_fraction: float = 0.25):
+    """Which denoising steps of a sampling run use full attention: the paper's training-free setting runs the
+    first 25 % of the steps dense and the rest through VMoBA (Section 4.1, implementation details).  Returns a list
+    of n_steps booleans, True = dense; the number of dense steps is ceil(dense_fraction * n_steps)."""
+    import math
+    if n_steps < 0 or not (0.0 <= dense_fraction <= 1.0):
+        raise ValueError("n_steps >= 0 and 0 <= dense_fraction <= 1 required")
+    n_dense = min(n_steps, int(math.ceil(dense_fraction * n_steps - 1e-9)))
+    return [i < n_dense for i in range(n_steps)]
+
+
+class SteppedAttention:
+    """Host-side switch between the dense path and the sparse layer over the steps of a sampler: step i of
+    n_steps calls vmoba_full_attn while dense_step_schedule says so, the VMoBA layer afterwards (forward only:
+    this is the inference setting).  Tensors are raster-order [B, S, heads, d] on the device."""
+
+    def __init__(self, layer: VmobaLayer, tau: float, n_steps: int, dense_fraction: float = 0.25):
+        self.layer, self.tau = layer, tau
+        self.schedule = dense_step_schedule(n_steps, dense_fraction)
+        s = layer.shape
+        self._lse = torch.empty(s.B * s.heads * s.S, dtype=torch.float32, device=layer.device)
+
+    def forward(self, step: int, q, k, v, o_out) -> str:
+        """Runs step `step`; returns which path ran ("dense" or "sparse")."""
+        if self.schedule[step]:
+            # the dense kernels take [B, heads, S, d] in any one token order
+            qd, kd, vd = (x.permute(0, 2, 1, 3).contiguous() for x in (q, k, v))
+            od = torch.empty_like(qd)
+            vb.vmoba_full_attn(self.layer.shape, qd, kd, vd, od, self._lse, dev_status=self.layer.dev_status)
+            o_out.copy_(od.permute(0, 2, 1, 3))
+            return "dense"
+        self.layer.forward(q, k, v, self.tau, o_out)
+        return "sparse"
+
+
 def lists_from_mask(mask_bh, capacity=None, device="cuda"):
     """Builds kb_ptr / q_idx / q_ptr / q_pairs on the host from a boolean mask [BH, S, Nb]
     (used by tests to feed the attention kernels a selection that did not come from

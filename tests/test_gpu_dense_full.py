@@ -120,3 +120,32 @@ def test_config3_threshold_one_equals_dense_at_full_size(name):
     assert U.max_abs(lse, lse_ref) <= 2e-2
     dense = _dense_run(w, data, False)
     U.assert_close(U.to_numpy_f32(o[0, :, 0]), U.to_numpy_f32(dense["o"][0, 0]), w.dtype, "o sparse route vs dense path")
+
+
+def test_sampler_switch_runs_dense_then_sparse():
+    """The host-side rule of Section 4.1 (first quarter of the steps dense): step 0 of 4 must give dense attention,
+    the later steps the sparse layer's output."""
+    from paper_2506_23858_b200.layer import SteppedAttention, default_capacity
+    w = gen.Workload("mid", 1, 2, 128, 6, 12, 26, (3, 6, 13), 0.25, "bf16", "smooth", 5)
+    data = gen.make_inputs(w, with_do=False)
+    shape = vb.shape_of(w)
+    L = VmobaLayer(shape, capacity=default_capacity(shape, w.tau))
+    sw = SteppedAttention(L, w.tau, n_steps=4)
+    q, k, v = (U.to_device(w, data, n) for n in "qkv")
+    outs, paths = [], []
+    for step in range(4):
+        o = torch.empty_like(q)
+        paths.append(sw.forward(step, q, k, v, o))
+        outs.append(o)
+    torch.cuda.synchronize()
+    L.check_status()
+    assert paths == ["dense", "sparse", "sparse", "sparse"]
+    scale = w.head_dim ** -0.5
+    for h in range(w.heads):
+        od, _ = orc.dense_attn_fwd(data["q"][0, :, h], data["k"][0, :, h], data["v"][0, :, h], scale)
+        U.assert_close(U.to_numpy_f32(outs[0][0, :, h]), od, w.dtype, "o dense step")
+    ref = torch.empty_like(q)
+    L.forward(q, k, v, w.tau, ref)
+    torch.cuda.synchronize()
+    assert torch.equal(outs[1], ref) and torch.equal(outs[3], ref)
+    assert not torch.equal(outs[0], ref)

@@ -311,3 +311,14 @@ def test_config5_all_40_heads_one_layer(name):
     rng = np.random.default_rng(2)
     for (b, h) in [(0, 0), (0, 39)]:
         _check_head(w, data, res, b, h, rng, 32, 1, True)
+
+
+@pytest.mark.parametrize("grid", ["t55k", "t56k"])
+@pytest.mark.parametrize("name", ["1d", "2d", "3d"])
+def test_paper_training_grids_forward_backward(grid, name):
+    """The paper's two fine-tuning grids with its own block sizes (Table 4): latent 24 x 36 x 64 with 8 / 48 / 72
+    blocks of 6912 / 1152 / 768 keys, latent 36 x 30 x 52 with 12 / 24 / 36 blocks of 4680 / 2340 / 1560 keys;
+    tau = 0.25, forward and backward, four heads, one of them against the oracle on sampled rows and a key block."""
+    base, blocks = (gen.T55, gen.T55_BLOCKS) if grid == "t55k" else (gen.T56, gen.T56_BLOCKS)
+    w = base.with_(name=f"{grid}_{name}", block=blocks[name], heads=4)
+    _full_size(w, True, [(0, 3)], n_rows=48, n_blocks=1)
