@@ -266,6 +266,8 @@ def main():
                     help="partition dO and inverse-partition dq, dk, dv in passes of their own (instead of the backward reading / writing raster order)")
     ap.add_argument("--fold-do", action="store_true",
                     help="also let the backward read dO in raster order (pays with few heads: c4 yes, c5 no)")
+    ap.add_argument("--fold-o", action="store_true",
+                    help="let the forward write o in raster order (saves the inverse partition pass of o; measured slower)")
     ap.add_argument("--heads", type=int, default=0, help="override the number of heads (small profiling runs)")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -337,6 +339,7 @@ def main():
     stage_ms = {s: 0.0 for s in stage_names}
 
     fold = with_bwd and not args.no_fold and L[0].can_fold_inverse(outs["dq"], outs["dk"], outs["dv"])
+    fold_o = args.fold_o and L[0].can_fold_o()            # the forward writes o in raster order itself
 
     def step(record, dev=dev, outs=outs):
         evs = []
@@ -352,8 +355,11 @@ def main():
             mark("partition")
             layer.block_scores(); mark("scores")
             do_select(layer, layer_w[id(layer)], layer_pos[id(layer)]); mark("select")
-            layer.attn_fwd(); mark("attn_fwd")
-            layer.partition(outs["o"], layer.o_bm, inverse=True); mark("partition")
+            if fold_o:
+                layer.attn_fwd_raster(outs["o"]); mark("attn_fwd")
+            else:
+                layer.attn_fwd(); mark("attn_fwd")
+                layer.partition(outs["o"], layer.o_bm, inverse=True); mark("partition")
             if with_bwd:
                 if fold and args.fold_do:
                     # the backward kernels read dO and write dq, dk, dv in raster order themselves (Eq. 1 folded in)
@@ -363,6 +369,8 @@ def main():
                     layer.attn_bwd_raster(None, outs["dq"], outs["dk"], outs["dv"]); mark("attn_bwd")
                 else:
                     layer.partition(dev["do"], layer.do_bm); mark("partition")
+                    if layer.o_raster is not None:
+                        layer.partition(layer.o_raster, layer.o_bm)
                     layer.attn_bwd(); mark("attn_bwd")
                     layer.partition(outs["dq"], layer.dq_bm, inverse=True)
                     layer.partition(outs["dk"], layer.dk_bm, inverse=True)
@@ -495,7 +503,10 @@ def main():
 
     es = 2 if w0.dtype == "bf16" else 4
     tensor_bytes = w0.B * w0.S * w0.heads * w0.head_dim * es
-    n_part = len(layers) * (((4 if args.fold_do else 5) if fold else 8) if with_bwd else 4)     # partition passes of a step
+    # partition passes of a step: q, k, v in; o out unless the forward writes raster order; dO in unless the backward
+    # reads raster order; dq, dk, dv out unless the backward writes raster order
+    n_part = len(layers) * (3 + (0 if fold_o else 1)
+                            + ((0 if (fold and args.fold_do) else 1) + (0 if fold else 3) if with_bwd else 0))
     alg = {
         "partition": ("hbm", 2.0 * tensor_bytes * n_part),
         "scores": ("hbm", sum(2.0 * tensor_bytes + 4.0 * w.B * w.heads * (w.S * w.n_blocks + w.n_blocks * w.head_dim)

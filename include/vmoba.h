@@ -210,6 +210,20 @@ int vmoba_attn_fwd(const vmoba_shape* shape, const void* q_bm, const void* k_bm,
                    float* lse, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * The same forward with the inverse of Eq. 1 folded into the kernels that write o: o is written in RASTER order,
+ * [B, S, heads, head_dim] addressed by element strides o_strides_bsh = {batch, token, head} (head_dim contiguous,
+ * every stride a multiple of 16 bytes), the row of block-major position p being token perm[p] (perm: device int32
+ * [S], as produced by vmoba_partition).  Saves the inverse partition pass of o.  The rounding residual, if asked
+ * for, stays block-major (it only feeds vmoba_attn_bwd*), as does lse.  bf16 with head_dim 128 only
+ * (VMOBA_ERR_NOT_IMPLEMENTED otherwise); everything else as for vmoba_attn_fwd.
+ */
+int vmoba_attn_fwd_raster(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
+                          const int32_t* kb_ptr, const int32_t* q_idx, const int32_t* q_ptr, const int32_t* q_pairs,
+                          int64_t capacity, void* o, const int64_t o_strides_bsh[3], const int32_t* perm,
+                          void* o_resid_bm_or_null, float* lse, int32_t* dev_status, void* ws, size_t ws_bytes,
+                          void* stream);
+
+/*
  * Training backward of Step 3 with the selection held constant (TopkMask has zero gradient):
  * dq, dk, dv [B, heads, S, head_dim] (dtype) from do_bm, the forward's o_bm (+ o_resid) and lse.
  * Queries without a selected block get dq = 0.  The paper states no gradient formula; this is
@@ -223,19 +237,19 @@ int vmoba_attn_bwd(const vmoba_shape* shape, const void* q_bm, const void* k_bm,
                    void* dv_bm, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
 
 /*
- * The same backward with Eq. 1 and its inverse folded into the kernels that read dO and write the gradients:
- * d_o is read and dq, dk, dv are written in RASTER order, [B, S, heads, head_dim] addressed by element strides
- * {batch, token, head} (do_strides_bsh for d_o, grad_strides_bsh for the three gradients; head_dim contiguous,
- * every stride a multiple of 16 bytes), the row of block-major position p being token perm[p] (perm: device
- * int32 [S], as produced by vmoba_partition).  do_strides_bsh may be NULL: d_o is then block-major like the
- * other inputs.  Saves the three inverse partition passes of a training step and, with a raster d_o, the
+ * The same backward with Eq. 1 and its inverse folded into the kernels that read o and dO and write the gradients:
+ * o and d_o are read and dq, dk, dv are written in RASTER order, [B, S, heads, head_dim] addressed by element
+ * strides {batch, token, head} (o_strides_bsh for o, do_strides_bsh for d_o, grad_strides_bsh for the three
+ * gradients; head_dim contiguous, every stride a multiple of 16 bytes), the row of block-major position p being
+ * token perm[p] (perm: device int32 [S], as produced by vmoba_partition).  o_strides_bsh and do_strides_bsh may
+ * each be NULL: that tensor is then block-major like the other inputs (o_resid always is).  Saves the three inverse partition passes of a training step and, with a raster d_o, the
  * partition pass of dO (its gathered reads from raster order cost more than that pass when the head count is
  * large: see the design notes).  The other inputs, the workspace and the errors are those of vmoba_attn_bwd; bf16
  * with head_dim 128 only (VMOBA_ERR_NOT_IMPLEMENTED otherwise).
  */
 int vmoba_attn_bwd_raster(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
-                          const void* o_bm, const void* o_resid_or_null, const float* lse, const void* d_o,
-                          const int64_t do_strides_bsh[3], const int32_t* kb_ptr, const int32_t* q_idx,
+                          const void* o, const int64_t o_strides_bsh[3], const void* o_resid_or_null, const float* lse,
+                          const void* d_o, const int64_t do_strides_bsh[3], const int32_t* kb_ptr, const int32_t* q_idx,
                           const int32_t* q_ptr, int64_t capacity, void* dq, void* dk, void* dv,
                           const int64_t grad_strides_bsh[3], const int32_t* perm, int32_t* dev_status, void* ws,
                           size_t ws_bytes, void* stream);

@@ -17,7 +17,8 @@ STAGE_SCORES, STAGE_SELECT, STAGE_ATTN_FWD, STAGE_ATTN_BWD, STAGE_FULL_FWD, STAG
 
 EXPORTS = (
     "vmoba_status_string", "vmoba_kernel_launches", "vmoba_workspace_bytes", "vmoba_partition", "vmoba_block_scores",
-    "vmoba_select", "vmoba_select_static", "vmoba_select_static_scratch_bytes", "vmoba_attn_fwd", "vmoba_attn_bwd", "vmoba_attn_bwd_raster", "vmoba_full_attn",
+    "vmoba_select", "vmoba_select_rule_apply", "vmoba_select_static", "vmoba_select_static_scratch_bytes", "vmoba_attn_fwd",
+    "vmoba_attn_fwd_raster", "vmoba_attn_bwd", "vmoba_attn_bwd_raster", "vmoba_full_attn",
     "vmoba_debug_wait_profile",
 )
 
@@ -109,8 +110,11 @@ def lib():
     L.vmoba_attn_bwd.restype = ctypes.c_int
     L.vmoba_attn_bwd.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, sz, vp]
     L.vmoba_attn_bwd_raster.restype = ctypes.c_int
-    L.vmoba_attn_bwd_raster.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(ctypes.c_int64), vp, vp, vp, i64,
-                                        vp, vp, vp, ctypes.POINTER(ctypes.c_int64), vp, vp, vp, sz, vp]
+    p64 = ctypes.POINTER(ctypes.c_int64)
+    L.vmoba_attn_bwd_raster.argtypes = [sp, vp, vp, vp, vp, p64, vp, vp, vp, p64, vp, vp, vp, i64,
+                                        vp, vp, vp, p64, vp, vp, vp, sz, vp]
+    L.vmoba_attn_fwd_raster.restype = ctypes.c_int
+    L.vmoba_attn_fwd_raster.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, i64, vp, p64, vp, vp, vp, vp, vp, sz, vp]
     L.vmoba_debug_wait_profile.restype = None
     L.vmoba_debug_wait_profile.argtypes = [vp]
     L.vmoba_full_attn.restype = ctypes.c_int
@@ -217,12 +221,23 @@ def vmoba_attn_bwd(shape, q_bm, k_bm, v_bm, o_bm, o_resid, lse, do_bm, kb_ptr, q
                                 _ptr(dk_bm), _ptr(dv_bm), _ptr(dev_status), p, n, _stream(stream)), "vmoba_attn_bwd")
 
 
-def vmoba_attn_bwd_raster(shape, q_bm, k_bm, v_bm, o_bm, o_resid, lse, d_o, do_strides_bsh, kb_ptr, q_idx, q_ptr, capacity,
-                          dq, dk, dv, grad_strides_bsh, perm, dev_status, ws, stream=None):
+def vmoba_attn_fwd_raster(shape, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o, o_strides_bsh, perm,
+                          o_resid_bm, lse, dev_status, ws, stream=None):
+    p, n = _ws_args(ws)
+    os_ = (ctypes.c_int64 * 3)(*[int(x) for x in o_strides_bsh])
+    _check(lib().vmoba_attn_fwd_raster(ctypes.byref(shape), _ptr(q_bm), _ptr(k_bm), _ptr(v_bm), _ptr(kb_ptr), _ptr(q_idx),
+                                       _ptr(q_ptr), _ptr(q_pairs), int(capacity), _ptr(o), os_, _ptr(perm),
+                                       _ptr(o_resid_bm), _ptr(lse), _ptr(dev_status), p, n, _stream(stream)),
+           "vmoba_attn_fwd_raster")
+
+
+def vmoba_attn_bwd_raster(shape, q_bm, k_bm, v_bm, o, o_strides_bsh, o_resid, lse, d_o, do_strides_bsh, kb_ptr, q_idx,
+                          q_ptr, capacity, dq, dk, dv, grad_strides_bsh, perm, dev_status, ws, stream=None):
     p, n = _ws_args(ws)
     dos = None if do_strides_bsh is None else (ctypes.c_int64 * 3)(*[int(x) for x in do_strides_bsh])
+    os_ = None if o_strides_bsh is None else (ctypes.c_int64 * 3)(*[int(x) for x in o_strides_bsh])
     gs = (ctypes.c_int64 * 3)(*[int(x) for x in grad_strides_bsh])
-    _check(lib().vmoba_attn_bwd_raster(ctypes.byref(shape), _ptr(q_bm), _ptr(k_bm), _ptr(v_bm), _ptr(o_bm),
+    _check(lib().vmoba_attn_bwd_raster(ctypes.byref(shape), _ptr(q_bm), _ptr(k_bm), _ptr(v_bm), _ptr(o), os_,
                                        _ptr(o_resid), _ptr(lse), _ptr(d_o), dos, _ptr(kb_ptr), _ptr(q_idx),
                                        _ptr(q_ptr), int(capacity), _ptr(dq), _ptr(dk), _ptr(dv), gs, _ptr(perm),
                                        _ptr(dev_status), p, n, _stream(stream)), "vmoba_attn_bwd_raster")

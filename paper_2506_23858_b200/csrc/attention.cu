@@ -15,7 +15,7 @@ size_t scores_ws_bytes(const Dims& D);   // scores.cu
 int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                   const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
                   int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o, float* part_lse,
-                  cudaStream_t st);
+                  cudaStream_t st, const RowMap& o_map);
 int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, void* o, void* o_resid, float* lse,
                  int32_t* status, cudaStream_t st);
 
@@ -82,26 +82,28 @@ template <typename T, int DH>
 static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* o,
                            const void* o_resid, const float* lse, const void* d_o, const int* kb_ptr, const int* q_idx,
                            const int* q_ptr, long long cap, void* dq, void* dk, void* dv, int32_t* status, void* ws,
-                           cudaStream_t st, const RowMap& out_map, const RowMap& do_map) {
-  // raster-order dO / gradients (perm set) are handled by the tensor-core kernels only
-  if ((out_map.perm || do_map.perm) && !use_tensor_cores(D)) return VMOBA_ERR_NOT_IMPLEMENTED;
+                           cudaStream_t st, const RowMap& out_map, const RowMap& do_map, const RowMap& o_map) {
+  // raster-order o / dO / gradients (perm set) are handled by the tensor-core kernels only
+  if ((out_map.perm || do_map.perm || o_map.perm) && !use_tensor_cores(D)) return VMOBA_ERR_NOT_IMPLEMENTED;
   BwdWs w = carve_bwd(D, false, ws, cap);
   const long long n_kb = (long long)D.BH * D.Nb;
   const long long nq = (long long)D.BH * D.S;
-  simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>((const T*)o, (const T*)o_resid,
-                                                                        (const T*)d_o, nq, w.Dv, do_map);
   if (use_tensor_cores(D)) {
-    // the backward kernel adds every dQ contribution into the fp32 accumulator: clear the rows of all
-    // selecting queries, convert them afterwards (rows of queries without a block become zero)
+    // the backward kernel adds every dQ contribution into the fp32 accumulator: the row-dot pass also clears the
+    // rows of all selecting queries; they are converted afterwards (rows of queries without a block become zero)
     const int min_nb = 1;
-    simt::zero_multi_rows_kernel<DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, q_ptr, nq, min_nb);
-    count_launches(2);
+    simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(
+        (const T*)o, (const T*)o_resid, (const T*)d_o, nq, w.Dv, do_map, o_map, w.dq_acc, q_ptr);
+    count_launches(1);
     int rc = tc_sparse_bwd(D, q, k, v, d_o, lse, w.Dv, kb_ptr, q_idx, cap, w.dq_acc, dk, dv, status, st, out_map, do_map);
     if (rc) return rc;
     simt::cast_rows_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, q_ptr, nq, 1, min_nb, out_map);
     VMOBA_LAUNCH_OK(1);
     return VMOBA_OK;
   }
+  simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>((const T*)o, (const T*)o_resid,
+                                                                        (const T*)d_o, nq, w.Dv, do_map);
+  count_launches(1);
   VMOBA_CUDA_OK(cudaMemsetAsync(w.dq_acc, 0, (size_t)nq * DH * sizeof(float), st));
   simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, simt::kRows, cap, w.item_ptr);
   long long tiles = (D.sb + simt::kRows - 1) / simt::kRows;
@@ -112,7 +114,7 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
       (const T*)q, (const T*)k, (const T*)v, (const T*)d_o, lse, w.Dv, kb_ptr, q_idx, w.item_ptr, (int)n_kb, D.S,
       D.Nb, D.sb, D.BH, D.scale, cap, w.dq_acc, (T*)dq);
   simt::cast_kernel<T><<<grid_for((nq * DH / 4 + 255) / 256, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, nq * DH / 4);
-  VMOBA_LAUNCH_OK(5);
+  VMOBA_LAUNCH_OK(4);
   return VMOBA_OK;
 }
 
@@ -214,7 +216,8 @@ extern "C" int vmoba_attn_fwd(const vmoba_shape* shape, const void* q_bm, const 
   if (use_tensor_cores(D)) {
     FwdWs w = carve_fwd(D, capacity, ws);
     return tc_sparse_fwd(D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null, lse,
-                         dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse, st);
+                         dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse, st,
+                         RowMap());
   }
   VMOBA_DISPATCH(simt_sparse_fwd, D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null,
                  lse, ws, st);
@@ -240,12 +243,41 @@ extern "C" int vmoba_attn_bwd(const vmoba_shape* shape, const void* q_bm, const 
   if (D.dtype != VMOBA_BF16) o_resid_or_null = nullptr;
   if (!aligned16(o_resid_or_null)) return VMOBA_ERR_ARG;
   VMOBA_DISPATCH(simt_sparse_bwd, D, q_bm, k_bm, v_bm, o_bm, o_resid_or_null, lse, do_bm, kb_ptr, q_idx, q_ptr,
-                 capacity, dq_bm, dk_bm, dv_bm, dev_status, ws, st, RowMap(), RowMap());
+                 capacity, dq_bm, dk_bm, dv_bm, dev_status, ws, st, RowMap(), RowMap(), RowMap());
+}
+
+extern "C" int vmoba_attn_fwd_raster(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
+                                     const int32_t* kb_ptr, const int32_t* q_idx, const int32_t* q_ptr,
+                                     const int32_t* q_pairs, int64_t capacity, void* o, const int64_t o_strides_bsh[3],
+                                     const int32_t* perm, void* o_resid_bm_or_null, float* lse, int32_t* dev_status,
+                                     void* ws, size_t ws_bytes, void* stream) {
+  Dims D;
+  int rc = make_dims(shape, &D);
+  if (rc) return rc;
+  if (!q_bm || !k_bm || !v_bm || !kb_ptr || !q_idx || !q_ptr || !q_pairs || !o || !o_strides_bsh || !perm || !lse ||
+      !dev_status || !ws)
+    return VMOBA_ERR_ARG;
+  if (!aligned16(q_bm) || !aligned16(k_bm) || !aligned16(v_bm) || !aligned16(o) || !aligned16(ws) ||
+      !aligned16(o_resid_bm_or_null))
+    return VMOBA_ERR_ARG;
+  for (int i = 0; i < 3; ++i)
+    if (o_strides_bsh[i] < 0 || o_strides_bsh[i] % (16 / D.es)) return VMOBA_ERR_ARG;     // rows stay 16-byte aligned
+  if (capacity <= 0 || capacity > (int64_t)INT32_MAX) return VMOBA_ERR_ARG;
+  if (ws_bytes < carve_fwd(D, capacity, nullptr).bytes) return VMOBA_ERR_WORKSPACE;
+  if (!use_tensor_cores(D)) return VMOBA_ERR_NOT_IMPLEMENTED;
+  RowMap o_map;
+  o_map.perm = perm; o_map.heads = D.heads; o_map.S = D.S;
+  o_map.sb = o_strides_bsh[0]; o_map.st = o_strides_bsh[1]; o_map.sh = o_strides_bsh[2];
+  FwdWs w = carve_fwd(D, capacity, ws);
+  return tc_sparse_fwd(D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o, o_resid_bm_or_null, lse,
+                       dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse,
+                       static_cast<cudaStream_t>(stream), o_map);
 }
 
 extern "C" int vmoba_attn_bwd_raster(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
-                                     const void* o_bm, const void* o_resid_or_null, const float* lse,
-                                     const void* d_o, const int64_t do_strides_bsh[3], const int32_t* kb_ptr,
+                                     const void* o_bm, const int64_t o_strides_bsh[3], const void* o_resid_or_null,
+                                     const float* lse, const void* d_o, const int64_t do_strides_bsh[3],
+                                     const int32_t* kb_ptr,
                                      const int32_t* q_idx, const int32_t* q_ptr, int64_t capacity, void* dq, void* dk,
                                      void* dv, const int64_t grad_strides_bsh[3], const int32_t* perm,
                                      int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
@@ -263,23 +295,28 @@ extern "C" int vmoba_attn_bwd_raster(const vmoba_shape* shape, const void* q_bm,
   for (int i = 0; i < 3; ++i) {
     if (grad_strides_bsh[i] < 0 || grad_strides_bsh[i] % per16) return VMOBA_ERR_ARG;
     if (do_strides_bsh && (do_strides_bsh[i] < 0 || do_strides_bsh[i] % per16)) return VMOBA_ERR_ARG;
+    if (o_strides_bsh && (o_strides_bsh[i] < 0 || o_strides_bsh[i] % per16)) return VMOBA_ERR_ARG;
   }
   if (capacity <= 0 || capacity > (int64_t)INT32_MAX) return VMOBA_ERR_ARG;
   if (ws_bytes < carve_bwd(D, false, nullptr, capacity).bytes) return VMOBA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (D.dtype != VMOBA_BF16) o_resid_or_null = nullptr;
   if (!aligned16(o_resid_or_null)) return VMOBA_ERR_ARG;
-  RowMap out_map, do_map;
+  RowMap out_map, do_map, o_map;
   out_map.perm = perm;
-  out_map.heads = do_map.heads = D.heads;
-  out_map.S = do_map.S = D.S;
+  out_map.heads = do_map.heads = o_map.heads = D.heads;
+  out_map.S = do_map.S = o_map.S = D.S;
+  if (o_strides_bsh) {      // else o is block-major
+    o_map.perm = perm;
+    o_map.sb = o_strides_bsh[0]; o_map.st = o_strides_bsh[1]; o_map.sh = o_strides_bsh[2];
+  }
   out_map.sb = grad_strides_bsh[0]; out_map.st = grad_strides_bsh[1]; out_map.sh = grad_strides_bsh[2];
   if (do_strides_bsh) {     // else d_o is block-major
     do_map.perm = perm;
     do_map.sb = do_strides_bsh[0]; do_map.st = do_strides_bsh[1]; do_map.sh = do_strides_bsh[2];
   }
   VMOBA_DISPATCH(simt_sparse_bwd, D, q_bm, k_bm, v_bm, o_bm, o_resid_or_null, lse, d_o, kb_ptr, q_idx, q_ptr,
-                 capacity, dq, dk, dv, dev_status, ws, st, out_map, do_map);
+                 capacity, dq, dk, dv, dev_status, ws, st, out_map, do_map, o_map);
 }
 
 extern "C" int vmoba_full_attn(const vmoba_shape* shape, const void* q, const void* k, const void* v, void* o,

@@ -203,7 +203,7 @@ template <typename T, int DH, typename PT>
 __global__ void __launch_bounds__(256)
 merge_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pairs, long long n_queries,
              const PT* __restrict__ part_o, const float* __restrict__ part_lse, long long capacity,
-             T* __restrict__ o, T* __restrict__ o_resid, float* __restrict__ lse) {
+             T* __restrict__ o, T* __restrict__ o_resid, float* __restrict__ lse, const RowMap o_map = RowMap()) {
   constexpr int C = DH / 32;   // channels per lane
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -260,14 +260,16 @@ merge_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pairs, lon
       for (int c = 0; c < C; ++c) acc[c] *= inv;
       out_lse = mx + logf(tot);
     }
+    // o goes to the caller's layout (block-major, or raster order through perm); the residual stays block-major
+    T* o_row = o + o_map.off(g, DH);
     if constexpr (C == 4) {
-      store4_resid(o + g * DH + lane * 4, o_resid ? o_resid + g * DH + lane * 4 : nullptr,
+      store4_resid(o_row + lane * 4, o_resid ? o_resid + g * DH + lane * 4 : nullptr,
                    make_float4(acc[0], acc[1], acc[2], acc[3]));
     } else {
 #pragma unroll
       for (int c = 0; c < C; ++c) {
         const T hi_ = from_f32<T>(acc[c]);
-        o[g * DH + lane * C + c] = hi_;
+        o_row[lane * C + c] = hi_;
         if (o_resid) o_resid[g * DH + lane * C + c] = from_f32<T>(acc[c] - to_f32<T>(hi_));
       }
     }
@@ -276,11 +278,14 @@ merge_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pairs, lon
 }
 
 // ------------------------------------------------------------------------------ backward
-// D = rowsum(dO * O), one warp per query.
+// D = rowsum(dO * O), one warp per query; o and dO block-major or in raster order through their maps, the
+// rounding residual of o always block-major.  If zero_acc is given, the fp32 dQ accumulator rows of the queries
+// with at least one selected block are cleared in the same pass (the only rows the backward kernel adds into).
 template <typename T, int DH>
 __global__ void __launch_bounds__(256)
 rowdot_kernel(const T* __restrict__ o, const T* __restrict__ o_resid, const T* __restrict__ d_o, long long n_queries,
-              float* __restrict__ Dv, const RowMap do_map = RowMap()) {
+              float* __restrict__ Dv, const RowMap do_map = RowMap(), const RowMap o_map = RowMap(),
+              float* __restrict__ zero_acc = nullptr, const int* __restrict__ q_ptr = nullptr) {
   constexpr int C = DH / 32;
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -288,9 +293,14 @@ rowdot_kernel(const T* __restrict__ o, const T* __restrict__ o_resid, const T* _
   for (long long g = warp; g < n_queries; g += nwarps) {
     float a = 0.f;
     const T* do_row = d_o + do_map.off(g, DH);
+    const T* o_row = o + o_map.off(g, DH);
+    if (zero_acc && __ldg(q_ptr + g + 1) - __ldg(q_ptr + g) >= 1) {
+      float4* row = reinterpret_cast<float4*>(zero_acc + g * DH);
+      for (int c = lane; c < DH / 4; c += 32) row[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
 #pragma unroll
     for (int c = 0; c < C; ++c) {
-      float ov = to_f32<T>(o[g * DH + lane * C + c]);
+      float ov = to_f32<T>(o_row[lane * C + c]);
       if (o_resid) ov += to_f32<T>(o_resid[g * DH + lane * C + c]);
       a = fmaf(ov, to_f32<T>(do_row[lane * C + c]), a);
     }
@@ -526,21 +536,6 @@ cast_rows_kernel(const float* __restrict__ src, T* __restrict__ dst, const int* 
 #pragma unroll
       for (int c = 0; c < C; ++c) out[lane * C + c] = from_f32<T>(nb == 0 ? 0.f : src[g * DH + lane * C + c]);
     }
-  }
-}
-
-// Zeroes the accumulator rows of the queries with at least min_nb selected blocks (the only rows the
-// attention kernel adds into), instead of clearing the whole [queries, head_dim] fp32 buffer.
-template <int DH>
-__global__ void __launch_bounds__(256)
-zero_multi_rows_kernel(float* __restrict__ acc, const int* __restrict__ q_ptr, long long n_queries, int min_nb) {
-  const int lane = threadIdx.x & 31;
-  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
-  for (long long g = warp; g < n_queries; g += nwarps) {
-    if (q_ptr[g + 1] - q_ptr[g] < min_nb) continue;
-    float4* row = reinterpret_cast<float4*>(acc + g * DH);
-    for (int c = lane; c < DH / 4; c += 32) row[c] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
 }
 

@@ -65,6 +65,7 @@ struct Params {
   float scale_log2;      // softmax scale * log2(e)
   __nv_bfloat16* o;
   __nv_bfloat16* o_resid;
+  RowMap o_map;          // where the rows of o go (block-major, or raster order through perm); o_resid is block-major
   float* lse;
   float* part_o;
   float* part_lse;
@@ -161,7 +162,9 @@ __device__ __forceinline__ void store_resid(__nv_bfloat16* dst, __nv_bfloat16* r
   }
 }
 
-template <bool DENSE>
+// RASTER: the directly written rows of o go through p.o_map (a kernel of its own: with the map's address
+// arithmetic compiled into the one kernel, the block-major case ran 6 % slower on the 720p-shaped layers).
+template <bool DENSE, bool RASTER = false>
 __global__ void __launch_bounds__(THREADS, 1)
 attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
   extern __shared__ uint8_t smem_raw[];
@@ -463,6 +466,7 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
       const float row_lse = (m_used + log2f(l)) * 0.6931471805599453f;
       const bool row_ok = qpos >= 0;
       const long long G_ = it.head_off + (row_ok ? qpos : 0);
+      const long long o_row_off = RASTER ? ((row_ok && direct) ? p.o_map.off(G_, DH) : 0) : G_ * DH;
       const long long pos = (long long)it.list_lo + row;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
@@ -472,7 +476,7 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         if (row_ok) {
           const int col = 32 * c;
           if (direct) {
-            __nv_bfloat16* dst = p.o + G_ * DH + col;
+            __nv_bfloat16* dst = p.o + o_row_off + col;
             __nv_bfloat16* rdst = p.o_resid ? p.o_resid + G_ * DH + col : nullptr;
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {     // 16-byte stores (32-byte ones were slower here: more values live at once)
@@ -522,7 +526,7 @@ static int grid_items(long long items) { return (int)std::max<long long>(1, std:
 int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                        const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
                        int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o,
-                       float* part_lse, cudaStream_t st) {
+                       float* part_lse, cudaStream_t st, const RowMap& o_map) {
   using namespace tcw;
   CUtensorMap tmK, tmV;
   const uint64_t rows = (uint64_t)D.BH * D.S;
@@ -539,13 +543,20 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
   p.scale_log2 = D.scale * 1.4426950408889634f;
   p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
   p.capacity = cap; p.status = status; p.prof = debug_wait_profile();
+  p.o_map = o_map;
   p.part_o_32 = (reinterpret_cast<uintptr_t>(part_o) % 32) == 0;
-  VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_wide_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)SMEM_BYTES));
-  attn_fwd_wide_kernel<false><<<grid_items(cap / IM + n_kb), THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
+  if (o_map.perm) {
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_wide_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)SMEM_BYTES));
+    attn_fwd_wide_kernel<false, true><<<grid_items(cap / IM + n_kb), THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
+  } else {
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_wide_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)SMEM_BYTES));
+    attn_fwd_wide_kernel<false><<<grid_items(cap / IM + n_kb), THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
+  }
   const long long nq = (long long)D.BH * D.S;
   simt::merge_kernel<__nv_bfloat16, 128, float><<<(int)std::min<long long>((nq + 7) / 8, sm_count() * 16), 256, 0, st>>>(
-      q_ptr, q_pairs, nq, part_o, part_lse, cap, (__nv_bfloat16*)o, (__nv_bfloat16*)o_resid, lse);
+      q_ptr, q_pairs, nq, part_o, part_lse, cap, (__nv_bfloat16*)o, (__nv_bfloat16*)o_resid, lse, o_map);
   VMOBA_LAUNCH_OK(4);
   return VMOBA_OK;
 }
@@ -563,7 +574,7 @@ int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, voi
   p.n_kb = 0; p.S = D.S; p.Nb = 1; p.sb = D.S; p.BH = D.BH;
   p.scale_log2 = D.scale * 1.4426950408889634f;
   p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = nullptr; p.part_lse = nullptr;
-  p.capacity = 0; p.part_o_32 = 0;
+  p.capacity = 0; p.part_o_32 = 0; p.o_map = RowMap();
   p.status = status; p.prof = debug_wait_profile();
   VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_wide_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)SMEM_BYTES));

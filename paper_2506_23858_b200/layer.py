@@ -58,6 +58,7 @@ class VmobaLayer:
         ws_bytes = max(vb.workspace_bytes(s, st, self.capacity) for st in stages)
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
         self.with_backward = with_backward
+        self.o_raster = None          # the raster-order o of the last attn_fwd_raster, if that is how o was written
 
     # ---- stage wrappers -----------------------------------------------------------------
     @staticmethod
@@ -91,6 +92,7 @@ class VmobaLayer:
                                    self.cutoff, self.dev_status, ws)
 
     def attn_fwd(self):
+        self.o_raster = None
         vb.vmoba_attn_fwd(self.shape, self.q_bm, self.k_bm, self.v_bm, self.kb_ptr, self.q_idx, self.q_ptr,
                           self.q_pairs, self.capacity, self.o_bm, self.o_resid, self.lse, self.dev_status, self.ws)
 
@@ -105,23 +107,45 @@ class VmobaLayer:
         return (self.shape.dtype == vb.BF16 and self.d == 128 and self.raster_strides(dk_out) == strides
                 and self.raster_strides(dv_out) == strides)
 
+    def can_fold_o(self) -> bool:
+        """Whether the forward kernels can write o in raster order themselves."""
+        return self.shape.dtype == vb.BF16 and self.d == 128
+
+    def attn_fwd_raster(self, o_out):
+        """Forward writing o straight into the raster-order tensor o_out (needs self.perm from the partition of q).
+        The tensor is remembered: a following attn_bwd_raster reads o from it."""
+        vb.vmoba_attn_fwd_raster(self.shape, self.q_bm, self.k_bm, self.v_bm, self.kb_ptr, self.q_idx, self.q_ptr,
+                                 self.q_pairs, self.capacity, o_out, self.raster_strides(o_out), self.perm,
+                                 self.o_resid, self.lse, self.dev_status, self.ws)
+        self.o_raster = o_out
+
     def attn_bwd_raster(self, do_raster_or_none, dq_out, dk_out, dv_out):
         """Backward writing dq, dk, dv in raster order (needs self.perm from the forward's partition of q); dO is
-        read in raster order too if given, else from self.do_bm."""
+        read in raster order too if given, else from self.do_bm; o is read from the raster-order tensor the last
+        attn_fwd_raster wrote, else from self.o_bm."""
         do = self.do_bm if do_raster_or_none is None else do_raster_or_none
         dos = None if do_raster_or_none is None else self.raster_strides(do)
-        vb.vmoba_attn_bwd_raster(self.shape, self.q_bm, self.k_bm, self.v_bm, self.o_bm, self.o_resid, self.lse, do,
+        o = self.o_bm if self.o_raster is None else self.o_raster
+        os_ = None if self.o_raster is None else self.raster_strides(o)
+        vb.vmoba_attn_bwd_raster(self.shape, self.q_bm, self.k_bm, self.v_bm, o, os_, self.o_resid, self.lse, do,
                                  dos, self.kb_ptr, self.q_idx, self.q_ptr, self.capacity, dq_out,
                                  dk_out, dv_out, self.raster_strides(dq_out), self.perm, self.dev_status, self.ws)
 
     # ---- whole layer --------------------------------------------------------------------
-    def forward(self, q, k, v, tau, o_out):
-        """q, k, v, o_out: [B, S, heads, d] raster-order tensors on the device."""
+    def forward(self, q, k, v, tau, o_out, fold_o=None):
+        """q, k, v, o_out: [B, S, heads, d] raster-order tensors on the device.
+
+        fold_o: let the forward kernels write o in raster order themselves (bf16, head_dim 128) instead of an inverse
+        partition pass; off by default (measured on B200: the scattered 256-byte row writes cost the attention kernel
+        more than the pass they save, at 12 heads as at 40).  o_out must then stay alive and unchanged until backward()."""
         self.partition(q, self.q_bm, perm=self.perm)
         self.partition(k, self.k_bm)
         self.partition(v, self.v_bm)
         self.block_scores()
         self.select(tau)
+        if fold_o:
+            self.attn_fwd_raster(o_out)
+            return
         self.attn_fwd()
         self.partition(o_out, self.o_bm, inverse=True)
 
@@ -140,6 +164,8 @@ class VmobaLayer:
         if fold_inverse:
             self.attn_bwd_raster(None, dq_out, dk_out, dv_out)
             return
+        if self.o_raster is not None:      # the block-major backward reads o_bm, which the raster forward did not write
+            self.partition(self.o_raster, self.o_bm)
         self.attn_bwd()
         self.partition(dq_out, self.dq_bm, inverse=True)
         self.partition(dk_out, self.dk_bm, inverse=True)

@@ -180,6 +180,44 @@ def test_backward_writing_raster_order_equals_inverse_partition(block):
     assert torch.equal(fused[:, :, :, 1], ref[1]) and torch.equal(fused[:, :, :, 2], ref[2])
 
 
+@pytest.mark.parametrize("block", [(1, 12, 26), (3, 6, 13)], ids=["1d", "3d"])
+def test_forward_writing_raster_order_equals_inverse_partition(block):
+    """vmoba_attn_fwd_raster folds the inverse of Eq. 1 into the forward's row writes (directly written rows and merged
+    rows): o must equal vmoba_attn_fwd + inverse partition bit for bit, lse and the rounding residual must not change,
+    and the backward reading that raster-order o must give the gradients of the block-major route (dK, dV bit for
+    bit, dQ up to the order of its fp32 sum)."""
+    w = MID.with_(block=block)
+    data = gen.make_inputs(w)
+    shape = vb.shape_of(w)
+    L = VmobaLayer(shape, capacity=default_capacity(shape, w.tau), with_backward=True)
+    q, k, v, do = (U.to_device(w, data, n) for n in ("q", "k", "v", "do"))
+    o_ref = torch.empty_like(q)
+    L.forward(q, k, v, w.tau, o_ref, fold_o=False)
+    g_ref = [torch.empty_like(q) for _ in range(3)]
+    L.backward(do, *g_ref)
+    torch.cuda.synchronize()
+    lse_ref, resid_ref = L.lse.clone(), L.o_resid.clone()
+    # a strided destination: o as one slice of a [B, S, heads, 2, d] buffer
+    buf = torch.full((w.B, w.S, w.heads, 2, w.head_dim), float("nan"), dtype=q.dtype, device=q.device)
+    o_got = buf[:, :, :, 1]
+    L.forward(q, k, v, w.tau, o_got, fold_o=True)
+    g_got = [torch.empty_like(q) for _ in range(3)]
+    L.backward(do, *g_got)
+    torch.cuda.synchronize()
+    L.check_status()
+    assert torch.equal(o_got, o_ref)
+    assert torch.isnan(buf[:, :, :, 0].float()).all()
+    assert torch.equal(L.lse, lse_ref) and torch.equal(L.o_resid, resid_ref)
+    assert torch.equal(g_got[1], g_ref[1]) and torch.equal(g_got[2], g_ref[2])
+    diff = (g_got[0].float() - g_ref[0].float()).abs().max().item()
+    assert diff <= 2.0 ** -6 * max(1.0, g_ref[0].float().abs().max().item())
+    # and the block-major backward after a raster forward (o_bm rebuilt from the raster tensor)
+    g_bm = [torch.empty_like(q) for _ in range(3)]
+    L.backward(do, *g_bm, fold_inverse=False)
+    torch.cuda.synchronize()
+    assert torch.equal(g_bm[1], g_ref[1]) and torch.equal(g_bm[2], g_ref[2])
+
+
 def test_repeated_runs_reproduce():
     """Everything but dQ is written once, by one owner: repeated runs must agree bit for bit (a race between the
     roles of a kernel shows up here first).  dQ is an fp32 sum of per-key-tile parts whose order is not fixed."""
