@@ -109,6 +109,16 @@ int vmoba_block_scores(const vmoba_shape* shape, const void* q_bm, const void* k
                        void* stream);
 
 /*
+ * vmoba_block_scores that also hands over what the selection's first pass would look for: score_range
+ * [B*heads][2] fp32 receives the smallest and the largest score of each head's pool, taken in the epilogue of
+ * the scores kernel while the values are still in registers (Eq. 4's normalisation is relative to the pool's
+ * largest score, and the cutoff search starts from the pool's range).  Give it to vmoba_select_ranged.
+ */
+int vmoba_block_scores_range(const vmoba_shape* shape, const void* q_bm, const void* k_bm, float* centroids,
+                             float* scores, float* score_range, int32_t* dev_status, void* ws, size_t ws_bytes,
+                             void* stream);
+
+/*
  * Step 2b, Eq. 3 + Eq. 4: global threshold selection per (batch, head).
  * The head's S*N_b scores are normalised with a softmax at temperature softmax_scale over the
  * whole pool; pairs are taken in descending score order until the cumulative mass is >= tau
@@ -167,6 +177,19 @@ int vmoba_select_rule_apply(const vmoba_shape* shape, const float* scores, int32
                             uint32_t* mask_bits, int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr,
                             int32_t* q_pairs, int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
                             int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * vmoba_select_rule_apply for a caller that already knows each head's score range (score_range [B*heads][2] =
+ * minimum, maximum, exactly as vmoba_block_scores_range wrote them for these scores): the head-wide rules then
+ * skip their own pass over the score matrix that looks for it (four traversals instead of five).  The results are
+ * those of vmoba_select_rule_apply bit for bit.  A range that does not bound the scores gives an unspecified
+ * selection (every access still stays inside the buffers).  The per-query rules and the row-normalised rule
+ * ignore the range.
+ */
+int vmoba_select_ranged(const vmoba_shape* shape, const float* scores, const float* score_range, int32_t rule, float tau,
+                        int32_t topk, uint32_t* mask_bits, int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr,
+                        int32_t* q_pairs, int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
+                        int32_t* dev_status, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * vmoba_select for callers that cannot hand over scratch memory.  (The paper has no counterpart:

@@ -17,7 +17,7 @@ STAGE_SCORES, STAGE_SELECT, STAGE_ATTN_FWD, STAGE_ATTN_BWD, STAGE_FULL_FWD, STAG
 
 EXPORTS = (
     "vmoba_status_string", "vmoba_kernel_launches", "vmoba_workspace_bytes", "vmoba_partition", "vmoba_block_scores",
-    "vmoba_select", "vmoba_select_rule_apply", "vmoba_select_static", "vmoba_select_static_scratch_bytes", "vmoba_attn_fwd",
+    "vmoba_block_scores_range", "vmoba_select", "vmoba_select_rule_apply", "vmoba_select_ranged", "vmoba_select_static", "vmoba_select_static_scratch_bytes", "vmoba_attn_fwd",
     "vmoba_attn_fwd_raster", "vmoba_attn_bwd", "vmoba_attn_bwd_raster", "vmoba_full_attn",
     "vmoba_debug_wait_profile",
 )
@@ -96,6 +96,11 @@ def lib():
     L.vmoba_partition.argtypes = [sp, ctypes.c_int, vp, vp, ctypes.POINTER(i64), vp, vp, vp]
     L.vmoba_block_scores.restype = ctypes.c_int
     L.vmoba_block_scores.argtypes = [sp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.vmoba_block_scores_range.restype = ctypes.c_int
+    L.vmoba_block_scores_range.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.vmoba_select_ranged.restype = ctypes.c_int
+    L.vmoba_select_ranged.argtypes = [sp, vp, vp, ctypes.c_int32, ctypes.c_float, ctypes.c_int32, vp, vp, vp, vp, vp, i64, vp,
+                                      vp, vp, vp, sz, vp]
     L.vmoba_select.restype = ctypes.c_int
     L.vmoba_select.argtypes = [sp, vp, ctypes.c_float, vp, vp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp]
     L.vmoba_select_static.restype = ctypes.c_int
@@ -166,6 +171,22 @@ def vmoba_block_scores(shape, q_bm, k_bm, centroids, scores, dev_status, ws, str
     p, n = _ws_args(ws)
     _check(lib().vmoba_block_scores(ctypes.byref(shape), _ptr(q_bm), _ptr(k_bm), _ptr(centroids), _ptr(scores),
                                     _ptr(dev_status), p, n, _stream(stream)), "vmoba_block_scores")
+
+
+def vmoba_block_scores_range(shape, q_bm, k_bm, centroids, scores, score_range, dev_status, ws, stream=None):
+    p, n = _ws_args(ws)
+    _check(lib().vmoba_block_scores_range(ctypes.byref(shape), _ptr(q_bm), _ptr(k_bm), _ptr(centroids), _ptr(scores),
+                                          _ptr(score_range), _ptr(dev_status), p, n, _stream(stream)),
+           "vmoba_block_scores_range")
+
+
+def vmoba_select_ranged(shape, scores, score_range, rule, tau, topk, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity,
+                        k_per_head, cutoff_per_head, dev_status, ws, stream=None):
+    p, n = _ws_args(ws)
+    _check(lib().vmoba_select_ranged(ctypes.byref(shape), _ptr(scores), _ptr(score_range), int(rule), float(tau),
+                                     int(topk), _ptr(mask_bits), _ptr(kb_ptr), _ptr(q_idx), _ptr(q_ptr), _ptr(q_pairs),
+                                     int(capacity), _ptr(k_per_head), _ptr(cutoff_per_head), _ptr(dev_status), p, n,
+                                     _stream(stream)), "vmoba_select_ranged")
 
 
 def vmoba_select(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity, k_per_head,

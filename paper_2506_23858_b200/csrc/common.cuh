@@ -187,6 +187,17 @@ __device__ __forceinline__ void store4_resid(__nv_bfloat16* p, __nv_bfloat16* re
   }
 }
 
+// Atomic minimum / maximum of fp32 values in global memory (the integer order of the bit patterns agrees with
+// the float order for non-negative values and is reversed for negative ones).  The word starts at +inf / -inf.
+__device__ __forceinline__ void atomic_min_f32(float* addr, float v) {
+  if (!(v < 0.f)) atomicMin(reinterpret_cast<int*>(addr), __float_as_int(v));
+  else atomicMax(reinterpret_cast<unsigned int*>(addr), __float_as_uint(v));
+}
+__device__ __forceinline__ void atomic_max_f32(float* addr, float v) {
+  if (!(v < 0.f)) atomicMax(reinterpret_cast<int*>(addr), __float_as_int(v));
+  else atomicMin(reinterpret_cast<unsigned int*>(addr), __float_as_uint(v));
+}
+
 // Order-preserving map from fp32 to uint32 (larger float <-> larger key).
 __device__ __forceinline__ uint32_t float_key(float f) {
   uint32_t u = __float_as_uint(f);

@@ -5,14 +5,16 @@
 // scores, and the [S, N_b] fp32 score matrix is written once.  The contraction itself
 // (2 * S * N_b * d flops) is small next to that and runs on the fp32 FMA pipe so that the
 // scores carry fp32 accuracy (the selection cutoff is compared in fp32).
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace vmoba {
 
 // scores_tc.cu: tensor-core scores for bf16 / head_dim 128
 size_t scores_tc_ws_bytes(const Dims& D);
-int scores_tc(const Dims& D, const void* q_bm, const float* cent, float* scores, void* ws, int32_t* status,
-              cudaStream_t st);
+int scores_tc(const Dims& D, const void* q_bm, const float* cent, float* scores, float* range, void* ws,
+              int32_t* status, cudaStream_t st);
 
 size_t scores_ws_bytes(const Dims& D) {
   return (D.dtype == VMOBA_BF16 && D.d == 128) ? scores_tc_ws_bytes(D) : 256;
@@ -115,17 +117,46 @@ scores_kernel(const T* __restrict__ q_bm, const float* __restrict__ cent, float*
   }
 }
 
+// Smallest and largest score of each head (the paths whose scores kernel does not take them on the way).
+__global__ void range_init_kernel(float* __restrict__ range, int BH) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < BH) { range[2 * i] = INFINITY; range[2 * i + 1] = -INFINITY; }
+}
+__global__ void __launch_bounds__(256)
+range_kernel(const float* __restrict__ scores, long long P, float* __restrict__ range) {
+  const int bh = blockIdx.y;
+  const float* base = scores + (long long)bh * P;
+  float lo = INFINITY, hi = -INFINITY;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < P; i += (long long)gridDim.x * blockDim.x) {
+    const float s = base[i];
+    lo = fminf(lo, s); hi = fmaxf(hi, s);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+  }
+  if ((threadIdx.x & 31) == 0 && lo <= hi) { atomic_min_f32(range + 2 * bh, lo); atomic_max_f32(range + 2 * bh + 1, hi); }
+}
+
 template <typename T, int DH>
-static int run_scores(const Dims& D, const void* q, const void* k, float* cent, float* scores, void* ws,
+static int run_scores(const Dims& D, const void* q, const void* k, float* cent, float* scores, float* range, void* ws,
                       int32_t* status, cudaStream_t st) {
   centroid_kernel<T, DH><<<D.BH * D.Nb, 256, 0, st>>>(static_cast<const T*>(k), cent, D.sb);
   VMOBA_LAUNCH_OK(1);
-  if (D.dtype == VMOBA_BF16 && DH == 128) return scores_tc(D, q, cent, scores, ws, status, st);
+  if (D.dtype == VMOBA_BF16 && DH == 128) return scores_tc(D, q, cent, scores, range, ws, status, st);
   size_t smem = 2 * DH * (64 + 4) * sizeof(float);
   VMOBA_CUDA_OK(cudaFuncSetAttribute(scores_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid((D.S + 63) / 64, 1, D.BH);
   scores_kernel<T, DH><<<grid, 256, smem, st>>>(static_cast<const T*>(q), cent, scores, D.S, D.Nb);
   VMOBA_LAUNCH_OK(1);
+  if (range) {
+    const long long P = (long long)D.S * D.Nb;
+    range_init_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(range, D.BH);
+    const int gx = (int)std::min<long long>(std::max<long long>(P / 2048, 1), std::max(1, sm_count() * 8 / D.BH));
+    range_kernel<<<dim3(gx, D.BH), 256, 0, st>>>(scores, P, range);
+    VMOBA_LAUNCH_OK(2);
+  }
   return VMOBA_OK;
 }
 
@@ -133,9 +164,8 @@ static int run_scores(const Dims& D, const void* q, const void* k, float* cent, 
 
 using namespace vmoba;
 
-extern "C" int vmoba_block_scores(const vmoba_shape* shape, const void* q_bm, const void* k_bm,
-                                  float* centroids, float* scores, int32_t* dev_status, void* ws,
-                                  size_t ws_bytes, void* stream) {
+static int block_scores_impl(const vmoba_shape* shape, const void* q_bm, const void* k_bm, float* centroids,
+                             float* scores, float* range, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
   Dims D;
   int rc = make_dims(shape, &D);
   if (rc) return rc;
@@ -145,9 +175,22 @@ extern "C" int vmoba_block_scores(const vmoba_shape* shape, const void* q_bm, co
   if (ws_bytes < scores_ws_bytes(D)) return VMOBA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (D.dtype == VMOBA_BF16) {
-    if (D.d == 128) return run_scores<__nv_bfloat16, 128>(D, q_bm, k_bm, centroids, scores, ws, dev_status, st);
-    return run_scores<__nv_bfloat16, 64>(D, q_bm, k_bm, centroids, scores, ws, dev_status, st);
+    if (D.d == 128) return run_scores<__nv_bfloat16, 128>(D, q_bm, k_bm, centroids, scores, range, ws, dev_status, st);
+    return run_scores<__nv_bfloat16, 64>(D, q_bm, k_bm, centroids, scores, range, ws, dev_status, st);
   }
-  if (D.d == 128) return run_scores<float, 128>(D, q_bm, k_bm, centroids, scores, ws, dev_status, st);
-  return run_scores<float, 64>(D, q_bm, k_bm, centroids, scores, ws, dev_status, st);
+  if (D.d == 128) return run_scores<float, 128>(D, q_bm, k_bm, centroids, scores, range, ws, dev_status, st);
+  return run_scores<float, 64>(D, q_bm, k_bm, centroids, scores, range, ws, dev_status, st);
+}
+
+extern "C" int vmoba_block_scores(const vmoba_shape* shape, const void* q_bm, const void* k_bm,
+                                  float* centroids, float* scores, int32_t* dev_status, void* ws,
+                                  size_t ws_bytes, void* stream) {
+  return block_scores_impl(shape, q_bm, k_bm, centroids, scores, nullptr, dev_status, ws, ws_bytes, stream);
+}
+
+extern "C" int vmoba_block_scores_range(const vmoba_shape* shape, const void* q_bm, const void* k_bm,
+                                        float* centroids, float* scores, float* score_range, int32_t* dev_status,
+                                        void* ws, size_t ws_bytes, void* stream) {
+  if (!score_range) return VMOBA_ERR_ARG;
+  return block_scores_impl(shape, q_bm, k_bm, centroids, scores, score_range, dev_status, ws, ws_bytes, stream);
 }

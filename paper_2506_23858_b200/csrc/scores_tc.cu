@@ -47,13 +47,19 @@ struct Params {
   int S, Nb, Nb_pad, BH;
   int n_pass, rows_pass;    // block ranges per head, rows per range (multiple of 16, <= NT_MAX)
   int tma_store;            // rows are multiples of 16 bytes: the epilogue writes through tmS
+  float* range;             // optional [BH][2]: smallest and largest score of each head (starts at +inf, -inf)
   int32_t* status;
 };
 
 // Splits fp32 centroids into three bf16 parts: parts[part][bh][Nb_pad][128]; pad rows are zero.
 __global__ void __launch_bounds__(256)
-split_centroids_kernel(const float* __restrict__ cent, __nv_bfloat16* __restrict__ parts, int Nb, int Nb_pad, int BH) {
+split_centroids_kernel(const float* __restrict__ cent, __nv_bfloat16* __restrict__ parts, int Nb, int Nb_pad, int BH,
+                       float* __restrict__ range) {
   const long long n = (long long)BH * Nb_pad * DH;
+  if (range) {     // the scores kernel that follows takes minima / maxima into these words
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < BH) { range[2 * t] = INFINITY; range[2 * t + 1] = -INFINITY; }
+  }
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
     const int c = (int)(i % DH);
     const long long row = i / DH;
@@ -193,11 +199,30 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int r = quad * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     uint32_t qn = 0, slabs = 0;
+    // smallest / largest score seen by this thread for the current head (the selection's first pass, taken
+    // here while the scores are in registers); handed over with one atomic pair per warp when the head changes
+    float rmin = INFINITY, rmax = -INFINITY;
+    long long range_bh = -1;
+    auto flush_range = [&]() {
+      if (p.range && range_bh >= 0) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          rmin = fminf(rmin, __shfl_xor_sync(0xffffffffu, rmin, o));
+          rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
+        }
+        if (lane == 0 && rmin <= rmax) {
+          atomic_min_f32(p.range + 2 * range_bh, rmin);
+          atomic_max_f32(p.range + 2 * range_bh + 1, rmax);
+        }
+      }
+      rmin = INFINITY; rmax = -INFINITY;
+    };
     for (long long it = it0; it < it1; ++it, ++qn) {
       const int tile = (int)(it % tiles);
       const long long group = it / tiles;
       const int pass = (int)(group % p.n_pass);
       const long long bh = group / p.n_pass;
+      if (bh != range_bh) { flush_range(); range_bh = bh; }
       const int s = qn & 1;
       mbar_wait(&sm->acc_full[s], (qn >> 1) & 1, abort_flag, p.status);
       tc_fence_after();
@@ -213,6 +238,11 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           uint32_t v[32];
           tmem_ld32(a_tmem + c0, v);
           tmem_ld_wait();
+          if (p.range && row < p.S) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c0 + i < ncols) { rmin = fminf(rmin, __uint_as_float(v[i])); rmax = fmaxf(rmax, __uint_as_float(v[i])); }
+          }
           uint8_t* slab = sOut + (slabs & 1) * SLAB;
           // the slab's previous store (two slabs ago) must have read it
           if (threadIdx.x == 64) bulk_wait_group_read<1>();
@@ -237,13 +267,17 @@ scores_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (row < p.S) {
 #pragma unroll
           for (int i = 0; i < 32; ++i)
-            if (c0 + i < ncols) out[c0 + i] = __uint_as_float(v[i]);
+            if (c0 + i < ncols) {
+              out[c0 + i] = __uint_as_float(v[i]);
+              rmin = fminf(rmin, __uint_as_float(v[i])); rmax = fmaxf(rmax, __uint_as_float(v[i]));
+            }
         }
       }
       }
       tc_fence_before();
       mbar_arrive(&sm->acc_empty[s]);
     }
+    flush_range();
     if (threadIdx.x == 64) bulk_wait_group<0>();      // shared memory must outlive the last stores' reads
   }
   tc_fence_before();
@@ -259,8 +293,8 @@ size_t scores_tc_ws_bytes(const Dims& D) {
 }
 
 // scores [BH, S, Nb] fp32 from block-major bf16 q and fp32 centroids (already computed).
-int scores_tc(const Dims& D, const void* q_bm, const float* cent, float* scores, void* ws, int32_t* status,
-              cudaStream_t st) {
+int scores_tc(const Dims& D, const void* q_bm, const float* cent, float* scores, float* range, void* ws,
+              int32_t* status, cudaStream_t st) {
   using namespace sct;
   // ranges of whole 32-column slabs (the epilogue's store unit)
   const int Nb_pad = (D.Nb + 31) / 32 * 32;
@@ -268,7 +302,7 @@ int scores_tc(const Dims& D, const void* q_bm, const float* cent, float* scores,
   const int rows_pass = ((Nb_pad + n_pass - 1) / n_pass + 31) / 32 * 32;
   __nv_bfloat16* parts = reinterpret_cast<__nv_bfloat16*>((reinterpret_cast<uintptr_t>(ws) + 1023) & ~uintptr_t(1023));
   const long long n = (long long)D.BH * Nb_pad * DH;
-  split_centroids_kernel<<<(int)std::min<long long>((n + 255) / 256, sm_count() * 8), 256, 0, st>>>(cent, parts, D.Nb, Nb_pad, D.BH);
+  split_centroids_kernel<<<(int)std::min<long long>((n + 255) / 256, sm_count() * 8), 256, 0, st>>>(cent, parts, D.Nb, Nb_pad, D.BH, range);
   CUtensorMap tmQ, tmB, tmS;
   const int tma_store = (D.Nb % 4 == 0) && (reinterpret_cast<uintptr_t>(scores) % 16 == 0);
   if (tma_store) {
@@ -282,6 +316,7 @@ int scores_tc(const Dims& D, const void* q_bm, const float* cent, float* scores,
   Params p;
   p.scores = scores; p.S = D.S; p.Nb = D.Nb; p.Nb_pad = Nb_pad; p.BH = D.BH; p.n_pass = n_pass; p.rows_pass = rows_pass;
   p.tma_store = tma_store;
+  p.range = range;
   p.status = status;
   VMOBA_CUDA_OK(cudaFuncSetAttribute(scores_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
   const long long items = (long long)D.BH * n_pass * ((D.S + BM - 1) / BM);

@@ -94,14 +94,29 @@ minmax_kernel(const float* __restrict__ scores, long long P, HeadState* __restri
   }
 }
 
-__global__ void init_state_kernel(HeadState* st, int BH) {
-  int i = blockIdx.x * blockDim.x + threadIdx.x;
+// Start of a call: the per-head state and, for the head-wide rules, the histogram arrays (one kernel instead of
+// a memset per array).  If the caller knows each head's score range (range: [BH][2] = minimum, maximum, as
+// vmoba_block_scores_range writes them), the level-0 bins are laid over it here and no pass of the selection's
+// own has to look for it.
+__global__ void init_state_kernel(HeadState* st, int BH, const float* __restrict__ range, unsigned int* __restrict__ g_cnt,
+                                  double* __restrict__ g_w, uint32_t* __restrict__ g_minkey,
+                                  uint32_t* __restrict__ g_maxkey) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (g_cnt && i < (long long)BH * kBins) { g_cnt[i] = 0u; g_w[i] = 0.0; g_minkey[i] = 0xffffffffu; g_maxkey[i] = 0u; }
   if (i >= BH) return;
   HeadState h;
   memset(&h, 0, sizeof(h));
   h.min_key = 0xffffffffu;
   h.max_key = 0u;
   h.cutoff_key = 0xffffffffu;      // the per-query rules take the minimum of their row cutoffs into it
+  if (range) {
+    const float lo = range[2 * i], hi = range[2 * i + 1];
+    h.min_key = float_key(lo);
+    h.max_key = float_key(hi);
+    const float span = hi - lo;
+    h.anchor[0] = lo;
+    h.inv[0] = span > 0.f ? (float)kBins0 / span : 0.f;
+  }
   st[i] = h;
 }
 
@@ -771,7 +786,7 @@ size_t select_rownorm_ws_bytes(const Dims& D) {
 
 using namespace vmoba;
 
-static int select_impl(const vmoba_shape* shape, const float* scores, int rule, float tau, int topk, uint32_t* mask_bits,
+static int select_impl(const vmoba_shape* shape, const float* scores, const float* range, int rule, float tau, int topk, uint32_t* mask_bits,
                        int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr, int32_t* q_pairs, int64_t capacity,
                        int64_t* k_per_head, float* cutoff_per_head, int32_t* dev_status, void* ws, size_t ws_bytes,
                        void* stream) {
@@ -806,14 +821,15 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
     VMOBA_LAUNCH_OK(1);
     scores = lp;
     sigma = 1.0f;
+    range = nullptr;      // the range of the raw scores says nothing about the transformed matrix
   }
   const int QSEG = seg_queries(D.mask_words);
   const int nseg = (D.S + QSEG - 1) / QSEG;
   const size_t smem = (size_t)QSEG * D.mask_words * 4 + (size_t)std::max(D.Nb, QSEG) * 4 + (size_t)D.Nb * (QSEG >> 5) * 4;
   const dim3 sgrid(nseg, D.BH);
 
-  init_state_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH);
   if (local) {
+    init_state_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH, nullptr, nullptr, nullptr, nullptr, nullptr);
     // per-query rules: the mask comes straight from the rows; cutoff_key collects the smallest selected key
     const long long n_rows = (long long)D.BH * D.S;
     const int blocks = (int)std::min<long long>((n_rows + 7) / 8, sm_count() * 8);
@@ -841,17 +857,18 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
       tau = count_target >= (double)P ? 1.0f : 0.5f;      // tau only tells the scan whether everything is taken
     }
     const int unit_w = by_topk ? 1 : 0;
-    VMOBA_CUDA_OK(cudaMemsetAsync(w.g_cnt, 0, (size_t)D.BH * kBins * sizeof(unsigned int), st));
-    VMOBA_CUDA_OK(cudaMemsetAsync(w.g_w, 0, (size_t)D.BH * kBins * sizeof(double), st));
-    VMOBA_CUDA_OK(cudaMemsetAsync(w.g_minkey, 0xff, (size_t)D.BH * kBins * sizeof(uint32_t), st));
-    VMOBA_CUDA_OK(cudaMemsetAsync(w.g_maxkey, 0, (size_t)D.BH * kBins * sizeof(uint32_t), st));
+    init_state_kernel<<<(unsigned)(((long long)D.BH * kBins + 255) / 256), 256, 0, st>>>(w.state, D.BH, range, w.g_cnt, w.g_w,
+                                                                                        w.g_minkey, w.g_maxkey);
 
     // enough CTAs per head to fill the machine, few enough that the per-CTA flush stays small
     long long per_head = (P / 4 + 255) / 256;
     int gx = (int)std::min<long long>(std::max<long long>(per_head / 8, 1), std::max(1, sm_count() * 8 / D.BH));
     dim3 grid(gx, D.BH);
-    minmax_kernel<<<grid, 256, 0, st>>>(scores, P, w.state);
-    setup_level0_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH);
+    if (!range) {
+      minmax_kernel<<<grid, 256, 0, st>>>(scores, P, w.state);
+      setup_level0_kernel<<<(D.BH + 127) / 128, 128, 0, st>>>(w.state, D.BH);
+      count_launches(2);
+    }
     {
       constexpr int smem0 = kBins0 * kRep * (int)sizeof(float);
       VMOBA_CUDA_OK(cudaFuncSetAttribute(hist0_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem0));
@@ -867,7 +884,7 @@ static int select_impl(const vmoba_shape* shape, const float* scores, int rule, 
     hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, sigma, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
     scan_kernel<2><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,
                                          cutoff_per_head);
-    VMOBA_LAUNCH_OK(9);
+    VMOBA_LAUNCH_OK(7);
     VMOBA_CUDA_OK(cudaFuncSetAttribute(mark_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     mark_kernel<<<sgrid, kSegThreads, smem, st>>>(scores, w.state, D.S, D.Nb, D.mask_words, QSEG, nseg, own_sb, mask_bits,
                                                   w.seg_cnt, w.seg_total, w.tmask);
@@ -889,7 +906,16 @@ extern "C" int vmoba_select(const vmoba_shape* shape, const float* scores, float
                             int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr, int32_t* q_pairs,
                             int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
                             int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
-  return select_impl(shape, scores, VMOBA_SELECT_THRESHOLD_GLOBAL, tau, 0, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity,
+  return select_impl(shape, scores, nullptr, VMOBA_SELECT_THRESHOLD_GLOBAL, tau, 0, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs,
+                     capacity, k_per_head, cutoff_per_head, dev_status, ws, ws_bytes, stream);
+}
+
+extern "C" int vmoba_select_ranged(const vmoba_shape* shape, const float* scores, const float* score_range, int32_t rule,
+                                   float tau, int32_t topk, uint32_t* mask_bits, int32_t* kb_ptr, int32_t* q_idx,
+                                   int32_t* q_ptr, int32_t* q_pairs, int64_t capacity, int64_t* k_per_head,
+                                   float* cutoff_per_head, int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
+  if (!score_range) return VMOBA_ERR_ARG;
+  return select_impl(shape, scores, score_range, rule, tau, topk, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity,
                      k_per_head, cutoff_per_head, dev_status, ws, ws_bytes, stream);
 }
 
@@ -897,7 +923,7 @@ extern "C" int vmoba_select_rule_apply(const vmoba_shape* shape, const float* sc
                                        uint32_t* mask_bits, int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr,
                                        int32_t* q_pairs, int64_t capacity, int64_t* k_per_head, float* cutoff_per_head,
                                        int32_t* dev_status, void* ws, size_t ws_bytes, void* stream) {
-  return select_impl(shape, scores, rule, tau, topk, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity, k_per_head,
+  return select_impl(shape, scores, nullptr, rule, tau, topk, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity, k_per_head,
                      cutoff_per_head, dev_status, ws, ws_bytes, stream);
 }
 

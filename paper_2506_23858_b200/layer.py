@@ -46,6 +46,8 @@ class VmobaLayer:
         self.q_pairs = torch.empty(self.capacity, dtype=torch.int32, device=dev)
         self.k_per_head = torch.empty(BH, dtype=torch.int64, device=dev)
         self.cutoff = torch.empty(BH, dtype=torch.float32, device=dev)
+        self.score_range = torch.empty((BH, 2), dtype=torch.float32, device=dev)   # per head: smallest, largest score
+        self.range_valid = False
         self.lse = torch.empty(BH * S, dtype=torch.float32, device=dev)
         self.perm = torch.empty(S, dtype=torch.int32, device=dev)     # raster token of block-major position p (Eq. 1)
         self.dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
@@ -71,10 +73,26 @@ class VmobaLayer:
         src, dst = (bm, raster) if inverse else (raster, bm)
         vb.vmoba_partition(self.shape, int(inverse), src, dst, self.raster_strides(raster), perm, inv_perm)
 
-    def block_scores(self):
-        vb.vmoba_block_scores(self.shape, self.q_bm, self.k_bm, self.centroids, self.scores, self.dev_status, self.ws)
+    def block_scores(self, with_range=True):
+        """Centroids and scores; with_range: the scores kernel also takes each head's smallest and largest score,
+        which lets select() skip its own pass for them (valid until self.scores is overwritten by other means)."""
+        if with_range:
+            vb.vmoba_block_scores_range(self.shape, self.q_bm, self.k_bm, self.centroids, self.scores, self.score_range,
+                                        self.dev_status, self.ws)
+        else:
+            vb.vmoba_block_scores(self.shape, self.q_bm, self.k_bm, self.centroids, self.scores, self.dev_status, self.ws)
+        self.range_valid = bool(with_range)
 
-    def select(self, tau, scores=None):
+    def select(self, tau, scores=None, use_range=None):
+        """Eq. 3 + Eq. 4.  use_range: take the score range the last block_scores() left (default: if it left one and
+        the scores are the layer's own)."""
+        if use_range is None:
+            use_range = self.range_valid and scores is None
+        if use_range:
+            vb.vmoba_select_ranged(self.shape, self.scores, self.score_range, vb.SELECT_THRESHOLD_GLOBAL, tau, 0,
+                                   self.mask_bits, self.kb_ptr, self.q_idx, self.q_ptr, self.q_pairs, self.capacity,
+                                   self.k_per_head, self.cutoff, self.dev_status, self.ws)
+            return
         vb.vmoba_select(self.shape, self.scores if scores is None else scores, tau, self.mask_bits, self.kb_ptr,
                         self.q_idx, self.q_ptr, self.q_pairs, self.capacity, self.k_per_head, self.cutoff,
                         self.dev_status, self.ws)

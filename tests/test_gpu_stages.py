@@ -258,3 +258,40 @@ def test_dense_attention_forward_backward(w):
         ref = orc.dense_attn_bwd(hd["q"], hd["k"], hd["v"], ora["scale"], data["do"][b, :, h][ora["perm"]])
         for name, got, want in zip(("dq", "dk", "dv"), g, ref):
             U.assert_close(got[i], want, w.dtype, name)
+
+
+@pytest.mark.parametrize("w", [CASES[0], CASES[3], CASES[4], CASES[6], CASES[7], CASES[8]],
+                         ids=[IDS[0], IDS[3], IDS[4], IDS[6], IDS[7], IDS[8]])
+def test_score_range_from_the_scores_kernel_and_ranged_selection(w):
+    """vmoba_block_scores_range must report exactly the smallest and largest score of every head, and
+    vmoba_select_ranged, which skips its own search for them, must return what vmoba_select returns, bit for bit."""
+    data, ora = _prep(w)
+    shape = vb.shape_of(w)
+    cap = w.B * w.heads * w.S * w.n_blocks
+    L = VmobaLayer(shape, capacity=cap)
+    L.q_bm.copy_(U.bm_to_device(w, U.block_major(w, data, "q", ora["perm"])))
+    L.k_bm.copy_(U.bm_to_device(w, U.block_major(w, data, "k", ora["perm"])))
+    L.score_range.fill_(float("nan"))
+    L.block_scores(with_range=True)
+    torch.cuda.synchronize()
+    sc = L.scores.view(w.B * w.heads, -1)
+    assert torch.equal(L.score_range[:, 0], sc.amin(dim=1)) and torch.equal(L.score_range[:, 1], sc.amax(dim=1))
+    plain = L.scores.clone()
+    L.block_scores(with_range=False)
+    assert torch.equal(L.scores, plain)                       # the scores themselves do not depend on the entry point
+    names = ("mask_bits", "kb_ptr", "q_ptr", "k_per_head", "cutoff")
+    for tau in (w.tau, 0.6):
+        L.select(tau, use_range=False)
+        torch.cuda.synchronize()
+        n = L.n_selected()
+        ref = {k: getattr(L, k).clone() for k in names}
+        ref["q_idx"], ref["q_pairs"] = L.q_idx[:n].clone(), L.q_pairs[:n].clone()
+        for k in names:
+            getattr(L, k).fill_(0)
+        L.q_idx.fill_(-1); L.q_pairs.fill_(-1)
+        L.select(tau, use_range=True)
+        torch.cuda.synchronize()
+        L.check_status()
+        for k in names:
+            assert torch.equal(getattr(L, k), ref[k]), (tau, k)
+        assert torch.equal(L.q_idx[:n], ref["q_idx"]) and torch.equal(L.q_pairs[:n], ref["q_pairs"])
