@@ -13,7 +13,10 @@
  * Conventions shared by every entry point
  *   - All data pointers are DEVICE pointers, 16-byte aligned, owned by the caller.  The
  *     library allocates no device memory and keeps no state between calls; scratch memory
- *     is passed in as `ws` and must hold vmoba_workspace_bytes() bytes.
+ *     is passed in as `ws` and must hold vmoba_workspace_bytes() bytes.  Two entry points are
+ *     exceptions and say so: vmoba_select_static keeps a 16 MiB device array inside the library
+ *     image and a per-device cache of its address, and vmoba_debug_wait_profile keeps the pointer
+ *     it was given until it is cleared.
  *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work on it and
  *     return; they never synchronise.
  *   - The return value reports errors the host can see (bad arguments, shapes, workspace
@@ -206,7 +209,11 @@ int vmoba_select_ranged(const vmoba_shape* shape, const float* scores, const flo
  *   - The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
  *   - The first call on each device looks up the array's device address (one
  *     cudaGetSymbolAddress, with that device current); make that first call outside of any stream
- *     capture.  Later calls on the device reuse the address.
+ *     capture.  Later calls on the device reuse the address.  The address cache is filled without a
+ *     lock: two host threads that make the first call on one device at the same time both look the
+ *     address up and store the same value.
+ *   - The current device must be the device of `stream` and of every buffer: the address that is
+ *     used is the current device's copy of the array.
  *   - All calls on one device share the one array.  Every call re-initialises what it needs, so
  *     stale contents are harmless, but two calls whose kernels can overlap on the GPU (different
  *     streams, no ordering between them) race on it: serialise them.
@@ -304,6 +311,16 @@ int vmoba_full_attn(const vmoba_shape* shape, const void* q, const void* k, cons
  *     [13] total; writer warp: [9] wait for dQ^T, [14] reading it from TMEM, [15] waiting at the staging barrier.
  */
 void vmoba_debug_wait_profile(void* dev_counters16);
+
+/*
+ * Diagnostics; not part of the method.  Exercises the failure path of the kernels' bounded device-side waits
+ * without starving a real kernel: one CTA waits on a barrier that nothing arrives at, with a limit of `polls`
+ * polls (1 .. 65536; the attention kernels use 2^22).  The wait gives up, dev_status receives
+ * VMOBA_ERR_TIMEOUT (if it was 0), the CTA's later waits give up after a few polls and the kernel ends by itself.
+ * out2_or_null (device int32 [2]) receives the number of waits that gave up (128: two per thread) and a 1 written
+ * by the kernel's last instruction.
+ */
+int vmoba_debug_wait_timeout(int32_t* dev_status, uint32_t polls, int32_t* out2_or_null, void* stream);
 
 #ifdef __cplusplus
 }

@@ -19,7 +19,7 @@ EXPORTS = (
     "vmoba_status_string", "vmoba_kernel_launches", "vmoba_workspace_bytes", "vmoba_partition", "vmoba_block_scores",
     "vmoba_block_scores_range", "vmoba_select", "vmoba_select_rule_apply", "vmoba_select_ranged", "vmoba_select_static", "vmoba_select_static_scratch_bytes", "vmoba_attn_fwd",
     "vmoba_attn_fwd_raster", "vmoba_attn_bwd", "vmoba_attn_bwd_raster", "vmoba_full_attn",
-    "vmoba_debug_wait_profile",
+    "vmoba_debug_wait_profile", "vmoba_debug_wait_timeout",
 )
 
 
@@ -120,6 +120,8 @@ def lib():
                                         vp, vp, vp, p64, vp, vp, vp, sz, vp]
     L.vmoba_attn_fwd_raster.restype = ctypes.c_int
     L.vmoba_attn_fwd_raster.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, i64, vp, p64, vp, vp, vp, vp, vp, sz, vp]
+    L.vmoba_debug_wait_timeout.restype = ctypes.c_int
+    L.vmoba_debug_wait_timeout.argtypes = [vp, ctypes.c_uint32, vp, vp]
     L.vmoba_debug_wait_profile.restype = None
     L.vmoba_debug_wait_profile.argtypes = [vp]
     L.vmoba_full_attn.restype = ctypes.c_int
@@ -270,6 +272,12 @@ def vmoba_full_attn(shape, q, k, v, o, lse, do=None, dq=None, dk=None, dv=None, 
     _check(lib().vmoba_full_attn(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(do),
                                  _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dev_status), p, n, _stream(stream)),
            "vmoba_full_attn")
+
+
+def vmoba_debug_wait_timeout(dev_status, polls, out2=None, stream=None):
+    """Runs the one-CTA kernel whose bounded wait is made to run out (see include/vmoba.h)."""
+    _check(lib().vmoba_debug_wait_timeout(_ptr(dev_status), int(polls), _ptr(out2), _stream(stream)),
+           "vmoba_debug_wait_timeout")
 
 
 def vmoba_debug_wait_profile(counters=None):

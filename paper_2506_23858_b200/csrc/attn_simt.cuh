@@ -290,6 +290,44 @@ rowdot_kernel(const T* __restrict__ o, const T* __restrict__ o_resid, const T* _
   const int lane = threadIdx.x & 31;
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
+  if constexpr (C == 4 && sizeof(T) == 2) {
+    // Four rows per warp and trip, in phases (row offsets, loads, sums, stores), so that the twelve 8-byte
+    // loads of a lane are in flight together.
+    constexpr int R = 4;
+    for (long long g0 = warp * R; g0 < n_queries; g0 += nwarps * R) {
+      uint2 ov[R], rv[R], dv[R];
+      bool zero[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const long long g = min(g0 + r, n_queries - 1);
+        ov[r] = *reinterpret_cast<const uint2*>(o + o_map.off(g, DH) + lane * 4);
+        dv[r] = *reinterpret_cast<const uint2*>(d_o + do_map.off(g, DH) + lane * 4);
+        rv[r] = o_resid ? *reinterpret_cast<const uint2*>(o_resid + g * DH + lane * 4) : make_uint2(0u, 0u);
+        zero[r] = zero_acc && g0 + r < n_queries && __ldg(q_ptr + g + 1) - __ldg(q_ptr + g) >= 1;
+      }
+      float a[R];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        auto lo = [](uint32_t u) { return __uint_as_float(u << 16); };
+        auto hi = [](uint32_t u) { return __uint_as_float(u & 0xffff0000u); };
+        a[r] = (lo(ov[r].x) + lo(rv[r].x)) * lo(dv[r].x);
+        a[r] = fmaf(hi(ov[r].x) + hi(rv[r].x), hi(dv[r].x), a[r]);
+        a[r] = fmaf(lo(ov[r].y) + lo(rv[r].y), lo(dv[r].y), a[r]);
+        a[r] = fmaf(hi(ov[r].y) + hi(rv[r].y), hi(dv[r].y), a[r]);
+      }
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1)
+#pragma unroll
+        for (int r = 0; r < R; ++r) a[r] += __shfl_xor_sync(0xffffffffu, a[r], s);
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if (g0 + r >= n_queries) break;
+        if (lane == 0) Dv[g0 + r] = a[r];
+        if (zero[r]) reinterpret_cast<float4*>(zero_acc + (g0 + r) * DH)[lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    return;
+  }
   for (long long g = warp; g < n_queries; g += nwarps) {
     float a = 0.f;
     const T* do_row = d_o + do_map.off(g, DH);

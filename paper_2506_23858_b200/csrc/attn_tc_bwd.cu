@@ -584,12 +584,10 @@ static int grid_items(long long items) { return (int)std::max<long long>(1, std:
 }  // namespace tcb
 
 // attn_tc_bwd_long.cu
-int tc_long_dkdv(const Dims& D, bool dense, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
-                 const float* Dv, const int* kb_ptr, const int* q_idx, long long cap, void* dk, void* dv, int32_t* status,
-                 unsigned long long* prof, cudaStream_t st);
-int tc_long_dq(const Dims& D, bool dense, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
-               const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap, const int* item_ptr,
-               const int* item_tab, float* dq_acc, void* dq, int32_t* status, cudaStream_t st);
+int tc_long_dkdv(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                 const float* Dv, void* dk, void* dv, int32_t* status, unsigned long long* prof, cudaStream_t st);
+int tc_long_dq(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+               const float* Dv, void* dq, int32_t* status, cudaStream_t st);
 // Backward over the work lists (bf16, head_dim 128).  Dv holds rowsum(dO * O) per query; dq_acc is
 // an fp32 accumulator whose rows of selecting queries are zero; the caller converts it to bf16.
 int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
@@ -622,9 +620,9 @@ int tc_sparse_bwd(const Dims& D, const void* q, const void* k, const void* v, co
 // Dense backward: the kernels with 128-query units (one key range spanning the sequence).
 int tc_dense_bwd(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
                  const float* Dv, void* dq, void* dk, void* dv, int32_t* status, cudaStream_t st) {
-  int rc = tc_long_dkdv(D, true, q, k, v, d_o, lse, Dv, nullptr, nullptr, 0, dk, dv, status, tcb::g_wait_profile, st);
+  int rc = tc_long_dkdv(D, q, k, v, d_o, lse, Dv, dk, dv, status, tcb::g_wait_profile, st);
   if (rc) return rc;
-  return tc_long_dq(D, true, q, k, v, d_o, lse, Dv, nullptr, nullptr, nullptr, 0, nullptr, nullptr, nullptr, dq, status, st);
+  return tc_long_dq(D, q, k, v, d_o, lse, Dv, dq, status, st);
 }
 
 }  // namespace vmoba

@@ -12,8 +12,6 @@
 //        rows).  TMEM: S^T | dP^T | dV | dK, 128 columns each.  K/V tile single-buffered, Q/dO ring of 2.
 // dQ:    item = 128 queries x the key range, in units of 128 keys.
 //        TMEM: S | dP | dQ (x2, alternating by item).  Q/dO tile single-buffered, K/V ring of 2.
-// The kernels also carry index-list (gathered) variants of their loads from the time they served the
-// sparse path; those template branches are not instantiated any more.
 #include <algorithm>
 
 #include "attn_simt.cuh"
@@ -38,10 +36,6 @@ __device__ __forceinline__ constexpr uint32_t mnoff(int ks) { return (uint32_t)(
 __device__ __forceinline__ uint64_t desc_k0(uint32_t tile_addr) { return make_smem_desc(tile_addr, 16, 1024); }
 __device__ __forceinline__ uint64_t desc_mn0(uint32_t tile_addr) { return make_smem_desc(tile_addr, PANEL, 1024); }
 
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-
 // Order in which the four 32-column groups become ready: warps 2-5 do groups 0 then 1, warps 6-9 do
 // groups 2 then 3, so the MMA warp consumes 0, 2, 1, 3.
 __device__ __forceinline__ constexpr int group_order(int i) { return i == 0 ? 0 : i == 1 ? 2 : i == 2 ? 1 : 3; }
@@ -65,10 +59,8 @@ constexpr size_t KV_SMEM_BYTES = 1024 + 2 * TILE + 2 * 2 * TILE + sizeof(KvSmem)
 struct KvParams {
   const __nv_bfloat16 *q, *d_o;
   const float *lse, *Dv;
-  const int *kb_ptr, *q_idx;
-  int S, Nb, sb, BH;
+  int S, BH;
   float scale, scale_log2;
-  long long capacity;
   __nv_bfloat16 *dk, *dv;
   int32_t* status;
   unsigned long long* prof;    // optional wait-time counters (diagnostics), or null
@@ -79,26 +71,19 @@ struct KvItem {
   long long list_lo, list_hi, head_off;
 };
 
-template <bool DENSE>
-__device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, int tiles, int span) {
+// item = (batch * heads + head, key tile); every query of the head meets the tile
+__device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, int tiles) {
   KvItem it;
   const int tile = (int)(item % tiles);
-  const long long kbi = item / tiles;
-  it.bh = DENSE ? (int)kbi : (int)(kbi / p.Nb);
-  const int j = DENSE ? 0 : (int)(kbi - (long long)it.bh * p.Nb);
-  it.key0 = j * p.sb + tile * BN;
-  it.valid = min(BN, span - tile * BN);
+  it.bh = (int)(item / tiles);
+  it.key0 = tile * BN;
+  it.valid = min(BN, p.S - tile * BN);
   it.list_lo = 0; it.list_hi = p.S;
-  if (!DENSE) {
-    it.list_lo = min((long long)p.kb_ptr[kbi], p.capacity);
-    it.list_hi = min((long long)p.kb_ptr[kbi + 1], p.capacity);
-  }
   it.n_units = (int)((it.list_hi - it.list_lo + BM - 1) / BM);
   it.head_off = (long long)it.bh * p.S;
   return it;
 }
 
-template <bool DENSE>
 __global__ void __launch_bounds__(KV_THREADS, 1)
 dkdv_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                  const __grid_constant__ CUtensorMap tmQrow, const __grid_constant__ CUtensorMap tmOrow, const KvParams p) {
@@ -149,16 +134,15 @@ dkdv_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
   const uint32_t tmem = sm->tmem_base;
   constexpr uint32_t ST_COL = 0, DPT_COL = 128, DV_COL = 256, DK_COL = 384;
 
-  const int span = DENSE ? p.S : p.sb;
-  const int tiles = (span + BN - 1) / BN;
-  const long long n_items = (long long)p.BH * (DENSE ? 1 : p.Nb) * tiles;
+  const int tiles = (p.S + BN - 1) / BN;
+  const long long n_items = (long long)p.BH * tiles;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer: the item's K and V tiles
     if (lane == 0) {
       uint32_t n = 0;
       for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+        const KvItem it = kv_decode(p, item, tiles);
         if (it.n_units == 0) continue;
         if (n >= 1) twait(0, &sm->kv_empty, (n - 1) & 1);
         const int y = (int)it.head_off + it.key0;
@@ -180,7 +164,7 @@ dkdv_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
       uint32_t n = 0, u0 = 0;
       const uint64_t dK0 = desc_k0(smem_u32(sK)), dV0 = desc_k0(smem_u32(sV));
       for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+        const KvItem it = kv_decode(p, item, tiles);
         if (it.n_units == 0) continue;
         wwait(0, &sm->kv_full, n & 1);
         for (int i = 0; i < it.n_units; ++i) {
@@ -233,7 +217,7 @@ dkdv_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const int chunk = lt & 15, panel = chunk >> 3, cc = chunk & 7;
     uint32_t u0 = 0;
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-      const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+      const KvItem it = kv_decode(p, item, tiles);
       const __nv_bfloat16* qh = p.q + it.head_off * DH;
       const __nv_bfloat16* oh = p.d_o + it.head_off * DH;
       for (int i = 0; i < it.n_units; ++i) {
@@ -248,14 +232,14 @@ dkdv_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
           vq[k2] = make_uint4(0u, 0u, 0u, 0u);
           vo[k2] = vq[k2];
           if (row < rows) {
-            const long long src = DENSE ? lo + row : (long long)__ldg(p.q_idx + lo + row);
+            const long long src = lo + row;
             vq[k2] = __ldg(reinterpret_cast<const uint4*>(qh + src * DH) + chunk);
             vo[k2] = __ldg(reinterpret_cast<const uint4*>(oh + src * DH) + chunk);
           }
         }
         float l2 = INFINITY, dd = 0.f;     // padded queries: P = exp2(-inf) = 0
         if (lt < rows) {
-          const long long G_ = it.head_off + (DENSE ? lo + lt : (long long)__ldg(p.q_idx + lo + lt));
+          const long long G_ = it.head_off + lo + lt;
           l2 = p.lse[G_] * 1.4426950408889634f;
           dd = p.Dv[G_];
         }
@@ -283,7 +267,7 @@ dkdv_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant_
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     uint32_t n = 0, u0 = 0;
     for (long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-      const KvItem it = kv_decode<DENSE>(p, item, tiles, span);
+      const KvItem it = kv_decode(p, item, tiles);
       __nv_bfloat16* dv_row = p.dv + (it.head_off + it.key0 + r) * DH;
       __nv_bfloat16* dk_row = p.dk + (it.head_off + it.key0 + r) * DH;
       if (it.n_units == 0) {
@@ -381,17 +365,13 @@ struct DqSmem {
   float lse2[128];
   float Dr[128];
   int G[128];                  // flat output row of each query (b*heads+head)*S + p, -1 for padding rows
-  int direct[128];             // query has a single block: write bf16 directly
 };
 constexpr size_t DQ_SMEM_BYTES = 1024 + 2 * TILE + 2 * 2 * TILE + sizeof(DqSmem) + 32;
 
 struct DqParams {
   const float *lse, *Dv;
-  const int *kb_ptr, *q_idx, *q_ptr, *item_ptr, *item_tab;
-  int n_kb, S, Nb, sb, BH;
+  int S, BH;
   float scale, scale_log2;
-  long long capacity;
-  float* dq_acc;
   __nv_bfloat16* dq;
   int32_t* status;
 };
@@ -401,30 +381,18 @@ struct DqItem {
   long long head_off;
 };
 
-template <bool DENSE>
+// item = (batch * heads + head, tile of 128 consecutive queries) against all keys of the head
 __device__ __forceinline__ DqItem dq_decode(const DqParams& p, int item) {
   DqItem it;
-  if (DENSE) {
-    const int tiles = (p.S + BM - 1) / BM;
-    it.bh = item / tiles;
-    const int t = item - it.bh * tiles;
-    it.key_begin = 0; it.n_keys = p.S; it.list_lo = t * BM; it.n_rows = min(BM, p.S - it.list_lo);
-  } else {
-    const int kbi = __ldg(p.item_tab + item);
-    const int chunk = item - __ldg(p.item_ptr + kbi);
-    it.bh = kbi / p.Nb;
-    const int j = kbi - it.bh * p.Nb;
-    it.key_begin = j * p.sb; it.n_keys = p.sb;
-    const long long end = min((long long)__ldg(p.kb_ptr + kbi + 1), p.capacity);
-    it.list_lo = __ldg(p.kb_ptr + kbi) + chunk * BM;
-    it.n_rows = (int)min((long long)BM, end - it.list_lo);
-  }
+  const int tiles = (p.S + BM - 1) / BM;
+  it.bh = item / tiles;
+  const int t = item - it.bh * tiles;
+  it.key_begin = 0; it.n_keys = p.S; it.list_lo = t * BM; it.n_rows = min(BM, p.S - it.list_lo);
   it.n_units = (it.n_keys + BN - 1) / BN;
   it.head_off = (long long)it.bh * p.S;
   return it;
 }
 
-template <bool DENSE>
 __global__ void __launch_bounds__(THREADS, 1)
 dq_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                const __grid_constant__ CUtensorMap tmQrow, const __grid_constant__ CUtensorMap tmOrow, const DqParams p) {
@@ -458,31 +426,30 @@ dq_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem = sm->tmem_base;
   constexpr uint32_t S_COL = 0, DP_COL = 128, DQ_COL = 256;
-  const int n_items = DENSE ? p.BH * ((p.S + BM - 1) / BM) : p.item_ptr[p.n_kb];
+  const int n_items = p.BH * ((p.S + BM - 1) / BM);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer: gathered Q / dO of the item, K/V units
     uint32_t n = 0, f = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
-      const DqItem it = dq_decode<DENSE>(p, item);
-      int rc[4], gi[4], dr[4];
+      const DqItem it = dq_decode(p, item);
+      int rc[4], gi[4];
       float l2[4], dd[4];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const int r = 4 * lane + k;
         const bool ok = r < it.n_rows;
-        const int qpos = DENSE ? it.list_lo + (ok ? r : 0) : __ldg(p.q_idx + it.list_lo + (ok ? r : 0));
+        const int qpos = it.list_lo + (ok ? r : 0);
         const long long G_ = it.head_off + qpos;
         rc[k] = (int)G_;
         gi[k] = ok ? (int)G_ : -1;
         l2[k] = ok ? p.lse[G_] * 1.4426950408889634f : INFINITY;
         dd[k] = ok ? p.Dv[G_] : 0.f;
-        dr[k] = DENSE ? 1 : (ok ? ((p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1) : 0);
       }
       if (n >= 1) mbar_wait(&sm->qdo_empty, (n - 1) & 1, abort_flag, p.status);
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        sm->lse2[4 * lane + k] = l2[k]; sm->Dr[4 * lane + k] = dd[k]; sm->G[4 * lane + k] = gi[k]; sm->direct[4 * lane + k] = dr[k];
+        sm->lse2[4 * lane + k] = l2[k]; sm->Dr[4 * lane + k] = dd[k]; sm->G[4 * lane + k] = gi[k];
       }
       __syncwarp();
       if (lane == 0) mbar_expect_tx(&sm->qdo_full, 2 * TILE);
@@ -517,7 +484,7 @@ dq_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       uint32_t n = 0, f = 0;
       const uint64_t dQ0 = desc_k0(smem_u32(sQ)), dO0 = desc_k0(smem_u32(sdO));
       for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
-        const DqItem it = dq_decode<DENSE>(p, item);
+        const DqItem it = dq_decode(p, item);
         const int acc = n & 1;
         mbar_wait_warp(&sm->qdo_full, n & 1, abort_flag, p.status);
         for (int t = 0; t < it.n_units; ++t, ++f) {
@@ -563,12 +530,11 @@ dq_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
     uint32_t n = 0, f = 0;
     for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
-      const DqItem it = dq_decode<DENSE>(p, item);
+      const DqItem it = dq_decode(p, item);
       const int acc = n & 1;
       mbar_wait(&sm->qdo_full, n & 1, abort_flag, p.status);     // publishes the per-row scalars
       const float lse2 = sm->lse2[r], Dr = sm->Dr[r];
       const int G_ = sm->G[r];
-      const int direct = sm->direct[r];
       for (int t = 0; t < it.n_units; ++t, ++f) {
         const int valid_t = min(BN, it.n_keys - t * BN);
         mbar_wait(&sm->sdp_full, f & 1, abort_flag, p.status);
@@ -606,20 +572,12 @@ dq_long_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         uint32_t a[32];
         tmem_ld32(tmem + lane_addr + DQ_COL + acc * 128 + cgrp * 32, a);
         tmem_ld_wait();
-        if (G_ >= 0) {
-          if (direct) {
-            __nv_bfloat16* dst = p.dq + (long long)G_ * DH + cgrp * 32;
+        if (G_ >= 0) {      // the item holds every key of the row: the result is final
+          __nv_bfloat16* dst = p.dq + (long long)G_ * DH + cgrp * 32;
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              store4(dst + i, make_float4(__uint_as_float(a[i]) * p.scale, __uint_as_float(a[i + 1]) * p.scale,
-                                          __uint_as_float(a[i + 2]) * p.scale, __uint_as_float(a[i + 3]) * p.scale));
-          } else {
-            float* dst = p.dq_acc + (long long)G_ * DH + cgrp * 32;
-#pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              red_add_v4(dst + i, __uint_as_float(a[i]) * p.scale, __uint_as_float(a[i + 1]) * p.scale,
-                         __uint_as_float(a[i + 2]) * p.scale, __uint_as_float(a[i + 3]) * p.scale);
-          }
+          for (int i = 0; i < 32; i += 4)
+            store4(dst + i, make_float4(__uint_as_float(a[i]) * p.scale, __uint_as_float(a[i + 1]) * p.scale,
+                                        __uint_as_float(a[i + 2]) * p.scale, __uint_as_float(a[i + 3]) * p.scale));
         }
       }
       tc_fence_before();
@@ -635,10 +593,9 @@ static int grid_items(long long items) { return (int)std::max<long long>(1, std:
 
 }  // namespace tcl
 
-// dK, dV for long lists (sparse) or the dense path.  q / d_o row gathers need one-row tensor maps.
-int tc_long_dkdv(const Dims& D, bool dense, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
-                 const float* Dv, const int* kb_ptr, const int* q_idx, long long cap, void* dk, void* dv, int32_t* status,
-                 unsigned long long* prof, cudaStream_t st) {
+// dK, dV of the dense path.  The q / d_o rows are fetched as row gathers, which need one-row tensor maps.
+int tc_long_dkdv(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                 const float* Dv, void* dk, void* dv, int32_t* status, unsigned long long* prof, cudaStream_t st) {
   using namespace tcl;
   CUtensorMap tmK, tmV, tmQ, tmO;
   const uint64_t rows = (uint64_t)D.BH * D.S;
@@ -646,26 +603,19 @@ int tc_long_dkdv(const Dims& D, bool dense, const void* q, const void* k, const 
       !sm100::make_tmap_bf16_rows(&tmQ, q, rows, DH, 1) || !sm100::make_tmap_bf16_rows(&tmO, d_o, rows, DH, 1))
     return VMOBA_ERR_CUDA;
   KvParams kp;
-  kp.q = (const __nv_bfloat16*)q; kp.d_o = (const __nv_bfloat16*)d_o; kp.lse = lse; kp.Dv = Dv; kp.kb_ptr = kb_ptr; kp.q_idx = q_idx; kp.S = D.S; kp.BH = D.BH;
-  kp.Nb = dense ? 1 : D.Nb; kp.sb = dense ? D.S : D.sb;
-  kp.scale = D.scale; kp.scale_log2 = D.scale * 1.4426950408889634f; kp.capacity = cap;
+  kp.q = (const __nv_bfloat16*)q; kp.d_o = (const __nv_bfloat16*)d_o; kp.lse = lse; kp.Dv = Dv; kp.S = D.S; kp.BH = D.BH;
+  kp.scale = D.scale; kp.scale_log2 = D.scale * 1.4426950408889634f;
   kp.dk = (__nv_bfloat16*)dk; kp.dv = (__nv_bfloat16*)dv; kp.status = status; kp.prof = prof;
-  // Only the dense instantiation is dispatched: the sparse lists go through the fused kernel.
-  if (!dense) return VMOBA_ERR_ARG;
-  VMOBA_CUDA_OK(cudaFuncSetAttribute(dkdv_long_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KV_SMEM_BYTES));
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(dkdv_long_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)KV_SMEM_BYTES));
   const long long items = (long long)D.BH * ((D.S + BN - 1) / BN);
-  dkdv_long_kernel<true><<<grid_items(items), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, tmQ, tmO, kp);
+  dkdv_long_kernel<<<grid_items(items), KV_THREADS, KV_SMEM_BYTES, st>>>(tmK, tmV, tmQ, tmO, kp);
   VMOBA_LAUNCH_OK(1);
   return VMOBA_OK;
 }
 
-}  // namespace vmoba
-
-namespace vmoba {
-// dQ for long key blocks (sparse) or the dense path.
-int tc_long_dq(const Dims& D, bool dense, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
-               const float* Dv, const int* kb_ptr, const int* q_idx, const int* q_ptr, long long cap, const int* item_ptr,
-               const int* item_tab, float* dq_acc, void* dq, int32_t* status, cudaStream_t st) {
+// dQ of the dense path.
+int tc_long_dq(const Dims& D, const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+               const float* Dv, void* dq, int32_t* status, cudaStream_t st) {
   using namespace tcl;
   CUtensorMap tmK, tmV, tmQ, tmO;
   const uint64_t rows = (uint64_t)D.BH * D.S;
@@ -673,15 +623,14 @@ int tc_long_dq(const Dims& D, bool dense, const void* q, const void* k, const vo
       !sm100::make_tmap_bf16_rows(&tmQ, q, rows, DH, 1) || !sm100::make_tmap_bf16_rows(&tmO, d_o, rows, DH, 1))
     return VMOBA_ERR_CUDA;
   DqParams qp;
-  qp.lse = lse; qp.Dv = Dv; qp.kb_ptr = kb_ptr; qp.q_idx = q_idx; qp.q_ptr = q_ptr; qp.item_ptr = item_ptr; qp.item_tab = item_tab;
-  qp.n_kb = dense ? 0 : D.BH * D.Nb; qp.S = D.S; qp.BH = D.BH; qp.Nb = dense ? 1 : D.Nb; qp.sb = dense ? D.S : D.sb;
-  qp.scale = D.scale; qp.scale_log2 = D.scale * 1.4426950408889634f; qp.capacity = cap;
-  qp.dq_acc = dq_acc; qp.dq = (__nv_bfloat16*)dq; qp.status = status;
-  if (!dense) return VMOBA_ERR_ARG;     // see tc_long_dkdv
-  VMOBA_CUDA_OK(cudaFuncSetAttribute(dq_long_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DQ_SMEM_BYTES));
+  qp.lse = lse; qp.Dv = Dv; qp.S = D.S; qp.BH = D.BH;
+  qp.scale = D.scale; qp.scale_log2 = D.scale * 1.4426950408889634f;
+  qp.dq = (__nv_bfloat16*)dq; qp.status = status;
+  VMOBA_CUDA_OK(cudaFuncSetAttribute(dq_long_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DQ_SMEM_BYTES));
   const long long items = (long long)D.BH * ((D.S + BM - 1) / BM);
-  dq_long_kernel<true><<<grid_items(items), THREADS, DQ_SMEM_BYTES, st>>>(tmK, tmV, tmQ, tmO, qp);
+  dq_long_kernel<<<grid_items(items), THREADS, DQ_SMEM_BYTES, st>>>(tmK, tmV, tmQ, tmO, qp);
   VMOBA_LAUNCH_OK(1);
   return VMOBA_OK;
 }
+
 }  // namespace vmoba

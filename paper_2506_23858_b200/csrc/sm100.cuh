@@ -42,9 +42,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 
 // Bounded wait.  `abort_flag` (shared memory) is set on the first timeout of the CTA; once set,
 // later waits give up after a few polls so that the kernel drains quickly.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  constexpr uint32_t kPolls = 1u << 22;   // each failed poll suspends for up to ~a microsecond in hardware
-  const uint32_t limit = *abort_flag ? 16u : kPolls;
+__device__ __forceinline__ bool mbar_wait_polls(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                                uint32_t polls) {
+  const uint32_t limit = *abort_flag ? 16u : polls;
   for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if (i > 4096) __nanosleep(64);
@@ -52,6 +52,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   *abort_flag = 1;
   set_status(status, VMOBA_ERR_TIMEOUT);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  constexpr uint32_t kPolls = 1u << 22;   // each failed poll suspends for up to ~a microsecond in hardware
+  return mbar_wait_polls(bar, parity, abort_flag, status, kPolls);
 }
 
 // One lane of a converged warp.  A role whose loop runs on all 32 lanes with only the tcgen05.mma /

@@ -360,3 +360,23 @@ def test_paper_training_grids_forward_backward(grid, name):
     base, blocks = (gen.T55, gen.T55_BLOCKS) if grid == "t55k" else (gen.T56, gen.T56_BLOCKS)
     w = base.with_(name=f"{grid}_{name}", block=blocks[name], heads=4)
     _full_size(w, True, [(0, 3)], n_rows=48, n_blocks=1)
+
+
+def test_bounded_wait_runs_out_cleanly_and_the_library_keeps_working():
+    """The device-side failure detector: a wait on a barrier that nothing arrives at gives up after its poll limit,
+    the status word receives VMOBA_ERR_TIMEOUT, the CTA's later waits drain at once and the kernel ends by itself
+    (no trap, no hang); the context stays usable: a forward + backward right afterwards still matches the oracle."""
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.zeros(2, dtype=torch.int32, device="cuda")
+    vb.vmoba_debug_wait_timeout(st, 300, out)
+    torch.cuda.synchronize()
+    assert int(st.item()) == vb.ERR_TIMEOUT
+    assert out.tolist() == [128, 1]            # both waits of all 64 threads gave up; the kernel ran to its end
+    with pytest.raises(vb.VmobaError):
+        vb.vmoba_debug_wait_timeout(st, 0, out)        # host-side argument check
+    w = MID.with_(block=(3, 6, 13), B=1, heads=2)
+    data = gen.make_inputs(w)
+    res = _run_layer(w, data, with_bwd=True)
+    rng = np.random.default_rng(4)
+    for h in range(w.heads):
+        _check_head(w, data, res, 0, h, rng, n_rows=200, n_blocks=2, with_bwd=True)
