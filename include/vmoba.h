@@ -54,7 +54,9 @@ typedef enum {
   VMOBA_ERR_CAPACITY = 4,       /* (dev_status) more selected pairs than the lists can hold         */
   VMOBA_ERR_TIMEOUT = 5,        /* (dev_status) a bounded device-side wait expired                  */
   VMOBA_ERR_CUDA = 6,           /* a CUDA runtime / driver call failed                              */
-  VMOBA_ERR_NOT_IMPLEMENTED = 7 /* combination of dtype / head_dim without a kernel                 */
+  VMOBA_ERR_NOT_IMPLEMENTED = 7,/* combination of dtype / head_dim without a kernel                 */
+  VMOBA_ERR_BOUNDS = 8          /* (dev_status, debug build only) an index read from a work list was out of
+                                   range, or a guard zone between two slices of the workspace was overwritten */
 } vmoba_status;
 
 typedef enum { VMOBA_F32 = 0, VMOBA_BF16 = 1 } vmoba_dtype;

@@ -11,7 +11,7 @@ import os
 
 from . import build as _build
 
-OK, ERR_ARG, ERR_SHAPE, ERR_WORKSPACE, ERR_CAPACITY, ERR_TIMEOUT, ERR_CUDA, ERR_NOT_IMPLEMENTED = range(8)
+OK, ERR_ARG, ERR_SHAPE, ERR_WORKSPACE, ERR_CAPACITY, ERR_TIMEOUT, ERR_CUDA, ERR_NOT_IMPLEMENTED, ERR_BOUNDS = range(9)
 F32, BF16 = 0, 1
 STAGE_SCORES, STAGE_SELECT, STAGE_ATTN_FWD, STAGE_ATTN_BWD, STAGE_FULL_FWD, STAGE_FULL_BWD, STAGE_SELECT_ROWNORM = range(7)
 

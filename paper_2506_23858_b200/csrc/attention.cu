@@ -30,7 +30,7 @@ static bool use_tensor_cores(const Dims& D) { return D.dtype == VMOBA_BF16 && D.
 
 static long long max_items_128(const Dims& D, long long cap) { return cap / 128 + (long long)D.BH * D.Nb + 1; }
 
-struct FwdWs { int* item_ptr; int* item_tab; float* part_o; float* part_lse; size_t bytes; };
+struct FwdWs { int* item_ptr; int* item_tab; float* part_o; float* part_lse; size_t bytes; Guards guards; };
 static FwdWs carve_fwd(const Dims& D, long long cap, void* ws) {
   Carver c(ws);
   FwdWs w;
@@ -39,10 +39,11 @@ static FwdWs carve_fwd(const Dims& D, long long cap, void* ws) {
   w.part_lse = c.take<float>((size_t)cap);
   w.part_o = c.take<float>((size_t)cap * D.d);
   w.bytes = c.total();
+  w.guards = c.guards;
   return w;
 }
 
-struct BwdWs { int* item_ptr; int* item_tab; float* Dv; float* dq_acc; void* o_resid; size_t bytes; };
+struct BwdWs { int* item_ptr; int* item_tab; float* Dv; float* dq_acc; void* o_resid; size_t bytes; Guards guards; };
 static BwdWs carve_bwd(const Dims& D, bool dense, void* ws, long long cap = 0) {
   Carver c(ws);
   BwdWs w;
@@ -52,6 +53,7 @@ static BwdWs carve_bwd(const Dims& D, bool dense, void* ws, long long cap = 0) {
   w.dq_acc = dense ? nullptr : c.take<float>((size_t)D.BH * D.S * D.d);
   w.o_resid = (dense && D.dtype == VMOBA_BF16) ? c.take<__nv_bfloat16>((size_t)D.BH * D.S * D.d) : nullptr;
   w.bytes = c.total();
+  w.guards = c.guards;
   return w;
 }
 
@@ -63,8 +65,9 @@ static int grid_for(long long items, int per_sm) {
 template <typename T, int DH>
 static int simt_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr,
                            const int* q_idx, const int* q_ptr, const int* q_pairs, long long cap, void* o,
-                           void* o_resid, float* lse, void* ws, cudaStream_t st) {
+                           void* o_resid, float* lse, int32_t* status, void* ws, cudaStream_t st) {
   FwdWs w = carve_fwd(D, cap, ws);
+  VMOBA_GUARDS_ARM(w.guards, st);
   const long long n_kb = (long long)D.BH * D.Nb;
   simt::item_ptr_kernel<<<1, 1024, 0, st>>>(kb_ptr, n_kb, simt::kRows, cap, w.item_ptr);
   long long max_items = cap / simt::kRows + n_kb;
@@ -75,6 +78,7 @@ static int simt_sparse_fwd(const Dims& D, const void* q, const void* k, const vo
   simt::merge_kernel<T, DH, float><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(
       q_ptr, q_pairs, nq, w.part_o, w.part_lse, cap, (T*)o, (T*)o_resid, lse);
   VMOBA_LAUNCH_OK(3);
+  VMOBA_GUARDS_CHECK(w.guards, status, st);
   return VMOBA_OK;
 }
 
@@ -86,6 +90,7 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
   // raster-order o / dO / gradients (perm set) are handled by the tensor-core kernels only
   if ((out_map.perm || do_map.perm || o_map.perm) && !use_tensor_cores(D)) return VMOBA_ERR_NOT_IMPLEMENTED;
   BwdWs w = carve_bwd(D, false, ws, cap);
+  VMOBA_GUARDS_ARM(w.guards, st);
   const long long n_kb = (long long)D.BH * D.Nb;
   const long long nq = (long long)D.BH * D.S;
   if (use_tensor_cores(D)) {
@@ -99,6 +104,7 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
     if (rc) return rc;
     simt::cast_rows_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, q_ptr, nq, 1, min_nb, out_map);
     VMOBA_LAUNCH_OK(1);
+    VMOBA_GUARDS_CHECK(w.guards, status, st);
     return VMOBA_OK;
   }
   simt::rowdot_kernel<T, DH><<<grid_for((nq + 7) / 8, 16), 256, 0, st>>>((const T*)o, (const T*)o_resid,
@@ -115,6 +121,7 @@ static int simt_sparse_bwd(const Dims& D, const void* q, const void* k, const vo
       D.Nb, D.sb, D.BH, D.scale, cap, w.dq_acc, (T*)dq);
   simt::cast_kernel<T><<<grid_for((nq * DH / 4 + 255) / 256, 16), 256, 0, st>>>(w.dq_acc, (T*)dq, nq * DH / 4);
   VMOBA_LAUNCH_OK(4);
+  VMOBA_GUARDS_CHECK(w.guards, status, st);
   return VMOBA_OK;
 }
 
@@ -175,6 +182,7 @@ extern "C" const char* vmoba_status_string(int status) {
     case VMOBA_ERR_TIMEOUT: return "device-side wait timed out";
     case VMOBA_ERR_CUDA: return "CUDA error";
     case VMOBA_ERR_NOT_IMPLEMENTED: return "not implemented";
+    case VMOBA_ERR_BOUNDS: return "index out of range or workspace guard overwritten (debug build)";
     default: return "unknown status";
   }
 }
@@ -215,12 +223,14 @@ extern "C" int vmoba_attn_fwd(const vmoba_shape* shape, const void* q_bm, const 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (use_tensor_cores(D)) {
     FwdWs w = carve_fwd(D, capacity, ws);
-    return tc_sparse_fwd(D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null, lse,
-                         dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse, st,
-                         RowMap());
+    VMOBA_GUARDS_ARM(w.guards, st);
+    rc = tc_sparse_fwd(D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null, lse,
+                       dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse, st, RowMap());
+    VMOBA_GUARDS_CHECK(w.guards, dev_status, st);
+    return rc;
   }
   VMOBA_DISPATCH(simt_sparse_fwd, D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null,
-                 lse, ws, st);
+                 lse, dev_status, ws, st);
 }
 
 extern "C" int vmoba_attn_bwd(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
@@ -269,9 +279,12 @@ extern "C" int vmoba_attn_fwd_raster(const vmoba_shape* shape, const void* q_bm,
   o_map.perm = perm; o_map.heads = D.heads; o_map.S = D.S;
   o_map.sb = o_strides_bsh[0]; o_map.st = o_strides_bsh[1]; o_map.sh = o_strides_bsh[2];
   FwdWs w = carve_fwd(D, capacity, ws);
-  return tc_sparse_fwd(D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o, o_resid_bm_or_null, lse,
-                       dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse,
-                       static_cast<cudaStream_t>(stream), o_map);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  VMOBA_GUARDS_ARM(w.guards, st);
+  rc = tc_sparse_fwd(D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o, o_resid_bm_or_null, lse,
+                     dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse, st, o_map);
+  VMOBA_GUARDS_CHECK(w.guards, dev_status, st);
+  return rc;
 }
 
 extern "C" int vmoba_attn_bwd_raster(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,

@@ -139,6 +139,12 @@ __device__ __forceinline__ KvItem kv_decode(const KvParams& p, long long item, i
   it.valid = min(BN, p.sb - tile * BN);
   it.list_lo = min((long long)p.kb_ptr[kbi], p.capacity);
   it.list_hi = min((long long)p.kb_ptr[kbi + 1], p.capacity);
+#ifdef VMOBA_DEBUG
+  if (it.list_lo < 0 || it.list_hi < it.list_lo) {      // offsets must be non-negative and ascending
+    set_status(p.status, VMOBA_ERR_BOUNDS);
+    it.list_lo = it.list_hi = 0;
+  }
+#endif
   it.n_units = (int)((it.list_hi - it.list_lo + QC - 1) / QC);
   it.head_off = (long long)it.bh * p.S;
   return it;
@@ -334,7 +340,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         const int cb = u % NQ;
         const long long lo = it.list_lo + (long long)i * QC;
         const int rows = (int)min((long long)QC, it.list_hi - lo);
-        auto row_of = [&](int r) { return __ldg(p.q_idx + lo + r); };
+        auto row_of = [&](int r) { return checked_index(__ldg(p.q_idx + lo + r), p.S, p.status); };
         int idx[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -414,7 +420,7 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         const int tb = u & 1;
         // accumulator row of query 32 qhalf + lane of the unit (-1 beyond the list)
         const long long lo = it.list_lo + (long long)i * QC + 32 * qhalf;
-        const int row_lane = lo + lane < it.list_hi ? __ldg(p.q_idx + lo + lane) : -1;
+        const int row_lane = lo + lane < it.list_hi ? checked_index(__ldg(p.q_idx + lo + lane), p.S, p.status) : -1;
         long long tw0 = p.prof ? clock64() : 0;
         mbar_wait(&sm->dq_full[tb], (u >> 1) & 1, abort_flag, p.status);
         if (p.prof) { const long long t = clock64(); wp[0] += t - tw0; tw0 = t; }

@@ -89,7 +89,7 @@ __device__ __forceinline__ FwdItem decode_item(const Params& p, int item) {
     const int t = item - it.bh * tiles;
     it.key_begin = 0; it.n_keys = p.S; it.list_lo = t * IM; it.n_rows = min(IM, p.S - it.list_lo);
   } else {
-    const int kbi = __ldg(p.item_tab + item);
+    const int kbi = checked_index(__ldg(p.item_tab + item), p.n_kb, p.status);
     const int chunk = item - __ldg(p.item_ptr + kbi);
     it.bh = kbi / p.Nb;
     const int j = kbi - it.bh * p.Nb;
@@ -346,7 +346,7 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
           const int row = x * BM + (lt >> 4) + 8 * i;
           v[i] = make_uint4(0u, 0u, 0u, 0u);
           if (row < it.n_rows) {
-            const int qp = DENSE ? it.list_lo + row : __ldg(p.q_idx + it.list_lo + row);
+            const int qp = DENSE ? it.list_lo + row : checked_index(__ldg(p.q_idx + it.list_lo + row), p.S, p.status);
             v[i] = __ldg(reinterpret_cast<const uint4*>(qh + (long long)qp * DH) + chunk);
           }
         }
@@ -365,7 +365,7 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
         const int row = x * BM + lt;
         int my_qpos = -1, my_direct = DENSE ? 1 : 0;
         if (row < it.n_rows) {
-          my_qpos = DENSE ? it.list_lo + row : __ldg(p.q_idx + it.list_lo + row);
+          my_qpos = DENSE ? it.list_lo + row : checked_index(__ldg(p.q_idx + it.list_lo + row), p.S, p.status);
           if (!DENSE) {
             const long long G_ = it.head_off + my_qpos;
             my_direct = (p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1;

@@ -101,16 +101,38 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// The debug build (-DVMOBA_DEBUG, lib/libvmoba_debug.so) stands in for a memory checker: every index read from a
+// work list is range-checked before it is used (a violation records VMOBA_ERR_BOUNDS in the status word and the
+// access goes to element 0 instead: no trap, the kernel carries on), and every slice of a workspace is followed by
+// a 256-byte guard zone that is filled with a pattern before the stage's kernels run and verified after them.
+#ifdef VMOBA_DEBUG
+constexpr size_t kGuardBytes = 256;
+#else
+constexpr size_t kGuardBytes = 0;
+#endif
+constexpr uint32_t kGuardWord = 0xC0FFEE5Au;
+struct Guards {
+  char* base = nullptr;
+  size_t off[16] = {};
+  int n = 0;
+};
+
 // Carves 256-byte aligned slices out of a caller-provided workspace.
 struct Carver {
   char* base;
   size_t off = 0;
-  explicit Carver(void* p) : base(static_cast<char*>(p)) {}
+  Guards guards;
+  explicit Carver(void* p) : base(static_cast<char*>(p)) { guards.base = base; }
   template <typename T>
   T* take(size_t n) {
     off = align_up(off, 256);
     T* r = reinterpret_cast<T*>(base ? base + off : nullptr);
     off += n * sizeof(T);
+    if (kGuardBytes) {
+      off = align_up(off, 256);
+      if (guards.n < 16) guards.off[guards.n++] = off;
+      off += kGuardBytes;
+    }
     return r;
   }
   size_t total() const { return align_up(off, 256); }
@@ -141,6 +163,34 @@ inline void count_launches(int n) { g_kernel_launches.fetch_add((unsigned long l
 __device__ __forceinline__ void set_status(int32_t* st, int code) {
   if (st) atomicCAS(st, 0, code);
 }
+
+// An index read from a work list, about to address one of n elements.
+__device__ __forceinline__ int checked_index(int v, int n, int32_t* st) {
+#ifdef VMOBA_DEBUG
+  if ((unsigned)v >= (unsigned)n) {
+    set_status(st, VMOBA_ERR_BOUNDS);
+    return 0;
+  }
+#endif
+  return v;
+}
+
+#ifdef VMOBA_DEBUG
+static __global__ void guard_arm_kernel(Guards g) {
+  reinterpret_cast<uint32_t*>(g.base + g.off[blockIdx.x])[threadIdx.x] = kGuardWord;
+}
+static __global__ void guard_check_kernel(Guards g, int32_t* status) {
+  if (reinterpret_cast<const uint32_t*>(g.base + g.off[blockIdx.x])[threadIdx.x] != kGuardWord)
+    set_status(status, VMOBA_ERR_BOUNDS);
+}
+#define VMOBA_GUARDS_ARM(g, st) \
+  do { if ((g).n && (g).base) guard_arm_kernel<<<(g).n, (int)(kGuardBytes / 4), 0, st>>>(g); } while (0)
+#define VMOBA_GUARDS_CHECK(g, status, st) \
+  do { if ((g).n && (g).base) guard_check_kernel<<<(g).n, (int)(kGuardBytes / 4), 0, st>>>(g, status); } while (0)
+#else
+#define VMOBA_GUARDS_ARM(g, st) do { } while (0)
+#define VMOBA_GUARDS_CHECK(g, status, st) do { } while (0)
+#endif
 
 template <typename T>
 __device__ __forceinline__ float to_f32(T x);

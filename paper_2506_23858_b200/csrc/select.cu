@@ -755,6 +755,7 @@ struct SelectWs {
   int* seg_qoff;
   int* kb_total;
   size_t bytes;
+  Guards guards;
 };
 
 static SelectWs carve_select(const Dims& D, void* ws) {
@@ -773,6 +774,7 @@ static SelectWs carve_select(const Dims& D, void* ws) {
   w.seg_qoff = c.take<int>((size_t)D.BH * nseg + 1);
   w.kb_total = c.take<int>((size_t)D.BH * D.Nb);
   w.bytes = c.total();
+  w.guards = c.guards;
   return w;
 }
 
@@ -823,6 +825,7 @@ static int select_impl(const vmoba_shape* shape, const float* scores, const floa
     sigma = 1.0f;
     range = nullptr;      // the range of the raw scores says nothing about the transformed matrix
   }
+  VMOBA_GUARDS_ARM(w.guards, st);
   const int QSEG = seg_queries(D.mask_words);
   const int nseg = (D.S + QSEG - 1) / QSEG;
   const size_t smem = (size_t)QSEG * D.mask_words * 4 + (size_t)std::max(D.Nb, QSEG) * 4 + (size_t)D.Nb * (QSEG >> 5) * 4;
@@ -899,6 +902,7 @@ static int select_impl(const vmoba_shape* shape, const float* scores, const floa
   fill_kernel<<<sgrid, kSegThreads, smem, st>>>(mask_bits, w.tmask, D.S, D.Nb, D.mask_words, QSEG, nseg, kb_ptr, w.seg_cnt,
                                                 w.seg_qoff, q_idx, q_ptr, q_pairs, capacity);
   VMOBA_LAUNCH_OK(3);
+  VMOBA_GUARDS_CHECK(w.guards, dev_status, st);
   return VMOBA_OK;
 }
 
