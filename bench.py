@@ -581,6 +581,9 @@ def main():
         "attn_tflops": (alg["attn_fwd"][1] + (alg["attn_bwd"][1] if with_bwd else 0.0))
                        / ((stage_ms["attn_fwd"] + stage_ms.get("attn_bwd", 0.0)) * 1e-3) / 1e12,
         "dense_ms": dense_ms,
+        # which build of the library was timed (binding.lib() rebuilds it when a source is newer)
+        "library": {"path": os.path.relpath(vb.lib_path(), ROOT), "mtime": int(os.path.getmtime(vb.lib_path())),
+                    "bytes": os.path.getsize(vb.lib_path())},
     }
     if dense_ms is not None:
         # one dense layer against one sparse layer (the step's time over its layers, every stage included)
