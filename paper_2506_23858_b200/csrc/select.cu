@@ -9,7 +9,8 @@
 // masses), after which the mask is one comparison per pair.  Every kernel streams the score
 // matrix with 16-byte loads; the stage is bound by HBM bandwidth.
 //
-//   minmax  -> hist level 0 -> scan -> hist level 1 -> scan -> hist level 2 -> scan (cutoff)
+//   init (+ minmax, unless the caller hands over each head's score range)
+//           -> hist level 0 -> scan -> hist level 1 -> scan -> hist level 2 -> scan (cutoff)
 //   mark    : mask bits + per (segment, block) counts + per-segment pair totals
 //   offsets : CSR offsets by key block (kb_ptr) and by query (q_ptr)
 //   fill    : q_idx (queries of each key block, ascending) and q_pairs (pairs of each query)
