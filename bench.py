@@ -257,7 +257,9 @@ def main():
     ap.add_argument("--dense", action="store_true",
                     help="also time the dense vmoba_full_attn path on the same inputs (always done for c5)")
     ap.add_argument("--no-dense", action="store_true", help="skip the dense comparison of c5")
-    ap.add_argument("--e2e-steps", type=int, default=6)
+    ap.add_argument("--e2e-steps", type=int, default=0,
+                    help="steps of the end-to-end loop (default: as many as --steps); the first step's input copy and the last\n"
+                         "step's read-back are not overlapped with anything, so a short loop reads slower than a long one")
     ap.add_argument("--rule", default="threshold_global",
                     choices=["threshold_global", "topk_global", "threshold_local", "topk_local"],
                     help="block-choice rule (Table 3b); the paper's training-free runs use topk_local")
@@ -456,6 +458,8 @@ def main():
                 ev_out[i % 2].record(s_out)
         main_s.wait_stream(s_out); main_s.wait_stream(s_in)
 
+    if args.e2e_steps <= 0:
+        args.e2e_steps = args.steps
     e2e_run(2); barrier()
     e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
     e0.record()
