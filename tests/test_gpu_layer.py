@@ -124,6 +124,23 @@ def test_mid_size_layer_forward_backward(block):
             _check_head(w, data, res, b, h, rng, n_rows=400, n_blocks=3, with_bwd=True)
 
 
+@pytest.mark.parametrize("block", [(1, 12, 26), (3, 6, 13)], ids=["1d", "3d"])
+def test_mid_size_layer_unstructured_inputs(block):
+    """Inputs without any locality component: the selection pattern is unstructured and a large share of the
+    queries own several pairs (about 1.4 per query with 6 blocks, 11 with 48), so most output rows go through the
+    partial rows and the merge instead of being written directly by the forward kernel."""
+    w = MID.with_(block=block, recipe="white", heads=2, B=1)
+    data = gen.make_inputs(w)
+    res = _run_layer(w, data, with_bwd=True, capacity=w.S * w.n_blocks)
+    L = res["L"]
+    q_ptr = L.q_ptr.cpu().numpy().astype(np.int64)
+    per_query = np.diff(q_ptr.reshape(-1))[: w.S]
+    assert (per_query >= 2).mean() > 0.3, "the recipe is meant to give a large share of the queries several pairs"
+    rng = np.random.default_rng(3)
+    for h in range(w.heads):
+        _check_head(w, data, res, 0, h, rng, n_rows=400, n_blocks=3, with_bwd=True)
+
+
 @pytest.mark.parametrize("grid,block", [((6, 9, 20), (3, 9, 10)), ((4, 43, 3), (1, 43, 3)), ((2, 16, 32), (1, 16, 16))],
                          ids=["270keys_tail14", "129keys_tail1", "256keys_no_tail"])
 def test_key_block_tails_forward_backward(grid, block):
