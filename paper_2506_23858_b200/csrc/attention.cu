@@ -35,7 +35,7 @@ static FwdWs carve_fwd(const Dims& D, long long cap, void* ws) {
   Carver c(ws);
   FwdWs w;
   w.item_ptr = c.take<int>((size_t)D.BH * D.Nb + 1);
-  w.item_tab = c.take<int>((size_t)max_items_128(D, cap));
+  w.item_tab = c.take<int>(4 * (size_t)max_items_128(D, cap));   // one int per item, or a 16-byte descriptor
   w.part_lse = c.take<float>((size_t)cap);
   w.part_o = c.take<float>((size_t)cap * D.d);
   w.bytes = c.total();

@@ -277,6 +277,127 @@ merge_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pairs, lon
   }
 }
 
+// The same merge for head_dim 128 and fp32 partials, 32 consecutive queries per warp and trip.  With one
+// query per warp the four dependent loads of a query (list bounds, pair positions, partial lse, rows) are
+// paid one after the other for every query; here lane l reads the bounds, the first kInLane pair positions
+// and their lse of query g0 + l, works out the weights on its own, and the warp then walks the queries that
+// need a row written, fetching all rows of a query at once.  Queries with more pairs than a lane keeps take
+// the warp-wide loop of merge_kernel.
+constexpr int kInLane = 8;
+template <typename T>
+__global__ void __launch_bounds__(256)
+merge_batched_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pairs, long long n_queries,
+                     const float* __restrict__ part_o, const float* __restrict__ part_lse, long long capacity,
+                     T* __restrict__ o, T* __restrict__ o_resid, float* __restrict__ lse, const RowMap o_map = RowMap()) {
+  constexpr int DH = 128;
+  const int lane = threadIdx.x & 31;
+  const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
+  const int last = (int)(capacity - 1);
+  for (long long g0 = warp * 32; g0 < n_queries; g0 += nwarps * 32) {
+    const long long g = g0 + lane;
+    int lo = 0, n = 1, n_raw = 1;        // lanes beyond the last query behave like a directly written row
+    if (g < n_queries) {
+      lo = q_ptr[g];
+      const int hi_raw = q_ptr[g + 1];
+      n_raw = hi_raw - lo;
+      n = (int)(min((long long)hi_raw, capacity) - lo);
+      if (n < 0) n = 0;
+    }
+    const bool direct = n == 1 && n_raw == 1;
+    int pos[kInLane];
+    float w[kInLane];
+    float out_lse = -INFINITY;
+    if (!direct && n > 0 && n <= kInLane) {
+      float mx = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < kInLane; ++k) {
+        pos[k] = 0; w[k] = -INFINITY;
+        if (k < n) pos[k] = min(max(q_pairs[lo + k], 0), last);
+      }
+#pragma unroll
+      for (int k = 0; k < kInLane; ++k)
+        if (k < n) { w[k] = part_lse[pos[k]]; mx = fmaxf(mx, w[k]); }
+      float tot = 0.f;
+#pragma unroll
+      for (int k = 0; k < kInLane; ++k) {
+        w[k] = k < n ? expf(w[k] - mx) : 0.f;
+        tot += w[k];
+      }
+      const float inv = 1.0f / tot;
+#pragma unroll
+      for (int k = 0; k < kInLane; ++k) w[k] *= inv;
+      out_lse = mx + logf(tot);
+    } else {
+#pragma unroll
+      for (int k = 0; k < kInLane; ++k) { pos[k] = 0; w[k] = 0.f; }
+    }
+    uint32_t todo = __ballot_sync(0xffffffffu, !direct);
+    while (todo) {
+      const int b = __ffs(todo) - 1;
+      todo &= todo - 1;
+      const long long gq = g0 + b;
+      const int nb = __shfl_sync(0xffffffffu, n, b);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      float row_lse = __shfl_sync(0xffffffffu, out_lse, b);
+      if (nb <= kInLane) {
+        float4 v[kInLane];
+        float wk[kInLane];
+#pragma unroll
+        for (int k = 0; k < kInLane; ++k) {
+          const int pk = __shfl_sync(0xffffffffu, pos[k], b);
+          wk[k] = __shfl_sync(0xffffffffu, w[k], b);
+          v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (k < nb) v[k] = *reinterpret_cast<const float4*>(part_o + (long long)pk * DH + lane * 4);
+        }
+#pragma unroll
+        for (int k = 0; k < kInLane; ++k) {
+          acc.x = fmaf(wk[k], v[k].x, acc.x); acc.y = fmaf(wk[k], v[k].y, acc.y);
+          acc.z = fmaf(wk[k], v[k].z, acc.z); acc.w = fmaf(wk[k], v[k].w, acc.w);
+        }
+      } else {
+        // many pairs: lane i of each group of 32 pairs fetches position and lse of pair i, the weights travel by shuffle
+        const long long qlo = __shfl_sync(0xffffffffu, lo, b), qhi = qlo + nb;
+        float mx = -INFINITY;
+        for (long long i0 = qlo; i0 < qhi; i0 += 32) {
+          const long long i = i0 + lane;
+          mx = fmaxf(mx, i < qhi ? part_lse[min(max(q_pairs[i], 0), last)] : -INFINITY);
+        }
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, s));
+        float tot = 0.f;
+        for (long long i0 = qlo; i0 < qhi; i0 += 32) {
+          const long long i = i0 + lane;
+          int my_pos = 0;
+          float my_w = 0.f;
+          if (i < qhi) {
+            my_pos = min(max(q_pairs[i], 0), last);
+            my_w = expf(part_lse[my_pos] - mx);
+          }
+          tot += my_w;
+          const int m = (int)min((long long)32, qhi - i0);
+#pragma unroll 4
+          for (int k = 0; k < m; ++k) {
+            const long long pk = __shfl_sync(0xffffffffu, my_pos, k);
+            const float wgt = __shfl_sync(0xffffffffu, my_w, k);
+            const float4 v = *reinterpret_cast<const float4*>(part_o + pk * DH + lane * 4);
+            acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
+            acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
+          }
+        }
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, s);
+        const float inv = 1.0f / tot;
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        row_lse = mx + logf(tot);
+      }
+      T* o_row = o + o_map.off(gq, DH);
+      store4_resid(o_row + lane * 4, o_resid ? o_resid + gq * DH + lane * 4 : nullptr, acc);
+      if (lane == 0) lse[gq] = row_lse;
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------ backward
 // D = rowsum(dO * O), one warp per query; o and dO block-major or in raster order through their maps, the
 // rounding residual of o always block-major.  If zero_acc is given, the fp32 dQ accumulator rows of the queries

@@ -521,13 +521,22 @@ static int grid_items(long long items) { return (int)std::max<long long>(1, std:
 
 }  // namespace tcw
 
-// Forward over the work lists (bf16, head_dim 128).  Returns VMOBA_ERR_CUDA if the tensor maps or
-// the launch fail.
+int tc_sparse_fwd_narrow(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
+                         const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
+                         int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o,
+                         float* part_lse, cudaStream_t st, const RowMap& o_map);   // attn_tc_fwd_narrow.cu
+
+// Forward over the work lists (bf16, head_dim 128).  Key blocks of up to four 128-key tiles go to the kernel for
+// short items (two CTAs of one query tile per SM), longer ones to the wide kernel of this file.  Returns
+// VMOBA_ERR_CUDA if the tensor maps or the launch fail.
 int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                        const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
                        int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o,
                        float* part_lse, cudaStream_t st, const RowMap& o_map) {
   using namespace tcw;
+  if (D.sb <= 4 * BN)
+    return tc_sparse_fwd_narrow(D, q, k, v, kb_ptr, q_idx, q_ptr, q_pairs, cap, o, o_resid, lse, status, item_ptr, item_tab,
+                                max_items, part_o, part_lse, st, o_map);
   CUtensorMap tmK, tmV;
   const uint64_t rows = (uint64_t)D.BH * D.S;
   if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN))
@@ -555,7 +564,7 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
     attn_fwd_wide_kernel<false><<<grid_items(cap / IM + n_kb), THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
   }
   const long long nq = (long long)D.BH * D.S;
-  simt::merge_kernel<__nv_bfloat16, 128, float><<<(int)std::min<long long>((nq + 7) / 8, sm_count() * 16), 256, 0, st>>>(
+  simt::merge_batched_kernel<__nv_bfloat16><<<(int)std::min<long long>((nq + 255) / 256, sm_count() * 8), 256, 0, st>>>(
       q_ptr, q_pairs, nq, part_o, part_lse, cap, (__nv_bfloat16*)o, (__nv_bfloat16*)o_resid, lse, o_map);
   VMOBA_LAUNCH_OK(4);
   return VMOBA_OK;

@@ -230,11 +230,16 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, float4 v) {
 // Store 4 values and, for bf16 with a residual buffer, the rounding residual bf16(v - bf16(v)).
 __device__ __forceinline__ void store4_resid(float* p, float* /*resid*/, float4 v) { store4(p, v); }
 __device__ __forceinline__ void store4_resid(__nv_bfloat16* p, __nv_bfloat16* resid, float4 v) {
-  store4(p, v);
-  if (resid) {
-    float4 h = load4(p);
-    store4(resid, make_float4(v.x - h.x, v.y - h.y, v.z - h.z, v.w - h.w));
-  }
+  // the rounded values are rebuilt from the packed words in registers (no read-back of the row just stored)
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y);
+  __nv_bfloat162 b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<uint32_t*>(&a);
+  u.y = *reinterpret_cast<uint32_t*>(&b);
+  *reinterpret_cast<uint2*>(p) = u;
+  if (resid)
+    store4(resid, make_float4(v.x - __uint_as_float(u.x << 16), v.y - __uint_as_float(u.x & 0xffff0000u),
+                              v.z - __uint_as_float(u.y << 16), v.w - __uint_as_float(u.y & 0xffff0000u)));
 }
 
 // Atomic minimum / maximum of fp32 values in global memory (the integer order of the bit patterns agrees with
