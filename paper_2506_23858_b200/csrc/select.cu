@@ -11,6 +11,8 @@
 //
 //   init (+ minmax, unless the caller hands over each head's score range)
 //           -> hist level 0 -> scan -> hist level 1 -> scan -> hist level 2 -> scan (cutoff)
+//   (level 1 copies the pairs of the level-0 crossing bin aside, and level 2 reads that short list instead of the
+//    score matrix: three traversals of the matrix, levels 0 and 1 and mark)
 //   mark    : mask bits + per (segment, block) counts + per-segment pair totals
 //   offsets : CSR offsets by key block (kb_ptr) and by query (q_ptr)
 //   fill    : q_idx (queries of each key block, ascending) and q_pairs (pairs of each query)
@@ -36,7 +38,9 @@ struct HeadState {
   double mass_above;           // weight of everything above the crossing bin so far
   unsigned long long cnt_above;
   uint32_t cutoff_key;
-  uint32_t pad;
+  unsigned int cand_cnt;       // pairs of the level-0 crossing bin, copied aside by the level-1 pass
+  int cand_ok;                 // every one of them found room in the list: level 2 reads the list
+  uint32_t pad[2];
 };
 
 // bin of a score at refinement level L given the state; monotone non-decreasing in s.
@@ -129,7 +133,7 @@ template <int L>
 __global__ void __launch_bounds__(256)
 hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __restrict__ st, float sigma, int unit_w,
             unsigned int* __restrict__ g_cnt, double* __restrict__ g_w, uint32_t* __restrict__ g_minkey,
-            uint32_t* __restrict__ g_maxkey) {
+            uint32_t* __restrict__ g_maxkey, float* __restrict__ cand, long long ccap, unsigned int* __restrict__ cand_cnt) {
   __shared__ unsigned int s_cnt[kBins];
   __shared__ float s_w[kBins];
   __shared__ uint32_t s_min[kBins];
@@ -144,8 +148,18 @@ hist_kernel(const float* __restrict__ scores, long long P, const HeadState* __re
   }
   __syncthreads();
   const float smax = key_float(hs.max_key);
-  for_each_score(scores + (long long)bh * P, P, [&](float s) {
+  // level 1 copies the pairs of the level-0 crossing bin (one bin of 512: few) to the head's list; level 2 reads
+  // the list instead of the matrix if all of them found room
+  float* list = cand ? cand + (long long)bh * ccap : nullptr;
+  const bool from_list = L == 2 && hs.cand_ok;
+  const float* src = from_list ? list : scores + (long long)bh * P;
+  const long long n_src = from_list ? (long long)hs.cand_cnt : P;
+  for_each_score(src, n_src, [&](float s) {
     if (L >= 1 && bin_at(hs, 0, s) != hs.bin[0]) return;
+    if (L == 1 && list) {
+      const unsigned int pos = atomicAdd(cand_cnt + bh * (sizeof(HeadState) / sizeof(unsigned int)), 1u);
+      if (pos < ccap) list[pos] = s;
+    }
     if (L >= 2 && bin_at(hs, 1, s) != hs.bin[1]) return;
     int b = bin_at(hs, L, s);
     atomicAdd(&s_cnt[b], 1u);
@@ -199,7 +213,7 @@ __global__ void __launch_bounds__(1024)
 scan_kernel(HeadState* __restrict__ st, float tau, double count_target, unsigned int* __restrict__ g_cnt,
             double* __restrict__ g_w,
             uint32_t* __restrict__ g_minkey, uint32_t* __restrict__ g_maxkey, int64_t* __restrict__ k_per_head,
-            float* __restrict__ cutoff_per_head) {
+            float* __restrict__ cutoff_per_head, long long ccap) {
   __shared__ double s_wsum[32];
   __shared__ unsigned long long s_csum[32];
   __shared__ int s_cross;
@@ -289,6 +303,8 @@ scan_kernel(HeadState* __restrict__ st, float tau, double count_target, unsigned
   __syncthreads();
   if (t == 0) {
     hs.bin[L] = cross_bin;
+    // level 2 may read the list if level 1 copied the level-0 crossing bin to it in full
+    if (L == 1) hs.cand_ok = (long long)hs.cand_cnt <= ccap ? 1 : 0;
     hs.mass_above += s_above_w;
     hs.cnt_above += s_above_c;
     if (L < 2) {
@@ -408,11 +424,15 @@ __global__ void seg_prefix_kernel(int* __restrict__ seg_cnt, int* __restrict__ k
   if (i >= (long long)BH * Nb) return;
   int bh = (int)(i / Nb), j = (int)(i % Nb);
   int run = 0;
-  for (int s = 0; s < nseg; ++s) {
-    int* p = seg_cnt + ((long long)bh * nseg + s) * Nb + j;
-    int c = *p;
-    *p = run;
-    run += c;
+  // eight segments per trip: their loads go out together (the stores of a trip would otherwise order them)
+  for (int s0 = 0; s0 < nseg; s0 += 8) {
+    int* p = seg_cnt + ((long long)bh * nseg + s0) * Nb + j;
+    int c[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) c[k] = s0 + k < nseg ? p[(long long)k * Nb] : 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (s0 + k < nseg) { p[(long long)k * Nb] = run; run += c[k]; }
   }
   kb_total[i] = run;
 }
@@ -755,9 +775,18 @@ struct SelectWs {
   int* seg_total;
   int* seg_qoff;
   int* kb_total;
+  float* cand;          // [BH][ccap] scores copied aside by the level-0 pass (optional: the last slice)
+  long long ccap;
+  size_t base_bytes;    // without the candidate lists
   size_t bytes;
   Guards guards;
 };
+
+// Room for the list of one head: the pairs of one of the 512 level-0 bins.
+static long long cand_capacity(const Dims& D) {
+  const long long P = (long long)D.S * D.Nb;
+  return std::max<long long>(4096, ((P / 32 + 3) / 4) * 4);
+}
 
 static SelectWs carve_select(const Dims& D, void* ws) {
   SelectWs w;
@@ -774,12 +803,17 @@ static SelectWs carve_select(const Dims& D, void* ws) {
   w.seg_total = c.take<int>((size_t)D.BH * nseg);
   w.seg_qoff = c.take<int>((size_t)D.BH * nseg + 1);
   w.kb_total = c.take<int>((size_t)D.BH * D.Nb);
+  w.base_bytes = c.total();
+  w.ccap = cand_capacity(D);
+  w.cand = c.take<float>((size_t)D.BH * w.ccap);
   w.bytes = c.total();
   w.guards = c.guards;
   return w;
 }
 
 size_t select_ws_bytes(const Dims& D) { return carve_select(D, nullptr).bytes; }
+// the least the selection can work with (no candidate lists: levels 1 and 2 read the score matrix)
+size_t select_base_ws_bytes(const Dims& D) { return carve_select(D, nullptr).base_bytes; }
 // the row-normalised rule also keeps a transformed copy of the score matrix behind the common scratch
 size_t select_rownorm_ws_bytes(const Dims& D) {
   return ((carve_select(D, nullptr).bytes + 255) / 256) * 256 + (size_t)D.BH * D.S * D.Nb * sizeof(float);
@@ -792,7 +826,7 @@ using namespace vmoba;
 static int select_impl(const vmoba_shape* shape, const float* scores, const float* range, int rule, float tau, int topk, uint32_t* mask_bits,
                        int32_t* kb_ptr, int32_t* q_idx, int32_t* q_ptr, int32_t* q_pairs, int64_t capacity,
                        int64_t* k_per_head, float* cutoff_per_head, int32_t* dev_status, void* ws, size_t ws_bytes,
-                       void* stream) {
+                       void* stream, bool allow_base_ws = false) {
   Dims D;
   int rc = make_dims(shape, &D);
   if (rc) return rc;
@@ -812,7 +846,10 @@ static int select_impl(const vmoba_shape* shape, const float* scores, const floa
   if (capacity <= 0 || capacity > (int64_t)INT32_MAX) return VMOBA_ERR_ARG;
   if (D.Nb > 8192 || (local && D.Nb > 32 * kLocalMaxWords)) return VMOBA_ERR_SHAPE;
   SelectWs w = carve_select(D, ws);
-  if (ws_bytes < (rownorm ? select_rownorm_ws_bytes(D) : w.bytes)) return VMOBA_ERR_WORKSPACE;
+  if (ws_bytes < (rownorm ? select_rownorm_ws_bytes(D) : (allow_base_ws ? w.base_bytes : w.bytes))) return VMOBA_ERR_WORKSPACE;
+  // the candidate lists are the last slice: a caller with a fixed scratch area may have no room for them
+  const bool use_cand = ws_bytes >= w.bytes;
+  if (!use_cand) { w.cand = nullptr; w.ccap = -1; if (w.guards.n > 0) w.guards.n -= 1; }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const long long P = (long long)D.S * D.Nb;
   float sigma = D.scale;
@@ -881,13 +918,15 @@ static int select_impl(const vmoba_shape* shape, const float* scores, const floa
       hist0_kernel<<<dim3(gx0, D.BH), 512, smem0, st>>>(scores, P, w.state, sigma, unit_w, w.g_w);
     }
     scan_kernel<0><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,
-                                         cutoff_per_head);
-    hist_kernel<1><<<grid, 256, 0, st>>>(scores, P, w.state, sigma, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
+                                         cutoff_per_head, w.ccap);
+    hist_kernel<1><<<grid, 256, 0, st>>>(scores, P, w.state, sigma, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, w.cand,
+                                        w.ccap, &w.state->cand_cnt);
     scan_kernel<1><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,
-                                         cutoff_per_head);
-    hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, sigma, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey);
+                                         cutoff_per_head, w.ccap);
+    hist_kernel<2><<<grid, 256, 0, st>>>(scores, P, w.state, sigma, unit_w, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, w.cand,
+                                        w.ccap, &w.state->cand_cnt);
     scan_kernel<2><<<D.BH, 1024, 0, st>>>(w.state, tau, count_target, w.g_cnt, w.g_w, w.g_minkey, w.g_maxkey, k_per_head,
-                                         cutoff_per_head);
+                                         cutoff_per_head, w.ccap);
     VMOBA_LAUNCH_OK(7);
     VMOBA_CUDA_OK(cudaFuncSetAttribute(mark_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     mark_kernel<<<sgrid, kSegThreads, smem, st>>>(scores, w.state, D.S, D.Nb, D.mask_words, QSEG, nseg, own_sb, mask_bits,
@@ -960,7 +999,7 @@ extern "C" int vmoba_select_static(const vmoba_shape* shape, const float* scores
   if (rc) return rc;
   if (D.Nb > 8192) return VMOBA_ERR_SHAPE;
   // The shape's scratch need must fit the fixed array; larger problems have to use vmoba_select.
-  if (select_ws_bytes(D) > kStaticSelectScratchBytes) return VMOBA_ERR_WORKSPACE;
+  if (select_base_ws_bytes(D) > kStaticSelectScratchBytes) return VMOBA_ERR_WORKSPACE;
   int dev = -1;
   VMOBA_CUDA_OK(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kMaxDevices) return VMOBA_ERR_CUDA;
@@ -976,6 +1015,7 @@ extern "C" int vmoba_select_static(const vmoba_shape* shape, const float* scores
   }
   // vmoba_select clears everything in its scratch that has to start at zero, so the contents
   // left by an earlier call do not matter.
-  return vmoba_select(shape, scores, tau, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs, capacity, k_per_head,
-                      cutoff_per_head, dev_status, g_select_scratch_addr[dev], kStaticSelectScratchBytes, stream);
+  return select_impl(shape, scores, nullptr, VMOBA_SELECT_THRESHOLD_GLOBAL, tau, 0, mask_bits, kb_ptr, q_idx, q_ptr, q_pairs,
+                     capacity, k_per_head, cutoff_per_head, dev_status, g_select_scratch_addr[dev], kStaticSelectScratchBytes,
+                     stream, /*allow_base_ws=*/true);
 }

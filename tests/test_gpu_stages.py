@@ -155,6 +155,32 @@ def test_select_matches_oracle_outside_the_cutoff_band(w):
     assert got.all()          # tau = 1 selects every pair
 
 
+def test_select_when_the_crossing_bin_does_not_fit_the_side_list():
+    """Level 1 of the cutoff search copies the pairs of the level-0 crossing bin to a short list that level 2 reads
+    instead of the matrix.  Here nearly all pairs fall into that one bin (a tight cluster between two far outliers),
+    far more than the list holds, so level 2 has to go back to the matrix: same answer as the oracle."""
+    w = gen.Workload("sel_cluster", 1, 1, 64, 8, 32, 32, (1, 8, 32), 0.25, "bf16", "smooth", 3)
+    rng = np.random.default_rng(11)
+    sc = (rng.standard_normal((w.S, w.n_blocks)) * 1e-3).astype(np.float32)
+    sc[0, 0], sc[1, 1] = 12.0, -12.0           # stretch the range: one level-0 bin is 0.047 wide
+    sc[5, 3], sc[7, 9] = 0.5, 0.25
+    L = VmobaLayer(vb.shape_of(w), capacity=w.S * w.n_blocks)
+    L.scores.copy_(torch.from_numpy(sc.reshape(1, 1, w.S, w.n_blocks)))
+    scale = w.head_dim ** -0.5
+    for tau in (0.25, 0.6):
+        L.dev_status.zero_()
+        L.select(tau)
+        L.check_status()
+        got = U.unpack_mask(L.mask_bits, 1, w.S, w.n_blocks)[0]
+        m_ref, k_ref, c_ref = orc.select(sc, tau, scale)
+        cut = float(L.cutoff.cpu().numpy()[0])
+        decided = np.abs(sc - c_ref) > 1e-5       # the cluster is 1e-3 wide: compare much closer than the usual band
+        assert np.array_equal(got[decided], m_ref[decided]), tau
+        assert abs(cut - float(c_ref)) <= 1e-5
+        assert abs(int(L.k_per_head.cpu().numpy()[0]) - k_ref) <= 64
+        assert np.all(sc[got] >= cut) and np.all(sc[~got] < cut)
+
+
 def test_select_reports_capacity_overflow():
     w = MID
     data, ora = _prep(w)
