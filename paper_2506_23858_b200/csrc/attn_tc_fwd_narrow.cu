@@ -1,5 +1,5 @@
-// Tensor-core attention forward for SHORT key blocks (bf16, head_dim 128; Step 3 of VMoBA): key blocks of a few
-// 128-key tiles, where a work item is over after two or three tiles.
+// Tensor-core attention forward for short and medium key blocks (bf16, head_dim 128; Step 3 of VMoBA): written for
+// key blocks of a few 128-key tiles, where a work item is over after two or three tiles, and used up to thirteen.
 //
 // The wide kernel (attn_tc_fwd.cu) keeps the tensor pipe busy by running two query tiles of one item in opposite
 // phase; that phase needs many key tiles to establish itself.  On a 270-key block both tiles run their softmax at
@@ -486,7 +486,7 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 
 }  // namespace tcn
 
-// Forward over the work lists for key blocks of up to four 128-key tiles (bf16, head_dim 128).
+// Forward over the work lists with one 128-row query tile per item (bf16, head_dim 128).
 // item_tab must hold four ints per item.  Returns VMOBA_ERR_CUDA if the tensor maps or the launch fail.
 int tc_sparse_fwd_narrow(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                          const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
