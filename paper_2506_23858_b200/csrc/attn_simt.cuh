@@ -417,14 +417,23 @@ rowdot_kernel(const T* __restrict__ o, const T* __restrict__ o_resid, const T* _
     constexpr int R = 4;
     for (long long g0 = warp * R; g0 < n_queries; g0 += nwarps * R) {
       uint2 ov[R], rv[R], dv[R];
-      bool zero[R];
+      bool zero[R], used[R];
+      // with the lists at hand, a query without a selected block is skipped: nothing reads its D
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         const long long g = min(g0 + r, n_queries - 1);
-        ov[r] = *reinterpret_cast<const uint2*>(o + o_map.off(g, DH) + lane * 4);
-        dv[r] = *reinterpret_cast<const uint2*>(d_o + do_map.off(g, DH) + lane * 4);
-        rv[r] = o_resid ? *reinterpret_cast<const uint2*>(o_resid + g * DH + lane * 4) : make_uint2(0u, 0u);
-        zero[r] = zero_acc && g0 + r < n_queries && __ldg(q_ptr + g + 1) - __ldg(q_ptr + g) >= 1;
+        used[r] = !q_ptr || __ldg(q_ptr + g + 1) - __ldg(q_ptr + g) >= 1;
+        zero[r] = zero_acc && q_ptr && g0 + r < n_queries && used[r];
+      }
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const long long g = min(g0 + r, n_queries - 1);
+        ov[r] = dv[r] = rv[r] = make_uint2(0u, 0u);
+        if (used[r]) {
+          ov[r] = *reinterpret_cast<const uint2*>(o + o_map.off(g, DH) + lane * 4);
+          dv[r] = *reinterpret_cast<const uint2*>(d_o + do_map.off(g, DH) + lane * 4);
+          if (o_resid) rv[r] = *reinterpret_cast<const uint2*>(o_resid + g * DH + lane * 4);
+        }
       }
       float a[R];
 #pragma unroll
