@@ -206,8 +206,12 @@ int vmoba_select_ranged(const vmoba_shape* shape, const float* scores, const flo
  * Same arguments and results as vmoba_select minus `ws`: the scratch is a fixed
  * vmoba_select_static_scratch_bytes() = 16 MiB array inside the library image, which every GPU
  * that loads the library keeps resident until the process exits.
- *   - Shapes whose vmoba_workspace_bytes(shape, VMOBA_STAGE_SELECT, 0) exceeds that size are
- *     rejected with VMOBA_ERR_WORKSPACE; use vmoba_select with your own buffer for those.
+ *   - Shapes whose vmoba_workspace_bytes(shape, VMOBA_STAGE_SELECT, 0) fits that size run exactly
+ *     as vmoba_select does.  The last slice of that workspace is an optional side list (the larger of
+ *     4096 and S * N_b / 32 floats per (batch, head)) that saves the cutoff search one pass over the
+ *     scores; a shape that fits only without it still runs, one pass slower, with the same results.
+ *     Shapes that do not fit even so are rejected with VMOBA_ERR_WORKSPACE; use vmoba_select with
+ *     your own buffer for those.
  *   - The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
  *   - The first call on each device looks up the array's device address (one
  *     cudaGetSymbolAddress, with that device current); make that first call outside of any stream

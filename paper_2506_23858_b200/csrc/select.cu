@@ -40,7 +40,8 @@ struct HeadState {
   uint32_t cutoff_key;
   unsigned int cand_cnt;       // pairs of the level-0 crossing bin, copied aside by the level-1 pass
   int cand_ok;                 // every one of them found room in the list: level 2 reads the list
-  uint32_t pad[2];
+  float bin0_off;              // -anchor[0] * inv[0]: the level-0 bin of s is floor(s * inv[0] + bin0_off)
+  uint32_t pad;
 };
 
 // bin of a score at refinement level L given the state; monotone non-decreasing in s.
@@ -48,11 +49,22 @@ struct HeadState {
 // in descending score order).  One definition for every histogram level and for the final exact
 // steps, so that the masses they hand to each other are sums of the same numbers; the fast
 // exponential (one multiply, one ex2) is within a few ulp of expf over the range that carries mass.
-__device__ __forceinline__ float pair_weight(float sigma, float s, float smax) { return __expf(sigma * (s - smax)); }
+// One fused multiply-add and one ex2 per pair: exp(sigma (s - smax)) = 2^(s c - smax c) with c = sigma log2(e);
+// c and smax c do not depend on the pair and leave the loops.
+__device__ __forceinline__ float pair_weight(float sigma, float s, float smax) {
+  const float c = sigma * 1.4426950408889634f;
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(fmaf(s, c, -smax * c)));
+  return y;
+}
 
+// Level 0 sees every pair: its bin is one fused multiply-add (bin0_off = -anchor[0] * inv[0], a number of bins, so
+// its rounding moves a bin edge by a few millionths of a bin) and an integer clamp.  The finer levels keep the
+// subtraction first: their inv is so large that the product form would cancel.
 __device__ __forceinline__ int bin_at(const HeadState& hs, int L, float s) {
+  if (L == 0) return min(max(__float2int_rd(fmaf(s, hs.inv[0], hs.bin0_off)), 0), kBins0 - 1);
   float t = (s - hs.anchor[L]) * hs.inv[L];
-  int b = t > 0.f ? (int)fminf(t, (float)((L == 0 ? kBins0 : kBins) - 1)) : 0;
+  int b = t > 0.f ? (int)fminf(t, (float)(kBins - 1)) : 0;
   return b;
 }
 
@@ -121,6 +133,7 @@ __global__ void init_state_kernel(HeadState* st, int BH, const float* __restrict
     const float span = hi - lo;
     h.anchor[0] = lo;
     h.inv[0] = span > 0.f ? (float)kBins0 / span : 0.f;
+    h.bin0_off = -lo * h.inv[0];
   }
   st[i] = h;
 }
@@ -334,6 +347,7 @@ __global__ void setup_level0_kernel(HeadState* st, int BH) {
   float range = hi - lo;
   st[i].anchor[0] = lo;
   st[i].inv[0] = range > 0.f ? (float)kBins0 / range : 0.f;
+  st[i].bin0_off = -lo * st[i].inv[0];
 }
 
 // mark: a CTA takes a segment of QSEG consecutive queries of one head (a contiguous run of
