@@ -328,6 +328,18 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
           const long long G_ = it.head_off + qp;
           info[half] = 2 * qp + ((p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1 ? 1 : 0);
         }
+        // the second half's rows are fetched only after the first half has been stored: ask the L2 for them now
+        // (one request per 128-byte line)
+        if (half == 0 && (chunk & 7) == 0) {
+#pragma unroll 4
+          for (int i = 0; i < 16; ++i) {
+            const int row = 64 + (lt >> 4) + 4 * i;
+            if (row < it.n_rows) {
+              const int qp = checked_index(__ldg(p.q_idx + it.list_lo + row), p.S, p.status);
+              asm volatile("prefetch.global.L2 [%0];" ::"l"(qh + (long long)qp * DH + chunk * 8));
+            }
+          }
+        }
         // the Q tile is free once the previous item's last Q K^T has run
         if (half == 0 && n >= 1) mbar_wait(&sm->q_empty, (n - 1) & 1, abort_flag, p.status);
 #pragma unroll
