@@ -239,6 +239,49 @@ def test_sparse_attention_forward_backward(w):
         U.assert_close(dv[i], r["dv"], w.dtype, f"dv head {i}")
 
 
+@pytest.mark.parametrize("block", [(1, 4, 16), (1, 5, 13), (1, 8, 16), (1, 10, 13), (2, 12, 8)],
+                         ids=["64keys", "65keys", "128keys", "130keys", "192keys"])
+def test_sparse_attention_item_and_tile_edges(block):
+    """Hand-built lists whose lengths sit on the work-item edges of the tensor-core kernels (0, 1, 63, 64, 65, 127,
+    128, 129, 255, 256, 257 and 300 queries per key block) against key blocks whose tail tile is full, one key
+    long, or absent: forward and backward against the oracle, empty queries zero-filled."""
+    grid = {(1, 4, 16): (6, 8, 16), (1, 5, 13): (6, 10, 13), (1, 8, 16): (6, 8, 16), (1, 10, 13): (6, 10, 13),
+            (2, 12, 8): (12, 12, 8)}[block]
+    w = gen.Workload("edges", 1, 1, 128, *grid, block, 0.25, "bf16", "smooth", 9)
+    data = gen.make_inputs(w)
+    perm, _ = orc.partition_perm(w.T, w.H, w.W, *w.block)
+    q, k, v, do = (data[n][0, :, 0][perm] for n in ("q", "k", "v", "do"))
+    rng = np.random.default_rng(3)
+    counts = [0, 1, 63, 64, 65, 127, 128, 129, 255, 256, 257, 300] if w.n_blocks >= 12 else [0, 1, 127, 128, 129, 300]
+    mask = np.zeros((1, w.S, w.n_blocks), dtype=bool)
+    for j in range(w.n_blocks):
+        c = min(counts[j % len(counts)], w.S)
+        mask[0, rng.choice(w.S, size=c, replace=False), j] = True
+    kb_ptr, q_idx, q_ptr, q_pairs, n = lists_from_mask(mask)
+    L = VmobaLayer(vb.shape_of(w), capacity=max(n, 1), with_backward=True)
+    for name, buf in (("q", L.q_bm), ("k", L.k_bm), ("v", L.v_bm), ("do", L.do_bm)):
+        buf.copy_(U.bm_to_device(w, U.block_major(w, data, name, perm)))
+    L.kb_ptr.copy_(kb_ptr); L.q_idx.copy_(q_idx); L.q_ptr.copy_(q_ptr); L.q_pairs.copy_(q_pairs)
+    L.o_bm.fill_(7.0); L.lse.fill_(7.0)
+    L.attn_fwd()
+    L.attn_bwd()
+    L.check_status()
+    scale = w.head_dim ** -0.5
+    o_ref, lse_ref = orc.sparse_attn_fwd(q, k, v, mask[0], scale)
+    dq_ref, dk_ref, dv_ref = orc.sparse_attn_bwd(q, k, v, mask[0], scale, do)
+    o = U.to_numpy_f32(L.o_bm).reshape(w.S, w.head_dim)
+    lse = L.lse.cpu().numpy().reshape(w.S)
+    dq, dk, dv = (U.to_numpy_f32(t).reshape(w.S, w.head_dim) for t in (L.dq_bm, L.dk_bm, L.dv_bm))
+    empty = ~mask[0].any(axis=1)
+    assert empty.any() and (~empty).any()
+    assert np.all(o[empty] == 0) and np.all(np.isneginf(lse[empty])) and np.all(dq[empty] == 0)
+    U.assert_close(o, o_ref, w.dtype, "o")
+    assert U.max_abs(lse[~empty], lse_ref[~empty]) <= 2e-2
+    U.assert_close(dq, dq_ref, w.dtype, "dq")
+    U.assert_close(dk, dk_ref, w.dtype, "dk")
+    U.assert_close(dv, dv_ref, w.dtype, "dv")
+
+
 @pytest.mark.parametrize("w", [CASES[0], CASES[3], CASES[8]], ids=[IDS[0], IDS[3], IDS[8]])
 def test_sparse_attention_full_mask_equals_dense_oracle(w):
     """tau = 1: the sparse path over every pair must reproduce dense softmax attention."""
