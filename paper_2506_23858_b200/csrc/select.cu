@@ -569,18 +569,43 @@ select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, flo
   const long long warp = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const long long nwarps = (long long)gridDim.x * (blockDim.x >> 5);
   const uint32_t lt_mask = (1u << lane) - 1u;
-  for (long long row = warp; row < n_rows; row += nwarps) {
+  // A warp takes a run of consecutive rows: they belong to one head (or two), so the smallest cutoff of the run
+  // reaches the head's state with one atomic per run instead of one per row, and the next row's scores are
+  // requested while the current row is worked on.
+  const long long per_warp = (n_rows + nwarps - 1) / nwarps;
+  const long long row_begin = warp * per_warp, row_end = min(n_rows, row_begin + per_warp);
+  uint32_t run_cut = 0xffffffffu;
+  long long run_head = -1;
+  auto note_cutoff = [&](long long row, uint32_t c) {
+    const long long head = row / S;
+    if (head != run_head) {
+      if (lane == 0 && run_head >= 0) atomicMin(&st[run_head].cutoff_key, run_cut);
+      run_head = head;
+      run_cut = 0xffffffffu;
+    }
+    run_cut = min(run_cut, c);
+  };
+  auto load_row = [&](long long row, uint32_t (&k)[MW]) {
     const float* sr = scores + row * Nb;
+#pragma unroll
+    for (int i = 0; i < MW; ++i) {
+      const int j = lane + 32 * i;
+      k[i] = (i < mw && j < Nb) ? float_key(__ldg(sr + j)) : 0u;     // 0 is below every real score's key
+    }
+  };
+  uint32_t next_key[MW];
+  if (row_begin < row_end) load_row(row_begin, next_key);
+  for (long long row = row_begin; row < row_end; ++row) {
     const int own = own_sb > 0 ? (int)(row % S) / own_sb : -1;      // the query's own block, if it is to be kept
     const uint32_t own_bit = (own >= 0 && (own >> 5) == lane) ? 1u << (own & 31) : 0u;
     uint32_t key[MW];
     uint32_t kmax = 0u;
 #pragma unroll
     for (int i = 0; i < MW; ++i) {
-      const int j = lane + 32 * i;
-      key[i] = (i < mw && j < Nb) ? float_key(__ldg(sr + j)) : 0u;     // 0 is below every real score's key
+      key[i] = next_key[i];
       kmax = max(kmax, key[i]);
     }
+    if (row + 1 < row_end) load_row(row + 1, next_key);
     kmax = __reduce_max_sync(0xffffffffu, kmax);
     double w[TOPK ? 1 : MW];
     double target;
@@ -617,8 +642,10 @@ select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, flo
     // best first, lowest block index among equals, exactly the order the rule is stated in; the
     // cumulative mass of the threshold rule is the running sum of the winners' weights.
     {
-      constexpr int kRounds = 24;
-      const int rounds = TOPK ? ((int)target <= kRounds ? (int)target : 0) : (tau < 1.0f ? min(kRounds, Nb) : 0);
+      // (a round costs about as much as two steps of the 32-step bitwise search below: beyond eight blocks the
+      // top-k rule, whose count is known, goes there directly)
+      constexpr int kRounds = 24, kTopkRounds = 8;
+      const int rounds = TOPK ? ((int)target <= kTopkRounds ? (int)target : 0) : (tau < 1.0f ? min(kRounds, Nb) : 0);
       uint32_t taken = 0u;              // bit i: this lane's block lane + 32 i is selected
       uint32_t c_last = 0u;
       double acc = 0.0;
@@ -651,7 +678,7 @@ select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, flo
           if (lane == i) my_word = word;
         }
         if (lane < mw) mask_bits[row * mw + lane] = my_word | own_bit;
-        if (lane == 0) atomicMin(&st[row / S].cutoff_key, c_last);
+        note_cutoff(row, c_last);
         continue;
       }
     }
@@ -660,9 +687,18 @@ select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, flo
     if (!TOPK && tau >= 1.0f) {
       c = 1u;                                  // everything: every real key is >= 1
     } else {
+      // the top-k rule counts in integers (its measure is a number of blocks)
+      const int k_target = TOPK ? (int)target : 0;
+      auto count_ge = [&](uint32_t cc) {
+        int n = 0;
+#pragma unroll
+        for (int i = 0; i < MW; ++i) n += (i < mw && key[i] >= cc) ? 1 : 0;
+        return __reduce_add_sync(0xffffffffu, n);
+      };
       for (int b = 31; b >= 0; --b) {
         const uint32_t cand = c | (1u << b);
-        if (cand <= kmax && measure_ge(cand) >= target) c = cand;
+        if (cand > kmax) continue;
+        if (TOPK ? count_ge(cand) >= k_target : measure_ge(cand) >= target) c = cand;
       }
       if (c == 0u) c = 1u;                     // rounding kept the mass below the target: take the row
     }
@@ -697,8 +733,9 @@ select_local_kernel(const float* __restrict__ scores, int S, int Nb, int mw, flo
       }
     }
     if (lane < mw) mask_bits[row * mw + lane] = my_word | own_bit;
-    if (lane == 0) atomicMin(&st[row / S].cutoff_key, c);
+    note_cutoff(row, c);
   }
+  if (lane == 0 && run_head >= 0) atomicMin(&st[run_head].cutoff_key, run_cut);
 }
 
 __global__ void local_cutoff_kernel(const HeadState* __restrict__ st, float* __restrict__ cutoff_per_head, int BH) {
@@ -893,7 +930,9 @@ static int select_impl(const vmoba_shape* shape, const float* scores, const floa
           scores, D.S, D.Nb, D.mask_words, D.scale, tau, topk, own_sb, mask_bits, w.state, n_rows);
     };
     auto by_words = [&](auto topk_tag) {
-      if (D.mask_words <= 4) launch_local(topk_tag, std::integral_constant<int, 4>());
+      if (D.mask_words <= 1) launch_local(topk_tag, std::integral_constant<int, 1>());
+      else if (D.mask_words <= 2) launch_local(topk_tag, std::integral_constant<int, 2>());
+      else if (D.mask_words <= 4) launch_local(topk_tag, std::integral_constant<int, 4>());
       else if (D.mask_words <= 8) launch_local(topk_tag, std::integral_constant<int, 8>());
       else if (D.mask_words <= 16) launch_local(topk_tag, std::integral_constant<int, 16>());
       else launch_local(topk_tag, std::integral_constant<int, kLocalMaxWords>());
