@@ -35,6 +35,7 @@ constexpr int DH = 128;              // head dim
 constexpr int PANEL = BM * 128;      // bytes of one 64-column panel of a 128-row tile (16 KB)
 constexpr int TILE = 2 * PANEL;      // bytes of a [128 x 128] bf16 tile (32 KB)
 constexpr int THREADS = 256;
+constexpr int THREADS_SPLIT = 384;   // with four epilogue warps
 constexpr uint32_t TMEM_COLS = 256;
 constexpr uint32_t O_COL = 128;      // S at 0, P at 64, O at 128
 constexpr float RESCALE_LOG2 = 8.0f;
@@ -44,8 +45,11 @@ struct Smem {
   uint64_t s_full, p_ready;          // scores written (commit) / P written (128 arrivals)
   uint64_t o_done;                   // P V of a key tile complete (commit)
   uint64_t q_full, q_empty;          // Q tile of an item gathered (64 arrivals) / no longer needed (commit)
+  uint64_t ep_ready;                 // SPLIT: an item's normalisers are in ep_inv / ep_lse (128 softmax arrivals)
+  uint64_t o_free;                   // SPLIT: the epilogue warps have read the accumulator (128 arrivals)
   uint32_t tmem_base;
   int abort_flag;
+  float ep_inv[2][BM], ep_lse[2][BM];   // SPLIT, [item % 2][row]: 1 / sum of the rounded weights, natural-log lse
   int qinfo[4][BM];                  // [item % 4][row]: 2 * in-head position + (query has a single block), -1 for padding rows
 };
 // two CTAs per SM: each may use half of the SM's shared memory
@@ -157,8 +161,13 @@ __device__ __forceinline__ void store8_resid(__nv_bfloat16* dst, __nv_bfloat16* 
 }
 
 // RASTER: the directly written rows of o go through p.o_map.
-template <bool RASTER>
-__global__ void __launch_bounds__(THREADS, 2)
+// SPLIT: four more warps (8-11) take the epilogue: they read the accumulator and write the rows while the softmax
+// warps are already on the next item's first tile.  With 384 threads two CTAs leave 80 registers per thread, so the
+// warp groups trade registers at the start: the softmax group takes 128, the first group keeps 72, the epilogue
+// group 40.  Its loaders then have no room to hold rows in registers: they ask the L2 for an item's rows ahead of
+// time and, once the Q tile is free, bring them in as asynchronous 16-byte copies straight into the swizzled tile.
+template <bool RASTER, bool SPLIT>
+__global__ void __launch_bounds__(SPLIT ? THREADS_SPLIT : THREADS, 2)
 attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -192,6 +201,7 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     mbar_init(&sm->s_full, 1); mbar_init(&sm->p_ready, 128);
     mbar_init(&sm->o_done, 1);
     mbar_init(&sm->q_full, 64); mbar_init(&sm->q_empty, 1);
+    mbar_init(&sm->ep_ready, 128); mbar_init(&sm->o_free, 128);
     sm->abort_flag = 0;
     fence_barrier_init();
     prefetch_tmap(&tmK);
@@ -217,6 +227,10 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
     return item_from_desc(p, d);
   };
 
+  // SPLIT: every role starts by taking or giving back registers (the whole warp group executes the same one)
+  if (warp < 4) {
+    if constexpr (SPLIT) asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+  }
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -284,6 +298,11 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         lap(2);
         mbar_wait_warp(&sm->v_full, f & 1, abort_flag, p.status);
         lap(3);
+        if constexpr (SPLIT) {
+          // the accumulator still holds the item before until the epilogue warps have read it
+          if (t == 0 && n >= 1) mbar_wait_warp(&sm->o_free, (n - 1) & 1, abort_flag, p.status);
+          lap(4);
+        }
         tc_fence_after();
         {
           const int ksteps = (keys + 15) >> 4;
@@ -310,41 +329,83 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       // Four bookkeeping slots: the softmax warps read slot n % 4 in the epilogue of item n, and the loaders can be
       // at most two items ahead of an epilogue.
       int info[2];
-      for (int half = 0; half < 2; ++half) {       // rows 0..63, then rows 64..127
-        uint4 v[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int row = half * 64 + (lt >> 4) + 4 * i;
-          v[i] = make_uint4(0u, 0u, 0u, 0u);
-          if (row < it.n_rows) {
-            const int qp = checked_index(__ldg(p.q_idx + it.list_lo + row), p.S, p.status);
-            v[i] = __ldg(reinterpret_cast<const uint4*>(qh + (long long)qp * DH) + chunk);
-          }
-        }
-        // per-row bookkeeping of row 64 half + lt, fetched while the rows are in flight
-        info[half] = -1;
-        if (half * 64 + lt < it.n_rows) {
-          const int qp = checked_index(__ldg(p.q_idx + it.list_lo + half * 64 + lt), p.S, p.status);
-          const long long G_ = it.head_off + qp;
-          info[half] = 2 * qp + ((p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1 ? 1 : 0);
-        }
-        // the second half's rows are fetched only after the first half has been stored: ask the L2 for them now
-        // (one request per 128-byte line)
-        if (half == 0 && (chunk & 7) == 0) {
+      if constexpr (SPLIT) {
+        if ((chunk & 7) == 0) {       // one L2 request per 128-byte line of every row of the item
 #pragma unroll 4
-          for (int i = 0; i < 16; ++i) {
-            const int row = 64 + (lt >> 4) + 4 * i;
+          for (int i = 0; i < BM / 4; ++i) {
+            const int row = (lt >> 4) + 4 * i;
             if (row < it.n_rows) {
               const int qp = checked_index(__ldg(p.q_idx + it.list_lo + row), p.S, p.status);
               asm volatile("prefetch.global.L2 [%0];" ::"l"(qh + (long long)qp * DH + chunk * 8));
             }
           }
         }
-        // the Q tile is free once the previous item's last Q K^T has run
-        if (half == 0 && n >= 1) mbar_wait(&sm->q_empty, (n - 1) & 1, abort_flag, p.status);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int row = half * 64 + (lt >> 4) + 4 * i;
+        for (int h = 0; h < 2; ++h) {
+          info[h] = -1;
+          if (h * 64 + lt < it.n_rows) {
+            const int qp = checked_index(__ldg(p.q_idx + it.list_lo + h * 64 + lt), p.S, p.status);
+            const long long G_ = it.head_off + qp;
+            info[h] = 2 * qp + ((p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1 ? 1 : 0);
+          }
+        }
+        if (n >= 1) mbar_wait(&sm->q_empty, (n - 1) & 1, abort_flag, p.status);
+        const uint32_t q_base = smem_u32(sQ) + panel * PANEL;
+#pragma unroll 8
+        for (int i = 0; i < BM / 4; ++i) {
+          const int row = (lt >> 4) + 4 * i;
+          const bool ok = row < it.n_rows;
+          const int qp = ok ? checked_index(__ldg(p.q_idx + it.list_lo + row), p.S, p.status) : 0;
+          // rows beyond the item's are zero-filled (source size 0)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(q_base + row * 128 + ((cc ^ (row & 7)) << 4)),
+                       "l"(reinterpret_cast<const uint4*>(qh + (long long)qp * DH) + chunk), "r"(ok ? 16u : 0u)
+                       : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+      }
+      constexpr int RR = 64;                       // rows per round (a round's rows wait in registers)
+      constexpr int NI = RR / 4;
+      for (int rnd = 0; rnd < (SPLIT ? 0 : BM / RR); ++rnd) {
+        uint4 v[NI];
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+          const int row = rnd * RR + (lt >> 4) + 4 * i;
+          v[i] = make_uint4(0u, 0u, 0u, 0u);
+          if (row < it.n_rows) {
+            const int qp = checked_index(__ldg(p.q_idx + it.list_lo + row), p.S, p.status);
+            v[i] = __ldg(reinterpret_cast<const uint4*>(qh + (long long)qp * DH) + chunk);
+          }
+        }
+        if (rnd == 0) {
+          // per-row bookkeeping of rows lt and 64 + lt, fetched while the rows are in flight
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            info[h] = -1;
+            if (h * 64 + lt < it.n_rows) {
+              const int qp = checked_index(__ldg(p.q_idx + it.list_lo + h * 64 + lt), p.S, p.status);
+              const long long G_ = it.head_off + qp;
+              info[h] = 2 * qp + ((p.q_ptr[G_ + 1] - p.q_ptr[G_]) == 1 ? 1 : 0);
+            }
+          }
+          // the later rounds' rows are fetched only after this round has been stored: ask the L2 for them now
+          // (one request per 128-byte line)
+          if ((chunk & 7) == 0) {
+#pragma unroll 4
+            for (int i = 0; i < (BM - RR) / 4; ++i) {
+              const int row = RR + (lt >> 4) + 4 * i;
+              if (row < it.n_rows) {
+                const int qp = checked_index(__ldg(p.q_idx + it.list_lo + row), p.S, p.status);
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(qh + (long long)qp * DH + chunk * 8));
+              }
+            }
+          }
+          // the Q tile is free once the previous item's last Q K^T has run
+          if (n >= 1) mbar_wait(&sm->q_empty, (n - 1) & 1, abort_flag, p.status);
+        }
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+          const int row = rnd * RR + (lt >> 4) + 4 * i;
           *reinterpret_cast<uint4*>(sQ + panel * PANEL + row * 128 + ((cc ^ (row & 7)) << 4)) = v[i];
         }
       }
@@ -353,8 +414,74 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       fence_async_proxy();
       mbar_arrive(&sm->q_full);
     }
+  } else if (SPLIT && warp >= 8) {
+    // ------------------------------------------------------------------ epilogue warps (SPLIT): thread = one query row
+    if constexpr (SPLIT) asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
+    const int quad = warp & 3;
+    const int r = quad * 32 + lane;
+    const uint32_t o_tmem = tmem + ((uint32_t)(quad * 32) << 16) + O_COL;
+    uint32_t tc = 0, n = 0;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x, ++n) {
+      const Item it = get_item(item);
+      tc += it.ntiles;
+      mbar_wait(&sm->ep_ready, n & 1, abort_flag, p.status);
+      mbar_wait(&sm->o_done, (tc - 1) & 1, abort_flag, p.status);
+      tc_fence_after();
+      const int info = sm->qinfo[n & 3][r];
+      const float inv = sm->ep_inv[n & 1][r];
+      const float row_lse = sm->ep_lse[n & 1][r];
+      const bool row_ok = info >= 0;
+      const int qpos = row_ok ? info >> 1 : 0;
+      const bool direct = (info & 1) != 0;
+      const long long G_ = it.head_off + qpos;
+      const long long o_row_off = RASTER ? ((row_ok && direct) ? p.o_map.off(G_, DH) : 0) : G_ * DH;
+      const long long pos = (long long)it.list_lo + r;
+#pragma unroll 1
+      for (int c = 0; c < 8; ++c) {
+        uint32_t ov[16];
+        tmem_ld16(o_tmem + c * 16, ov);
+        tmem_ld_wait();
+        if (c == 7) {          // the accumulator has been read: the next item's first P V may overwrite it
+          tc_fence_before();
+          mbar_arrive(&sm->o_free);
+        }
+        if (row_ok) {
+          const int col = 16 * c;
+          if (direct) {
+            __nv_bfloat16* dst = p.o + o_row_off + col;
+            __nv_bfloat16* rdst = p.o_resid ? p.o_resid + G_ * DH + col : nullptr;
+#pragma unroll
+            for (int i = 0; i < 16; i += 8) {
+              float v8[8];
+#pragma unroll
+              for (int k = 0; k < 8; ++k) v8[k] = __uint_as_float(ov[i + k]) * inv;
+              store8_resid(dst + i, rdst ? rdst + i : nullptr, v8);
+            }
+          } else {
+            float* dst = p.part_o + pos * DH + col;
+            if (!p.part_o_32) {
+#pragma unroll
+              for (int i = 0; i < 16; i += 4)
+                *reinterpret_cast<float4*>(dst + i) =
+                    make_float4(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
+                                __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv);
+            } else
+#pragma unroll
+            for (int i = 0; i < 16; i += 8)
+              st_global_v8(dst + i, __uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
+                           __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv,
+                           __uint_as_float(ov[i + 4]) * inv, __uint_as_float(ov[i + 5]) * inv,
+                           __uint_as_float(ov[i + 6]) * inv, __uint_as_float(ov[i + 7]) * inv);
+          }
+        }
+      }
+      if (row_ok) {
+        if (direct) p.lse[G_] = row_lse; else p.part_lse[pos] = row_lse;
+      }
+    }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue
+    if constexpr (SPLIT) asm volatile("setmaxnreg.inc.sync.aligned.u32 128;");
     const int quad = warp & 3;                      // TMEM lane quarter this warp may access
     const int r = quad * 32 + lane;                 // query row inside the tile
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
@@ -432,6 +559,14 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         tmem_st_wait();
         tc_fence_before();
         mbar_arrive(&sm->p_ready);
+      }
+      if constexpr (SPLIT) {
+        // hand the row's normalisers to the epilogue warps and go on with the next item
+        sm->ep_inv[n & 1][r] = 1.0f / l_r;
+        sm->ep_lse[n & 1][r] = (m_used + log2f(l)) * 0.6931471805599453f;
+        mbar_arrive(&sm->ep_ready);
+        lap(4);
+        continue;
       }
       // ---- epilogue: wait for the last P V, normalise, write the row
       lap(3);
@@ -523,12 +658,19 @@ int tc_sparse_fwd_narrow(const Dims& D, const void* q, const void* k, const void
   p.part_o_32 = (reinterpret_cast<uintptr_t>(part_o) % 32) == 0;
   p.o_map = o_map;
   const long long items = std::max<long long>(1, std::min<long long>(cap / BM + n_kb, 2LL * sm_count()));
+  // Epilogue warps pay when an item is a few tiles long and its epilogue a quarter of it (C4 forward stage 0.42 ->
+  // 0.37 ms, C2 0.212 -> 0.190 ms, 3D layer of C5 with 4 heads 0.84 -> 0.81 ms); on key blocks of 1560 and 1638
+  // keys the plain variant is 2 % faster.
+  const bool split_mode = D.sb <= 4 * BN;
   if (o_map.perm) {
-    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_narrow_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-    attn_fwd_narrow_kernel<true><<<(int)items, THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_narrow_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    attn_fwd_narrow_kernel<true, false><<<(int)items, THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
+  } else if (split_mode) {
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_narrow_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    attn_fwd_narrow_kernel<false, true><<<(int)items, THREADS_SPLIT, SMEM_BYTES, st>>>(tmK, tmV, p);
   } else {
-    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_narrow_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-    attn_fwd_narrow_kernel<false><<<(int)items, THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
+    VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_narrow_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    attn_fwd_narrow_kernel<false, false><<<(int)items, THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
   }
   const long long nq = (long long)D.BH * D.S;
   simt::merge_batched_kernel<__nv_bfloat16><<<(int)std::min<long long>((nq + 255) / 256, sm_count() * 8), 256, 0, st>>>(
