@@ -186,7 +186,7 @@ int vmoba_select_rule_apply(const vmoba_shape* shape, const float* scores, int32
 /*
  * vmoba_select_rule_apply for a caller that already knows each head's score range (score_range [B*heads][2] =
  * minimum, maximum, exactly as vmoba_block_scores_range wrote them for these scores): the head-wide rules then
- * skip their own pass over the score matrix that looks for it (four traversals instead of five).  The results are
+ * skip their own pass over the score matrix that looks for it (one traversal fewer).  The results are
  * those of vmoba_select_rule_apply bit for bit.  A range that does not bound the scores gives an unspecified
  * selection (every access still stays inside the buffers).  The per-query rules and the row-normalised rule
  * ignore the range.

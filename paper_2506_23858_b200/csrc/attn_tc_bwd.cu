@@ -228,6 +228,16 @@ attn_bwd_dkdv_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_co
         tma_load_2d(sV, &tmV, &sm->kv_full[0], 0, y);
         tma_load_2d(sV + PANEL, &tmV, &sm->kv_full[0], 64, y);
         ++n;
+        // The one K / V pair is reloaded only when the item's last MMA has run: ask the L2 for the next item's
+        // tiles now, so that the reload finds them there.
+        if (item + gridDim.x < n_items) {
+          const KvItem nx = kv_decode(p, item + gridDim.x, tiles);
+          const int yn = (int)nx.head_off + nx.key0;
+          if (nx.n_units > 0) {
+            tma_prefetch_2d(&tmK, 0, yn); tma_prefetch_2d(&tmK, 64, yn);
+            tma_prefetch_2d(&tmV, 0, yn); tma_prefetch_2d(&tmV, 64, yn);
+          }
+        }
       }
       if (*abort_flag)
         for (uint32_t f = n > 2 ? n - 2 : 0; f < n; ++f) mbar_wait(&sm->kv_full[0], f & 1, abort_flag, p.status);

@@ -98,6 +98,12 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
       : "memory");
 }
+// The same box requested into the L2 only (no shared-memory destination, no barrier).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x),
+               "r"(y)
+               : "memory");
+}
 // Row gather: four rows (given by their row coordinates) of a 2D tensor whose map has a one-row
 // box of 64 columns; the rows land in four consecutive 128-byte rows at smem_dst with the same
 // 128-byte swizzle a tiled load produces, so a 128-row operand tile is 32 of these per panel.
