@@ -238,7 +238,8 @@ int vmoba_select_static(const vmoba_shape* shape, const float* scores, float tau
  * bf16(o_exact - o_bm).  The backward needs rowsum(dO * O) to better than bf16 accuracy of O
  * (taken from the rounded output alone, dQ loses about 6e-3 relative accuracy); training
  * callers keep this tensor with o_bm and lse for vmoba_attn_bwd.
- * `capacity` is the one given to vmoba_select (bounds the per-pair partial results in ws).
+ * `capacity` is the one given to vmoba_select (bounds the per-pair partial results in ws: for bf16 with
+ * head_dim 128 a row of fp16 values with a power-of-two scale per row, else an fp32 row).
  */
 int vmoba_attn_fwd(const vmoba_shape* shape, const void* q_bm, const void* k_bm, const void* v_bm,
                    const int32_t* kb_ptr, const int32_t* q_idx, const int32_t* q_ptr,

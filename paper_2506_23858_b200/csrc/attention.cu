@@ -15,7 +15,7 @@ size_t scores_ws_bytes(const Dims& D);   // scores.cu
 int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                   const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
                   int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o, float* part_lse,
-                  cudaStream_t st, const RowMap& o_map);
+                  float* part_scale, cudaStream_t st, const RowMap& o_map);
 int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, void* o, void* o_resid, float* lse,
                  int32_t* status, cudaStream_t st);
 
@@ -30,14 +30,16 @@ static bool use_tensor_cores(const Dims& D) { return D.dtype == VMOBA_BF16 && D.
 
 static long long max_items_128(const Dims& D, long long cap) { return cap / 128 + (long long)D.BH * D.Nb + 1; }
 
-struct FwdWs { int* item_ptr; int* item_tab; float* part_o; float* part_lse; size_t bytes; Guards guards; };
+struct FwdWs { int* item_ptr; int* item_tab; float* part_o; float* part_lse; float* part_scale; size_t bytes; Guards guards; };
 static FwdWs carve_fwd(const Dims& D, long long cap, void* ws) {
   Carver c(ws);
   FwdWs w;
   w.item_ptr = c.take<int>((size_t)D.BH * D.Nb + 1);
   w.item_tab = c.take<int>(4 * (size_t)max_items_128(D, cap));   // one int per item, or a 16-byte descriptor
   w.part_lse = c.take<float>((size_t)cap);
-  w.part_o = c.take<float>((size_t)cap * D.d);
+  w.part_scale = c.take<float>((size_t)cap);     // per partial row: the power of two its fp16 values are scaled by
+  // fp32 rows on the CUDA-core path, fp16 rows (scaled per row) on the tensor-core path
+  w.part_o = c.take<float>((size_t)cap * D.d / (use_tensor_cores(D) ? 2 : 1));
   w.bytes = c.total();
   w.guards = c.guards;
   return w;
@@ -225,7 +227,8 @@ extern "C" int vmoba_attn_fwd(const vmoba_shape* shape, const void* q_bm, const 
     FwdWs w = carve_fwd(D, capacity, ws);
     VMOBA_GUARDS_ARM(w.guards, st);
     rc = tc_sparse_fwd(D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o_bm, o_resid_or_null, lse,
-                       dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse, st, RowMap());
+                       dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse, w.part_scale, st,
+                       RowMap());
     VMOBA_GUARDS_CHECK(w.guards, dev_status, st);
     return rc;
   }
@@ -282,7 +285,8 @@ extern "C" int vmoba_attn_fwd_raster(const vmoba_shape* shape, const void* q_bm,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   VMOBA_GUARDS_ARM(w.guards, st);
   rc = tc_sparse_fwd(D, q_bm, k_bm, v_bm, kb_ptr, q_idx, q_ptr, q_pairs, capacity, o, o_resid_bm_or_null, lse,
-                     dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse, st, o_map);
+                     dev_status, w.item_ptr, w.item_tab, max_items_128(D, capacity), w.part_o, w.part_lse, w.part_scale, st,
+                     o_map);
   VMOBA_GUARDS_CHECK(w.guards, dev_status, st);
   return rc;
 }

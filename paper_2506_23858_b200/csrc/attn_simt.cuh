@@ -9,6 +9,8 @@
 // directly, queries with none are zero-filled by the merge kernel.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace vmoba {
@@ -283,11 +285,27 @@ merge_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pairs, lon
 // and their lse of query g0 + l, works out the weights on its own, and the warp then walks the queries that
 // need a row written, fetching all rows of a query at once.  Queries with more pairs than a lane keeps take
 // the warp-wide loop of merge_kernel.
+//
+// PT = __half: a partial row is stored as fp16 values times a power of two (part_scale, one per row; the row's
+// largest magnitude rounded up), which halves the bytes the forward writes and this pass reads; a value is then off
+// by at most 2^-11 of its row's largest one.  The scale is folded into the row's merge weight.
 constexpr int kInLane = 8;
-template <typename T>
+template <typename PT>
+__device__ __forceinline__ float4 load_part4(const PT* p);
+template <>
+__device__ __forceinline__ float4 load_part4<float>(const float* p) { return *reinterpret_cast<const float4*>(p); }
+template <>
+__device__ __forceinline__ float4 load_part4<__half>(const __half* p) {
+  const uint2 u = *reinterpret_cast<const uint2*>(p);
+  const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&u.x));
+  const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&u.y));
+  return make_float4(a.x, a.y, b.x, b.y);
+}
+template <typename T, typename PT>
 __global__ void __launch_bounds__(256)
 merge_batched_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pairs, long long n_queries,
-                     const float* __restrict__ part_o, const float* __restrict__ part_lse, long long capacity,
+                     const PT* __restrict__ part_o, const float* __restrict__ part_lse,
+                     const float* __restrict__ part_scale, long long capacity,
                      T* __restrict__ o, T* __restrict__ o_resid, float* __restrict__ lse, const RowMap o_map = RowMap()) {
   constexpr int DH = 128;
   const int lane = threadIdx.x & 31;
@@ -306,7 +324,7 @@ merge_batched_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pa
     }
     const bool direct = n == 1 && n_raw == 1;
     int pos[kInLane];
-    float w[kInLane];
+    float w[kInLane], sc[kInLane];
     float out_lse = -INFINITY;
     if (!direct && n > 0 && n <= kInLane) {
       float mx = -INFINITY;
@@ -316,8 +334,14 @@ merge_batched_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pa
         if (k < n) pos[k] = min(max(q_pairs[lo + k], 0), last);
       }
 #pragma unroll
-      for (int k = 0; k < kInLane; ++k)
-        if (k < n) { w[k] = part_lse[pos[k]]; mx = fmaxf(mx, w[k]); }
+      for (int k = 0; k < kInLane; ++k) {
+        sc[k] = 1.0f;
+        if (k < n) {
+          w[k] = part_lse[pos[k]];
+          if (part_scale) sc[k] = part_scale[pos[k]];
+          mx = fmaxf(mx, w[k]);
+        }
+      }
       float tot = 0.f;
 #pragma unroll
       for (int k = 0; k < kInLane; ++k) {
@@ -326,7 +350,7 @@ merge_batched_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pa
       }
       const float inv = 1.0f / tot;
 #pragma unroll
-      for (int k = 0; k < kInLane; ++k) w[k] *= inv;
+      for (int k = 0; k < kInLane; ++k) w[k] *= inv * sc[k];
       out_lse = mx + logf(tot);
     } else {
 #pragma unroll
@@ -348,7 +372,7 @@ merge_batched_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pa
           const int pk = __shfl_sync(0xffffffffu, pos[k], b);
           wk[k] = __shfl_sync(0xffffffffu, w[k], b);
           v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (k < nb) v[k] = *reinterpret_cast<const float4*>(part_o + (long long)pk * DH + lane * 4);
+          if (k < nb) v[k] = load_part4<PT>(part_o + (long long)pk * DH + lane * 4);
         }
 #pragma unroll
         for (int k = 0; k < kInLane; ++k) {
@@ -369,18 +393,19 @@ merge_batched_kernel(const int* __restrict__ q_ptr, const int* __restrict__ q_pa
         for (long long i0 = qlo; i0 < qhi; i0 += 32) {
           const long long i = i0 + lane;
           int my_pos = 0;
-          float my_w = 0.f;
+          float my_w = 0.f, my_ws = 0.f;
           if (i < qhi) {
             my_pos = min(max(q_pairs[i], 0), last);
             my_w = expf(part_lse[my_pos] - mx);
+            my_ws = part_scale ? my_w * part_scale[my_pos] : my_w;
           }
           tot += my_w;
           const int m = (int)min((long long)32, qhi - i0);
 #pragma unroll 4
           for (int k = 0; k < m; ++k) {
             const long long pk = __shfl_sync(0xffffffffu, my_pos, k);
-            const float wgt = __shfl_sync(0xffffffffu, my_w, k);
-            const float4 v = *reinterpret_cast<const float4*>(part_o + pk * DH + lane * 4);
+            const float wgt = __shfl_sync(0xffffffffu, my_ws, k);
+            const float4 v = load_part4<PT>(part_o + pk * DH + lane * 4);
             acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
             acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
           }

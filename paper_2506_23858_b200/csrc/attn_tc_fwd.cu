@@ -21,6 +21,8 @@
 // half, so that it never holds more than 64 scores.
 #include <algorithm>
 
+#include <cuda_fp16.h>
+
 #include "attn_simt.cuh"
 #include "sm100.cuh"
 
@@ -67,8 +69,9 @@ struct Params {
   __nv_bfloat16* o_resid;
   RowMap o_map;          // where the rows of o go (block-major, or raster order through perm); o_resid is block-major
   float* lse;
-  float* part_o;
+  __half* part_o;        // partial rows: fp16 values times part_scale[row]
   float* part_lse;
+  float* part_scale;
   long long capacity;
   int part_o_32;         // part_o is 32-byte aligned: rows go out with 32-byte stores
   int32_t* status;
@@ -141,6 +144,17 @@ __device__ __forceinline__ void exp_pack64(const uint32_t (&sv)[64], float scale
     pk[i] = pack_bf16(p0, p1);
     add2(r0, r1, r0, r1, __uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u));
   }
+}
+
+// Partial rows are stored as fp16 times a power of two per row: the smallest one at or above the row's largest
+// magnitude (1 for a row of zeros), so that the values use the format's full precision whatever the scale of V.
+__device__ __forceinline__ float pow2_at_or_above(float x) {
+  const uint32_t u = (__float_as_uint(x) + 0x007fffffu) & 0x7f800000u;
+  return u ? __uint_as_float(u) : 1.0f;
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
 }
 
 // N (8 or 16) consecutive outputs as bf16 (one 16- or 32-byte store) and, if asked for, their rounding
@@ -468,6 +482,26 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
       const long long G_ = it.head_off + (row_ok ? qpos : 0);
       const long long o_row_off = RASTER ? ((row_ok && direct) ? p.o_map.off(G_, DH) : 0) : G_ * DH;
       const long long pos = (long long)it.list_lo + row;
+      // a partial row goes out as fp16 times a power of two: find the row's largest magnitude first
+      float mul = inv, row_scale = 1.0f;
+      if constexpr (!DENSE) {
+        const bool partial = row_ok && !direct;
+        if (__any_sync(0xffffffffu, partial)) {
+          float amax = 0.f;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            uint32_t ov[32];
+            tmem_ld32(o_tmem + c * 32, ov);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(ov[i])));
+          }
+          if (partial) {
+            row_scale = pow2_at_or_above(amax * inv);
+            mul = inv / row_scale;
+          }
+        }
+      }
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         uint32_t ov[32];
@@ -486,25 +520,25 @@ attn_fwd_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_const
               store_resid<8>(dst + i, rdst ? rdst + i : nullptr, v8);
             }
           } else {
-            float* dst = p.part_o + pos * DH + col;
-            if (!p.part_o_32) {
+            __half* dst = p.part_o + pos * DH + col;
 #pragma unroll
-              for (int i = 0; i < 32; i += 4)
-                *reinterpret_cast<float4*>(dst + i) =
-                    make_float4(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
-                                __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv);
-            } else
+            for (int i = 0; i < 32; i += 16) {
+              uint32_t h[8];
 #pragma unroll
-            for (int i = 0; i < 32; i += 8)       // 32-byte stores: a thread's row is 512 contiguous bytes
-              st_global_v8(dst + i, __uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
-                           __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv,
-                           __uint_as_float(ov[i + 4]) * inv, __uint_as_float(ov[i + 5]) * inv,
-                           __uint_as_float(ov[i + 6]) * inv, __uint_as_float(ov[i + 7]) * inv);
+              for (int k = 0; k < 8; ++k)
+                h[k] = pack_half2(__uint_as_float(ov[i + 2 * k]) * mul, __uint_as_float(ov[i + 2 * k + 1]) * mul);
+              if (p.part_o_32) {       // one 32-byte store, else two of 16 bytes
+                st_global_v8(dst + i, h[0], h[1], h[2], h[3], h[4], h[5], h[6], h[7]);
+              } else {
+                reinterpret_cast<uint4*>(dst + i)[0] = make_uint4(h[0], h[1], h[2], h[3]);
+                reinterpret_cast<uint4*>(dst + i)[1] = make_uint4(h[4], h[5], h[6], h[7]);
+              }
+            }
           }
         }
       }
       if (row_ok) {
-        if (direct) p.lse[G_] = row_lse; else p.part_lse[pos] = row_lse;
+        if (direct) p.lse[G_] = row_lse; else { p.part_lse[pos] = row_lse; p.part_scale[pos] = row_scale; }
       }
       tc_fence_before();
       mbar_arrive(&sm->o_free[x]);
@@ -524,7 +558,7 @@ static int grid_items(long long items) { return (int)std::max<long long>(1, std:
 int tc_sparse_fwd_narrow(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                          const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
                          int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o,
-                         float* part_lse, cudaStream_t st, const RowMap& o_map);   // attn_tc_fwd_narrow.cu
+                         float* part_lse, float* part_scale, cudaStream_t st, const RowMap& o_map);   // attn_tc_fwd_narrow.cu
 
 // Forward over the work lists (bf16, head_dim 128).  Key blocks of up to thirteen 128-key tiles go to the narrow
 // kernel (two CTAs of one query tile per SM), longer ones to the wide kernel of this file.  Returns
@@ -532,14 +566,14 @@ int tc_sparse_fwd_narrow(const Dims& D, const void* q, const void* k, const void
 int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                        const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
                        int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o,
-                       float* part_lse, cudaStream_t st, const RowMap& o_map) {
+                       float* part_lse, float* part_scale, cudaStream_t st, const RowMap& o_map) {
   using namespace tcw;
   // Measured: with blocks of 234 to 1638 keys the narrow kernel is 4 to 14 % faster; from about 1900 keys on the
   // two run level, and the narrow one reads every K / V tile twice as often from the L2, which costs a
   // power-capped step more clock than the forward gains.
   if (D.sb <= 13 * BN)
     return tc_sparse_fwd_narrow(D, q, k, v, kb_ptr, q_idx, q_ptr, q_pairs, cap, o, o_resid, lse, status, item_ptr, item_tab,
-                                max_items, part_o, part_lse, st, o_map);
+                                max_items, part_o, part_lse, part_scale, st, o_map);
   CUtensorMap tmK, tmV;
   const uint64_t rows = (uint64_t)D.BH * D.S;
   if (!sm100::make_tmap_bf16_rows(&tmK, k, rows, DH, BN) || !sm100::make_tmap_bf16_rows(&tmV, v, rows, DH, BN))
@@ -553,7 +587,8 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
   p.item_tab = item_tab;
   p.n_kb = (int)n_kb; p.S = D.S; p.Nb = D.Nb; p.sb = D.sb; p.BH = D.BH;
   p.scale_log2 = D.scale * 1.4426950408889634f;
-  p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
+  p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse;
+  p.part_o = reinterpret_cast<__half*>(part_o); p.part_lse = part_lse; p.part_scale = part_scale;
   p.capacity = cap; p.status = status; p.prof = debug_wait_profile();
   p.o_map = o_map;
   p.part_o_32 = (reinterpret_cast<uintptr_t>(part_o) % 32) == 0;
@@ -567,8 +602,8 @@ int tc_sparse_fwd(const Dims& D, const void* q, const void* k, const void* v, co
     attn_fwd_wide_kernel<false><<<grid_items(cap / IM + n_kb), THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
   }
   const long long nq = (long long)D.BH * D.S;
-  simt::merge_batched_kernel<__nv_bfloat16><<<(int)std::min<long long>((nq + 255) / 256, sm_count() * 8), 256, 0, st>>>(
-      q_ptr, q_pairs, nq, part_o, part_lse, cap, (__nv_bfloat16*)o, (__nv_bfloat16*)o_resid, lse, o_map);
+  simt::merge_batched_kernel<__nv_bfloat16, __half><<<(int)std::min<long long>((nq + 255) / 256, sm_count() * 8), 256, 0, st>>>(
+      q_ptr, q_pairs, nq, p.part_o, part_lse, part_scale, cap, (__nv_bfloat16*)o, (__nv_bfloat16*)o_resid, lse, o_map);
   VMOBA_LAUNCH_OK(4);
   return VMOBA_OK;
 }
@@ -585,7 +620,7 @@ int tc_dense_fwd(const Dims& D, const void* q, const void* k, const void* v, voi
   p.item_tab = nullptr;
   p.n_kb = 0; p.S = D.S; p.Nb = 1; p.sb = D.S; p.BH = D.BH;
   p.scale_log2 = D.scale * 1.4426950408889634f;
-  p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = nullptr; p.part_lse = nullptr;
+  p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = nullptr; p.part_lse = nullptr; p.part_scale = nullptr;
   p.capacity = 0; p.part_o_32 = 0; p.o_map = RowMap();
   p.status = status; p.prof = debug_wait_profile();
   VMOBA_CUDA_OK(cudaFuncSetAttribute(attn_fwd_wide_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,

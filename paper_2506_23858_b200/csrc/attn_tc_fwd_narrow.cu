@@ -21,6 +21,8 @@
 // item ahead.
 #include <algorithm>
 
+#include <cuda_fp16.h>
+
 #include "attn_simt.cuh"
 #include "sm100.cuh"
 
@@ -69,8 +71,9 @@ struct Params {
   __nv_bfloat16* o_resid;
   RowMap o_map;            // where the rows of o go (block-major, or raster order through perm); o_resid is block-major
   float* lse;
-  float* part_o;
+  __half* part_o;          // partial rows: fp16 values times part_scale[row]
   float* part_lse;
+  float* part_scale;
   int part_o_32;           // part_o is 32-byte aligned: rows go out with 32-byte stores
   int32_t* status;
   unsigned long long* prof;   // optional per-section cycle counters (diagnostics), or null
@@ -144,6 +147,27 @@ __device__ __forceinline__ void exp_pack64(const uint32_t (&sv)[64], float scale
     add2(s0, s1, s0, s1, p0, p1);
     pk[i] = pack_bf16(p0, p1);
     add2(r0, r1, r0, r1, __uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u));
+  }
+}
+
+// Partial rows are stored as fp16 times a power of two per row: the smallest one at or above the row's largest
+// magnitude (1 for a row of zeros), so that the values use the format's full precision whatever the scale of V.
+__device__ __forceinline__ float pow2_at_or_above(float x) {
+  const uint32_t u = (__float_as_uint(x) + 0x007fffffu) & 0x7f800000u;
+  return u ? __uint_as_float(u) : 1.0f;
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  const __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+// sixteen fp16 values of a partial row: one 32-byte store if the buffer allows it, else two of 16 bytes
+__device__ __forceinline__ void store_part16(__half* dst, const uint32_t (&h)[8], int aligned32) {
+  if (aligned32) {
+    st_global_v8(dst, h[0], h[1], h[2], h[3], h[4], h[5], h[6], h[7]);
+  } else {
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(h[0], h[1], h[2], h[3]);
+    reinterpret_cast<uint4*>(dst)[1] = make_uint4(h[4], h[5], h[6], h[7]);
   }
 }
 
@@ -436,6 +460,24 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       const long long G_ = it.head_off + qpos;
       const long long o_row_off = RASTER ? ((row_ok && direct) ? p.o_map.off(G_, DH) : 0) : G_ * DH;
       const long long pos = (long long)it.list_lo + r;
+      const bool partial = row_ok && !direct;
+      // a partial row goes out as fp16 times a power of two: find the row's largest magnitude first
+      float mul = inv, row_scale = 1.0f;
+      if (__any_sync(0xffffffffu, partial)) {
+        float amax = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+          uint32_t ov[16];
+          tmem_ld16(o_tmem + c * 16, ov);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(ov[i])));
+        }
+        if (partial) {
+          row_scale = pow2_at_or_above(amax * inv);
+          mul = inv / row_scale;
+        }
+      }
 #pragma unroll 1
       for (int c = 0; c < 8; ++c) {
         uint32_t ov[16];
@@ -458,25 +500,15 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
               store8_resid(dst + i, rdst ? rdst + i : nullptr, v8);
             }
           } else {
-            float* dst = p.part_o + pos * DH + col;
-            if (!p.part_o_32) {
+            uint32_t h[8];
 #pragma unroll
-              for (int i = 0; i < 16; i += 4)
-                *reinterpret_cast<float4*>(dst + i) =
-                    make_float4(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
-                                __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv);
-            } else
-#pragma unroll
-            for (int i = 0; i < 16; i += 8)
-              st_global_v8(dst + i, __uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
-                           __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv,
-                           __uint_as_float(ov[i + 4]) * inv, __uint_as_float(ov[i + 5]) * inv,
-                           __uint_as_float(ov[i + 6]) * inv, __uint_as_float(ov[i + 7]) * inv);
+            for (int i = 0; i < 8; ++i) h[i] = pack_half2(__uint_as_float(ov[2 * i]) * mul, __uint_as_float(ov[2 * i + 1]) * mul);
+            store_part16(p.part_o + pos * DH + col, h, p.part_o_32);
           }
         }
       }
       if (row_ok) {
-        if (direct) p.lse[G_] = row_lse; else p.part_lse[pos] = row_lse;
+        if (direct) p.lse[G_] = row_lse; else { p.part_lse[pos] = row_lse; p.part_scale[pos] = row_scale; }
       }
     }
   } else {
@@ -581,6 +613,24 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
       const long long G_ = it.head_off + qpos;
       const long long o_row_off = RASTER ? ((row_ok && direct) ? p.o_map.off(G_, DH) : 0) : G_ * DH;
       const long long pos = (long long)it.list_lo + r;
+      const bool partial = row_ok && !direct;
+      // a partial row goes out as fp16 times a power of two: find the row's largest magnitude first
+      float mul = inv, row_scale = 1.0f;
+      if (__any_sync(0xffffffffu, partial)) {
+        float amax = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t ov[32];
+          tmem_ld32(o_tmem + c * 32, ov);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(__uint_as_float(ov[i])));
+        }
+        if (partial) {
+          row_scale = pow2_at_or_above(amax * inv);
+          mul = inv / row_scale;
+        }
+      }
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         uint32_t ov[32];
@@ -599,25 +649,19 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
               store8_resid(dst + i, rdst ? rdst + i : nullptr, v8);
             }
           } else {
-            float* dst = p.part_o + pos * DH + col;
-            if (!p.part_o_32) {
 #pragma unroll
-              for (int i = 0; i < 32; i += 4)
-                *reinterpret_cast<float4*>(dst + i) =
-                    make_float4(__uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
-                                __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv);
-            } else
+            for (int i = 0; i < 32; i += 16) {
+              uint32_t h[8];
 #pragma unroll
-            for (int i = 0; i < 32; i += 8)       // 32-byte stores: a thread's row is 512 contiguous bytes
-              st_global_v8(dst + i, __uint_as_float(ov[i]) * inv, __uint_as_float(ov[i + 1]) * inv,
-                           __uint_as_float(ov[i + 2]) * inv, __uint_as_float(ov[i + 3]) * inv,
-                           __uint_as_float(ov[i + 4]) * inv, __uint_as_float(ov[i + 5]) * inv,
-                           __uint_as_float(ov[i + 6]) * inv, __uint_as_float(ov[i + 7]) * inv);
+              for (int k = 0; k < 8; ++k)
+                h[k] = pack_half2(__uint_as_float(ov[i + 2 * k]) * mul, __uint_as_float(ov[i + 2 * k + 1]) * mul);
+              store_part16(p.part_o + pos * DH + col + i, h, p.part_o_32);
+            }
           }
         }
       }
       if (row_ok) {
-        if (direct) p.lse[G_] = row_lse; else p.part_lse[pos] = row_lse;
+        if (direct) p.lse[G_] = row_lse; else { p.part_lse[pos] = row_lse; p.part_scale[pos] = row_scale; }
       }
       // No barrier tells the MMA warp that the accumulator has been read: the next thing it waits for from these
       // threads is the P of the next item's first tile, which they write after this point.
@@ -638,7 +682,7 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
 int tc_sparse_fwd_narrow(const Dims& D, const void* q, const void* k, const void* v, const int* kb_ptr, const int* q_idx,
                          const int* q_ptr, const int* q_pairs, long long cap, void* o, void* o_resid, float* lse,
                          int32_t* status, int* item_ptr, int* item_tab, long long max_items, float* part_o,
-                         float* part_lse, cudaStream_t st, const RowMap& o_map) {
+                         float* part_lse, float* part_scale, cudaStream_t st, const RowMap& o_map) {
   using namespace tcn;
   CUtensorMap tmK, tmV;
   const uint64_t rows = (uint64_t)D.BH * D.S;
@@ -653,7 +697,8 @@ int tc_sparse_fwd_narrow(const Dims& D, const void* q, const void* k, const void
   p.item_desc = reinterpret_cast<const int4*>(item_tab);
   p.n_kb = (int)n_kb; p.S = D.S; p.Nb = D.Nb; p.sb = D.sb;
   p.scale_log2 = D.scale * 1.4426950408889634f;
-  p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse; p.part_o = part_o; p.part_lse = part_lse;
+  p.o = (__nv_bfloat16*)o; p.o_resid = (__nv_bfloat16*)o_resid; p.lse = lse;
+  p.part_o = reinterpret_cast<__half*>(part_o); p.part_lse = part_lse; p.part_scale = part_scale;
   p.status = status; p.prof = debug_wait_profile();
   p.part_o_32 = (reinterpret_cast<uintptr_t>(part_o) % 32) == 0;
   p.o_map = o_map;
@@ -673,8 +718,8 @@ int tc_sparse_fwd_narrow(const Dims& D, const void* q, const void* k, const void
     attn_fwd_narrow_kernel<false, false><<<(int)items, THREADS, SMEM_BYTES, st>>>(tmK, tmV, p);
   }
   const long long nq = (long long)D.BH * D.S;
-  simt::merge_batched_kernel<__nv_bfloat16><<<(int)std::min<long long>((nq + 255) / 256, sm_count() * 8), 256, 0, st>>>(
-      q_ptr, q_pairs, nq, part_o, part_lse, cap, (__nv_bfloat16*)o, (__nv_bfloat16*)o_resid, lse, o_map);
+  simt::merge_batched_kernel<__nv_bfloat16, __half><<<(int)std::min<long long>((nq + 255) / 256, sm_count() * 8), 256, 0, st>>>(
+      q_ptr, q_pairs, nq, p.part_o, part_lse, part_scale, cap, (__nv_bfloat16*)o, (__nv_bfloat16*)o_resid, lse, o_map);
   VMOBA_LAUNCH_OK(4);
   return VMOBA_OK;
 }
