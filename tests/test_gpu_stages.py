@@ -282,6 +282,33 @@ def test_sparse_attention_item_and_tile_edges(block):
     U.assert_close(dv, dv_ref, w.dtype, "dv")
 
 
+@pytest.mark.parametrize("block", [(3, 6, 13), (1, 12, 26), (6, 12, 13)], ids=["234keys", "312keys", "936keys"])
+def test_partial_rows_follow_the_scale_of_v(block):
+    """The forward keeps one partial result per (query, block) pair as fp16 values times a power of two chosen per
+    row.  Multiplying v by a power of two (exact in bf16) must therefore multiply o by the same factor bit for bit,
+    far beyond the range of fp16 itself (v reaches about 5 * 2^20 here) and far below it."""
+    w = MID.with_(name="mid_vscale_%d_%d_%d" % block, block=block, tau=0.5)
+    data, ora = _prep(w)
+    shape = vb.shape_of(w)
+    # a random half of all pairs: most queries hold several blocks, so their rows go through the merge
+    masks = np.random.default_rng(17).random((w.B * w.heads, w.S, w.n_blocks)) < 0.5
+    assert (masks.sum(axis=2) >= 2).any()
+    kb_ptr, q_idx, q_ptr, q_pairs, n = lists_from_mask(masks)
+    L = VmobaLayer(shape, capacity=max(n, 1))
+    for name, buf in (("q", L.q_bm), ("k", L.k_bm), ("v", L.v_bm)):
+        buf.copy_(U.bm_to_device(w, U.block_major(w, data, name, ora["perm"])))
+    L.kb_ptr.copy_(kb_ptr); L.q_idx.copy_(q_idx); L.q_ptr.copy_(q_ptr); L.q_pairs.copy_(q_pairs)
+    v0 = L.v_bm.clone()
+    L.attn_fwd(); L.check_status()
+    o0, lse0 = L.o_bm.clone(), L.lse.clone()
+    for factor in (2.0 ** 20, 2.0 ** -20):
+        L.v_bm.copy_(v0 * factor)
+        assert torch.equal(L.v_bm.float(), v0.float() * factor)
+        L.attn_fwd(); L.check_status()
+        assert torch.equal(L.o_bm.float(), o0.float() * factor), factor
+        assert torch.equal(L.lse, lse0)
+
+
 @pytest.mark.parametrize("w", [CASES[0], CASES[3], CASES[8]], ids=[IDS[0], IDS[3], IDS[8]])
 def test_sparse_attention_full_mask_equals_dense_oracle(w):
     """tau = 1: the sparse path over every pair must reproduce dense softmax attention."""
