@@ -11,8 +11,12 @@
 //
 //   warp 0        TMA producer: K and V tiles, one stage each (a K tile is reloaded as soon as its Q K^T has run)
 //   warp 1        MMA issuer (all lanes walk the loop, one elected lane issues)
-//   warps 4-7     softmax + epilogue: thread = one query row
-//   warps 2,3     loaders: gather the 128 Q rows (and per-row output bookkeeping) of the NEXT item, 64 rows at a time
+//   warps 4-7     softmax (+ epilogue, unless warps 8-11 exist): thread = one query row
+//   warps 2,3     loaders: gather the 128 Q rows (and per-row output bookkeeping) of the NEXT item
+//   warps 8-11    (key blocks of up to four tiles only) epilogue: read the accumulator, write the rows
+//
+// Rows of queries with a single block are final and go to o; the others are partial results that the merge pass
+// combines: fp16 values times a power of two per row, beside the row's lse.
 //
 // TMEM: S (128 columns; the bf16 P is written over columns 64..127) and the accumulator O (128 columns).  A softmax
 // thread reads its row in two halves, first for the maximum and, after the second half has been turned into P,
@@ -388,9 +392,11 @@ attn_fwd_narrow_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_con
         asm volatile("cp.async.commit_group;" ::: "memory");
         asm volatile("cp.async.wait_group 0;" ::: "memory");
       }
-      constexpr int RR = 64;                       // rows per round (a round's rows wait in registers)
+      // without epilogue warps the loaders have 128 registers: two rounds of 64 rows that wait in registers
+      constexpr int RR = 64;
       constexpr int NI = RR / 4;
-      for (int rnd = 0; rnd < (SPLIT ? 0 : BM / RR); ++rnd) {
+      if constexpr (!SPLIT)
+      for (int rnd = 0; rnd < BM / RR; ++rnd) {
         uint4 v[NI];
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
