@@ -282,6 +282,29 @@ def test_sparse_attention_item_and_tile_edges(block):
     U.assert_close(dv, dv_ref, w.dtype, "dv")
 
 
+@pytest.mark.parametrize("block", [(3, 6, 13), (6, 12, 13), (6, 12, 26)], ids=["234keys", "936keys", "1872keys"])
+def test_attention_with_no_selected_pair(block):
+    """Empty work lists (no query selected any block): every kernel variant of the forward and the backward must
+    return with o = 0, lse = -inf and zero gradients."""
+    w = MID.with_(name="mid_empty_%d_%d_%d" % block, block=block)
+    shape = vb.shape_of(w)
+    masks = np.zeros((w.B * w.heads, w.S, w.n_blocks), dtype=bool)
+    kb_ptr, q_idx, q_ptr, q_pairs, n = lists_from_mask(masks)
+    assert n == 0
+    L = VmobaLayer(shape, capacity=1, with_backward=True)
+    for buf in (L.q_bm, L.k_bm, L.v_bm, L.do_bm):
+        buf.normal_()
+    L.kb_ptr.copy_(kb_ptr); L.q_idx.copy_(q_idx); L.q_ptr.copy_(q_ptr); L.q_pairs.copy_(q_pairs)
+    L.o_bm.fill_(7.0); L.lse.fill_(7.0)
+    for g in (L.dq_bm, L.dk_bm, L.dv_bm):
+        g.fill_(7.0)
+    L.attn_fwd()
+    L.attn_bwd()
+    L.check_status()
+    assert torch.all(L.o_bm == 0) and torch.all(torch.isneginf(L.lse))
+    assert torch.all(L.dq_bm == 0) and torch.all(L.dk_bm == 0) and torch.all(L.dv_bm == 0)
+
+
 @pytest.mark.parametrize("block", [(3, 6, 13), (1, 12, 26), (6, 12, 13)], ids=["234keys", "312keys", "936keys"])
 def test_partial_rows_follow_the_scale_of_v(block):
     """The forward keeps one partial result per (query, block) pair as fp16 values times a power of two chosen per
